@@ -1,0 +1,260 @@
+"""ctypes front end of the CPU oracle (``cstep_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by ``__graft_entry__.smoke()``
+and by the ``cpu_baseline`` / ``--impl reference`` legs of ``bench.py``. The
+product package never imports this module and this module never imports the
+product package.
+
+Arrays are numpy, on the host. Every call works on a list of tensors
+(``w`` and optional ``lam`` per tensor) and returns freshly allocated outputs.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "cstep_oracle.c")
+_LIB = os.path.join(_HERE, "libcstep_oracle.so")
+
+FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY = 1, 2, 4
+
+CFLAGS = ["-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
+          "-fno-unsafe-math-optimizations", "-Wall"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + ".tmp%d" % os.getpid()
+    subprocess.run(["gcc"] + CFLAGS + ["-o", tmp, _SRC, "-lm"], check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Tensor(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("lam", C.c_void_p), ("theta", C.c_void_p),
+                ("mask", C.c_void_p), ("lam_out", C.c_void_p), ("grad", C.c_void_p),
+                ("theta_h", C.c_void_p), ("numel", C.c_int64), ("ndim", C.c_int32),
+                ("shape", C.c_int64 * 4)]
+
+
+class _Result(C.Structure):
+    _fields_ = [("n_units", C.c_int64), ("n_zero", C.c_int64), ("n_keep", C.c_int64),
+                ("tau_key", C.c_uint64), ("tau_id", C.c_int64), ("n_gt", C.c_int64),
+                ("n_tie", C.c_int64), ("n_tie_kept", C.c_int64), ("tau_norm", C.c_float)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        assert L.orc_sizeof_tensor() == C.sizeof(_Tensor)
+        assert L.orc_sizeof_result() == C.sizeof(_Result)
+        L.orc_round_count.restype = C.c_int64
+        L.orc_round_count.argtypes = [C.c_double, C.c_int64]
+        L.orc_f32_to_f16.restype = C.c_uint16
+        L.orc_f32_to_f16.argtypes = [C.c_uint32]
+        L.orc_f16_to_f32.restype = C.c_uint32
+        L.orc_f16_to_f32.argtypes = [C.c_uint16]
+        L.orc_f32_to_f16_array.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+        L.orc_f32_to_f16_range.argtypes = [C.c_uint32, C.c_int64, C.c_void_p]
+        L.orc_form_u.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int64, C.c_void_p]
+        L.orc_lagrange.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_uint,
+                                   C.c_int64, C.c_void_p, C.c_void_p]
+        L.orc_structure_norms.restype = C.c_int64
+        L.orc_structure_norms.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_int, C.c_int,
+                                          C.c_int, C.c_void_p]
+        L.orc_cstep_prune.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_float, C.c_uint,
+                                      C.c_void_p]
+        L.orc_cstep_filter.argtypes = list(L.orc_cstep_prune.argtypes)
+        L.orc_cstep_block.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_float, C.c_int,
+                                      C.c_int, C.c_uint, C.c_void_p]
+        L.orc_cstep_quantize.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint]
+        L.orc_lagrange_update.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint]
+        if not L.orc_denormals_ok():
+            raise RuntimeError("subnormal fp32 arithmetic is flushed in this process; "
+                               "the oracle's results would not be IEEE")
+        _lib = L
+    return _lib
+
+
+@dataclass
+class Result:
+    n_units: int
+    n_zero: int
+    n_keep: int
+    tau_key: int
+    tau_id: int
+    n_gt: int
+    n_tie: int
+    n_tie_kept: int
+    tau_norm: float
+
+
+@dataclass
+class Outputs:
+    theta: List[np.ndarray]
+    mask: List[np.ndarray]
+    lam: List[np.ndarray]        # multipliers after the call (copy of the input if not updated)
+    grad: List[np.ndarray]
+    theta_h: List[np.ndarray]
+    result: Optional[Result] = None
+
+
+def fuse_bits(fuse: Sequence[str]) -> int:
+    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY}
+    b = 0
+    for f in fuse:
+        b |= table[f]
+    return b
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _table(ws, lams, thetas=None):
+    T = len(ws)
+    keep = []          # keeps every numpy buffer alive while the C call runs
+    tab = (_Tensor * max(T, 1))()
+    out = Outputs([], [], [], [], [])
+    for t in range(T):
+        w = np.ascontiguousarray(ws[t], dtype=np.float32)
+        lam = None if (lams is None or lams[t] is None) else np.ascontiguousarray(
+            lams[t], dtype=np.float32)
+        n = w.size
+        theta = (np.empty(w.shape, np.float32) if thetas is None
+                 else np.ascontiguousarray(thetas[t], dtype=np.float32).copy())
+        mask = np.empty(w.shape, np.uint8)
+        lam_out = np.zeros(w.shape, np.float32)
+        grad = np.zeros(w.shape, np.float32)
+        theta_h = np.zeros(w.shape, np.uint16)
+        keep += [w, lam]
+        e = tab[t]
+        e.w, e.lam, e.theta, e.mask = _ptr(w), _ptr(lam), _ptr(theta), _ptr(mask)
+        e.lam_out, e.grad, e.theta_h = _ptr(lam_out), _ptr(grad), _ptr(theta_h)
+        e.numel, e.ndim = n, w.ndim
+        assert 1 <= w.ndim <= 4
+        for d in range(4):
+            e.shape[d] = w.shape[d] if d < w.ndim else 1
+        out.theta.append(theta); out.mask.append(mask); out.lam.append(lam_out)
+        out.grad.append(grad); out.theta_h.append(theta_h)
+    return tab, out, keep
+
+
+def _result(r: _Result) -> Result:
+    return Result(r.n_units, r.n_zero, r.n_keep, r.tau_key, r.tau_id, r.n_gt, r.n_tie,
+                  r.n_tie_kept, float(r.tau_norm))
+
+
+def round_count(s: float, n: int) -> int:
+    return int(lib().orc_round_count(float(s), int(n)))
+
+
+def form_u(w: np.ndarray, lam: Optional[np.ndarray], mu: float) -> np.ndarray:
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    u = np.empty_like(w)
+    l = None if lam is None else np.ascontiguousarray(lam, dtype=np.float32)
+    lib().orc_form_u(_ptr(w), _ptr(l), C.c_float(mu), w.size, _ptr(u))
+    return u
+
+
+def f32_to_f16_bits(x: np.ndarray) -> np.ndarray:
+    """binary16 bits (uint16) of each fp32 value (or uint32 bit pattern) in x."""
+    b = np.ascontiguousarray(x)
+    if b.dtype == np.float32:
+        b = b.view(np.uint32)
+    assert b.dtype == np.uint32
+    out = np.empty(b.shape, np.uint16)
+    lib().orc_f32_to_f16_array(_ptr(b), b.size, _ptr(out))
+    return out
+
+
+def f32_to_f16_range(first: int, n: int) -> np.ndarray:
+    out = np.empty(n, np.uint16)
+    lib().orc_f32_to_f16_range(C.c_uint32(first), n, _ptr(out))
+    return out
+
+
+def f16_bits_to_f32(h: np.ndarray) -> np.ndarray:
+    h = np.ascontiguousarray(h, dtype=np.uint16)
+    out = np.empty(h.shape, np.uint32)
+    L = lib()
+    flat_h, flat_o = h.reshape(-1), out.reshape(-1)
+    for i in range(flat_h.size):
+        flat_o[i] = L.orc_f16_to_f32(int(flat_h[i]))
+    return out.view(np.float32)
+
+
+def structure_norms(ws, lams, mu: float, kind: str, block=(4, 4)) -> np.ndarray:
+    """fp64 nu of every ranked structure, in global structure order."""
+    tab, _, keep = _table(ws, lams)
+    k = {"filter": 0, "block": 1}[kind]
+    S = lib().orc_structure_norms(tab, len(ws), C.c_float(mu), k, block[0], block[1], None)
+    nu = np.empty(S, np.float64)
+    lib().orc_structure_norms(tab, len(ws), C.c_float(mu), k, block[0], block[1], _ptr(nu))
+    return nu
+
+
+def cstep_prune(ws, lams, s: float, mu: float, fuse: Sequence[str] = ()) -> Outputs:
+    tab, out, keep = _table(ws, lams)
+    r = _Result()
+    rc = lib().orc_cstep_prune(tab, len(ws), float(s), C.c_float(mu), fuse_bits(fuse), C.byref(r))
+    assert rc == 0
+    out.result = _result(r)
+    return out
+
+
+def cstep_filter(ws, lams, s: float, mu: float, fuse: Sequence[str] = ()) -> Outputs:
+    tab, out, keep = _table(ws, lams)
+    r = _Result()
+    rc = lib().orc_cstep_filter(tab, len(ws), float(s), C.c_float(mu), fuse_bits(fuse), C.byref(r))
+    assert rc == 0
+    out.result = _result(r)
+    return out
+
+
+def cstep_block(ws, lams, s: float, mu: float, block=(4, 4), fuse: Sequence[str] = ()) -> Outputs:
+    tab, out, keep = _table(ws, lams)
+    r = _Result()
+    rc = lib().orc_cstep_block(tab, len(ws), float(s), C.c_float(mu), int(block[0]), int(block[1]),
+                               fuse_bits(fuse), C.byref(r))
+    assert rc == 0
+    out.result = _result(r)
+    return out
+
+
+def cstep_quantize(ws, lams, mu: float, fuse: Sequence[str] = ()) -> Outputs:
+    tab, out, keep = _table(ws, lams)
+    rc = lib().orc_cstep_quantize(tab, len(ws), C.c_float(mu), fuse_bits(fuse))
+    assert rc == 0
+    return out
+
+
+def lagrange_update(ws, thetas, lams, mu: float, fuse: Sequence[str] = ("lambda",)) -> Outputs:
+    tab, out, keep = _table(ws, lams, thetas)
+    rc = lib().orc_lagrange_update(tab, len(ws), C.c_float(mu), fuse_bits(fuse))
+    assert rc == 0
+    return out
+
+
+def run_config(ws) -> Outputs:
+    """Run the call a ``workloads.WeightSet`` names (duck typed: only its fields are read)."""
+    if ws.op == "prune":
+        return cstep_prune(ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
+    if ws.op == "filter":
+        return cstep_filter(ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
+    if ws.op == "block":
+        return cstep_block(ws.w, ws.lam, ws.sparsity, ws.mu, ws.block, ws.fuse)
+    raise ValueError(ws.op)

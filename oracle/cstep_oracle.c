@@ -1,0 +1,435 @@
+/*
+ * CPU oracle for the C-step of the learning-compression (L-C) scheme.
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the slow, plain definition that the
+ * CUDA path is checked against. Nothing in the product path may include,
+ * link or call it; it shares no code, header, table or helper with the
+ * CUDA kernels.
+ *
+ * What it computes, with the passage each piece follows:
+ *
+ *  - compression mapping C(w) = argmin_Theta ||w - D(Theta)||^2 (Section 3.3,
+ *    text under Eq. 1). For pruning, D is the identity and Theta is limited
+ *    in its number of non-zeros, so the argmin keeps the entries (or whole
+ *    structures) of largest magnitude (largest L2 norm) and zeroes the rest.
+ *    Here that is written out literally: sort all units by magnitude and
+ *    keep the first k.
+ *  - target sparsity = proportion of zero-valued parameters (Introduction,
+ *    definition of "target sparsity"): exactly Z = round(s * units) units are
+ *    zeroed, one global ranking over all tensors ("global sparsity ...
+ *    across all the layers", Section 3).
+ *  - structured pruning aggregates filters (3-D blocks) or n-D blocks and
+ *    prunes whole structures (Table 1, FilterPrune / BlockPrune); the
+ *    criterion used here is the L2 norm, which is the argmin above.
+ *  - low-precision approximation: each parameter gets the nearest value of
+ *    the lower-precision format (Section 2, "quantization using a fixed
+ *    codebook"); 32-bit to 16-bit floating point, done by explicit bit
+ *    manipulation with round-to-nearest-even.
+ *  - scheme order for P+Q is prune, then quantise (Evaluation, Objective 1).
+ *  - augmented-Lagrangian quantities of the L-C algorithm (Section 3.3 cites
+ *    the AL method; the paper prints no formulas): u = w - lambda/mu,
+ *    lambda <- lambda - mu (w - theta), penalty gradient mu (w - theta) - lambda.
+ *
+ * All fp32 arithmetic is done one IEEE operation at a time (compile with
+ * -ffp-contract=off and without -ffast-math); norms accumulate in fp64 in
+ * index order.
+ *
+ * Pins: every function here is pinned by tests/test_oracle_pins.py (brute
+ * force ranking, all-supports enumeration of the argmin, closed forms,
+ * library routines, hand-computed binary16 values). The printed compression
+ * ratios of Table 2 depend on trained weights and pin nothing here.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+#define ORC_FUSE_FP16    1u
+#define ORC_FUSE_LAMBDA  2u
+#define ORC_FUSE_PENALTY 4u
+
+typedef struct {
+    const float *w;        /* weights, never written                          */
+    const float *lambda;   /* multipliers, may be NULL (treated as zero)      */
+    float *theta;          /* out: compressed weights                         */
+    uint8_t *mask;         /* out: 1 = kept, may be NULL                      */
+    float *lambda_out;     /* out: updated multipliers, may be NULL           */
+    float *grad;           /* out: penalty gradient, may be NULL              */
+    uint16_t *theta_h;     /* out: binary16 bits of theta, may be NULL        */
+    int64_t numel;
+    int32_t ndim;
+    int64_t shape[4];
+} orc_tensor;
+
+typedef struct {
+    int64_t n_units;   /* units that were ranked (elements or structures)     */
+    int64_t n_zero;    /* Z                                                    */
+    int64_t n_keep;    /* k = n_units - Z                                      */
+    uint64_t tau_key;  /* key of the weakest kept unit                         */
+    int64_t tau_id;    /* global id of the weakest kept unit, -1 if k == 0     */
+    int64_t n_gt;      /* units with key  > tau                                */
+    int64_t n_tie;     /* units with key == tau                                */
+    int64_t n_tie_kept;/* of those, how many are kept (lowest ids first)       */
+    float tau_norm;    /* structured: (float)sqrt(nu) of the weakest kept unit */
+} orc_result;
+
+/* ---- bit helpers ------------------------------------------------------- */
+static uint32_t f32_bits(float x) { uint32_t b; memcpy(&b, &x, 4); return b; }
+static float bits_f32(uint32_t b) { float x; memcpy(&x, &b, 4); return x; }
+static uint64_t f64_bits(double x) { uint64_t b; memcpy(&b, &x, 8); return b; }
+
+/* Z = round(s * n): half-up rounding of the product taken in double. */
+int64_t orc_round_count(double s, int64_t n)
+{
+    double z = floor(s * (double)n + 0.5);
+    if (z < 0.0) z = 0.0;
+    if (z > (double)n) z = (double)n;
+    return (int64_t)z;
+}
+
+/* ---- binary32 -> binary16, round to nearest even ------------------------ */
+/* Returns the 16 bits. NaN maps to a quiet NaN that keeps the sign and drops
+ * the payload; overflow goes to infinity; results below the smallest normal
+ * are denormalised gradually. */
+uint16_t orc_f32_to_f16(uint32_t b)
+{
+    uint32_t sign = (b >> 16) & 0x8000u;
+    uint32_t e = (b >> 23) & 0xFFu;
+    uint32_t m = b & 0x7FFFFFu;
+    if (e == 0xFFu) {
+        if (m != 0) return (uint16_t)(sign | 0x7E00u);
+        return (uint16_t)(sign | 0x7C00u);
+    }
+    int32_t eh = (int32_t)e - 127 + 15;          /* exponent in binary16 bias */
+    if (eh >= 31) return (uint16_t)(sign | 0x7C00u);
+    if (eh <= 0) {
+        /* subnormal half or zero: value = (1.m) * 2^(e-127); the half
+         * subnormal unit is 2^-24. Shift the 24-bit significand right. */
+        if (e == 0) return (uint16_t)sign;        /* fp32 subnormals are < 2^-126: round to 0 */
+        int32_t shift = 14 - eh;                  /* >= 14 */
+        if (shift > 25) return (uint16_t)sign;
+        uint32_t sig = m | 0x800000u;
+        uint32_t q = sig >> shift;
+        uint32_t rem = sig & ((1u << shift) - 1u);
+        uint32_t half = 1u << (shift - 1);
+        if (rem > half || (rem == half && (q & 1u))) q += 1u;
+        return (uint16_t)(sign | q);              /* q may carry into the normal range: still right */
+    }
+    uint32_t q = ((uint32_t)eh << 10) | (m >> 13);
+    uint32_t rem = m & 0x1FFFu;
+    if (rem > 0x1000u || (rem == 0x1000u && (q & 1u))) q += 1u;   /* may carry to the exponent / inf */
+    return (uint16_t)(sign | q);
+}
+
+/* binary16 -> binary32, exact. */
+uint32_t orc_f16_to_f32(uint16_t h)
+{
+    uint32_t sign = ((uint32_t)h & 0x8000u) << 16;
+    uint32_t e = (h >> 10) & 0x1Fu;
+    uint32_t m = h & 0x3FFu;
+    if (e == 31) return sign | 0x7F800000u | (m << 13);
+    if (e == 0) {
+        if (m == 0) return sign;
+        /* normalise the subnormal */
+        int32_t ex = -14;
+        while (!(m & 0x400u)) { m <<= 1; ex -= 1; }
+        m &= 0x3FFu;
+        return sign | ((uint32_t)(ex + 127) << 23) | (m << 13);
+    }
+    return sign | ((e - 15 + 127) << 23) | (m << 13);
+}
+
+void orc_f32_to_f16_array(const uint32_t *bits, int64_t n, uint16_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_f16(bits[i]);
+}
+
+/* Convert the contiguous range of bit patterns [first, first + n). */
+void orc_f32_to_f16_range(uint32_t first, int64_t n, uint16_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_f16(first + (uint32_t)i);
+}
+
+/* ---- elementwise pieces ------------------------------------------------ */
+/* u = w - lambda / mu, two fp32 operations. */
+void orc_form_u(const float *w, const float *lambda, float mu, int64_t n, float *u)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        if (lambda) {
+            volatile float q = lambda[i] / mu;
+            u[i] = w[i] - q;
+        } else {
+            u[i] = w[i];
+        }
+    }
+}
+
+/* Multiplier update and penalty gradient for one tensor, theta given.
+ *   d = w - theta;  p = mu * d;  lambda' = lambda - p   (if FUSE_LAMBDA)
+ *   g = p - lambda_used, lambda_used = lambda' when updated, else lambda. */
+void orc_lagrange(const float *w, const float *theta, const float *lambda, float mu,
+                  unsigned fuse, int64_t n, float *lambda_out, float *grad)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        float lam = lambda ? lambda[i] : 0.0f;
+        volatile float d = w[i] - theta[i];
+        volatile float p = mu * d;
+        float lam_used = lam;
+        if ((fuse & ORC_FUSE_LAMBDA) && lambda) {
+            volatile float l2 = lam - p;
+            lam_used = l2;
+        }
+        if (lambda_out) lambda_out[i] = lam_used;
+        if ((fuse & ORC_FUSE_PENALTY) && grad) {
+            volatile float g = p - lam_used;
+            grad[i] = g;
+        }
+    }
+}
+
+/* theta (and mask, fp16 bits) for one tensor from u and a 0/1 keep decision
+ * per element, then the multiplier / penalty arithmetic. */
+static void finish_tensor(const orc_tensor *t, const float *u, const uint8_t *keep, float mu,
+                          unsigned fuse)
+{
+    for (int64_t i = 0; i < t->numel; ++i) {
+        uint32_t tb = 0u;
+        uint16_t hb = 0u;
+        if (keep[i]) {
+            if (fuse & ORC_FUSE_FP16) {
+                hb = orc_f32_to_f16(f32_bits(u[i]));
+                tb = orc_f16_to_f32(hb);
+            } else {
+                tb = f32_bits(u[i]);
+                hb = orc_f32_to_f16(tb);
+            }
+        }
+        t->theta[i] = bits_f32(tb);
+        if (t->mask) t->mask[i] = keep[i];
+        if (t->theta_h) t->theta_h[i] = hb;
+    }
+    orc_lagrange(t->w, t->theta, t->lambda, mu, fuse, t->numel, t->lambda_out, t->grad);
+}
+
+/* ---- ranking ----------------------------------------------------------- */
+typedef struct { uint64_t key; int64_t id; } unit_t;
+
+/* Larger key first; among equal keys the lower id first. A total order, so
+ * any comparison sort gives the same sequence as a stable descending sort. */
+static int unit_cmp(const void *a, const void *b)
+{
+    const unit_t *x = (const unit_t *)a, *y = (const unit_t *)b;
+    if (x->key != y->key) return (x->key > y->key) ? -1 : 1;
+    if (x->id != y->id) return (x->id < y->id) ? -1 : 1;
+    return 0;
+}
+
+/* Sort units, mark the first k as kept in keep_unit[id], fill the record. */
+static void rank_units(unit_t *units, int64_t n, double s, uint8_t *keep_unit, orc_result *r,
+                       uint64_t inf_key)
+{
+    int64_t z = orc_round_count(s, n);
+    int64_t k = n - z;
+    qsort(units, (size_t)n, sizeof(unit_t), unit_cmp);
+    for (int64_t i = 0; i < n; ++i) keep_unit[units[i].id] = (uint8_t)(i < k);
+    memset(r, 0, sizeof(*r));
+    r->n_units = n; r->n_zero = z; r->n_keep = k;
+    if (k == 0) {
+        r->tau_key = inf_key; r->tau_id = -1;
+        return;
+    }
+    uint64_t tau = units[k - 1].key;
+    r->tau_key = tau;
+    r->tau_id = units[k - 1].id;
+    for (int64_t i = 0; i < n; ++i) {
+        if (units[i].key > tau) r->n_gt++;
+        else if (units[i].key == tau) { r->n_tie++; if (i < k) r->n_tie_kept++; }
+    }
+}
+
+/* Unstructured magnitude pruning over the whole list (Table 1, Prune()). */
+int orc_cstep_prune(const orc_tensor *ts, int32_t T, double s, float mu, unsigned fuse,
+                    orc_result *res)
+{
+    int64_t N = 0;
+    for (int32_t t = 0; t < T; ++t) N += ts[t].numel;
+    float *u = (float *)malloc(sizeof(float) * (size_t)(N ? N : 1));
+    unit_t *units = (unit_t *)malloc(sizeof(unit_t) * (size_t)(N ? N : 1));
+    uint8_t *keep = (uint8_t *)malloc((size_t)(N ? N : 1));
+    if (!u || !units || !keep) { free(u); free(units); free(keep); return -1; }
+    int64_t off = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        orc_form_u(ts[t].w, ts[t].lambda, mu, ts[t].numel, u + off);
+        for (int64_t i = 0; i < ts[t].numel; ++i) {
+            units[off + i].key = (uint64_t)(f32_bits(u[off + i]) & 0x7FFFFFFFu);
+            units[off + i].id = off + i;
+        }
+        off += ts[t].numel;
+    }
+    rank_units(units, N, s, keep, res, 0x7F800000ull);
+    off = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        finish_tensor(&ts[t], u + off, keep + off, mu, fuse);
+        off += ts[t].numel;
+    }
+    free(u); free(units); free(keep);
+    return 0;
+}
+
+/* nu of each structure of one tensor, fp64, accumulated in index order.
+ * kind 0: filters = slices [f, :, :, :] of a 4-D tensor.
+ * kind 1: bh x bw blocks of a 2-D tensor, numbered row-major; a block that
+ *         sticks out over the edge only sums the elements that exist. */
+static int64_t structure_count(const orc_tensor *t, int kind, int bh, int bw)
+{
+    if (kind == 0) return (t->ndim == 4) ? t->shape[0] : 0;
+    if (t->ndim != 2) return 0;
+    int64_t nbr = (t->shape[0] + bh - 1) / bh, nbc = (t->shape[1] + bw - 1) / bw;
+    return nbr * nbc;
+}
+
+static int64_t structure_of(const orc_tensor *t, int kind, int bh, int bw, int64_t i)
+{
+    if (kind == 0) {
+        int64_t len = t->shape[1] * t->shape[2] * t->shape[3];
+        return i / len;
+    }
+    int64_t C = t->shape[1];
+    int64_t nbc = (C + bw - 1) / bw;
+    int64_t r = i / C, c = i % C;
+    return (r / bh) * nbc + (c / bw);
+}
+
+static void structure_norms(const orc_tensor *t, const float *u, int kind, int bh, int bw,
+                            double *nu)
+{
+    if (kind == 0) {
+        int64_t len = t->shape[1] * t->shape[2] * t->shape[3];
+        for (int64_t f = 0; f < t->shape[0]; ++f) {
+            double acc = 0.0;
+            for (int64_t j = 0; j < len; ++j) {
+                double x = (double)u[f * len + j];
+                acc = acc + x * x;
+            }
+            nu[f] = acc;
+        }
+        return;
+    }
+    int64_t R = t->shape[0], C = t->shape[1];
+    int64_t nbr = (R + bh - 1) / bh, nbc = (C + bw - 1) / bw;
+    for (int64_t br = 0; br < nbr; ++br)
+        for (int64_t bc = 0; bc < nbc; ++bc) {
+            double acc = 0.0;
+            for (int64_t r = br * bh; r < (br + 1) * bh && r < R; ++r)
+                for (int64_t c = bc * bw; c < (bc + 1) * bw && c < C; ++c) {
+                    double x = (double)u[r * C + c];
+                    acc = acc + x * x;
+                }
+            nu[br * nbc + bc] = acc;
+        }
+}
+
+/* nu for every structure in the list, in global structure order; returns the
+ * count. nu may be NULL to only count. */
+int64_t orc_structure_norms(const orc_tensor *ts, int32_t T, float mu, int kind, int bh, int bw,
+                            double *nu)
+{
+    int64_t S = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        int64_t c = structure_count(&ts[t], kind, bh, bw);
+        if (c && nu) {
+            float *u = (float *)malloc(sizeof(float) * (size_t)ts[t].numel);
+            orc_form_u(ts[t].w, ts[t].lambda, mu, ts[t].numel, u);
+            structure_norms(&ts[t], u, kind, bh, bw, nu + S);
+            free(u);
+        }
+        S += c;
+    }
+    return S;
+}
+
+static int cstep_structured(const orc_tensor *ts, int32_t T, double s, float mu, unsigned fuse,
+                            int kind, int bh, int bw, orc_result *res)
+{
+    int64_t S = orc_structure_norms(ts, T, mu, kind, bh, bw, NULL);
+    double *nu = (double *)malloc(sizeof(double) * (size_t)(S ? S : 1));
+    unit_t *units = (unit_t *)malloc(sizeof(unit_t) * (size_t)(S ? S : 1));
+    uint8_t *keep_s = (uint8_t *)malloc((size_t)(S ? S : 1));
+    if (!nu || !units || !keep_s) { free(nu); free(units); free(keep_s); return -1; }
+    orc_structure_norms(ts, T, mu, kind, bh, bw, nu);
+    for (int64_t i = 0; i < S; ++i) { units[i].key = f64_bits(nu[i]); units[i].id = i; }
+    rank_units(units, S, s, keep_s, res, 0x7FF0000000000000ull);
+    if (res->n_keep > 0) res->tau_norm = (float)sqrt(nu[res->tau_id]);
+    int64_t sbase = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        int64_t n = ts[t].numel;
+        int64_t c = structure_count(&ts[t], kind, bh, bw);
+        float *u = (float *)malloc(sizeof(float) * (size_t)(n ? n : 1));
+        uint8_t *keep = (uint8_t *)malloc((size_t)(n ? n : 1));
+        orc_form_u(ts[t].w, ts[t].lambda, mu, n, u);
+        for (int64_t i = 0; i < n; ++i)
+            keep[i] = c ? keep_s[sbase + structure_of(&ts[t], kind, bh, bw, i)] : 1;
+        finish_tensor(&ts[t], u, keep, mu, fuse);
+        free(u); free(keep);
+        sbase += c;
+    }
+    free(nu); free(units); free(keep_s);
+    return 0;
+}
+
+/* Filter pruning (Table 1, FilterPrune): 4-D tensors are ranked by filter,
+ * every other tensor passes through unpruned (theta = u, mask = 1). */
+int orc_cstep_filter(const orc_tensor *ts, int32_t T, double s, float mu, unsigned fuse,
+                     orc_result *res)
+{
+    return cstep_structured(ts, T, s, mu, fuse, 0, 0, 0, res);
+}
+
+/* Block pruning (Table 1, BlockPrune): 2-D tensors are ranked by bh x bw
+ * block, every other tensor passes through unpruned. */
+int orc_cstep_block(const orc_tensor *ts, int32_t T, double s, float mu, int bh, int bw,
+                    unsigned fuse, orc_result *res)
+{
+    if (bh < 1 || bw < 1) return -2;
+    return cstep_structured(ts, T, s, mu, fuse, 1, bh, bw, res);
+}
+
+/* Quantisation only (Table 1, Quantize(float16)): theta = Q(u), mask = 1. */
+int orc_cstep_quantize(const orc_tensor *ts, int32_t T, float mu, unsigned fuse)
+{
+    for (int32_t t = 0; t < T; ++t) {
+        int64_t n = ts[t].numel;
+        float *u = (float *)malloc(sizeof(float) * (size_t)(n ? n : 1));
+        uint8_t *keep = (uint8_t *)malloc((size_t)(n ? n : 1));
+        orc_form_u(ts[t].w, ts[t].lambda, mu, n, u);
+        memset(keep, 1, (size_t)n);
+        finish_tensor(&ts[t], u, keep, mu, fuse | ORC_FUSE_FP16);
+        free(u); free(keep);
+    }
+    return 0;
+}
+
+/* Multiplier update / penalty gradient with theta supplied by the caller. */
+int orc_lagrange_update(const orc_tensor *ts, int32_t T, float mu, unsigned fuse)
+{
+    for (int32_t t = 0; t < T; ++t)
+        orc_lagrange(ts[t].w, ts[t].theta, ts[t].lambda, mu, fuse, ts[t].numel,
+                     ts[t].lambda_out, ts[t].grad);
+    return 0;
+}
+
+/* 1 when subnormal fp32 arithmetic is intact in this process (no flush to
+ * zero, no denormals-are-zero), which every function above relies on. */
+int orc_denormals_ok(void)
+{
+    volatile float tiny = bits_f32(0x00000001u);
+    volatile float two = 2.0f;
+    volatile float r = tiny * two;
+    volatile float mn = bits_f32(0x00800000u);
+    volatile float half = 0.5f;
+    volatile float r2 = mn * half;
+    return f32_bits(r) == 0x00000002u && f32_bits(r2) == 0x00400000u;
+}
+
+unsigned orc_sizeof_tensor(void) { return (unsigned)sizeof(orc_tensor); }
+unsigned orc_sizeof_result(void) { return (unsigned)sizeof(orc_result); }
