@@ -1,0 +1,202 @@
+/*
+ * condensa_cstep.h - C ABI of the B200 (sm_100a) C-step library.
+ *
+ * The C-step of the learning-compression (L-C) scheme (paper Section 3.3): given
+ * the current weights w, the multipliers lambda and the penalty weight mu, form
+ *
+ *      u = w - lambda / mu
+ *
+ * and replace theta by the compression mapping C(u) = argmin_Theta ||u - D(Theta)||^2
+ * (Section 3.3, text under Eq. 1), followed by the augmented-Lagrangian updates
+ *
+ *      lambda <- lambda - mu (w - theta)          (multiplier update)
+ *      g       = mu (w - theta) - lambda          (penalty gradient the L step adds)
+ *
+ * The compression mappings offered are the paper's pre-built schemes (Table 1):
+ * Prune() (unstructured magnitude pruning), FilterPrune (3-D blocks),
+ * BlockPrune (2-D blocks), Quantize(float16) and Compose([Prune, Quantize]).
+ * One sparsity is applied globally over the whole tensor list (Section 3: the
+ * L-C optimizer "distributes this global sparsity across all the layers").
+ *
+ * Conventions
+ *  - Every function returns CONDENSA_OK (0) or a negative CONDENSA_ERR_* code and
+ *    never throws. condensa_last_error() gives a text for the last failure of a
+ *    context.
+ *  - All tensor pointers in condensa_tensor are DEVICE pointers on the context's
+ *    device unless a function says "host". They are owned by the caller, must
+ *    stay valid until the stream has run the call, are contiguous row-major, and
+ *    need only their natural alignment (4 bytes for fp32): 16-byte alignment is
+ *    faster but not required.
+ *  - Calls are asynchronous and ordered on the `stream` argument (a cudaStream_t
+ *    passed as void*; NULL is the legacy default stream). A context may be used
+ *    by one stream at a time. The library allocates device memory only in
+ *    condensa_create() and when a call needs a larger workspace than any call
+ *    before it on that context (this synchronises the device once); steady-state
+ *    calls allocate nothing and do not synchronise.
+ *  - Arguments are checked on the host before anything is launched; on an
+ *    argument error no caller buffer has been touched.
+ *  - Arithmetic: every fp32 value is produced by single IEEE-754 operations,
+ *    round-to-nearest-even, no fused multiply-add, subnormals kept:
+ *        q = lambda / mu;  u = w - q;
+ *        d = w - theta;    p = mu * d;   lambda' = lambda - p;   g = p - lambda_used
+ *    where lambda_used is lambda' when CONDENSA_FUSE_LAMBDA is set and the given
+ *    lambda otherwise. Structure norms are accumulated in fp64.
+ *  - Ranking: units (elements, filters or blocks) are ordered by key, larger
+ *    first, and among equal keys by global index, lower first. With n ranked
+ *    units, Z = floor(sparsity * n + 0.5) (computed in double, clamped to [0, n])
+ *    units are zeroed: exactly the last Z of that order. "Target sparsity" is the
+ *    proportion of zeroed units (Introduction).
+ */
+#ifndef CONDENSA_CSTEP_H
+#define CONDENSA_CSTEP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define CONDENSA_API __attribute__((visibility("default")))
+#else
+#define CONDENSA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct condensa_ctx condensa_ctx;   /* opaque: workspace + descriptor cache of one device */
+
+/* One weight tensor of the list. Global element index of element i of tensor t
+ * is (sum of numel of tensors before t) + i; structures are numbered the same
+ * way, tensor by tensor. */
+typedef struct {
+    const float *w;       /* in : weights, fp32, never written                              */
+    float *lambda;        /* i/o: multipliers, fp32. NULL: treated as 0 and never written    */
+    float *theta;         /* out: compressed weights, fp32 (in: for _lagrange_update)        */
+    uint8_t *mask;        /* out: 1 byte per element, 1 = in the kept set. NULL: not written */
+    float *grad;          /* out: penalty gradient g, fp32, overwritten. NULL: not written   */
+    uint16_t *theta_h;    /* out: IEEE binary16 bits of theta. NULL: not written             */
+    int64_t numel;        /* number of elements, >= 0                                        */
+    int32_t ndim;         /* 1..4; product of shape[0..ndim-1] must equal numel              */
+    int64_t shape[4];     /* dim 0 = filters (4-D) or rows (2-D)                             */
+} condensa_tensor;
+
+/* `fuse` bits */
+enum {
+    CONDENSA_FUSE_FP16 = 1,     /* theta = fp16 round-to-nearest-even of kept u, widened back  */
+    CONDENSA_FUSE_LAMBDA = 2,   /* update lambda in place                                     */
+    CONDENSA_FUSE_PENALTY = 4,  /* write g to grad                                            */
+    CONDENSA_NO_SAMPLING = 64   /* do not bracket the threshold from a sample first: rank with
+                                   full histogram passes only (slower; same results)           */
+};
+
+/* return codes */
+enum {
+    CONDENSA_OK = 0,
+    CONDENSA_ERR_INVALID_ARG = -1,   /* bad pointer, size, shape, sparsity, mu, aliasing       */
+    CONDENSA_ERR_WORKSPACE = -2,     /* workspace could not be allocated                       */
+    CONDENSA_ERR_CUDA = -3,          /* CUDA runtime error, text in condensa_last_error()      */
+    CONDENSA_ERR_UNSUPPORTED = -4,   /* dtype or block shape not built                         */
+    CONDENSA_ERR_INTERNAL = -5       /* a device-side consistency check failed (reported by
+                                        condensa_get_result)                                   */
+};
+
+enum { CONDENSA_DTYPE_FP16 = 1 };
+
+/* Record of the last ranking call, filled on the device. */
+typedef struct {
+    int32_t status;        /* CONDENSA_OK or CONDENSA_ERR_INTERNAL                             */
+    int32_t passes;        /* histogram passes the selection took (over the source or a list) */
+    int64_t n_units;       /* ranked units: elements, filters or blocks                       */
+    int64_t n_zero;        /* Z                                                                */
+    int64_t n_keep;        /* n_units - Z                                                      */
+    uint64_t tau_key;      /* key of the weakest kept unit: bits(|u|) for _prune, the fp64
+                              bits of the squared L2 norm for _filter/_block; the bits of
+                              +infinity in that format when nothing is kept                   */
+    int64_t tau_id;        /* global index of the weakest kept unit, -1 when nothing is kept  */
+    int64_t n_gt;          /* units with key  > tau_key                                       */
+    int64_t n_tie;         /* units with key == tau_key                                       */
+    int64_t n_tie_kept;    /* how many of those are kept (the lowest indices)                 */
+    float tau_norm;        /* _filter/_block: (float)sqrt of the weakest kept squared norm    */
+    int32_t sampled;       /* 1 when a sample bracket was used and held                       */
+    int64_t n_candidates;  /* units that had to be listed for the exact selection             */
+} condensa_result;
+
+/* Create a context on CUDA device `device`. workspace_bytes = 0 sizes the
+ * workspace on demand; otherwise that much is reserved up front. */
+CONDENSA_API int condensa_create(condensa_ctx **out, int device, size_t workspace_bytes);
+CONDENSA_API int condensa_destroy(condensa_ctx *ctx);
+
+/* Prune() - unstructured magnitude pruning (Table 1; Section 3.3 "pruning").
+ * key = bits(u) & 0x7FFFFFFF. theta = u (or fp16(u) with FUSE_FP16: Compose([Prune(),
+ * Quantize(float16)]), Evaluation, Objective 1: prune first, then quantise) on the
+ * kept set, +0 elsewhere. `tensors` is a HOST array of T entries. */
+CONDENSA_API int condensa_cstep_prune(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
+                         double sparsity, float mu, unsigned fuse, void *stream);
+
+/* FilterPrune - every 4-D tensor is ranked by output filter [f, :, :, :] on the
+ * fp64 sum of u^2 (Table 1, "filters (3D blocks)"); `sparsity` is the proportion
+ * of filters zeroed. Tensors with ndim != 4 pass through: theta = u, mask = 1. */
+CONDENSA_API int condensa_cstep_filter(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
+                          double sparsity, float mu, unsigned fuse, void *stream);
+
+/* BlockPrune - every 2-D tensor is cut into bh x bw blocks (row-major numbering,
+ * blocks that stick out over an edge hold fewer elements) ranked on the fp64 sum
+ * of u^2 taken row by row inside the block (Table 1, "n-D blocks of size bs").
+ * Only bh = bw = 4 is built; anything else returns CONDENSA_ERR_UNSUPPORTED.
+ * Tensors with ndim != 2 pass through. */
+CONDENSA_API int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
+                         double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream);
+
+/* Quantize(dtype) - theta = fp16 round-to-nearest-even of u for every element,
+ * mask = 1 (Table 1; Section 2 "low-precision approximation"). Overflow goes to
+ * infinity, underflow is gradual, NaN becomes a quiet NaN with the same sign. */
+CONDENSA_API int condensa_cstep_quantize(condensa_ctx *ctx, const condensa_tensor *tensors, int T, float mu,
+                            int dtype, unsigned fuse, void *stream);
+
+/* Multiplier update and/or penalty gradient with theta as given by the caller
+ * (augmented-Lagrangian method of the L-C algorithm, Section 3.3). `fuse` is
+ * CONDENSA_FUSE_LAMBDA and/or CONDENSA_FUSE_PENALTY. Reads w, theta, lambda. */
+CONDENSA_API int condensa_cstep_lagrange_update(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
+                                   float mu, unsigned fuse, void *stream);
+
+/* Operation selector for condensa_cstep_host(). */
+enum { CONDENSA_OP_PRUNE = 0, CONDENSA_OP_FILTER = 1, CONDENSA_OP_BLOCK = 2,
+       CONDENSA_OP_QUANTIZE = 3, CONDENSA_OP_LAGRANGE = 4 };
+
+/* Same operations for weights that live in HOST memory: every pointer in
+ * `tensors` is a host pointer (pinned memory makes the copies asynchronous).
+ * The call copies w and lambda (and theta for CONDENSA_OP_LAGRANGE) to device
+ * buffers the context keeps, runs the operation there, copies every non-NULL
+ * output back and returns after the stream has finished. bh/bw are read for
+ * CONDENSA_OP_BLOCK only, sparsity for the three pruning operations. */
+CONDENSA_API int condensa_cstep_host(condensa_ctx *ctx, int op, const condensa_tensor *tensors, int T,
+                        double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream);
+
+/* Waits for the stream of the last ranking call and copies its record. */
+CONDENSA_API int condensa_get_result(condensa_ctx *ctx, condensa_result *out);
+
+/* Per-kernel device time. While enabled, every kernel launch of this context is
+ * bracketed by a pair of CUDA events on its stream (this adds a little latency
+ * between kernels, so enable it only to measure). condensa_profile_read() waits
+ * for the recorded events and returns, per kernel name, the launches and the
+ * summed event time since profiling was enabled. `out` is a HOST array. */
+typedef struct {
+    char name[48];
+    int64_t launches;
+    double total_ms;
+} condensa_kernel_time;
+CONDENSA_API int condensa_profile_enable(condensa_ctx *ctx, int on);
+CONDENSA_API int condensa_profile_read(condensa_ctx *ctx, condensa_kernel_time *out, int max_entries,
+                                       int *n_out);
+
+/* Number of kernels this context has launched so far. */
+CONDENSA_API int64_t condensa_launch_count(const condensa_ctx *ctx);
+
+/* Text of the last error on this context (never NULL). ctx may be NULL to get
+ * the text of a failed condensa_create(). */
+CONDENSA_API const char *condensa_last_error(const condensa_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONDENSA_CSTEP_H */

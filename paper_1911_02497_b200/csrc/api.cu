@@ -1,0 +1,728 @@
+// C ABI of the C-step library: argument checks, descriptor table, workspace,
+// kernel sequencing. See include/condensa_cstep.h for the contract.
+#include "../../include/condensa_cstep.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "select.cuh"
+#include "structured.cuh"
+
+using namespace cs;
+
+static_assert(sizeof(condensa_result) == sizeof(cs::Result), "result layouts must agree");
+
+namespace {
+
+std::string g_create_error;
+
+struct KernelInfo {
+    int occ = 0;     // CTAs per SM
+};
+
+struct DeviceMirror {   // device copies used by condensa_cstep_host
+    char *buf = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace
+
+struct condensa_ctx {
+    int device = 0;
+    int num_sms = 0;
+    bool coop = false;
+    std::string err;
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    char *h_stage = nullptr;        // pinned staging of the descriptor upload
+    size_t h_stage_bytes = 0;
+    cudaEvent_t stage_ev = nullptr;
+    std::vector<char> last_upload;  // what the device descriptor area holds now
+    char *last_upload_dst = nullptr;
+    int64_t launches = 0;
+    cudaStream_t last_stream = nullptr;
+    bool has_result = false;
+    Ctl *ctl = nullptr;
+    int occ_select[3] = {0, 0, 0};
+    int occ_stream = 0;
+    DeviceMirror mirror;
+    // optional per-kernel timing (event pair around every launch)
+    bool prof_on = false;
+    std::vector<cudaEvent_t> prof_ev;       // start/stop pairs
+    std::vector<int> prof_name;             // index into prof_names per pair
+    std::vector<std::string> prof_names;
+    size_t prof_used = 0;                   // pairs recorded since the last read
+    std::vector<double> prof_ms;            // accumulated per name
+    std::vector<int64_t> prof_cnt;
+};
+
+namespace {
+
+int fail(condensa_ctx *c, int code, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    if (c) c->err = buf; else g_create_error = buf;
+    return code;
+}
+
+#define CU_TRY(ctx, call)                                                                   \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess)                                                              \
+            return fail(ctx, CONDENSA_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_));   \
+    } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Interval {
+    uintptr_t lo, hi;
+    bool out;
+};
+
+// Layout of one call's workspace.
+struct Layout {
+    size_t ctl, hist, fin_key, fin_id, desc, list_key, list_id, arr_key, partial, total;
+    size_t desc_bytes;
+};
+
+struct Plan {
+    std::vector<TensorDesc> td;
+    std::vector<long long> prefix_a, prefix_b;   // scan / apply work items
+    long long n_items_a = 0, n_items_b = 0;
+    long long S = 0, N = 0, n_seg = 0;
+    u64 cap = 0;
+};
+
+int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s, float mu,
+             unsigned fuse)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    if (!ts || T <= 0 || T > (1 << 20)) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor list is empty or NULL");
+    if (!(mu > 0.0f) || !std::isfinite(mu)) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "mu must be finite and > 0");
+    if (op <= CONDENSA_OP_BLOCK && !(s >= 0.0 && s <= 1.0))
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "sparsity must lie in [0, 1]");
+    const unsigned known = CONDENSA_FUSE_FP16 | CONDENSA_FUSE_LAMBDA | CONDENSA_FUSE_PENALTY | CONDENSA_NO_SAMPLING;
+    if (fuse & ~known) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "unknown fuse bits");
+    std::vector<Interval> iv;
+    iv.reserve((size_t)T * 6);
+    for (int t = 0; t < T; ++t) {
+        const condensa_tensor &x = ts[t];
+        if (x.numel < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: numel < 0", t);
+        if (x.ndim < 1 || x.ndim > 4) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: ndim must be 1..4", t);
+        long long prod = 1;
+        for (int d = 0; d < x.ndim; ++d) {
+            if (x.shape[d] < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: negative dimension", t);
+            prod *= x.shape[d];
+        }
+        if (prod != x.numel) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: shape does not match numel", t);
+        if (x.numel == 0) continue;
+        if (!x.w || !x.theta) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: w and theta must not be NULL", t);
+        const uintptr_t p4[4] = {(uintptr_t)x.w, (uintptr_t)x.lambda, (uintptr_t)x.theta, (uintptr_t)x.grad};
+        for (int i = 0; i < 4; ++i)
+            if (p4[i] % 4) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: fp32 pointer not 4-byte aligned", t);
+        if ((uintptr_t)x.theta_h % 2) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: theta_h not 2-byte aligned", t);
+        const size_t n = (size_t)x.numel;
+        const bool theta_out = op != CONDENSA_OP_LAGRANGE;
+        iv.push_back({(uintptr_t)x.w, (uintptr_t)x.w + 4 * n, false});
+        iv.push_back({(uintptr_t)x.theta, (uintptr_t)x.theta + 4 * n, theta_out});
+        if (x.lambda) iv.push_back({(uintptr_t)x.lambda, (uintptr_t)x.lambda + 4 * n, (fuse & CONDENSA_FUSE_LAMBDA) != 0});
+        if (x.grad && (fuse & CONDENSA_FUSE_PENALTY)) iv.push_back({(uintptr_t)x.grad, (uintptr_t)x.grad + 4 * n, true});
+        if (x.mask && theta_out) iv.push_back({(uintptr_t)x.mask, (uintptr_t)x.mask + n, true});
+        if (x.theta_h && theta_out) iv.push_back({(uintptr_t)x.theta_h, (uintptr_t)x.theta_h + 2 * n, true});
+    }
+    std::sort(iv.begin(), iv.end(), [](const Interval &a, const Interval &b) { return a.lo < b.lo; });
+    // an output range may overlap nothing else
+    uintptr_t reach = 0, reach_out = 0;
+    for (size_t i = 0; i < iv.size(); ++i) {
+        if (iv[i].lo < reach_out || (iv[i].out && iv[i].lo < reach))
+            return fail(ctx, CONDENSA_ERR_INVALID_ARG, "an output buffer overlaps another buffer of the call");
+        reach = std::max(reach, iv[i].hi);
+        if (iv[i].out) reach_out = std::max(reach_out, iv[i].hi);
+    }
+    return CONDENSA_OK;
+}
+
+void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl)
+{
+    pl.td.resize(T);
+    pl.prefix_a.assign(T + 1, 0);
+    pl.prefix_b.assign(T + 1, 0);
+    long long eoff = 0, uoff = 0, seg = 0;
+    for (int t = 0; t < T; ++t) {
+        const condensa_tensor &x = ts[t];
+        TensorDesc d;
+        memset(&d, 0, sizeof(d));
+        d.w = x.w; d.lam = x.lambda; d.theta = x.theta; d.mask = x.mask; d.grad = x.grad; d.theta_h = x.theta_h;
+        d.numel = x.numel;
+        d.elem_prefix = eoff;
+        d.unit_prefix = uoff;
+        // linear vector path: all arrays must reach 16-byte alignment at the same element
+        const uintptr_t aw = (uintptr_t)x.w;
+        const int pad = (int)((aw % 16) / 4);
+        bool ok = true;
+        const uintptr_t f32p[3] = {(uintptr_t)x.lambda, (uintptr_t)x.theta, (uintptr_t)x.grad};
+        for (int i = 0; i < 3; ++i)
+            if (f32p[i] && (f32p[i] % 16) != (aw % 16)) ok = false;
+        if (x.mask && ((uintptr_t)x.mask % 4) != (uintptr_t)(pad % 4)) ok = false;
+        if (x.theta_h && ((uintptr_t)x.theta_h % 8) != (uintptr_t)((2 * pad) % 8)) ok = false;
+        d.vec_ok = ok ? 1 : 0;
+        d.pad = ok ? pad : 0;
+        const long long n_groups = (x.numel + d.pad + 3) / 4;
+        const long long lin_items = (n_groups + GROUPS_PER_ITEM - 1) / GROUPS_PER_ITEM;
+        long long items_a = 0, items_b = lin_items;
+        if (op == OP_PRUNE) {
+            d.ranked = x.numel > 0;
+            d.n_units = x.numel;
+            items_a = lin_items;
+        } else if (op == OP_FILTER) {
+            d.ranked = (x.ndim == 4 && x.numel > 0) ? 1 : 0;
+            if (d.ranked) {
+                d.d0 = x.shape[0];
+                d.d1 = x.shape[1] * x.shape[2] * x.shape[3];
+                d.n_units = d.d0;
+                items_a = d.d0 * ((d.d1 + SEG - 1) / SEG);
+            }
+        } else if (op == OP_BLOCK) {
+            d.ranked = (x.ndim == 2 && x.numel > 0) ? 1 : 0;
+            if (d.ranked) {
+                d.d0 = x.shape[0];
+                d.d1 = x.shape[1];
+                d.nbc = (d.d1 + 3) / 4;
+                d.n_units = ((d.d0 + 3) / 4) * d.nbc;
+                bool bok = (d.d1 % 4) == 0 && (aw % 16) == 0;
+                for (int i = 0; i < 3; ++i)
+                    if (f32p[i] % 16) bok = false;
+                if ((uintptr_t)x.mask % 4) bok = false;
+                if ((uintptr_t)x.theta_h % 8) bok = false;
+                d.blk_vec_ok = bok ? 1 : 0;
+                items_a = (d.n_units + BLOCKS_PER_ITEM - 1) / BLOCKS_PER_ITEM;
+                items_b = items_a;
+            }
+        }
+        pl.td[t] = d;
+        pl.prefix_a[t + 1] = pl.prefix_a[t] + items_a;
+        pl.prefix_b[t + 1] = pl.prefix_b[t] + items_b;
+        eoff += x.numel;
+        if (op != OP_PRUNE) uoff += d.n_units;
+        if (op == OP_FILTER) seg += items_a;
+    }
+    pl.N = eoff;
+    pl.S = (op == OP_PRUNE) ? eoff : uoff;
+    pl.n_seg = seg;
+    pl.n_items_a = pl.prefix_a[T];
+    pl.n_items_b = pl.prefix_b[T];
+    const u64 S = (u64)pl.S;
+    u64 cap = S / 8;
+    if (cap < 65536) cap = 65536;
+    if (cap > (1ull << 22)) cap = 1ull << 22;
+    if (cap > S) cap = S ? S : 1;
+    pl.cap = cap;
+}
+
+Layout make_layout(int T, const Plan &pl, bool ranking, bool filter)
+{
+    Layout L;
+    size_t off = 0;
+    L.ctl = off; off = align_up(off + sizeof(Ctl), 256);
+    L.hist = off; off = align_up(off + sizeof(u64) * 3 * NBINS, 256);
+    L.fin_key = off; off = align_up(off + sizeof(u64) * FIN, 256);
+    L.fin_id = off; off = align_up(off + sizeof(u64) * FIN, 256);
+    L.desc = off;
+    L.desc_bytes = sizeof(TensorDesc) * (size_t)T + 2 * sizeof(long long) * (size_t)(T + 1);
+    off = align_up(off + L.desc_bytes, 256);
+    L.list_key = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
+    L.list_id = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
+    L.arr_key = off; if (filter) off = align_up(off + sizeof(u64) * (size_t)std::max<long long>(pl.S, 1), 256);
+    L.partial = off; if (filter) off = align_up(off + sizeof(double) * (size_t)std::max<long long>(pl.n_seg, 1), 256);
+    L.total = off;
+    return L;
+}
+
+int ensure_workspace(condensa_ctx *ctx, size_t bytes, cudaStream_t stream)
+{
+    if (bytes <= ctx->ws_bytes) return CONDENSA_OK;
+    CU_TRY(ctx, cudaStreamSynchronize(stream));
+    if (ctx->last_stream && ctx->last_stream != stream) CU_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
+    if (ctx->ws) cudaFree(ctx->ws);
+    ctx->ws = nullptr;
+    ctx->ws_bytes = 0;
+    ctx->last_upload.clear();
+    ctx->last_upload_dst = nullptr;
+    const size_t want = align_up(bytes + bytes / 4, 1 << 20);
+    cudaError_t e = cudaMalloc((void **)&ctx->ws, want);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ctx, CONDENSA_ERR_WORKSPACE, "cannot allocate %zu bytes of workspace: %s", want, cudaGetErrorString(e));
+    }
+    ctx->ws_bytes = want;
+    return CONDENSA_OK;
+}
+
+// Copies the descriptor table and both prefix arrays to the workspace unless
+// the device already holds exactly these bytes.
+int upload_desc(condensa_ctx *ctx, const Plan &pl, int T, char *dst, size_t bytes, cudaStream_t stream)
+{
+    std::vector<char> img(bytes);
+    char *p = img.data();
+    memcpy(p, pl.td.data(), sizeof(TensorDesc) * (size_t)T); p += sizeof(TensorDesc) * (size_t)T;
+    memcpy(p, pl.prefix_a.data(), sizeof(long long) * (size_t)(T + 1)); p += sizeof(long long) * (size_t)(T + 1);
+    memcpy(p, pl.prefix_b.data(), sizeof(long long) * (size_t)(T + 1));
+    if (ctx->last_upload_dst == dst && ctx->last_upload == img) return CONDENSA_OK;
+    CU_TRY(ctx, cudaEventSynchronize(ctx->stage_ev));    // the previous upload has left the staging area
+    if (bytes > ctx->h_stage_bytes) {
+        if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
+        ctx->h_stage = nullptr;
+        ctx->h_stage_bytes = 0;
+        CU_TRY(ctx, cudaMallocHost((void **)&ctx->h_stage, align_up(bytes * 2, 4096)));
+        ctx->h_stage_bytes = align_up(bytes * 2, 4096);
+    }
+    memcpy(ctx->h_stage, img.data(), bytes);
+    CU_TRY(ctx, cudaMemcpyAsync(dst, ctx->h_stage, bytes, cudaMemcpyHostToDevice, stream));
+    CU_TRY(ctx, cudaEventRecord(ctx->stage_ev, stream));
+    ctx->last_upload.swap(img);
+    ctx->last_upload_dst = dst;
+    return CONDENSA_OK;
+}
+
+template <class K>
+int occupancy(K kernel)
+{
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, THREADS, 0) != cudaSuccess) occ = 1;
+    return occ < 1 ? 1 : occ;
+}
+
+int stream_grid(condensa_ctx *ctx, long long n_items, int occ)
+{
+    long long g = (long long)ctx->num_sms * occ;
+    if (g > n_items) g = n_items;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+int prof_begin(condensa_ctx *ctx, const char *name, cudaStream_t stream)
+{
+    if (!ctx->prof_on) return 0;
+    if (ctx->prof_used * 2 + 2 > ctx->prof_ev.size()) {
+        for (int i = 0; i < 2; ++i) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return 0;
+            ctx->prof_ev.push_back(e);
+        }
+    }
+    int id = -1;
+    for (size_t i = 0; i < ctx->prof_names.size(); ++i)
+        if (ctx->prof_names[i] == name) id = (int)i;
+    if (id < 0) {
+        id = (int)ctx->prof_names.size();
+        ctx->prof_names.push_back(name);
+        ctx->prof_ms.push_back(0.0);
+        ctx->prof_cnt.push_back(0);
+    }
+    if (ctx->prof_name.size() <= ctx->prof_used) ctx->prof_name.resize(ctx->prof_used + 1);
+    ctx->prof_name[ctx->prof_used] = id;
+    cudaEventRecord(ctx->prof_ev[ctx->prof_used * 2], stream);
+    return 1;
+}
+
+void prof_end(condensa_ctx *ctx, int active, cudaStream_t stream)
+{
+    if (!active) return;
+    cudaEventRecord(ctx->prof_ev[ctx->prof_used * 2 + 1], stream);
+    ctx->prof_used += 1;
+}
+
+// Folds the recorded event pairs into the per-kernel totals (synchronises).
+void prof_collect(condensa_ctx *ctx)
+{
+    for (size_t i = 0; i < ctx->prof_used; ++i) {
+        float ms = 0.0f;
+        cudaEventSynchronize(ctx->prof_ev[2 * i + 1]);
+        if (cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]) == cudaSuccess) {
+            ctx->prof_ms[ctx->prof_name[i]] += ms;
+            ctx->prof_cnt[ctx->prof_name[i]] += 1;
+        }
+    }
+    ctx->prof_used = 0;
+}
+
+#define LAUNCH_CHECK(ctx)                                                                    \
+    do {                                                                                     \
+        cudaError_t e_ = cudaGetLastError();                                                 \
+        if (e_ != cudaSuccess)                                                               \
+            return fail(ctx, CONDENSA_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e_)); \
+        ctx->launches += 1;                                                                  \
+    } while (0)
+
+template <int SRC>
+int launch_select(condensa_ctx *ctx, Params &P, int first_listed, cudaStream_t stream)
+{
+    if (!ctx->occ_select[SRC]) ctx->occ_select[SRC] = occupancy(k_select<SRC>);
+    const int per_sm = std::min(ctx->occ_select[SRC], 2);
+    dim3 grid((unsigned)(ctx->num_sms * per_sm)), block(THREADS);
+    void *args[] = {(void *)&P, (void *)&first_listed};
+    const int pa_ = prof_begin(ctx, "k_select", stream);
+    CU_TRY(ctx, cudaLaunchCooperativeKernel((const void *)k_select<SRC>, grid, block, args, 0, stream));
+    ctx->launches += 1;
+    prof_end(ctx, pa_, stream);
+    return CONDENSA_OK;
+}
+
+Sel initial_state(long long S, long long k, int bits_key)
+{
+    Sel s;
+    memset(&s, 0, sizeof(s));
+    s.S = (u64)S;
+    s.k = (u64)k;
+    s.lo_key = 0;
+    s.hi_key = bits_key >= 63 ? 0x7FFFFFFFFFFFFFFFull : ((1ull << bits_key) - 1ull);
+    s.lo_id = 0;
+    s.hi_id = S > 0 ? (u64)S - 1 : 0;
+    s.pop = (u64)S;
+    s.above_known = 1;
+    s.shift = bits_key > LOG_NBINS ? bits_key - LOG_NBINS : 0;
+    s.done = (S == 0 || k == 0) ? 1 : 0;
+    return s;
+}
+
+int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double sparsity, float mu,
+           unsigned fuse, cudaStream_t stream)
+{
+    int rc = validate(ctx, op, ts, T, sparsity, mu, fuse);
+    if (rc) return rc;
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    Plan pl;
+    build_plan(op, ts, T, pl);
+    const bool ranking = op <= OP_BLOCK;
+    const Layout L = make_layout(T, pl, ranking, op == OP_FILTER);
+    rc = ensure_workspace(ctx, L.total, stream);
+    if (rc) return rc;
+    char *ws = ctx->ws;
+    rc = upload_desc(ctx, pl, T, ws + L.desc, L.desc_bytes, stream);
+    if (rc) return rc;
+
+    Params P;
+    memset(&P, 0, sizeof(P));
+    P.td = (const TensorDesc *)(ws + L.desc);
+    const long long *pa = (const long long *)(ws + L.desc + sizeof(TensorDesc) * (size_t)T);
+    const long long *pb = pa + (T + 1);
+    P.T = T;
+    P.mu = mu;
+    P.fuse = fuse & 7u;
+    if (op == OP_QUANTIZE) P.fuse |= FUSE_FP16;
+    if (op == OP_LAGRANGE) P.fuse &= ~(unsigned)FUSE_FP16;
+    P.ctl = (Ctl *)(ws + L.ctl);
+    P.hist = (u64 *)(ws + L.hist);
+    P.fin_key = (u64 *)(ws + L.fin_key);
+    P.fin_id = (u64 *)(ws + L.fin_id);
+    P.list_key = (u64 *)(ws + L.list_key);
+    P.list_id = (u64 *)(ws + L.list_id);
+    P.cap = pl.cap;
+    P.arr_key = (u64 *)(ws + L.arr_key);
+    P.partial = (double *)(ws + L.partial);
+    P.S = pl.S;
+    P.bits_key = (op == OP_PRUNE) ? 31 : 63;
+    ctx->ctl = P.ctl;
+    ctx->last_stream = stream;
+
+    if (!ctx->occ_stream) ctx->occ_stream = 4;
+
+    if (ranking) {
+        const long long Z = (long long)std::min<double>((double)pl.S, std::max(0.0, std::floor(sparsity * (double)pl.S + 0.5)));
+        const long long k = pl.S - Z;
+        Sel init = initial_state(pl.S, k, P.bits_key);
+        const int do_list0 = (u64)pl.S <= pl.cap ? 1 : 0;
+
+        Params Pa = P;
+        Pa.item_prefix = pa;
+        Pa.n_items = pl.n_items_a;
+        if (op == OP_FILTER && pl.S > 0) {
+            int pa_ = prof_begin(ctx, "k_filter_partial", stream);
+            k_filter_partial<<<stream_grid(ctx, (pl.n_items_a + WARPS - 1) / WARPS, 8), THREADS, 0, stream>>>(Pa);
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, pa_, stream);
+            pa_ = prof_begin(ctx, "k_filter_combine", stream);
+            k_filter_combine<<<stream_grid(ctx, (pl.S + THREADS - 1) / THREADS, 8), THREADS, 0, stream>>>(Pa);
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, pa_, stream);
+        }
+        int pi_ = prof_begin(ctx, "k_init", stream);
+        k_init<<<8, THREADS, 0, stream>>>(P, init);
+        LAUNCH_CHECK(ctx);
+        prof_end(ctx, pi_, stream);
+        if (!init.done) {
+            const int ps_ = prof_begin(ctx, op == OP_PRUNE ? "k_scan_elem" : op == OP_BLOCK ? "k_scan_block" : "k_scan_array", stream);
+            if (op == OP_PRUNE) {
+                k_scan<SRC_ELEM><<<stream_grid(ctx, pl.n_items_a, 4), THREADS, 0, stream>>>(Pa, do_list0);
+            } else if (op == OP_BLOCK) {
+                k_scan<SRC_BLOCK><<<stream_grid(ctx, pl.n_items_a, 4), THREADS, 0, stream>>>(Pa, do_list0);
+            } else {
+                k_scan<SRC_ARRAY><<<stream_grid(ctx, (pl.S + THREADS - 1) / THREADS, 4), THREADS, 0, stream>>>(Pa, do_list0);
+            }
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, ps_, stream);
+        }
+        if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, stream);
+        else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, stream);
+        else rc = launch_select<SRC_ARRAY>(ctx, Pa, do_list0, stream);
+        if (rc) return rc;
+        ctx->has_result = true;
+    }
+
+    Params Pb = P;
+    Pb.item_prefix = pb;
+    Pb.n_items = pl.n_items_b;
+    if (pl.n_items_b > 0) {
+        const int grid = stream_grid(ctx, pl.n_items_b, ctx->occ_stream);
+        static const char *apply_names[5] = {"k_apply_prune", "k_apply_filter", "k_apply_block", "k_quantize", "k_lagrange"};
+        const int pa_ = prof_begin(ctx, apply_names[op], stream);
+        switch (op) {
+        case OP_PRUNE: k_apply_linear<M_PRUNE><<<grid, THREADS, 0, stream>>>(Pb); break;
+        case OP_FILTER: k_apply_linear<M_FILTER><<<grid, THREADS, 0, stream>>>(Pb); break;
+        case OP_BLOCK: k_apply_block<<<grid, THREADS, 0, stream>>>(Pb); break;
+        case OP_QUANTIZE: k_apply_linear<M_KEEPALL><<<grid, THREADS, 0, stream>>>(Pb); break;
+        default: k_apply_linear<M_LAGRANGE><<<grid, THREADS, 0, stream>>>(Pb); break;
+        }
+        LAUNCH_CHECK(ctx);
+        prof_end(ctx, pa_, stream);
+    }
+    return CONDENSA_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- C ABI
+extern "C" {
+
+int condensa_create(condensa_ctx **out, int device, size_t workspace_bytes)
+{
+    if (!out) return fail(nullptr, CONDENSA_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    int n = 0;
+    cudaError_t e = cudaGetDeviceCount(&n);
+    if (e != cudaSuccess || n == 0) {
+        cudaGetLastError();
+        return fail(nullptr, CONDENSA_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(e));
+    }
+    if (device < 0 || device >= n) return fail(nullptr, CONDENSA_ERR_INVALID_ARG, "device %d out of range", device);
+    if ((e = cudaSetDevice(device)) != cudaSuccess) return fail(nullptr, CONDENSA_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(e));
+    condensa_ctx *c = new condensa_ctx();
+    c->device = device;
+    int coop = 0;
+    cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device);
+    c->coop = coop != 0;
+    if (!c->coop || c->num_sms <= 0) {
+        delete c;
+        return fail(nullptr, CONDENSA_ERR_UNSUPPORTED, "device lacks cooperative launch");
+    }
+    if ((e = cudaEventCreateWithFlags(&c->stage_ev, cudaEventDisableTiming)) != cudaSuccess) {
+        delete c;
+        return fail(nullptr, CONDENSA_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+    }
+    if (workspace_bytes) {
+        int rc = ensure_workspace(c, workspace_bytes, nullptr);
+        if (rc) {
+            g_create_error = c->err;
+            cudaEventDestroy(c->stage_ev);
+            delete c;
+            return rc;
+        }
+    }
+    *out = c;
+    return CONDENSA_OK;
+}
+
+int condensa_destroy(condensa_ctx *ctx)
+{
+    if (!ctx) return CONDENSA_OK;
+    cudaSetDevice(ctx->device);
+    if (ctx->last_stream) cudaStreamSynchronize(ctx->last_stream);
+    cudaDeviceSynchronize();
+    if (ctx->ws) cudaFree(ctx->ws);
+    if (ctx->mirror.buf) cudaFree(ctx->mirror.buf);
+    if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
+    if (ctx->stage_ev) cudaEventDestroy(ctx->stage_ev);
+    for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
+    delete ctx;
+    return CONDENSA_OK;
+}
+
+int condensa_cstep_prune(condensa_ctx *ctx, const condensa_tensor *tensors, int T, double sparsity,
+                         float mu, unsigned fuse, void *stream)
+{
+    return run_op(ctx, OP_PRUNE, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_cstep_filter(condensa_ctx *ctx, const condensa_tensor *tensors, int T, double sparsity,
+                          float mu, unsigned fuse, void *stream)
+{
+    return run_op(ctx, OP_FILTER, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T, double sparsity,
+                         float mu, int bh, int bw, unsigned fuse, void *stream)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    if (bh < 1 || bw < 1) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "block shape must be positive");
+    if (bh != 4 || bw != 4) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "only 4x4 blocks are built");
+    return run_op(ctx, OP_BLOCK, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_cstep_quantize(condensa_ctx *ctx, const condensa_tensor *tensors, int T, float mu,
+                            int dtype, unsigned fuse, void *stream)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    if (dtype != CONDENSA_DTYPE_FP16) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "only fp16 is built");
+    return run_op(ctx, OP_QUANTIZE, tensors, T, 0.0, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_cstep_lagrange_update(condensa_ctx *ctx, const condensa_tensor *tensors, int T, float mu,
+                                   unsigned fuse, void *stream)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    if (!(fuse & (CONDENSA_FUSE_LAMBDA | CONDENSA_FUSE_PENALTY)))
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "nothing to do: set FUSE_LAMBDA and/or FUSE_PENALTY");
+    return run_op(ctx, OP_LAGRANGE, tensors, T, 0.0, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_cstep_host(condensa_ctx *ctx, int op, const condensa_tensor *tensors, int T,
+                        double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream_)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    if (op < CONDENSA_OP_PRUNE || op > CONDENSA_OP_LAGRANGE) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "unknown op");
+    if (!tensors || T <= 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor list is empty or NULL");
+    cudaStream_t stream = (cudaStream_t)stream_;
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    // device mirror: w, lambda, theta, grad (fp32), theta_h (u16), mask (u8) per tensor
+    size_t total = 0;
+    std::vector<size_t> off(T);
+    for (int t = 0; t < T; ++t) {
+        if (tensors[t].numel < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: numel < 0", t);
+        off[t] = total;
+        total += align_up((size_t)tensors[t].numel * 4, 256) * 4 + align_up((size_t)tensors[t].numel * 2, 256) +
+                 align_up((size_t)tensors[t].numel, 256);
+    }
+    if (total > ctx->mirror.bytes) {
+        CU_TRY(ctx, cudaStreamSynchronize(stream));
+        if (ctx->mirror.buf) cudaFree(ctx->mirror.buf);
+        ctx->mirror.buf = nullptr;
+        ctx->mirror.bytes = 0;
+        cudaError_t e = cudaMalloc((void **)&ctx->mirror.buf, total);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(ctx, CONDENSA_ERR_WORKSPACE, "cannot allocate %zu bytes of device mirror", total);
+        }
+        ctx->mirror.bytes = total;
+    }
+    std::vector<condensa_tensor> dev(tensors, tensors + T);
+    for (int t = 0; t < T; ++t) {
+        const condensa_tensor &h = tensors[t];
+        const size_t n = (size_t)h.numel, a4 = align_up(n * 4, 256);
+        char *base = ctx->mirror.buf + off[t];
+        condensa_tensor &d = dev[t];
+        d.w = (const float *)base;
+        d.lambda = h.lambda ? (float *)(base + a4) : nullptr;
+        d.theta = (float *)(base + 2 * a4);
+        d.grad = h.grad ? (float *)(base + 3 * a4) : nullptr;
+        d.theta_h = h.theta_h ? (uint16_t *)(base + 4 * a4) : nullptr;
+        d.mask = h.mask ? (uint8_t *)(base + 4 * a4 + align_up(n * 2, 256)) : nullptr;
+        if (n == 0) continue;
+        if (!h.w || !h.theta) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: w and theta must not be NULL", t);
+        CU_TRY(ctx, cudaMemcpyAsync((void *)d.w, h.w, n * 4, cudaMemcpyHostToDevice, stream));
+        if (h.lambda) CU_TRY(ctx, cudaMemcpyAsync(d.lambda, h.lambda, n * 4, cudaMemcpyHostToDevice, stream));
+        if (op == CONDENSA_OP_LAGRANGE) CU_TRY(ctx, cudaMemcpyAsync(d.theta, h.theta, n * 4, cudaMemcpyHostToDevice, stream));
+    }
+    int rc;
+    switch (op) {
+    case CONDENSA_OP_PRUNE: rc = condensa_cstep_prune(ctx, dev.data(), T, sparsity, mu, fuse, stream); break;
+    case CONDENSA_OP_FILTER: rc = condensa_cstep_filter(ctx, dev.data(), T, sparsity, mu, fuse, stream); break;
+    case CONDENSA_OP_BLOCK: rc = condensa_cstep_block(ctx, dev.data(), T, sparsity, mu, bh, bw, fuse, stream); break;
+    case CONDENSA_OP_QUANTIZE: rc = condensa_cstep_quantize(ctx, dev.data(), T, mu, CONDENSA_DTYPE_FP16, fuse, stream); break;
+    default: rc = condensa_cstep_lagrange_update(ctx, dev.data(), T, mu, fuse, stream); break;
+    }
+    if (rc) return rc;
+    for (int t = 0; t < T; ++t) {
+        const condensa_tensor &h = tensors[t];
+        const condensa_tensor &d = dev[t];
+        const size_t n = (size_t)h.numel;
+        if (n == 0) continue;
+        if (op != CONDENSA_OP_LAGRANGE) {
+            CU_TRY(ctx, cudaMemcpyAsync(h.theta, d.theta, n * 4, cudaMemcpyDeviceToHost, stream));
+            if (h.mask) CU_TRY(ctx, cudaMemcpyAsync(h.mask, d.mask, n, cudaMemcpyDeviceToHost, stream));
+            if (h.theta_h) CU_TRY(ctx, cudaMemcpyAsync(h.theta_h, d.theta_h, n * 2, cudaMemcpyDeviceToHost, stream));
+        }
+        if (h.lambda && (fuse & CONDENSA_FUSE_LAMBDA))
+            CU_TRY(ctx, cudaMemcpyAsync(h.lambda, d.lambda, n * 4, cudaMemcpyDeviceToHost, stream));
+        if (h.grad && (fuse & CONDENSA_FUSE_PENALTY))
+            CU_TRY(ctx, cudaMemcpyAsync(h.grad, d.grad, n * 4, cudaMemcpyDeviceToHost, stream));
+    }
+    CU_TRY(ctx, cudaStreamSynchronize(stream));
+    return CONDENSA_OK;
+}
+
+int condensa_get_result(condensa_ctx *ctx, condensa_result *out)
+{
+    if (!ctx || !out) return CONDENSA_ERR_INVALID_ARG;
+    if (!ctx->has_result || !ctx->ctl) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "no ranking call has run on this context");
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    CU_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
+    CU_TRY(ctx, cudaMemcpy(out, &ctx->ctl->res, sizeof(*out), cudaMemcpyDeviceToHost));
+    if (out->status != 0) {
+        int code = 0;
+        cudaMemcpy(&code, &ctx->ctl->sel.error, sizeof(int), cudaMemcpyDeviceToHost);
+        return fail(ctx, CONDENSA_ERR_INTERNAL, "device-side selection check failed (check %d)", code);
+    }
+    return CONDENSA_OK;
+}
+
+int condensa_profile_enable(condensa_ctx *ctx, int on)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    if (ctx->prof_on) prof_collect(ctx);
+    ctx->prof_on = on != 0;
+    if (on) {
+        std::fill(ctx->prof_ms.begin(), ctx->prof_ms.end(), 0.0);
+        std::fill(ctx->prof_cnt.begin(), ctx->prof_cnt.end(), 0);
+    }
+    return CONDENSA_OK;
+}
+
+int condensa_profile_read(condensa_ctx *ctx, condensa_kernel_time *out, int max_entries, int *n_out)
+{
+    if (!ctx || !out || !n_out || max_entries < 0) return CONDENSA_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    prof_collect(ctx);
+    int n = 0;
+    for (size_t i = 0; i < ctx->prof_names.size() && n < max_entries; ++i) {
+        if (!ctx->prof_cnt[i]) continue;
+        memset(&out[n], 0, sizeof(out[n]));
+        strncpy(out[n].name, ctx->prof_names[i].c_str(), sizeof(out[n].name) - 1);
+        out[n].launches = ctx->prof_cnt[i];
+        out[n].total_ms = ctx->prof_ms[i];
+        ++n;
+    }
+    *n_out = n;
+    return CONDENSA_OK;
+}
+
+int64_t condensa_launch_count(const condensa_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const char *condensa_last_error(const condensa_ctx *ctx)
+{
+    return ctx ? ctx->err.c_str() : g_create_error.c_str();
+}
+
+}  // extern "C"

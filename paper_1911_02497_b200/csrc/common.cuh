@@ -1,0 +1,194 @@
+// Shared device-side definitions of the C-step kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cooperative_groups.h>
+#include <stdint.h>
+
+namespace cs {
+
+typedef unsigned long long u64;
+typedef unsigned int u32;
+
+constexpr int THREADS = 256;             // every kernel here runs 256-thread CTAs
+constexpr int WARPS = THREADS / 32;
+constexpr int GROUPS_PER_ITEM = 1024;    // linear work item = 1024 groups of 4 elements
+constexpr int BLOCKS_PER_ITEM = 512;     // block work item = 512 4x4 blocks
+constexpr int SEG = 2048;                // filter norm segment (elements)
+constexpr int LOG_NBINS = 11;
+constexpr int NBINS = 1 << LOG_NBINS;    // histogram bins per selection pass
+constexpr int FIN = 1024;                // bracket population finished by direct ranking
+constexpr int WSTG = 256;                // staged list entries per warp
+constexpr int MAX_SELECT_ITERS = 24;
+constexpr u64 KEY_NONE = ~0ull;          // cut-off key that keeps nothing
+
+enum { OP_PRUNE = 0, OP_FILTER = 1, OP_BLOCK = 2, OP_QUANTIZE = 3, OP_LAGRANGE = 4 };
+enum { FUSE_FP16 = 1, FUSE_LAMBDA = 2, FUSE_PENALTY = 4, NO_SAMPLING = 64 };
+enum { SRC_ELEM = 0, SRC_BLOCK = 1, SRC_ARRAY = 2 };
+
+// One tensor of the list as the kernels see it.
+struct TensorDesc {
+    const float *w;
+    float *lam;
+    float *theta;
+    uint8_t *mask;
+    float *grad;
+    uint16_t *theta_h;
+    long long numel;
+    long long elem_prefix;   // global index of element 0
+    long long unit_prefix;   // global id of this tensor's first ranked structure
+    long long n_units;       // ranked structures in this tensor (0: passes through)
+    long long d0, d1;        // block: rows, cols.  filter: filters, filter length
+    long long nbc;           // block: blocks per block row
+    int pad;                 // linear groups start at element -pad (0..3)
+    int vec_ok;              // linear path may use 128-bit accesses
+    int blk_vec_ok;          // block path may use 128-bit accesses
+    int ranked;              // takes part in the ranking of the current call
+};
+
+// Device-resident record of one ranking call.
+struct Result {
+    int status, passes;
+    long long n_units, n_zero, n_keep;
+    u64 tau_key;
+    long long tau_id, n_gt, n_tie, n_tie_kept;
+    float tau_norm;
+    int sampled;
+    long long n_candidates;
+};
+
+// Selection state: the bracket is the set of units whose (key, id) lies in
+// [lo_key, hi_key] and, when lo_key == hi_key, also in [lo_id, hi_id]. `n_above`
+// units are known to rank before the bracket, so the unit looked for (rank k
+// overall, 1-based, larger key first, lower id first) has rank k - n_above in it.
+struct Sel {
+    u64 lo_key, hi_key, lo_id, hi_id;
+    u64 n_above, pop;
+    u64 k, S;
+    u64 n_gt, n_tie;          // fixed when the key range collapses to one value
+    int shift;                // bin = (hi_key - key) >> shift, or (id - lo_id) >> shift
+    int slot;                 // histogram buffer the last scan filled
+    int list_valid;           // the candidate list covers the bracket
+    int list_sel;             // which list counter is live (0: first scan, 1: relist)
+    int above_known;          // n_above is exact (else taken from the scan's own count)
+    int done, error, passes;
+    int key_fixed;            // n_gt / n_tie are set
+    int sampled;
+};
+
+struct Ctl {
+    Sel sel;
+    u64 tau_key, tau_id;      // final cut-off: keep iff key > tau_key || (== && id <= tau_id)
+    u64 scan_above[3];        // per histogram slot: units above the bracket seen by that scan
+    u64 list_count[2];
+    u32 fin_count;
+    u32 pad0;
+    Result res;
+};
+
+// Kernel argument block.
+struct Params {
+    const TensorDesc *td;
+    const long long *item_prefix;   // [T+1] work items per tensor (kernel specific)
+    int T;
+    long long n_items;
+    float mu;
+    unsigned fuse;
+    Ctl *ctl;
+    u64 *hist;                      // [3][NBINS]
+    u64 *list_key, *list_id;        // [cap]
+    u64 cap;
+    u64 *fin_key, *fin_id;          // [FIN]
+    u64 *arr_key;                   // filter: fp64 bits of nu per structure
+    double *partial;                // filter: per segment partial sums
+    long long S;                    // ranked units
+    int bits_key;                   // width of the key in bits (31 or 63)
+};
+
+// ---------------------------------------------------------------- arithmetic
+// u = w - lambda / mu as two IEEE fp32 operations.
+__device__ __forceinline__ float form_u(float w, float lam, float mu, bool has_lam)
+{
+    return has_lam ? __fsub_rn(w, __fdiv_rn(lam, mu)) : w;
+}
+
+// binary32 -> binary16 bits, round to nearest even; NaN -> quiet NaN, sign kept.
+__device__ __forceinline__ unsigned short f32_to_f16_bits(float x)
+{
+    unsigned short h = __half_as_ushort(__float2half_rn(x));
+    if (x != x) h = (unsigned short)(((__float_as_uint(x) >> 16) & 0x8000u) | 0x7E00u);
+    return h;
+}
+
+// binary16 bits -> binary32, exact.
+__device__ __forceinline__ float f16_bits_to_f32(unsigned short h)
+{
+    float f = __half2float(__ushort_as_half(h));
+    if ((h & 0x7FFFu) > 0x7C00u)
+        f = __uint_as_float((((u32)h & 0x8000u) << 16) | 0x7F800000u | (((u32)h & 0x3FFu) << 13));
+    return f;
+}
+
+struct Out {
+    float theta, lam, grad;
+    unsigned short th;
+    unsigned char m;
+};
+
+// Everything that follows the keep decision for one element.
+__device__ __forceinline__ Out finish(float w, float lam, float u, bool keep, float mu,
+                                      unsigned fuse, bool has_lam)
+{
+    Out o;
+    unsigned short hb = keep ? f32_to_f16_bits(u) : (unsigned short)0;
+    float th = keep ? ((fuse & FUSE_FP16) ? f16_bits_to_f32(hb) : u) : 0.0f;
+    float d = __fsub_rn(w, th);
+    float p = __fmul_rn(mu, d);
+    float lu = has_lam ? lam : 0.0f;
+    if ((fuse & FUSE_LAMBDA) && has_lam) lu = __fsub_rn(lam, p);
+    o.theta = th;
+    o.th = hb;
+    o.m = keep ? 1 : 0;
+    o.lam = lu;
+    o.grad = __fsub_rn(p, lu);
+    return o;
+}
+
+// Same with theta supplied (multiplier update / penalty gradient only).
+__device__ __forceinline__ Out finish_given(float w, float lam, float th, float mu, unsigned fuse,
+                                            bool has_lam)
+{
+    Out o;
+    float d = __fsub_rn(w, th);
+    float p = __fmul_rn(mu, d);
+    float lu = has_lam ? lam : 0.0f;
+    if ((fuse & FUSE_LAMBDA) && has_lam) lu = __fsub_rn(lam, p);
+    o.theta = th;
+    o.th = 0;
+    o.m = 1;
+    o.lam = lu;
+    o.grad = __fsub_rn(p, lu);
+    return o;
+}
+
+__device__ __forceinline__ u64 key_of_u(float u) { return (u64)(__float_as_uint(u) & 0x7FFFFFFFu); }
+
+__device__ __forceinline__ bool keep_by_cutoff(u64 key, u64 id, u64 tau_key, u64 tau_id)
+{
+    return key > tau_key || (key == tau_key && id <= tau_id);
+}
+
+// Tensor that owns work item `item`: largest t with prefix[t] <= item.
+__device__ __forceinline__ int find_tensor(const long long *__restrict__ prefix, int T, long long item)
+{
+    int lo = 0, hi = T - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (prefix[mid] <= item) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ int bit_length(u64 x) { return x ? 64 - __clzll((long long)x) : 0; }
+
+}  // namespace cs

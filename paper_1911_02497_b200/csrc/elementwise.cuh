@@ -1,0 +1,165 @@
+// Elementwise passes over a multi-tensor descriptor table: projection with a
+// known cut-off, fp16 quantisation, multiplier update, penalty gradient.
+// A linear work item is GROUPS_PER_ITEM groups of 4 consecutive elements; groups
+// start at element -pad so that full groups are 16-byte aligned in every array.
+#pragma once
+#include "common.cuh"
+
+namespace cs {
+
+enum { M_KEEPALL = 0, M_PRUNE = 1, M_FILTER = 2, M_LAGRANGE = 3 };
+
+constexpr int LIN_UNROLL = GROUPS_PER_ITEM / THREADS;   // 4 groups per thread per item
+
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 ld4_ro(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ void st4(float *p, const float *v)
+{
+    *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+
+// One work item of tensor d. tau_* is the cut-off for M_PRUNE / M_FILTER.
+template <int MODE>
+__device__ __forceinline__ void process_linear_item(const Params &P, const TensorDesc &d,
+                                                    long long item_local, u64 tau_key, u64 tau_id)
+{
+    const long long ng = (d.numel + d.pad + 3) >> 2;
+    const long long g0 = item_local * GROUPS_PER_ITEM;
+    const long long g1 = (g0 + GROUPS_PER_ITEM < ng) ? g0 + GROUPS_PER_ITEM : ng;
+    const bool has_lam = d.lam != nullptr;
+    const unsigned fuse = P.fuse;
+    const float mu = P.mu;
+    const float *__restrict__ wp = d.w;
+    const float *lp = d.lam;
+
+    float w[LIN_UNROLL][4], l[LIN_UNROLL][4], t[LIN_UNROLL][4];
+    bool live[LIN_UNROLL], full[LIN_UNROLL];
+
+#pragma unroll
+    for (int it = 0; it < LIN_UNROLL; ++it) {
+        const long long g = g0 + it * THREADS + threadIdx.x;
+        const long long e0 = 4 * g - d.pad;
+        live[it] = g < g1;
+        full[it] = live[it] && d.vec_ok && e0 >= 0 && e0 + 4 <= d.numel;
+        if (full[it]) {
+            float4 a = ld4_ro(wp + e0);
+            w[it][0] = a.x; w[it][1] = a.y; w[it][2] = a.z; w[it][3] = a.w;
+            if (has_lam) {
+                float4 b = ld4(lp + e0);
+                l[it][0] = b.x; l[it][1] = b.y; l[it][2] = b.z; l[it][3] = b.w;
+            } else {
+                l[it][0] = l[it][1] = l[it][2] = l[it][3] = 0.0f;
+            }
+            if (MODE == M_LAGRANGE) {
+                float4 c = ld4(d.theta + e0);
+                t[it][0] = c.x; t[it][1] = c.y; t[it][2] = c.z; t[it][3] = c.w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const long long e = e0 + j;
+                const bool ok = live[it] && e >= 0 && e < d.numel;
+                w[it][j] = ok ? wp[e] : 0.0f;
+                l[it][j] = (ok && has_lam) ? lp[e] : 0.0f;
+                if (MODE == M_LAGRANGE) t[it][j] = ok ? d.theta[e] : 0.0f;
+            }
+        }
+    }
+
+#pragma unroll
+    for (int it = 0; it < LIN_UNROLL; ++it) {
+        if (!live[it]) continue;
+        const long long g = g0 + it * THREADS + threadIdx.x;
+        const long long e0 = 4 * g - d.pad;
+        Out o[4];
+        // structure id of lane 0 for the filter decision
+        long long f0 = 0, r0 = 0;
+        if (MODE == M_FILTER && d.ranked) {
+            const long long eb = e0 < 0 ? 0 : e0;
+            if (d.numel < 0x7FFFFFFFll) {
+                f0 = (long long)((u32)eb / (u32)d.d1);
+            } else {
+                f0 = eb / d.d1;
+            }
+            r0 = eb - f0 * d.d1;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const long long e = e0 + j;
+            if (MODE == M_LAGRANGE) {
+                o[j] = finish_given(w[it][j], l[it][j], t[it][j], mu, fuse, has_lam);
+            } else {
+                const float u = form_u(w[it][j], l[it][j], mu, has_lam);
+                bool keep = true;
+                if (MODE == M_PRUNE) {
+                    keep = keep_by_cutoff(key_of_u(u), (u64)(d.elem_prefix + e), tau_key, tau_id);
+                } else if (MODE == M_FILTER) {
+                    if (d.ranked && e >= 0 && e < d.numel) {
+                        long long f = f0, r = r0 + (e - (e0 < 0 ? 0 : e0));
+                        while (r >= d.d1) { r -= d.d1; ++f; }
+                        const u64 sid = (u64)(d.unit_prefix + f);
+                        keep = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
+                    }
+                }
+                o[j] = finish(w[it][j], l[it][j], u, keep, mu, fuse, has_lam);
+            }
+        }
+        const bool wr_lam = (fuse & FUSE_LAMBDA) && has_lam;
+        const bool wr_grad = (fuse & FUSE_PENALTY) && d.grad != nullptr;
+        if (full[it]) {
+            if (MODE != M_LAGRANGE) {
+                float v[4] = {o[0].theta, o[1].theta, o[2].theta, o[3].theta};
+                st4(d.theta + e0, v);
+                if (d.mask) {
+                    const u32 mm = (u32)o[0].m | ((u32)o[1].m << 8) | ((u32)o[2].m << 16) | ((u32)o[3].m << 24);
+                    *reinterpret_cast<u32 *>(d.mask + e0) = mm;
+                }
+                if (d.theta_h) {
+                    uint2 hh;
+                    hh.x = (u32)o[0].th | ((u32)o[1].th << 16);
+                    hh.y = (u32)o[2].th | ((u32)o[3].th << 16);
+                    *reinterpret_cast<uint2 *>(d.theta_h + e0) = hh;
+                }
+            }
+            if (wr_lam) {
+                float v[4] = {o[0].lam, o[1].lam, o[2].lam, o[3].lam};
+                st4(d.lam + e0, v);
+            }
+            if (wr_grad) {
+                float v[4] = {o[0].grad, o[1].grad, o[2].grad, o[3].grad};
+                st4(d.grad + e0, v);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const long long e = e0 + j;
+                if (e < 0 || e >= d.numel) continue;
+                if (MODE != M_LAGRANGE) {
+                    d.theta[e] = o[j].theta;
+                    if (d.mask) d.mask[e] = o[j].m;
+                    if (d.theta_h) d.theta_h[e] = o[j].th;
+                }
+                if (wr_lam) d.lam[e] = o[j].lam;
+                if (wr_grad) d.grad[e] = o[j].grad;
+            }
+        }
+    }
+}
+
+// Persistent CTAs stride over the linear work items of the whole list.
+template <int MODE>
+__global__ void __launch_bounds__(THREADS) k_apply_linear(Params P)
+{
+    u64 tau_key = 0, tau_id = 0;
+    if (MODE == M_PRUNE || MODE == M_FILTER) {
+        tau_key = P.ctl->tau_key;
+        tau_id = P.ctl->tau_id;
+    }
+    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        process_linear_item<MODE>(P, d, item - P.item_prefix[t], tau_key, tau_id);
+    }
+}
+
+}  // namespace cs

@@ -1,0 +1,614 @@
+// Exact selection of the rank-k unit in (key descending, id ascending) order
+// by range-partition histogram passes, without sorting.
+//
+// A pass ("scan") visits units, drops those outside the current bracket,
+// bins the rest into NBINS equal power-of-two-wide bins (by key, or by id once
+// the key range is a single value) and optionally appends them to a candidate
+// list. The "pick" finds the bin that holds the wanted rank and makes it the
+// new bracket. Passes run over the source until the bracket fits the list,
+// then over the list, until at most FIN units are left, which are ranked
+// directly. One cooperative kernel drives the loop with grid-wide barriers.
+#pragma once
+#include "common.cuh"
+
+namespace cs {
+
+namespace cg = cooperative_groups;
+
+struct ScanShared {
+    u32 hist[NBINS];
+    u64 stg_key[WARPS][WSTG];
+    u64 stg_id[WARPS][WSTG];
+    u64 red[WARPS];
+    Sel sel;
+    u64 pick_before;
+    u64 pick_count;
+    int pick_bin;
+    int fin_hit;
+};
+
+struct ScanCtx {
+    u64 n_above;     // per thread
+    u32 wc;          // staged entries of this warp (warp uniform)
+    bool sk;         // bracket is a single key: bin by id
+    bool do_list;
+    int list_sel;
+};
+
+__device__ __forceinline__ void scan_begin(ScanShared &sh, ScanCtx &c, bool do_list)
+{
+    for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
+    c.n_above = 0;
+    c.wc = 0;
+    c.sk = sh.sel.lo_key == sh.sel.hi_key;
+    c.do_list = do_list;
+    c.list_sel = sh.sel.list_sel;
+    __syncthreads();
+}
+
+__device__ __forceinline__ void flush_warp(const Params &P, ScanShared &sh, ScanCtx &c)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    u64 base = 0;
+    if (lane == 0 && c.wc) base = atomicAdd(&P.ctl->list_count[c.list_sel], (u64)c.wc);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    for (u32 i = lane; i < c.wc; i += 32) {
+        const u64 pos = base + i;
+        if (pos < P.cap) {
+            P.list_key[pos] = sh.stg_key[warp][i];
+            P.list_id[pos] = sh.stg_id[warp][i];
+        }
+    }
+    c.wc = 0;
+    __syncwarp();
+}
+
+// Classify one unit per lane. Must be called by all 32 lanes of a warp together.
+__device__ __forceinline__ void scan_emit(const Params &P, ScanShared &sh, ScanCtx &c, u64 key,
+                                          u64 id, bool active)
+{
+    const Sel &s = sh.sel;
+    bool in = false;
+    if (active) {
+        const bool above = key > s.hi_key || (c.sk && key == s.hi_key && id < s.lo_id);
+        const bool below = key < s.lo_key || (c.sk && key == s.lo_key && id > s.hi_id);
+        in = !above && !below;
+        c.n_above += above ? 1 : 0;
+    }
+    if (in) {
+        u64 b = c.sk ? ((id - s.lo_id) >> s.shift) : ((s.hi_key - key) >> s.shift);
+        if (b > (u64)(NBINS - 1)) b = NBINS - 1;
+        atomicAdd(&sh.hist[(u32)b], 1u);
+    }
+    if (c.do_list) {
+        const unsigned bal = __ballot_sync(0xffffffffu, in);
+        if (bal) {
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            if (in) {
+                const u32 pos = c.wc + __popc(bal & ((1u << lane) - 1u));
+                sh.stg_key[warp][pos] = key;
+                sh.stg_id[warp][pos] = id;
+            }
+            c.wc += __popc(bal);
+            __syncwarp();
+            if (c.wc > WSTG - 32) flush_warp(P, sh, c);
+        }
+    }
+}
+
+__device__ __forceinline__ void scan_end(const Params &P, ScanShared &sh, ScanCtx &c, int slot)
+{
+    if (c.do_list) flush_warp(P, sh, c);
+    // units above the bracket seen by this CTA
+    u64 v = c.n_above;
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        u64 tot = 0;
+        for (int i = 0; i < WARPS; ++i) tot += sh.red[i];
+        if (tot) atomicAdd(&P.ctl->scan_above[slot], tot);
+    }
+    u64 *gh = P.hist + (size_t)slot * NBINS;
+    for (int i = threadIdx.x; i < NBINS; i += THREADS) {
+        const u32 h = sh.hist[i];
+        if (h) atomicAdd(&gh[i], (u64)h);
+    }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------- sources
+// Unstructured: key of every element of every tensor.
+__device__ __forceinline__ void scan_source_elem(const Params &P, ScanShared &sh, ScanCtx &c)
+{
+    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        const long long ng = (d.numel + d.pad + 3) >> 2;
+        const long long g0 = (item - P.item_prefix[t]) * GROUPS_PER_ITEM;
+        const long long g1 = (g0 + GROUPS_PER_ITEM < ng) ? g0 + GROUPS_PER_ITEM : ng;
+        const bool has_lam = d.lam != nullptr;
+        float w[GROUPS_PER_ITEM / THREADS][4], l[GROUPS_PER_ITEM / THREADS][4];
+#pragma unroll
+        for (int it = 0; it < GROUPS_PER_ITEM / THREADS; ++it) {
+            const long long g = g0 + it * THREADS + threadIdx.x;
+            const long long e0 = 4 * g - d.pad;
+            const bool live = g < g1;
+            const bool full = live && d.vec_ok && e0 >= 0 && e0 + 4 <= d.numel;
+            if (full) {
+                const float4 a = __ldg(reinterpret_cast<const float4 *>(d.w + e0));
+                w[it][0] = a.x; w[it][1] = a.y; w[it][2] = a.z; w[it][3] = a.w;
+                if (has_lam) {
+                    const float4 b = *reinterpret_cast<const float4 *>(d.lam + e0);
+                    l[it][0] = b.x; l[it][1] = b.y; l[it][2] = b.z; l[it][3] = b.w;
+                } else {
+                    l[it][0] = l[it][1] = l[it][2] = l[it][3] = 0.0f;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const long long e = e0 + j;
+                    const bool ok = live && e >= 0 && e < d.numel;
+                    w[it][j] = ok ? d.w[e] : 0.0f;
+                    l[it][j] = (ok && has_lam) ? d.lam[e] : 0.0f;
+                }
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < GROUPS_PER_ITEM / THREADS; ++it) {
+            const long long g = g0 + it * THREADS + threadIdx.x;
+            const long long e0 = 4 * g - d.pad;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const long long e = e0 + j;
+                const bool ok = g < g1 && e >= 0 && e < d.numel;
+                const float u = form_u(w[it][j], l[it][j], P.mu, has_lam);
+                scan_emit(P, sh, c, key_of_u(u), (u64)(d.elem_prefix + e), ok);
+            }
+        }
+    }
+}
+
+// nu of one 4x4 block: fp64 sum of u^2, row by row. Elements outside the tensor
+// count as zero. Returns the fp64 bit pattern.
+struct BlockData {
+    float w[16], l[16];
+    bool full;
+    long long r0, c0;
+};
+
+__device__ __forceinline__ void load_block(const TensorDesc &d, long long b, BlockData &bd)
+{
+    long long br;
+    if (d.n_units < 0x7FFFFFFFll) br = (long long)((u32)b / (u32)d.nbc);
+    else br = b / d.nbc;
+    const long long bc = b - br * d.nbc;
+    bd.r0 = br * 4;
+    bd.c0 = bc * 4;
+    bd.full = d.blk_vec_ok && bd.r0 + 4 <= d.d0;
+    const bool has_lam = d.lam != nullptr;
+    if (bd.full) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const long long off = (bd.r0 + i) * d.d1 + bd.c0;
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(d.w + off));
+            bd.w[4 * i + 0] = a.x; bd.w[4 * i + 1] = a.y; bd.w[4 * i + 2] = a.z; bd.w[4 * i + 3] = a.w;
+            if (has_lam) {
+                const float4 q = *reinterpret_cast<const float4 *>(d.lam + off);
+                bd.l[4 * i + 0] = q.x; bd.l[4 * i + 1] = q.y; bd.l[4 * i + 2] = q.z; bd.l[4 * i + 3] = q.w;
+            } else {
+                bd.l[4 * i + 0] = bd.l[4 * i + 1] = bd.l[4 * i + 2] = bd.l[4 * i + 3] = 0.0f;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const long long r = bd.r0 + i, cc = bd.c0 + j;
+                const bool ok = r < d.d0 && cc < d.d1;
+                const long long off = r * d.d1 + cc;
+                bd.w[4 * i + j] = ok ? d.w[off] : 0.0f;
+                bd.l[4 * i + j] = (ok && has_lam) ? d.lam[off] : 0.0f;
+            }
+    }
+}
+
+__device__ __forceinline__ u64 block_key(const BlockData &bd, float mu, bool has_lam, float *u)
+{
+    double acc = 0.0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        u[i] = form_u(bd.w[i], bd.l[i], mu, has_lam);
+        const double x = (double)u[i];
+        acc = __fma_rn(x, x, acc);     // x*x is exact in fp64, so this is (acc + x*x) rounded once
+    }
+    return (u64)__double_as_longlong(acc);
+}
+
+// Block items exist for ranked (2-D) tensors only in the scan decomposition.
+__device__ __forceinline__ void scan_source_block(const Params &P, ScanShared &sh, ScanCtx &c)
+{
+    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        const long long b0 = (item - P.item_prefix[t]) * BLOCKS_PER_ITEM;
+        const bool has_lam = d.lam != nullptr;
+#pragma unroll 1
+        for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it) {
+            const long long b = b0 + it * THREADS + threadIdx.x;
+            const bool ok = b < d.n_units;
+            u64 key = 0;
+            if (ok) {
+                BlockData bd;
+                float u[16];
+                load_block(d, b, bd);
+                key = block_key(bd, P.mu, has_lam, u);
+            }
+            scan_emit(P, sh, c, key, (u64)(d.unit_prefix + b), ok);
+        }
+    }
+}
+
+__device__ __forceinline__ void scan_source_array(const Params &P, ScanShared &sh, ScanCtx &c)
+{
+    const long long stride = (long long)gridDim.x * THREADS;
+    for (long long base = (long long)blockIdx.x * THREADS; base < P.S; base += stride) {
+        const long long i = base + threadIdx.x;
+        const bool ok = i < P.S;
+        scan_emit(P, sh, c, ok ? P.arr_key[i] : 0, (u64)i, ok);
+    }
+}
+
+template <int SRC>
+__device__ __forceinline__ void scan_source(const Params &P, ScanShared &sh, bool do_list, int slot)
+{
+    ScanCtx c;
+    scan_begin(sh, c, do_list);
+    if (SRC == SRC_ELEM) scan_source_elem(P, sh, c);
+    else if (SRC == SRC_BLOCK) scan_source_block(P, sh, c);
+    else scan_source_array(P, sh, c);
+    scan_end(P, sh, c, slot);
+}
+
+__device__ __forceinline__ void scan_list(const Params &P, ScanShared &sh, int slot, u64 n_list)
+{
+    ScanCtx c;
+    scan_begin(sh, c, false);
+    const u64 stride = (u64)gridDim.x * THREADS;
+    for (u64 base = (u64)blockIdx.x * THREADS; base < n_list; base += stride) {
+        const u64 i = base + threadIdx.x;
+        const bool ok = i < n_list;
+        scan_emit(P, sh, c, ok ? __ldcg(&P.list_key[i]) : 0, ok ? __ldcg(&P.list_id[i]) : 0, ok);
+    }
+    scan_end(P, sh, c, slot);
+}
+
+// ---------------------------------------------------------------- pick
+__device__ __forceinline__ void set_shift(Sel &s)
+{
+    const u64 range = (s.lo_key == s.hi_key) ? (s.hi_id - s.lo_id) : (s.hi_key - s.lo_key);
+    const int bl = bit_length(range);
+    s.shift = bl > LOG_NBINS ? bl - LOG_NBINS : 0;
+}
+
+// All threads of the CTA; every CTA computes the same new state from the same
+// global histogram. `src_scan`: the scan that filled the histogram visited the
+// whole source (its count of units above the bracket is then complete).
+__device__ __forceinline__ void block_pick(const Params &P, ScanShared &sh, bool src_scan, u64 max_key)
+{
+    Sel &s = sh.sel;
+    const u64 *gh = P.hist + (size_t)s.slot * NBINS;
+    constexpr int PER = NBINS / THREADS;
+    u64 cnt[PER];
+    u64 tsum = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        cnt[j] = __ldcg(&gh[threadIdx.x * PER + j]);
+        tsum += cnt[j];
+    }
+    // exclusive scan of tsum over the CTA
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    u64 inc = tsum;
+    for (int o = 1; o < 32; o <<= 1) {
+        const u64 v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += v;
+    }
+    if (lane == 31) sh.red[warp] = inc;
+    if (threadIdx.x == 0) sh.pick_bin = -1;
+    __syncthreads();
+    u64 wbase = 0, total = 0;
+    for (int i = 0; i < WARPS; ++i) {
+        if (i < warp) wbase += sh.red[i];
+        total += sh.red[i];
+    }
+    const u64 excl = wbase + inc - tsum;
+    const u64 above_scan = __ldcg(&P.ctl->scan_above[s.slot]);
+    const u64 n_above = s.above_known ? s.n_above : above_scan;
+    const bool valid = s.k > n_above && (s.k - n_above) <= total;
+    const u64 r = s.k - n_above;
+    if (valid && r > excl && r <= excl + tsum) {
+        u64 run = excl;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            if (r > run && r <= run + cnt[j]) {
+                sh.pick_bin = threadIdx.x * PER + j;
+                sh.pick_before = run;
+                sh.pick_count = cnt[j];
+            }
+            run += cnt[j];
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s.passes += 1;
+        if (s.above_known && src_scan && above_scan != s.n_above) s.error = 1;
+        const bool sk = s.lo_key == s.hi_key;
+        if (!valid) {
+            if (s.above_known) {
+                s.error = 2;        // a histogram-derived bracket must hold the rank
+                s.done = 1;
+            } else if (s.k <= n_above) {
+                // wanted unit ranks before the sampled bracket
+                if (sk && s.lo_id > 0) { s.error = 3; s.done = 1; }
+                s.lo_key = s.hi_key + 1;
+                s.hi_key = max_key;
+                s.n_above = 0;
+                s.pop = n_above;
+            } else {
+                if (s.lo_key == 0) { s.error = 4; s.done = 1; }
+                s.n_above = n_above + total;
+                s.hi_key = s.lo_key - 1;
+                s.lo_key = 0;
+                s.pop = s.S - s.n_above;
+            }
+            s.lo_id = 0;
+            s.hi_id = s.S - 1;
+            s.above_known = 1;
+            s.list_valid = 0;
+            s.sampled = 0;
+            if (s.lo_key > s.hi_key) { s.error = 4; s.done = 1; }
+        } else {
+            if (sk && !s.key_fixed) {
+                s.key_fixed = 1;
+                s.n_gt = n_above;
+                s.n_tie = total;
+            }
+            const int b = sh.pick_bin;
+            if (b < 0) { s.error = 5; s.done = 1; }
+            s.n_above = n_above + sh.pick_before;
+            s.above_known = 1;
+            s.pop = sh.pick_count;
+            if (!sk) {
+                const u64 width = 1ull << s.shift;
+                const u64 nh = s.hi_key - ((u64)b << s.shift);
+                u64 nl = (nh - s.lo_key >= width - 1) ? nh - (width - 1) : s.lo_key;
+                s.hi_key = nh;
+                s.lo_key = nl;
+                if (nl == nh && !s.key_fixed) {
+                    s.key_fixed = 1;
+                    s.n_gt = s.n_above;
+                    s.n_tie = s.pop;
+                    s.lo_id = 0;
+                    s.hi_id = s.S - 1;
+                }
+            } else {
+                const u64 width = 1ull << s.shift;
+                const u64 nl = s.lo_id + ((u64)b << s.shift);
+                const u64 nh = (s.hi_id - nl >= width - 1) ? nl + (width - 1) : s.hi_id;
+                s.lo_id = nl;
+                s.hi_id = nh;
+            }
+            if (s.lo_key == s.hi_key && s.lo_id == s.hi_id) {
+                s.done = 1;            // a single unit is left: it is the cut-off
+                if (s.pop != 1) s.error = 6;
+            }
+        }
+        set_shift(s);
+        if (s.passes >= MAX_SELECT_ITERS && !s.done) { s.error = 7; s.done = 1; }
+    }
+    __syncthreads();
+}
+
+// Rank the (at most FIN) bracket members directly. Entries are in fin_key/fin_id.
+__device__ __forceinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
+{
+    Sel &s = sh.sel;
+    u64 *k = &sh.stg_key[0][0];       // FIN <= WARPS * WSTG
+    u64 *d = &sh.stg_id[0][0];
+    if (n > FIN) n = FIN;
+    for (u32 i = threadIdx.x; i < n; i += THREADS) {
+        k[i] = __ldcg(&P.fin_key[i]);
+        d[i] = __ldcg(&P.fin_id[i]);
+    }
+    if (threadIdx.x == 0) sh.fin_hit = -1;
+    __syncthreads();
+    const u64 r = s.k - s.n_above;     // 1-based rank inside the bracket
+    // bitonic sort of the padded array into ranking order (first = strongest)
+    u32 n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    for (u32 i = n + threadIdx.x; i < n2; i += THREADS) { k[i] = 0; d[i] = ~0ull; }   // ranks last
+    __syncthreads();
+    for (u32 size = 2; size <= n2; size <<= 1) {
+        for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
+            for (u32 t = threadIdx.x; t < (n2 >> 1); t += THREADS) {
+                const u32 i = 2 * t - (t & (stride - 1));
+                const u32 j = i + stride;
+                const bool i_after_j = k[j] > k[i] || (k[j] == k[i] && d[j] < d[i]);
+                const bool j_after_i = k[i] > k[j] || (k[i] == k[j] && d[i] < d[j]);
+                const bool up = (i & size) == 0;
+                if (up ? i_after_j : j_after_i) {
+                    const u64 tk = k[i], td = d[i];
+                    k[i] = k[j]; d[i] = d[j];
+                    k[j] = tk; d[j] = td;
+                }
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0 && r >= 1 && r <= (u64)n) sh.fin_hit = (int)(r - 1);
+    __syncthreads();
+    if (sh.fin_hit >= 0) {
+        const u64 tk = k[sh.fin_hit];
+        u64 gt = 0, eq = 0;
+        for (u32 i = threadIdx.x; i < n; i += THREADS) {
+            gt += k[i] > tk ? 1 : 0;
+            eq += k[i] == tk ? 1 : 0;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            gt += __shfl_xor_sync(0xffffffffu, gt, o);
+            eq += __shfl_xor_sync(0xffffffffu, eq, o);
+        }
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) {
+            sh.red[threadIdx.x >> 5] = gt;
+            sh.hist[threadIdx.x >> 5] = (u32)eq;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            u64 g = 0, e = 0;
+            for (int i = 0; i < WARPS; ++i) { g += sh.red[i]; e += sh.hist[i]; }
+            if (!s.key_fixed) {
+                s.key_fixed = 1;
+                s.n_gt = s.n_above + g;
+                s.n_tie = e;
+            }
+            s.lo_key = s.hi_key = tk;
+            s.lo_id = s.hi_id = d[sh.fin_hit];
+            s.done = 1;
+        }
+    } else if (threadIdx.x == 0) {
+        s.error = 8;
+        s.done = 1;
+    }
+    __syncthreads();
+}
+
+// First pass of a ranking call: a plain (non-cooperative) scan at full grid.
+template <int SRC>
+__global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
+{
+    __shared__ ScanShared sh;
+    if (threadIdx.x == 0) sh.sel = P.ctl->sel;
+    __syncthreads();
+    scan_source<SRC>(P, sh, do_list != 0, sh.sel.slot);
+}
+
+// Cooperative driver: picks, further scans, direct ranking of the last few,
+// result record. Entered with the histogram of the first scan in slot 0.
+template <int SRC>
+__global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
+{
+    __shared__ ScanShared sh;
+    cg::grid_group grid = cg::this_grid();
+    const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
+    if (threadIdx.x == 0) sh.sel = P.ctl->sel;
+    __syncthreads();
+    bool src_scan = true;
+    if (!sh.sel.done) {
+        if (first_listed && threadIdx.x == 0) sh.sel.list_valid = 1;
+        __syncthreads();
+        for (int it = 0; it < MAX_SELECT_ITERS + 2; ++it) {
+            // a listing scan that overflowed the list does not count
+            if (threadIdx.x == 0 && sh.sel.list_valid &&
+                __ldcg(&P.ctl->list_count[sh.sel.list_sel]) > P.cap) sh.sel.list_valid = 0;
+            __syncthreads();
+            block_pick(P, sh, src_scan, max_key);
+            // clear the histogram slot that the scan after the next one will use
+            if (blockIdx.x == 0) {
+                const int z = (sh.sel.slot + 2) % 3;
+                for (int i = threadIdx.x; i < NBINS; i += THREADS) P.hist[(size_t)z * NBINS + i] = 0;
+                if (threadIdx.x == 0) P.ctl->scan_above[z] = 0;
+            }
+            if (sh.sel.done) break;
+            if (sh.sel.list_valid && sh.sel.pop <= FIN) {
+                // gather the bracket members from the list and rank them
+                const u64 n_list = __ldcg(&P.ctl->list_count[sh.sel.list_sel]);
+                const Sel &s = sh.sel;
+                const bool sk = s.lo_key == s.hi_key;
+                const u64 stride = (u64)gridDim.x * THREADS;
+                for (u64 i = (u64)blockIdx.x * THREADS + threadIdx.x; i < n_list; i += stride) {
+                    const u64 key = __ldcg(&P.list_key[i]), id = __ldcg(&P.list_id[i]);
+                    const bool above = key > s.hi_key || (sk && key == s.hi_key && id < s.lo_id);
+                    const bool below = key < s.lo_key || (sk && key == s.lo_key && id > s.hi_id);
+                    if (!above && !below) {
+                        const u32 pos = atomicAdd(&P.ctl->fin_count, 1u);
+                        if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; }
+                    }
+                }
+                grid.sync();
+                const u32 n = __ldcg(&P.ctl->fin_count);
+                if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
+                __syncthreads();
+                final_rank(P, sh, n);
+                break;
+            }
+            // next scan
+            if (threadIdx.x == 0) sh.sel.slot = (sh.sel.slot + 1) % 3;
+            __syncthreads();
+            if (sh.sel.list_valid) {
+                scan_list(P, sh, sh.sel.slot, __ldcg(&P.ctl->list_count[sh.sel.list_sel]));
+                src_scan = false;
+            } else {
+                const bool do_list = sh.sel.pop <= P.cap;
+                if (do_list && threadIdx.x == 0) sh.sel.list_sel = 1;
+                __syncthreads();
+                scan_source<SRC>(P, sh, do_list, sh.sel.slot);
+                if (do_list && threadIdx.x == 0) sh.sel.list_valid = 1;
+                __syncthreads();
+                src_scan = true;
+            }
+            grid.sync();
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        Ctl *c = P.ctl;
+        const Sel &s = sh.sel;
+        Result r;
+        r.status = s.error ? -5 : 0;
+        r.passes = s.passes;
+        r.n_units = (long long)s.S;
+        r.n_keep = (long long)s.k;
+        r.n_zero = (long long)(s.S - s.k);
+        r.sampled = s.sampled;
+        r.n_candidates = (long long)(c->list_count[0] + c->list_count[1]);
+        r.tau_norm = 0.0f;
+        if (s.k == 0 || s.S == 0 || s.error) {
+            c->tau_key = KEY_NONE;
+            c->tau_id = 0;
+            r.tau_key = (P.bits_key >= 63) ? 0x7FF0000000000000ull : 0x7F800000ull;
+            r.tau_id = -1;
+            r.n_gt = r.n_tie = r.n_tie_kept = 0;
+        } else {
+            c->tau_key = s.lo_key;
+            c->tau_id = s.lo_id;
+            r.tau_key = s.lo_key;
+            r.tau_id = (long long)s.lo_id;
+            r.n_gt = (long long)s.n_gt;
+            r.n_tie = (long long)s.n_tie;
+            r.n_tie_kept = (long long)(s.k - s.n_gt);
+            if (P.bits_key >= 63) r.tau_norm = (float)sqrt(__longlong_as_double((long long)s.lo_key));
+        }
+        c->sel = s;
+        c->res = r;
+    }
+}
+
+// Start of every ranking call: clears the histograms and counters and installs
+// the initial selection state.
+__global__ void __launch_bounds__(THREADS) k_init(Params P, Sel init)
+{
+    const int n = 3 * NBINS;
+    for (int i = blockIdx.x * THREADS + threadIdx.x; i < n; i += gridDim.x * THREADS) P.hist[i] = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        Ctl *c = P.ctl;
+        c->sel = init;
+        c->tau_key = KEY_NONE;
+        c->tau_id = 0;
+        c->scan_above[0] = c->scan_above[1] = c->scan_above[2] = 0;
+        c->list_count[0] = c->list_count[1] = 0;
+        c->fin_count = 0;
+    }
+}
+
+}  // namespace cs

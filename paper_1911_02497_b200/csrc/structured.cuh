@@ -1,0 +1,157 @@
+// Structured pruning kernels: 4x4 block projection with a known cut-off, and
+// the fp64 filter norms (segment partial sums + in-order combine).
+#pragma once
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "select.cuh"
+
+namespace cs {
+
+// Final write of one 4x4 block given the keep decision.
+__device__ __forceinline__ void store_block(const TensorDesc &d, const BlockData &bd, const float *u,
+                                            bool keep, float mu, unsigned fuse)
+{
+    const bool has_lam = d.lam != nullptr;
+    const bool wr_lam = (fuse & FUSE_LAMBDA) && has_lam;
+    const bool wr_grad = (fuse & FUSE_PENALTY) && d.grad != nullptr;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        Out o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            o[j] = finish(bd.w[4 * i + j], bd.l[4 * i + j], u[4 * i + j], keep, mu, fuse, has_lam);
+        const long long off = (bd.r0 + i) * d.d1 + bd.c0;
+        if (bd.full) {
+            float v[4] = {o[0].theta, o[1].theta, o[2].theta, o[3].theta};
+            st4(d.theta + off, v);
+            if (d.mask) {
+                const u32 mm = (u32)o[0].m | ((u32)o[1].m << 8) | ((u32)o[2].m << 16) | ((u32)o[3].m << 24);
+                *reinterpret_cast<u32 *>(d.mask + off) = mm;
+            }
+            if (d.theta_h) {
+                uint2 hh;
+                hh.x = (u32)o[0].th | ((u32)o[1].th << 16);
+                hh.y = (u32)o[2].th | ((u32)o[3].th << 16);
+                *reinterpret_cast<uint2 *>(d.theta_h + off) = hh;
+            }
+            if (wr_lam) {
+                float v2[4] = {o[0].lam, o[1].lam, o[2].lam, o[3].lam};
+                st4(d.lam + off, v2);
+            }
+            if (wr_grad) {
+                float v3[4] = {o[0].grad, o[1].grad, o[2].grad, o[3].grad};
+                st4(d.grad + off, v3);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (bd.r0 + i >= d.d0 || bd.c0 + j >= d.d1) continue;
+                d.theta[off + j] = o[j].theta;
+                if (d.mask) d.mask[off + j] = o[j].m;
+                if (d.theta_h) d.theta_h[off + j] = o[j].th;
+                if (wr_lam) d.lam[off + j] = o[j].lam;
+                if (wr_grad) d.grad[off + j] = o[j].grad;
+            }
+        }
+    }
+}
+
+// Projection pass of block pruning. Work items: BLOCKS_PER_ITEM blocks for
+// ranked (2-D) tensors, linear items for tensors that pass through.
+__global__ void __launch_bounds__(THREADS) k_apply_block(Params P)
+{
+    const u64 tau_key = P.ctl->tau_key, tau_id = P.ctl->tau_id;
+    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        const long long local = item - P.item_prefix[t];
+        if (!d.ranked) {
+            process_linear_item<M_KEEPALL>(P, d, local, 0, 0);
+            continue;
+        }
+        const bool has_lam = d.lam != nullptr;
+#pragma unroll 1
+        for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it) {
+            const long long b = local * BLOCKS_PER_ITEM + it * THREADS + threadIdx.x;
+            if (b >= d.n_units) continue;
+            BlockData bd;
+            float u[16];
+            load_block(d, b, bd);
+            const u64 key = block_key(bd, P.mu, has_lam, u);
+            const bool keep = keep_by_cutoff(key, (u64)(d.unit_prefix + b), tau_key, tau_id);
+            store_block(d, bd, u, keep, P.mu, P.fuse);
+        }
+    }
+}
+
+// Filter norms, step 1: one warp per segment of SEG elements of one filter.
+// Lane l adds elements l, l+32, ... of the segment in that order, then the 32
+// lane sums are combined by a fixed butterfly; the value depends only on the
+// segment's contents and length, never on where the filter sits.
+// Work items: (filter, segment) pairs of ranked tensors, WARPS per CTA step.
+__global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long n_work = P.n_items;
+    for (long long base = (long long)blockIdx.x * WARPS; base < n_work; base += (long long)gridDim.x * WARPS) {
+        const long long item = base + warp;
+        if (item >= n_work) continue;
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        const long long local = item - P.item_prefix[t];
+        const long long nseg = (d.d1 + SEG - 1) / SEG;
+        const long long f = local / nseg, sgm = local - f * nseg;
+        const long long j0 = sgm * SEG;
+        const long long j1 = (j0 + SEG < d.d1) ? j0 + SEG : d.d1;
+        const float *__restrict__ wp = d.w + f * d.d1;
+        const float *lp = d.lam ? d.lam + f * d.d1 : nullptr;
+        const bool has_lam = lp != nullptr;
+        double acc = 0.0;
+        long long j = j0 + lane;
+        for (; j + 7 * 32 < j1; j += 8 * 32) {
+            float wv[8], lv[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                wv[q] = __ldg(wp + j + q * 32);
+                lv[q] = has_lam ? lp[j + q * 32] : 0.0f;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const double x = (double)form_u(wv[q], lv[q], P.mu, has_lam);
+                acc = __fma_rn(x, x, acc);
+            }
+        }
+        for (; j < j1; j += 32) {
+            const double x = (double)form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam);
+            acc = __fma_rn(x, x, acc);
+        }
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) P.partial[item] = acc;
+    }
+}
+
+// Filter norms, step 2: nu_f = partial sums added in segment order.
+__global__ void __launch_bounds__(THREADS) k_filter_combine(Params P)
+{
+    const long long stride = (long long)gridDim.x * THREADS;
+    for (long long sid = (long long)blockIdx.x * THREADS + threadIdx.x; sid < P.S; sid += stride) {
+        // tensor that owns structure sid
+        int lo = 0, hi = P.T - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (P.td[mid].unit_prefix <= sid) lo = mid; else hi = mid - 1;
+        }
+        // skip tensors without ranked structures that share the same prefix
+        int t = lo;
+        while (t > 0 && P.td[t].n_units == 0) --t;
+        const TensorDesc d = P.td[t];
+        const long long f = sid - d.unit_prefix;
+        const long long nseg = (d.d1 + SEG - 1) / SEG;
+        const double *p = P.partial + P.item_prefix[t] + f * nseg;
+        double acc = 0.0;
+        for (long long sgm = 0; sgm < nseg; ++sgm) acc = __dadd_rn(acc, p[sgm]);
+        P.arr_key[sid] = (u64)__double_as_longlong(acc);
+    }
+}
+
+}  // namespace cs

@@ -1,0 +1,216 @@
+"""Thin ctypes binding of ``libcondensa_cstep.so`` (argument marshalling only).
+
+Every step of the C-step runs in the library's CUDA kernels; PyTorch is used
+by callers for device memory and streams. There is no CPU fallback: if the
+shared library is missing or no CUDA device is present the calls raise.
+Function names and arguments mirror ``include/condensa_cstep.h``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcondensa_cstep.so")
+
+FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, NO_SAMPLING = 1, 2, 4, 64
+OP_PRUNE, OP_FILTER, OP_BLOCK, OP_QUANTIZE, OP_LAGRANGE = 0, 1, 2, 3, 4
+DTYPE_FP16 = 1
+OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_UNSUPPORTED, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
+
+EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "condensa_cstep_filter",
+           "condensa_cstep_block", "condensa_cstep_quantize", "condensa_cstep_lagrange_update",
+           "condensa_cstep_host", "condensa_get_result", "condensa_launch_count",
+           "condensa_last_error", "condensa_profile_enable", "condensa_profile_read"]
+
+
+class CondensaError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__("condensa error %d: %s" % (code, text))
+        self.code = code
+
+
+class Tensor(C.Structure):
+    """Mirror of ``condensa_tensor``."""
+    _fields_ = [("w", C.c_void_p), ("lam", C.c_void_p), ("theta", C.c_void_p),
+                ("mask", C.c_void_p), ("grad", C.c_void_p), ("theta_h", C.c_void_p),
+                ("numel", C.c_int64), ("ndim", C.c_int32), ("shape", C.c_int64 * 4)]
+
+
+class Result(C.Structure):
+    """Mirror of ``condensa_result``."""
+    _fields_ = [("status", C.c_int32), ("passes", C.c_int32), ("n_units", C.c_int64),
+                ("n_zero", C.c_int64), ("n_keep", C.c_int64), ("tau_key", C.c_uint64),
+                ("tau_id", C.c_int64), ("n_gt", C.c_int64), ("n_tie", C.c_int64),
+                ("n_tie_kept", C.c_int64), ("tau_norm", C.c_float), ("sampled", C.c_int32),
+                ("n_candidates", C.c_int64)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class KernelTime(C.Structure):
+    """Mirror of ``condensa_kernel_time``."""
+    _fields_ = [("name", C.c_char * 48), ("launches", C.c_int64), ("total_ms", C.c_double)]
+
+
+_lib = None
+
+
+def load():
+    """Load the shared library (no GPU needed for this) and declare signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("%s is missing: run `python -m paper_1911_02497_b200.build`" % LIB_PATH)
+    L = C.CDLL(LIB_PATH)
+    vp, i32, u32, f32, f64 = C.c_void_p, C.c_int, C.c_uint, C.c_float, C.c_double
+    L.condensa_create.argtypes = [C.POINTER(vp), i32, C.c_size_t]
+    L.condensa_destroy.argtypes = [vp]
+    L.condensa_cstep_prune.argtypes = [vp, vp, i32, f64, f32, u32, vp]
+    L.condensa_cstep_filter.argtypes = [vp, vp, i32, f64, f32, u32, vp]
+    L.condensa_cstep_block.argtypes = [vp, vp, i32, f64, f32, i32, i32, u32, vp]
+    L.condensa_cstep_quantize.argtypes = [vp, vp, i32, f32, i32, u32, vp]
+    L.condensa_cstep_lagrange_update.argtypes = [vp, vp, i32, f32, u32, vp]
+    L.condensa_cstep_host.argtypes = [vp, i32, vp, i32, f64, f32, i32, i32, u32, vp]
+    L.condensa_get_result.argtypes = [vp, C.POINTER(Result)]
+    L.condensa_profile_enable.argtypes = [vp, i32]
+    L.condensa_profile_read.argtypes = [vp, C.POINTER(KernelTime), i32, C.POINTER(i32)]
+    L.condensa_launch_count.argtypes = [vp]
+    L.condensa_launch_count.restype = C.c_int64
+    L.condensa_last_error.argtypes = [vp]
+    L.condensa_last_error.restype = C.c_char_p
+    for name in EXPORTS:
+        getattr(L, name)
+    _lib = L
+    return L
+
+
+def fuse_bits(fuse) -> int:
+    if isinstance(fuse, int):
+        return fuse
+    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY,
+             "no_sampling": NO_SAMPLING}
+    b = 0
+    for f in fuse:
+        b |= table[f]
+    return b
+
+
+def _addr(x) -> Optional[int]:
+    """Address of a torch tensor, a numpy array, an int, or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    return int(x.ctypes.data)
+
+
+def tensor_table(w: Sequence, lam: Optional[Sequence] = None, theta: Optional[Sequence] = None,
+                 mask: Optional[Sequence] = None, grad: Optional[Sequence] = None,
+                 theta_h: Optional[Sequence] = None, shapes: Optional[Sequence] = None):
+    """Build a ``condensa_tensor[T]`` array from per-tensor buffers (torch tensors
+    on the device, or numpy arrays for the host entry point). Buffers must be
+    contiguous; the caller keeps them alive."""
+    T = len(w)
+    tab = (Tensor * max(T, 1))()
+    for t in range(T):
+        e = tab[t]
+        shp = tuple(shapes[t]) if shapes is not None else tuple(w[t].shape)
+        n = 1
+        for d in shp:
+            n *= int(d)
+        e.w = _addr(w[t])
+        e.lam = _addr(lam[t]) if lam is not None else None
+        e.theta = _addr(theta[t]) if theta is not None else None
+        e.mask = _addr(mask[t]) if mask is not None else None
+        e.grad = _addr(grad[t]) if grad is not None else None
+        e.theta_h = _addr(theta_h[t]) if theta_h is not None else None
+        e.numel, e.ndim = n, len(shp)
+        for d in range(4):
+            e.shape[d] = int(shp[d]) if d < len(shp) else 1
+    return tab
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)          # torch.cuda.Stream
+
+
+class Context:
+    """Owns a ``condensa_ctx`` (workspace and descriptor cache of one device)."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        self._lib = load()
+        h = C.c_void_p()
+        rc = self._lib.condensa_create(C.byref(h), int(device), int(workspace_bytes))
+        if rc != OK:
+            raise CondensaError(rc, (self._lib.condensa_last_error(None) or b"").decode())
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.condensa_destroy(self._h)
+            self._h = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != OK:
+            raise CondensaError(rc, (self._lib.condensa_last_error(self._h) or b"").decode())
+
+    def cstep_prune(self, tab, T, sparsity, mu, fuse=(), stream=None):
+        self._check(self._lib.condensa_cstep_prune(self._h, tab, T, float(sparsity), float(mu),
+                                                   fuse_bits(fuse), _stream_handle(stream)))
+
+    def cstep_filter(self, tab, T, sparsity, mu, fuse=(), stream=None):
+        self._check(self._lib.condensa_cstep_filter(self._h, tab, T, float(sparsity), float(mu),
+                                                    fuse_bits(fuse), _stream_handle(stream)))
+
+    def cstep_block(self, tab, T, sparsity, mu, bh=4, bw=4, fuse=(), stream=None):
+        self._check(self._lib.condensa_cstep_block(self._h, tab, T, float(sparsity), float(mu),
+                                                   int(bh), int(bw), fuse_bits(fuse),
+                                                   _stream_handle(stream)))
+
+    def cstep_quantize(self, tab, T, mu, dtype=DTYPE_FP16, fuse=(), stream=None):
+        self._check(self._lib.condensa_cstep_quantize(self._h, tab, T, float(mu), int(dtype),
+                                                      fuse_bits(fuse), _stream_handle(stream)))
+
+    def cstep_lagrange_update(self, tab, T, mu, fuse=("lambda",), stream=None):
+        self._check(self._lib.condensa_cstep_lagrange_update(self._h, tab, T, float(mu),
+                                                             fuse_bits(fuse), _stream_handle(stream)))
+
+    def cstep_host(self, op, tab, T, sparsity, mu, bh=4, bw=4, fuse=(), stream=None):
+        self._check(self._lib.condensa_cstep_host(self._h, int(op), tab, T, float(sparsity),
+                                                  float(mu), int(bh), int(bw), fuse_bits(fuse),
+                                                  _stream_handle(stream)))
+
+    def get_result(self) -> Result:
+        r = Result()
+        self._check(self._lib.condensa_get_result(self._h, C.byref(r)))
+        return r
+
+    def profile_enable(self, on: bool):
+        self._check(self._lib.condensa_profile_enable(self._h, 1 if on else 0))
+
+    def profile_read(self):
+        """{kernel name: (launches, total ms)} since profiling was enabled."""
+        buf = (KernelTime * 32)()
+        n = C.c_int(0)
+        self._check(self._lib.condensa_profile_read(self._h, buf, 32, C.byref(n)))
+        return {buf[i].name.decode(): (int(buf[i].launches), float(buf[i].total_ms))
+                for i in range(n.value)}
+
+    def launch_count(self) -> int:
+        return int(self._lib.condensa_launch_count(self._h))

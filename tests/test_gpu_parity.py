@@ -1,0 +1,333 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs. Integer / bit results must be identical; fp32 values are
+produced by the same single IEEE operations, so they are compared bit for bit as
+well (and within 1e-6 relative as the stated bar)."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_1911_02497_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+REL = 1e-6      # tolerance stated for fp32 norms and multiplier updates
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_1911_02497_b200 import cstep
+    c = cstep.Context(0)
+    yield c
+    c.close()
+
+
+def bits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def same_f32(a, b):
+    """Bit-identical, except that a NaN only has to be a NaN (IEEE leaves the
+    payload of a generated NaN to the implementation)."""
+    a = np.ascontiguousarray(a, np.float32); b = np.ascontiguousarray(b, np.float32)
+    na, nb = np.isnan(a), np.isnan(b)
+    return bool(np.array_equal(na, nb) and np.array_equal(bits(a)[~na], bits(b)[~nb]))
+
+
+def same_f16(a, b):
+    """binary16 bit patterns agree; a NaN only has to be a NaN."""
+    a = np.asarray(a, np.uint16); b = np.asarray(b, np.uint16)
+    na, nb = (a & 0x7FFF) > 0x7C00, (b & 0x7FFF) > 0x7C00
+    return bool(np.array_equal(na, nb) and np.array_equal(a[~na], b[~nb]))
+
+
+def rel_close(a, b):
+    a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
+    both_nan = np.isnan(a) & np.isnan(b)
+    ok = np.abs(a - b) <= REL * np.maximum(np.abs(b), 1e-30)
+    return bool(np.all(ok | both_nan | (a == b)))
+
+
+def run_gpu(ctx, op, w, lam, s, mu, fuse, block=(4, 4), elem_offset=0, skew=0, theta=None):
+    from paper_1911_02497_b200.device_set import DeviceSet
+    ds = DeviceSet(w, lam, elem_offset=elem_offset, skew=skew, theta=theta)
+    ds.poison_outputs() if theta is None else None
+    ds.run(ctx, op, s, mu, fuse, block)
+    out = ds.fetch()
+    res = ctx.get_result() if op in ("prune", "filter", "block") else None
+    return out, res
+
+
+def run_oracle(op, w, lam, s, mu, fuse, block=(4, 4), theta=None):
+    if op == "prune":
+        return oracle.cstep_prune(w, lam, s, mu, fuse)
+    if op == "filter":
+        return oracle.cstep_filter(w, lam, s, mu, fuse)
+    if op == "block":
+        return oracle.cstep_block(w, lam, s, mu, block, fuse)
+    if op == "quantize":
+        return oracle.cstep_quantize(w, lam, mu, fuse)
+    return oracle.lagrange_update(w, theta, lam, mu, fuse)
+
+
+def check(ctx, op, w, lam, s=0.0, mu=1e-3, fuse=("lambda",), block=(4, 4), elem_offset=0, skew=0,
+          theta=None, exact_key=True):
+    lam = lam if lam is not None else [None] * len(w)
+    got, res = run_gpu(ctx, op, w, lam, s, mu, fuse, block, elem_offset, skew, theta)
+    exp = run_oracle(op, w, lam, s, mu, fuse, block, theta)
+    T = len(w)
+    for t in range(T):
+        if op != "lagrange":
+            assert np.array_equal(got["mask"][t], exp.mask[t]), "mask, tensor %d" % t
+            assert same_f32(got["theta"][t], exp.theta[t]), "theta, tensor %d" % t
+            assert same_f16(got["theta_h"][t], exp.theta_h[t]), "theta_h, tensor %d" % t
+        if lam[t] is not None:
+            assert rel_close(got["lam"][t], exp.lam[t])
+            assert same_f32(got["lam"][t], exp.lam[t]), "lambda, tensor %d" % t
+        if "penalty" in fuse:
+            assert rel_close(got["grad"][t], exp.grad[t])
+            assert same_f32(got["grad"][t], exp.grad[t]), "grad, tensor %d" % t
+    if res is not None:
+        r = exp.result
+        assert res.status == 0
+        assert (res.n_units, res.n_zero, res.n_keep) == (r.n_units, r.n_zero, r.n_keep)
+        assert res.tau_id == r.tau_id
+        assert (res.n_gt, res.n_tie, res.n_tie_kept) == (r.n_gt, r.n_tie, r.n_tie_kept)
+        if exact_key:
+            assert res.tau_key == r.tau_key
+        else:   # filter norms: the fp64 summation order differs from the oracle's
+            a = np.array([res.tau_key], np.uint64).view(np.float64)[0]
+            b = np.array([r.tau_key], np.uint64).view(np.float64)[0]
+            assert a == b or abs(a - b) <= 1e-12 * abs(b)
+        if op != "prune" and r.n_keep > 0:
+            assert abs(res.tau_norm - r.tau_norm) <= REL * abs(r.tau_norm)
+    return got, res, exp
+
+
+# ---------------------------------------------------------------- elementwise
+@pytest.mark.parametrize("n", [1, 3, 4, 5, 1023, 4096, 4097, 100003])
+@pytest.mark.parametrize("off", [0, 1, 2, 3])
+def test_quantize_sizes_and_alignments(ctx, n, off):
+    ws = W.random_set([(n,)], seed=n + off, kind="normal", scale=3.0, lam_sigma=1e-2, mu=1e-2)
+    check(ctx, "quantize", ws.w, ws.lam, mu=ws.mu, fuse=("lambda", "penalty"), elem_offset=off)
+
+
+def test_quantize_special_values_and_skewed_alignment(ctx):
+    sp = np.array([0.0, -0.0, np.inf, -np.inf, np.nan, -np.nan, 65504.0, 65519.99, 65520.0, 1e-8,
+                   2.0 ** -24, 2.0 ** -25, 2.0 ** -25 * 1.0001, 6.1e-5, -6.0e-8, 1e-45, 3.4e38],
+                  np.float32)
+    w = np.tile(sp, 40)
+    got, _, exp = check(ctx, "quantize", [w], [None], mu=1.0, fuse=())
+    # no arithmetic touches u here, so even the NaN signs must come through
+    assert np.array_equal(got["theta_h"][0], exp.theta_h[0])
+    check(ctx, "quantize", [w], [np.zeros_like(w)], mu=1.0, fuse=("lambda", "penalty"), skew=1)
+    ws = W.random_set([(7, 9), (5,), (2, 3, 4, 5)], seed=3, kind="normal", scale=100.0, lam_sigma=1.0, mu=0.5)
+    check(ctx, "quantize", ws.w, ws.lam, mu=ws.mu, fuse=("penalty",), elem_offset=1, skew=2)
+
+
+@pytest.mark.parametrize("fuse", [("lambda",), ("penalty",), ("lambda", "penalty")])
+def test_lagrange_update(ctx, fuse):
+    ws = W.random_set([(33, 17), (4096,), (5, 3, 3, 3), (1,)], seed=8, kind="normal", scale=0.1,
+                      lam_sigma=1e-2, mu=1e-2)
+    th = [np.where(np.abs(a) > 0.08, a, 0).astype(np.float32) for a in ws.w]
+    got, _, exp = check(ctx, "lagrange", ws.w, ws.lam, mu=ws.mu, fuse=fuse, theta=th)
+    if "lambda" not in fuse:
+        for t in range(4):
+            assert np.array_equal(bits(got["lam"][t]), bits(ws.lam[t]))   # untouched
+    check(ctx, "lagrange", ws.w, [None] * 4, mu=ws.mu, fuse=fuse, theta=th, elem_offset=3)
+    # w == theta leaves lambda bit-identical and zero stays zero
+    got, _, _ = check(ctx, "lagrange", ws.w, [np.zeros_like(a) for a in ws.w], mu=ws.mu,
+                      fuse=("lambda",), theta=[a.copy() for a in ws.w])
+    assert all(np.all(bits(x) == 0) for x in got["lam"])
+
+
+# ---------------------------------------------------------------- unstructured
+@pytest.mark.parametrize("n,s", [(1, 0.0), (1, 1.0), (2, 0.5), (7, 0.5), (100, 0.01), (100, 0.99),
+                                 (4096, 0.9), (4099, 0.37), (70001, 0.95), (300007, 0.5)])
+def test_prune_small(ctx, n, s):
+    ws = W.random_set([(n,)], seed=n, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
+    check(ctx, "prune", ws.w, ws.lam, s, ws.mu, ("lambda", "penalty"))
+
+
+@pytest.mark.parametrize("off,skew", [(1, 0), (2, 0), (3, 0), (0, 1), (1, 2)])
+def test_prune_unaligned(ctx, off, skew):
+    ws = W.random_set([(5003,), (17, 13), (4, 3, 3, 3)], seed=off * 7 + skew, kind="normal",
+                      scale=0.05, lam_sigma=1e-2, mu=1e-2)
+    check(ctx, "prune", ws.w, ws.lam, 0.8, ws.mu, ("fp16", "lambda", "penalty"), elem_offset=off, skew=skew)
+
+
+def test_prune_ties_and_degenerate_inputs(ctx):
+    n = 300000          # larger than the candidate list: ties must be settled by index passes
+    check(ctx, "prune", [np.full(n, 0.5, np.float32)], None, 0.7, 1.0, ())
+    check(ctx, "prune", [np.zeros(n, np.float32)], None, 0.25, 1.0, ("lambda",))
+    two = np.where(np.arange(n) % 3 == 0, 1.0, -0.25).astype(np.float32)
+    check(ctx, "prune", [two], None, 0.5, 1.0, ())          # threshold inside the big tie group
+    check(ctx, "prune", [two], None, 0.8, 1.0, ())          # threshold inside the small one
+    pm = np.tile(np.array([1.0, -1.0, 0.0, -0.0], np.float32), 1000)
+    check(ctx, "prune", [pm], None, 0.6, 1.0, ())
+    a = np.array([2.0, 1.0], np.float32); b = np.array([1.0, 1.0, 3.0], np.float32)
+    check(ctx, "prune", [a, b], None, 0.4, 1.0, ())         # tie across a tensor boundary
+    w = np.array([1.0, np.inf, np.nan, -np.inf, 0.5], np.float32)
+    check(ctx, "prune", [w], None, 0.6, 1.0, ())
+    den = (np.arange(1, 2001, dtype=np.uint32) * 4099 % 8388607).view(np.float32)   # subnormals
+    check(ctx, "prune", [den], None, 0.5, 1.0, ())
+    q = np.round(W.draw(500000, "normal", 4.0, 1, 0, 0)).astype(np.float32)         # few distinct values
+    check(ctx, "prune", [q], None, 0.9, 1.0, ("lambda",))
+
+
+def test_prune_k_zero_keep_all_and_empty_tensors(ctx):
+    ws = W.random_set([(1000,), (0,), (37,)], seed=1, kind="normal", scale=1.0)
+    for s in (0.0, 1.0, 1e-9, 1 - 1e-9):
+        check(ctx, "prune", ws.w, None, s, 1.0, ("lambda", "penalty"))
+
+
+def test_prune_idempotent_and_unfused_sequence(ctx):
+    ws = W.config(2, scale=0.3)
+    got, res, _ = check(ctx, "prune", ws.w, ws.lam, 0.95, ws.mu, ("fp16", "lambda"))
+    again, _ = run_gpu(ctx, "prune", got["theta"], [None] * len(ws.w), 0.95, 1.0, ())
+    for a, b in zip(got["theta"], again["theta"]):
+        assert np.array_equal(bits(a), bits(b))
+    # unfused: prune, quantise theta, multiplier update == fused call
+    p, _ = run_gpu(ctx, "prune", ws.w, ws.lam, 0.95, ws.mu, ())
+    q, _ = run_gpu(ctx, "quantize", p["theta"], [None] * len(ws.w), 0.0, ws.mu, ())
+    l, _ = run_gpu(ctx, "lagrange", ws.w, ws.lam, 0.0, ws.mu, ("lambda",), theta=q["theta"])
+    for t in range(len(ws.w)):
+        assert np.array_equal(p["mask"][t], got["mask"][t])
+        assert np.array_equal(bits(q["theta"][t]), bits(got["theta"][t]))
+        assert np.array_equal(bits(l["lam"][t]), bits(got["lam"][t]))
+
+
+@pytest.mark.parametrize("cfg,scale", [(1, 1.0), (2, 1.0), (4, 0.12)])
+def test_prune_configurations(ctx, cfg, scale):
+    ws = W.config(cfg, scale=scale)
+    got, res, _ = check(ctx, "prune", ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
+    zeros = sum(int((m == 0).sum()) for m in got["mask"])
+    assert zeros == res.n_zero == math.floor(ws.sparsity * ws.numel + 0.5)
+
+
+# ---------------------------------------------------------------- filters
+def test_filter_small_and_ties(ctx):
+    ws = W.random_set([(7, 3, 3, 3), (10, 12), (9, 7, 1, 1), (6, 300, 3, 3), (3,)], seed=2,
+                      kind="normal", scale=0.2, lam_sigma=1e-2, mu=1e-2)
+    for s in (0.0, 0.3, 0.6, 1.0):
+        check(ctx, "filter", ws.w, ws.lam, s, ws.mu, ("lambda", "penalty"), exact_key=False)
+    check(ctx, "filter", ws.w, ws.lam, 0.5, ws.mu, ("fp16", "lambda"), elem_offset=1, exact_key=False)
+    f = W.draw(2 * 5 * 9, "normal", 1.0, 5, 0, 0).reshape(2, 5, 3, 3)
+    dup = np.concatenate([f, f, f], 0)                        # filters 0,2,4 and 1,3,5 identical
+    got, res, _ = check(ctx, "filter", [dup], None, 0.5, 1.0, (), exact_key=False)
+    assert res.n_tie == 3
+    ints = np.round(W.draw(8 * 3000, "normal", 3.0, 6, 0, 0)).reshape(8, 3000, 1, 1).astype(np.float32)
+    check(ctx, "filter", [ints, ints[::-1].copy()], None, 0.5, 1.0, ())   # integer data: sums exact
+    check(ctx, "filter", [np.ones((4, 5), np.float32)], None, 0.5, 1.0, ())   # nothing to rank
+
+
+@pytest.mark.parametrize("scale", [0.25, 1.0])
+def test_filter_configuration(ctx, scale):
+    ws = W.config(3, scale=scale)
+    nu = oracle.structure_norms(ws.w, ws.lam, ws.mu, "filter")
+    srt = np.sort(nu)[::-1]
+    k = nu.size - oracle.round_count(ws.sparsity, nu.size)
+    assert (srt[k - 1] - srt[k]) > 1e-9 * srt[k - 1]          # kept set is decided well above fp64 noise
+    check(ctx, "filter", ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse, exact_key=False)
+
+
+# ---------------------------------------------------------------- blocks
+@pytest.mark.parametrize("shape", [(4, 4), (1, 1), (3, 5), (8, 12), (10, 14), (33, 28), (64, 1500 // 4 * 4 + 2),
+                                   (130, 256)])
+def test_block_shapes(ctx, shape):
+    ws = W.random_set([shape, (11,), (shape[1], shape[0])], seed=sum(shape), kind="uniform", scale=0.1,
+                      lam_sigma=1e-3, mu=1e-2)
+    for s in (0.0, 0.5, 0.9, 1.0):
+        check(ctx, "block", ws.w, ws.lam, s, ws.mu, ("lambda", "penalty"))
+    check(ctx, "block", ws.w, ws.lam, 0.7, ws.mu, ("fp16", "lambda"), elem_offset=2)
+    check(ctx, "block", ws.w, ws.lam, 0.7, ws.mu, ("lambda",), skew=1)
+
+
+def test_block_ties(ctx):
+    blk = np.arange(16, dtype=np.float32).reshape(4, 4)
+    got, res, _ = check(ctx, "block", [np.tile(blk, (2, 3))], None, 0.5, 1.0, ())
+    assert (res.n_tie, res.n_tie_kept, res.tau_id) == (6, 3, 2)
+    big = np.tile(blk, (600, 300))                            # 180000 equal blocks
+    check(ctx, "block", [big], None, 0.9, 1.0, ("lambda",))
+    check(ctx, "block", [np.zeros((100, 100), np.float32)], None, 0.5, 1.0, ())
+
+
+@pytest.mark.parametrize("cfg,scale", [("5", 0.05), ("5t", 0.2)])
+def test_block_configuration_scaled(ctx, cfg, scale):
+    ws = W.config(cfg, scale=scale)
+    check(ctx, "block", ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
+
+
+# ---------------------------------------------------------------- full sizes
+@pytest.mark.parametrize("cfg", ["4", "5"])
+def test_full_size_configurations(ctx, cfg):
+    ws = W.config(cfg)
+    got, res, _ = check(ctx, ws.op, ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
+    assert res.n_units == {"4": 62367776, "5": 8490000}[cfg]
+
+
+# ---------------------------------------------------------------- arguments
+def test_argument_errors_leave_buffers_untouched(ctx):
+    from paper_1911_02497_b200 import cstep
+    from paper_1911_02497_b200.device_set import DeviceSet
+    ws = W.random_set([(64,), (8, 8)], seed=0)
+    ds = DeviceSet(ws.w, ws.lam)
+    ds.poison_outputs()
+    bad = [lambda: ds.run(ctx, "prune", 1.5, 1e-3), lambda: ds.run(ctx, "prune", float("nan"), 1e-3),
+           lambda: ds.run(ctx, "prune", 0.5, 0.0), lambda: ds.run(ctx, "prune", 0.5, float("inf")),
+           lambda: ds.run(ctx, "prune", 0.5, -1.0), lambda: ds.run(ctx, "prune", 0.5, 1e-3, fuse=8),
+           lambda: ds.run(ctx, "lagrange", 0.0, 1e-3, fuse=())]
+    for f in bad:
+        with pytest.raises(cstep.CondensaError) as e:
+            f()
+        assert e.value.code == cstep.ERR_INVALID_ARG
+    with pytest.raises(cstep.CondensaError) as e:
+        ds.run(ctx, "block", 0.5, 1e-3, block=(5, 5))
+    assert e.value.code == cstep.ERR_UNSUPPORTED
+    with pytest.raises(cstep.CondensaError) as e:
+        ctx.cstep_quantize(ds.table, ds.T, 1e-3, dtype=2)
+    assert e.value.code == cstep.ERR_UNSUPPORTED
+    # aliasing: theta on top of w; the same lambda twice
+    tab = cstep.tensor_table(ds.w, ds.lam, ds.w, shapes=ds.shapes)
+    with pytest.raises(cstep.CondensaError):
+        ctx.cstep_prune(tab, ds.T, 0.5, 1e-3, ("lambda",))
+    tab = cstep.tensor_table([ds.w[0], ds.w[0]], [ds.lam[0], ds.lam[0]], [ds.theta[0], ds.theta[1]],
+                             shapes=[(64,), (64,)])
+    with pytest.raises(cstep.CondensaError):
+        ctx.cstep_prune(tab, 2, 0.5, 1e-3, ("lambda",))
+    tab = cstep.tensor_table(ds.w, ds.lam, ds.theta, shapes=[(63,), (8, 8)])
+    tab[0].numel = 64
+    with pytest.raises(cstep.CondensaError):
+        ctx.cstep_prune(tab, ds.T, 0.5, 1e-3)
+    out = ds.fetch()
+    assert all(np.isnan(t).all() for t in out["theta"]) and all((m == 7).all() for m in out["mask"])
+
+
+def test_host_entry_point_matches_device_entry_point(ctx):
+    from paper_1911_02497_b200 import cstep
+    ws = W.config(2, scale=0.2)
+    exp = oracle.cstep_prune(ws.w, ws.lam, 0.95, ws.mu, ("fp16", "lambda", "penalty"))
+    w = [np.ascontiguousarray(a) for a in ws.w]
+    lam = [a.copy() for a in ws.lam]
+    theta = [np.empty_like(a) for a in w]
+    mask = [np.empty(a.shape, np.uint8) for a in w]
+    grad = [np.empty_like(a) for a in w]
+    th = [np.empty(a.shape, np.uint16) for a in w]
+    tab = cstep.tensor_table(w, lam, theta, mask, grad, th)
+    ctx.cstep_host(cstep.OP_PRUNE, tab, len(w), 0.95, ws.mu, fuse=("fp16", "lambda", "penalty"))
+    for t in range(len(w)):
+        assert np.array_equal(mask[t], exp.mask[t]) and np.array_equal(th[t], exp.theta_h[t])
+        assert np.array_equal(bits(theta[t]), bits(exp.theta[t]))
+        assert np.array_equal(bits(lam[t]), bits(exp.lam[t]))
+        assert np.array_equal(bits(grad[t]), bits(exp.grad[t]))
+
+
+def test_deterministic_across_runs(ctx):
+    ws = W.config(1, scale=0.5)
+    first, _ = run_gpu(ctx, "prune", ws.w, ws.lam, 0.9, ws.mu, ws.fuse)
+    for _ in range(5):
+        again, _ = run_gpu(ctx, "prune", ws.w, ws.lam, 0.9, ws.mu, ws.fuse)
+        for key in ("theta", "mask", "lam", "theta_h"):
+            for a, b in zip(first[key], again[key]):
+                assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
