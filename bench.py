@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Throughput of the C-step on B200: parameters per second and achieved HBM GB/s.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 5] [--impl ours|reference]
+
+A step is one whole C-step call (ranking, projection, multiplier update) over
+one synthetic weight set. With N > 1 (launched by torch.distributed.run, one
+process per GPU) every rank runs the same workload on its own GPU: the method
+ranks one global list on one GPU, so the ranks are independent replicas and
+`value` is the sum of what they processed over the slowest rank's time.
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+def algorithmic_bytes_per_param(fuse) -> int:
+    """Minimal traffic of one C-step: read w and lambda, write theta, mask, lambda
+    (+ the penalty gradient, + the fp16 copy when they are asked for)."""
+    b = 4 + 4 + 4 + 1 + 4
+    if "penalty" in fuse:
+        b += 4
+    return b
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier copy measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+def workload_name(ws) -> str:
+    return "%s: %s s=%.2f fuse=%s, %d tensors, %d params" % (
+        ws.name, ws.op, ws.sparsity, "+".join(ws.fuse) or "none", len(ws.w), ws.numel)
+
+
+# --------------------------------------------------------------------------- oracle arm
+def time_oracle(ws, steps: int, warmup: int):
+    import oracle
+    for _ in range(warmup):
+        oracle.run_config(ws)
+    t0 = time.perf_counter()
+    out = None
+    for _ in range(steps):
+        out = oracle.run_config(ws)
+    dt = time.perf_counter() - t0
+    return dt / max(steps, 1), out
+
+
+def run_reference(args):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_1911_02497_b200 import workloads as W
+    scale = args.ref_scale
+    ws = W.config(args.config, scale=scale)
+    sec, _ = time_oracle(ws, args.steps, args.warmup)
+    value = ws.numel / sec
+    sample = "config %s with every dimension scaled by %.3g (%d params), one oracle call per step" % (
+        args.config, scale, ws.numel)
+    line = {"impl": "reference", "metric": "cstep_params_per_s", "value": value, "unit": "params/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "config %s (%s)" % (args.config, ws.name), "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "params/s", "cores": 1, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "params/s", "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1911_02497_b200 import cstep, workloads as W
+    from paper_1911_02497_b200.device_set import DeviceSet
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the C-step has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    ws = W.config(args.config)
+    fuse = ws.fuse + (("no_sampling",) if args.no_sampling else ())
+    with_grad = "penalty" in ws.fuse
+    ds = DeviceSet(ws.w, ws.lam, device="cuda:%d" % local, with_grad=with_grad, with_theta_h=False)
+    ctx = cstep.Context(local)
+    N = ws.numel
+    bpp = algorithmic_bytes_per_param(ws.fuse)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        ds.run(ctx, ws.op, ws.sparsity, ws.mu, fuse, ws.block)
+
+    flush = None
+    if N * 8 < 2 * L2_BYTES:       # small workloads fit the L2: evict it between steps
+        flush = torch.empty(2 * L2_BYTES // 4, dtype=torch.float32, device=ds.device)
+
+    def between_steps():
+        ds.reset_lambda()
+        if flush is not None:
+            flush.fill_(1.0)
+
+    for _ in range(max(args.warmup, 3)):
+        between_steps()
+        step()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    launches0 = ctx.launch_count()
+    barrier()
+    with ClockSampler(physical_gpu_index(local)) as clocks:
+        for a, b in ev:
+            between_steps()
+            a.record(stream)
+            step()
+            b.record(stream)
+        barrier()
+    launches = ctx.launch_count() - launches0
+    per_step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(per_step_ms))
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=ds.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * N / (ms_per_step * 1e-3)
+
+    line = None
+    if rank == 0:
+        res = ctx.get_result()
+        # second pass over the same call with an event pair around every kernel
+        ctx.profile_enable(True)
+        for _ in range(args.steps):
+            between_steps()
+            step()
+        torch.cuda.synchronize()
+        prof = ctx.profile_read()
+        ctx.profile_enable(False)
+        peak, peak_src = measured_peak()
+        kernels = {k: {"launches": n, "avg_us": 1e3 * ms / n} for k, (n, ms) in prof.items()}
+        dom = max(prof.items(), key=lambda kv: kv[1][1])
+        dom_name, (dom_n, dom_ms) = dom
+        # the dominant kernel does the whole projection: its algorithmic bytes are the step's
+        achieved = (N * bpp) / (dom_ms / dom_n * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak,
+                    "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                    "peak_source": peak_src, "algorithmic_bytes_per_launch": N * bpp,
+                    "step_achieved": (N * bpp) / (ms_per_step * 1e-3) / 1e9,
+                    "step_frac": (N * bpp) / (ms_per_step * 1e-3) / 1e9 / peak,
+                    "kernels": kernels}
+
+        # end to end: host buffers through the host entry point (pinned memory)
+        hw = [torch.from_numpy(a).pin_memory() for a in ws.w]
+        hl = [torch.from_numpy(a.copy()).pin_memory() for a in ws.lam]
+        ht = [torch.empty_like(a).pin_memory() for a in hw]
+        hm = [torch.empty(a.shape, dtype=torch.uint8).pin_memory() for a in hw]
+        hg = [torch.empty_like(a).pin_memory() for a in hw] if with_grad else None
+        tab = cstep.tensor_table(hw, hl, ht, hm, hg, None, shapes=ws.shapes)
+        opn = {"prune": cstep.OP_PRUNE, "filter": cstep.OP_FILTER, "block": cstep.OP_BLOCK}[ws.op]
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        lam0 = [torch.from_numpy(a.copy()) for a in ws.lam]
+
+        def e2e_step():
+            ctx.cstep_host(opn, tab, len(hw), ws.sparsity, ws.mu, ws.block[0], ws.block[1], fuse)
+
+        e2e_step()
+        e2e_ms = 0.0
+        for _ in range(e2e_steps):
+            for a, b in zip(hl, lam0):
+                a.copy_(b)
+            t0 = time.perf_counter()
+            e2e_step()                       # returns after the stream has finished
+            e2e_ms += (time.perf_counter() - t0) * 1e3
+        e2e_ms /= e2e_steps
+        h2d = 8 * N
+        d2h = (9 + (4 if with_grad else 0)) * N
+        e2e = {"value": N / (e2e_ms * 1e-3), "unit": "params/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps}
+
+        # CPU oracle on the same workload (bounded), and a parity check of this very run
+        cpu = None
+        if not args.skip_cpu:
+            small = N > args.cpu_max_params
+            ows = W.config(args.config, scale=args.cpu_scale) if small else ws
+            sec, out = time_oracle(ows, 1, 0)
+            cpu = {"value": ows.numel / sec, "unit": "params/s", "cores": 1, "kind": "oracle",
+                   "sample": ("whole workload, one call" if not small else
+                              "config scaled by %.3g (%d params), one call" % (args.cpu_scale, ows.numel)),
+                   "seconds": sec}
+            if not small:
+                got_mask = [m.cpu().numpy().reshape(s) for m, s in zip(hm, ws.shapes)]
+                cpu["parity_mask_equal"] = bool(all(np.array_equal(a, b) for a, b in zip(got_mask, out.mask)))
+                cpu["parity_tau_equal"] = bool(res.tau_key == out.result.tau_key and
+                                               res.tau_id == out.result.tau_id)
+        line = {"metric": "cstep_params_per_s", "value": value, "unit": "params/s", "n_gpus": world,
+                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic",
+                "config": {"workload": workload_name(ws),
+                           "l2": ("inputs (%.0f MB) larger than L2" % (N * 8 / 1e6)) if flush is None
+                           else "L2 flushed between steps by writing a 252 MB buffer",
+                           "parallelism": "replicas" if world > 1 else "single GPU",
+                           "lambda": "restored between steps outside the timed windows"},
+                "hbm_gbs": (N * bpp) / (ms_per_step * 1e-3) / 1e9,
+                "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches,
+                "roofline": roofline, "cpu_baseline": cpu,
+                "result": {"passes": res.passes, "sampled": res.sampled,
+                           "n_candidates": res.n_candidates, "n_units": res.n_units}}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="5", help="1..5 or 5t; 5 (the largest) is the headline")
+    ap.add_argument("--no-sampling", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-max-params", type=int, default=200_000_000)
+    ap.add_argument("--cpu-scale", type=float, default=0.25)
+    ap.add_argument("--ref-scale", type=float, default=0.25)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -59,9 +59,12 @@ class DeviceSet:
     # -- state ---------------------------------------------------------------
     def reset_lambda(self):
         """Restore the multipliers (they are updated in place by the calls)."""
-        for t, l in zip(self.lam, self.lam_init):
+        if getattr(self, "_lam_pristine", None) is None:
+            self._lam_pristine = [None if t is None else torch.from_numpy(l.reshape(-1)).to(self.device)
+                                  for t, l in zip(self.lam, self.lam_init)]
+        for t, p in zip(self.lam, self._lam_pristine):
             if t is not None:
-                t.copy_(torch.from_numpy(l.reshape(-1)))
+                t.copy_(p)
 
     def poison_outputs(self):
         """Fill every output with a recognisable pattern so that skipped writes show."""
