@@ -96,8 +96,9 @@ enum {
     CONDENSA_ERR_WORKSPACE = -2,     /* workspace could not be allocated                       */
     CONDENSA_ERR_CUDA = -3,          /* CUDA runtime error, text in condensa_last_error()      */
     CONDENSA_ERR_UNSUPPORTED = -4,   /* dtype or block shape not built                         */
-    CONDENSA_ERR_INTERNAL = -5       /* a device-side consistency check failed (reported by
+    CONDENSA_ERR_INTERNAL = -5,      /* a device-side consistency check failed (reported by
                                         condensa_get_result)                                   */
+    CONDENSA_ERR_TOO_LARGE = -6      /* input larger than a fixed built-in limit               */
 };
 
 enum { CONDENSA_DTYPE_FP16 = 1 };
@@ -192,8 +193,43 @@ CONDENSA_API int condensa_profile_read(condensa_ctx *ctx, condensa_kernel_time *
 /* Number of kernels this context has launched so far. */
 CONDENSA_API int64_t condensa_launch_count(const condensa_ctx *ctx);
 
+/* condensa_cstep_prune() for callers that must not allocate device memory.
+ * (An addition of this library: the paper has no counterpart.)
+ *
+ * Who needs it: programs in which a pool allocator already owns all device
+ * memory, so that a cudaMalloc from a library may fail or eat into the pool's
+ * reserve; and latency-critical loops that cannot accept the device-wide
+ * synchronisation cudaMalloc/cudaFree imply. The context-based calls allocate
+ * a workspace the first time they see a problem size; this call never does:
+ * no cudaMalloc, cudaFree, cudaMallocHost or other allocating routine, on any
+ * call. Its scratch (selection state, histograms, candidate list: 2176 KiB) is
+ * a fixed array inside the library image, so every GPU that loads the library
+ * holds those bytes until the process exits.
+ *
+ * Operation: exactly condensa_cstep_prune() on a list of ONE tensor, with the
+ * same arithmetic, ranking and tie rule and bit-identical theta, mask, lambda,
+ * grad and theta_h. `tensor` is a HOST pointer to one condensa_tensor whose
+ * buffers are DEVICE pointers on the CURRENT device (cudaGetDevice); all
+ * outputs are the caller's. There is no context and no result record.
+ *
+ * Limits and rules:
+ *  - tensor->numel <= CONDENSA_NOALLOC_MAX_NUMEL, else CONDENSA_ERR_TOO_LARGE
+ *    and nothing is launched or written.
+ *  - The first call on each device looks up the scratch's device address (once
+ *    per device, with that device current). Make that first call outside any
+ *    stream capture.
+ *  - All calls on a device share the one scratch array, which still holds the
+ *    previous call's contents; each call clears the parts that must start at
+ *    zero on `stream` before using them. Two calls that may overlap on the GPU
+ *    (different streams without ordering, or several host threads) race on it
+ *    and give wrong results: keep calls on one device ordered.
+ *  - The error text of a failed call is condensa_last_error(NULL). */
+#define CONDENSA_NOALLOC_MAX_NUMEL 1048576
+CONDENSA_API int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
+                                              float mu, unsigned fuse, void *stream);
+
 /* Text of the last error on this context (never NULL). ctx may be NULL to get
- * the text of a failed condensa_create(). */
+ * the text of a failed condensa_create() or condensa_cstep_prune_noalloc(). */
 CONDENSA_API const char *condensa_last_error(const condensa_ctx *ctx);
 
 #ifdef __cplusplus

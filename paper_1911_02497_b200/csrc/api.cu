@@ -720,6 +720,125 @@ int condensa_profile_read(condensa_ctx *ctx, condensa_kernel_time *out, int max_
 
 int64_t condensa_launch_count(const condensa_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+// ---------------------------------------------------------------- no-allocation variant
+// Scratch of condensa_cstep_prune_noalloc(): selection state, histograms, the
+// one-tensor descriptor and a candidate list for up to
+// CONDENSA_NOALLOC_MAX_NUMEL elements. It is part of the loaded module, so
+// every GPU that loads this library holds these bytes until the process exits.
+constexpr size_t NOALLOC_SCRATCH_BYTES = 2176u * 1024u;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+unsigned char *g_noalloc_ptr[NOALLOC_MAX_DEVICES];   // device address of the scratch, per device
+int g_noalloc_occ[NOALLOC_MAX_DEVICES];
+int g_noalloc_sms[NOALLOC_MAX_DEVICES];
+
+// Writes the descriptor of the single tensor and its two work-item prefix
+// arrays into the scratch (the regular path copies them from pinned memory).
+__global__ void k_noalloc_setup(TensorDesc d, long long items, TensorDesc *td, long long *prefix)
+{
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *td = d;
+        prefix[0] = 0; prefix[1] = items;     // scan decomposition
+        prefix[2] = 0; prefix[3] = items;     // projection decomposition
+    }
+}
+
+int noalloc_fail(int code, const char *text)
+{
+    g_create_error = text;
+    return code;
+}
+
+}  // namespace
+
+int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity, float mu,
+                                 unsigned fuse, void *stream_)
+{
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!tensor) return noalloc_fail(CONDENSA_ERR_INVALID_ARG, "tensor is NULL");
+    if (tensor->numel > CONDENSA_NOALLOC_MAX_NUMEL)
+        return noalloc_fail(CONDENSA_ERR_TOO_LARGE,
+                            "condensa_cstep_prune_noalloc: numel exceeds CONDENSA_NOALLOC_MAX_NUMEL "
+                            "(the built-in scratch is fixed); use condensa_cstep_prune with a context");
+    {
+        condensa_ctx checker;      // host-only object: collects the text of an argument error
+        const int rc = validate(&checker, OP_PRUNE, tensor, 1, sparsity, mu, fuse);
+        if (rc) return noalloc_fail(rc, checker.err.c_str());
+    }
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return noalloc_fail(CONDENSA_ERR_UNSUPPORTED, "device index too large");
+    if (!g_noalloc_ptr[dev]) {
+        // Once per device, with that device current: the array's name is only a
+        // host-side handle here; kernels need the address the runtime maps it to.
+        unsigned char *p = nullptr;
+        e = cudaGetSymbolAddress((void **)&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+        int sms = 0, coop = 0;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        if (!coop || sms <= 0) return noalloc_fail(CONDENSA_ERR_UNSUPPORTED, "device lacks cooperative launch");
+        g_noalloc_occ[dev] = occupancy(k_select<SRC_ELEM>);
+        g_noalloc_sms[dev] = sms;
+        g_noalloc_ptr[dev] = p;
+    }
+    Plan pl;
+    build_plan(OP_PRUNE, tensor, 1, pl);
+    const Layout L = make_layout(1, pl, true, false);
+    if (L.total > NOALLOC_SCRATCH_BYTES) return noalloc_fail(CONDENSA_ERR_TOO_LARGE, "scratch layout exceeds the built-in array");
+    unsigned char *ws = g_noalloc_ptr[dev];
+
+    Params P;
+    memset(&P, 0, sizeof(P));
+    P.td = (const TensorDesc *)(ws + L.desc);
+    long long *prefix = (long long *)(ws + L.desc + sizeof(TensorDesc));
+    P.T = 1;
+    P.mu = mu;
+    P.fuse = fuse & 7u;
+    P.ctl = (Ctl *)(ws + L.ctl);
+    P.hist = (u64 *)(ws + L.hist);
+    P.fin_key = (u64 *)(ws + L.fin_key);
+    P.fin_id = (u64 *)(ws + L.fin_id);
+    P.list_key = (u64 *)(ws + L.list_key);
+    P.list_id = (u64 *)(ws + L.list_id);
+    P.cap = pl.cap;
+    P.S = pl.S;
+    P.bits_key = 31;
+    P.item_prefix = prefix;
+    P.n_items = pl.n_items_a;
+
+    const long long Z = (long long)std::min<double>((double)pl.S, std::max(0.0, std::floor(sparsity * (double)pl.S + 0.5)));
+    Sel init = initial_state(pl.S, pl.S - Z, 31);
+    int do_list0 = (u64)pl.S <= pl.cap ? 1 : 0;
+    const int sms = g_noalloc_sms[dev];
+    auto grid_for = [&](long long items, int per_sm) {
+        long long g = (long long)sms * per_sm;
+        if (g > items) g = items;
+        return (int)(g < 1 ? 1 : g);
+    };
+
+    k_noalloc_setup<<<1, 32, 0, stream>>>(pl.td[0], pl.n_items_a, (TensorDesc *)(ws + L.desc), prefix);
+    k_init<<<8, THREADS, 0, stream>>>(P, init);      // clears the histograms and counters the last call left
+    if (!init.done)
+        k_scan<SRC_ELEM><<<grid_for(pl.n_items_a, 4), THREADS, 0, stream>>>(P, do_list0);
+    if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    {
+        dim3 grid((unsigned)(sms * std::min(g_noalloc_occ[dev], 2))), block(THREADS);
+        void *args[] = {(void *)&P, (void *)&do_list0};
+        e = cudaLaunchCooperativeKernel((const void *)k_select<SRC_ELEM>, grid, block, args, 0, stream);
+        if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    }
+    if (pl.n_items_b > 0) {
+        k_apply_linear<M_PRUNE><<<grid_for(pl.n_items_b, 4), THREADS, 0, stream>>>(P);
+        if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    }
+    return CONDENSA_OK;
+}
+
 const char *condensa_last_error(const condensa_ctx *ctx)
 {
     return ctx ? ctx->err.c_str() : g_create_error.c_str();

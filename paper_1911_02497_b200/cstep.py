@@ -18,11 +18,14 @@ FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, NO_SAMPLING = 1, 2, 4, 64
 OP_PRUNE, OP_FILTER, OP_BLOCK, OP_QUANTIZE, OP_LAGRANGE = 0, 1, 2, 3, 4
 DTYPE_FP16 = 1
 OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_UNSUPPORTED, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
+ERR_TOO_LARGE = -6
+NOALLOC_MAX_NUMEL = 1048576
 
 EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "condensa_cstep_filter",
            "condensa_cstep_block", "condensa_cstep_quantize", "condensa_cstep_lagrange_update",
            "condensa_cstep_host", "condensa_get_result", "condensa_launch_count",
-           "condensa_last_error", "condensa_profile_enable", "condensa_profile_read"]
+           "condensa_last_error", "condensa_profile_enable", "condensa_profile_read",
+           "condensa_cstep_prune_noalloc"]
 
 
 class CondensaError(RuntimeError):
@@ -78,6 +81,7 @@ def load():
     L.condensa_get_result.argtypes = [vp, C.POINTER(Result)]
     L.condensa_profile_enable.argtypes = [vp, i32]
     L.condensa_profile_read.argtypes = [vp, C.POINTER(KernelTime), i32, C.POINTER(i32)]
+    L.condensa_cstep_prune_noalloc.argtypes = [vp, f64, f32, u32, vp]
     L.condensa_launch_count.argtypes = [vp]
     L.condensa_launch_count.restype = C.c_int64
     L.condensa_last_error.argtypes = [vp]
@@ -142,6 +146,19 @@ def _stream_handle(stream) -> Optional[int]:
     if isinstance(stream, int):
         return stream
     return int(stream.cuda_stream)          # torch.cuda.Stream
+
+
+def cstep_prune_noalloc(tab, sparsity, mu, fuse=(), stream=None):
+    """``condensa_cstep_prune_noalloc``: magnitude pruning of ONE tensor (entry 0 of
+    ``tab``) on the current CUDA device without any device allocation by the
+    library - for callers whose memory pool owns the whole device or who cannot
+    take cudaMalloc's synchronisation. At most ``NOALLOC_MAX_NUMEL`` elements;
+    calls on one device must not overlap (they share one built-in scratch)."""
+    L = load()
+    rc = L.condensa_cstep_prune_noalloc(tab, float(sparsity), float(mu), fuse_bits(fuse),
+                                        _stream_handle(stream))
+    if rc != OK:
+        raise CondensaError(rc, (L.condensa_last_error(None) or b"").decode())
 
 
 class Context:
