@@ -168,7 +168,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    ws = W.config(args.config)
+    ws = W.config(args.config, scale=args.scale)
     fuse = ws.fuse + (("no_sampling",) if args.no_sampling else ())
     with_grad = "penalty" in ws.fuse
     ds = DeviceSet(ws.w, ws.lam, device="cuda:%d" % local, with_grad=with_grad, with_theta_h=False)
@@ -276,7 +276,7 @@ def run_ours(args):
         cpu = None
         if not args.skip_cpu:
             small = N > args.cpu_max_params
-            ows = W.config(args.config, scale=args.cpu_scale) if small else ws
+            ows = W.config(args.config, scale=args.cpu_scale * args.scale) if small else ws
             sec, out = time_oracle(ows, 1, 0)
             cpu = {"value": ows.numel / sec, "unit": "params/s", "cores": 1, "kind": "oracle",
                    "sample": ("whole workload, one call" if not small else
@@ -322,6 +322,8 @@ def main():
     ap.add_argument("--cpu-max-params", type=int, default=200_000_000)
     ap.add_argument("--cpu-scale", type=float, default=0.25)
     ap.add_argument("--ref-scale", type=float, default=0.25)
+    ap.add_argument("--scale", type=float, default=1.0,
+                    help="shrink every dimension (profiling captures only; not a bench value)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -120,6 +120,8 @@ typedef struct {
     float tau_norm;        /* _filter/_block: (float)sqrt of the weakest kept squared norm    */
     int32_t sampled;       /* 1 when a sample bracket was used and held                       */
     int64_t n_candidates;  /* units that had to be listed for the exact selection             */
+    int64_t n_repaired;    /* single-pass path: listed units whose provisional decision was
+                              wrong and were rewritten                                        */
 } condensa_result;
 
 /* Create a context on CUDA device `device`. workspace_bytes = 0 sizes the

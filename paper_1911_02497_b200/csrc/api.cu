@@ -14,6 +14,8 @@
 #include "elementwise.cuh"
 #include "select.cuh"
 #include "structured.cuh"
+#include "fused.cuh"
+#include "sample.cuh"
 
 using namespace cs;
 
@@ -92,7 +94,7 @@ struct Interval {
 
 // Layout of one call's workspace.
 struct Layout {
-    size_t ctl, hist, fin_key, fin_id, desc, list_key, list_id, arr_key, partial, total;
+    size_t ctl, hist, fin_key, fin_id, desc, list_key, list_id, arr_key, partial, sample, journal, total;
     size_t desc_bytes;
 };
 
@@ -230,7 +232,10 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl)
     pl.cap = cap;
 }
 
-Layout make_layout(int T, const Plan &pl, bool ranking, bool filter)
+constexpr int N_SAMPLE = SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD;
+
+// journal_floats: floats of original lambda kept per listed unit (0: no single-pass path)
+Layout make_layout(int T, const Plan &pl, bool ranking, bool filter, int journal_floats = 0)
 {
     Layout L;
     size_t off = 0;
@@ -245,6 +250,8 @@ Layout make_layout(int T, const Plan &pl, bool ranking, bool filter)
     L.list_id = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
     L.arr_key = off; if (filter) off = align_up(off + sizeof(u64) * (size_t)std::max<long long>(pl.S, 1), 256);
     L.partial = off; if (filter) off = align_up(off + sizeof(double) * (size_t)std::max<long long>(pl.n_seg, 1), 256);
+    L.sample = off; if (journal_floats) off = align_up(off + sizeof(u64) * N_SAMPLE, 256);
+    L.journal = off; if (journal_floats) off = align_up(off + sizeof(float) * (size_t)journal_floats * pl.cap, 256);
     L.total = off;
     return L;
 }
@@ -266,6 +273,9 @@ int ensure_workspace(condensa_ctx *ctx, size_t bytes, cudaStream_t stream)
         return fail(ctx, CONDENSA_ERR_WORKSPACE, "cannot allocate %zu bytes of workspace: %s", want, cudaGetErrorString(e));
     }
     ctx->ws_bytes = want;
+    // counters that kernels expect to find at zero on first use
+    if ((e = cudaMemset(ctx->ws, 0, std::min<size_t>(want, 1 << 16))) != cudaSuccess)
+        return fail(ctx, CONDENSA_ERR_CUDA, "cudaMemset: %s", cudaGetErrorString(e));
     return CONDENSA_OK;
 }
 
@@ -405,7 +415,12 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     Plan pl;
     build_plan(op, ts, T, pl);
     const bool ranking = op <= OP_BLOCK;
-    const Layout L = make_layout(T, pl, ranking, op == OP_FILTER);
+    // single-pass path: unstructured and block pruning of lists too large to list whole
+    const bool sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) &&
+                          (u64)pl.S > pl.cap && pl.S >= 8ll * N_SAMPLE;
+    if (sampling && op == OP_BLOCK && pl.cap > (1ull << 20)) pl.cap = 1ull << 20;   // bounds the journal
+    const int journal_floats = sampling ? (op == OP_BLOCK ? 16 : 1) : 0;
+    const Layout L = make_layout(T, pl, ranking, op == OP_FILTER, journal_floats);
     rc = ensure_workspace(ctx, L.total, stream);
     if (rc) return rc;
     char *ws = ctx->ws;
@@ -433,6 +448,13 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     P.partial = (double *)(ws + L.partial);
     P.S = pl.S;
     P.bits_key = (op == OP_PRUNE) ? 31 : 63;
+    P.sample_key = (u64 *)(ws + L.sample);
+    P.n_sample = N_SAMPLE;
+    P.jr_lam = (float *)(ws + L.journal);
+    P.onepass_cap = pl.cap;
+    P.seed = 0x9E3779B97F4A7C15ull;
+    bool need_h = (fuse & CONDENSA_FUSE_FP16) != 0;
+    for (int t = 0; t < T; ++t) need_h = need_h || ts[t].theta_h != nullptr;
     ctx->ctl = P.ctl;
     ctx->last_stream = stream;
 
@@ -457,10 +479,32 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pa_, stream);
         }
-        int pi_ = prof_begin(ctx, "k_init", stream);
-        k_init<<<8, THREADS, 0, stream>>>(P, init);
-        LAUNCH_CHECK(ctx);
-        prof_end(ctx, pi_, stream);
+        Params Pf = P;                      // single-pass kernel runs on the projection decomposition
+        Pf.item_prefix = pb;
+        Pf.n_items = pl.n_items_b;
+        if (sampling && !init.done) {
+            int pi_ = prof_begin(ctx, "k_sample", stream);
+            if (op == OP_PRUNE) k_sample<SRC_ELEM><<<N_SAMPLE / SAMPLE_THREADS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            else k_sample<SRC_BLOCK><<<N_SAMPLE / SAMPLE_THREADS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, pi_, stream);
+            pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : "k_fused_block", stream);
+            const int gridf = stream_grid(ctx, pl.n_items_b, 4);
+            if (op == OP_PRUNE) {
+                if (need_h) k_fused_elem<true><<<gridf, THREADS, 0, stream>>>(Pf);
+                else k_fused_elem<false><<<gridf, THREADS, 0, stream>>>(Pf);
+            } else {
+                if (need_h) k_fused_block<true><<<gridf, THREADS, 0, stream>>>(Pf);
+                else k_fused_block<false><<<gridf, THREADS, 0, stream>>>(Pf);
+            }
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, pi_, stream);
+        } else {
+            int pi_ = prof_begin(ctx, "k_init", stream);
+            k_init<<<8, THREADS, 0, stream>>>(P, init);
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, pi_, stream);
+        }
         if (!init.done) {
             const int ps_ = prof_begin(ctx, op == OP_PRUNE ? "k_scan_elem" : op == OP_BLOCK ? "k_scan_block" : "k_scan_array", stream);
             if (op == OP_PRUNE) {

@@ -55,6 +55,7 @@ struct Result {
     float tau_norm;
     int sampled;
     long long n_candidates;
+    long long n_repaired;
 };
 
 // Selection state: the bracket is the set of units whose (key, id) lies in
@@ -73,7 +74,10 @@ struct Sel {
     int above_known;          // n_above is exact (else taken from the scan's own count)
     int done, error, passes;
     int key_fixed;            // n_gt / n_tie are set
-    int sampled;
+    int sampled;              // the bracket came from a sample (and held so far)
+    int onepass;              // the first pass also writes provisional outputs + journal
+    int pad1;
+    u64 guess;                // provisional rule of the one-pass path: keep iff key >= guess
 };
 
 struct Ctl {
@@ -82,7 +86,8 @@ struct Ctl {
     u64 scan_above[3];        // per histogram slot: units above the bracket seen by that scan
     u64 list_count[2];
     u32 fin_count;
-    u32 pad0;
+    u32 sample_done;          // CTAs of the sample kernel that have finished
+    u64 n_repaired;           // one-pass: provisional decisions that had to be rewritten
     Result res;
 };
 
@@ -103,6 +108,12 @@ struct Params {
     double *partial;                // filter: per segment partial sums
     long long S;                    // ranked units
     int bits_key;                   // width of the key in bits (31 or 63)
+    u64 *sample_key;                // [n_sample] keys of the sampled units
+    int n_sample;
+    float *jr_lam;                  // one-pass journal: original lambda of listed units
+                                    // (1 float per element, 16 per block)
+    u64 onepass_cap;                // candidates the one-pass path accepts (<= cap)
+    u64 seed;                       // sample positions
 };
 
 // ---------------------------------------------------------------- arithmetic
@@ -152,6 +163,52 @@ __device__ __forceinline__ Out finish(float w, float lam, float u, bool keep, fl
     o.lam = lu;
     o.grad = __fsub_rn(p, lu);
     return o;
+}
+
+// Lean form for the hot kernels: H = the binary16 bits are needed (fp16 fuse or
+// a theta_h output); `fp16`, `upd` (update lambda) are warp-uniform flags.
+template <bool H>
+__device__ __forceinline__ Out finish_lean(float w, float lam, float u, bool keep, float mu,
+                                           bool fp16, bool upd)
+{
+    Out o;
+    float th = keep ? u : 0.0f;
+    o.th = 0;
+    if (H) {
+        const unsigned short hb = keep ? f32_to_f16_bits(u) : (unsigned short)0;
+        o.th = hb;
+        if (fp16) th = keep ? f16_bits_to_f32(hb) : 0.0f;
+    }
+    const float p = __fmul_rn(mu, __fsub_rn(w, th));
+    const float lu = upd ? __fsub_rn(lam, p) : lam;
+    o.theta = th;
+    o.m = keep ? 1 : 0;
+    o.lam = lu;
+    o.grad = __fsub_rn(p, lu);
+    return o;
+}
+
+// u for four elements; skips the divisions when every lambda is +0 (u == w then).
+__device__ __forceinline__ void form_u4(const float *w, const float *l, float mu, bool has_lam, float *u)
+{
+    const bool nz = has_lam && ((__float_as_uint(l[0]) | __float_as_uint(l[1]) |
+                                 __float_as_uint(l[2]) | __float_as_uint(l[3])) != 0u);
+    if (__any_sync(0xffffffffu, nz)) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) u[j] = has_lam ? __fsub_rn(w[j], __fdiv_rn(l[j], mu)) : w[j];
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) u[j] = w[j];
+    }
+}
+
+// splitmix64 output function: position hash of the sampler.
+__device__ __forceinline__ u64 mix64(u64 z)
+{
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+    z ^= z >> 27; z *= 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z;
 }
 
 // Same with theta supplied (multiplier update / penalty gradient only).

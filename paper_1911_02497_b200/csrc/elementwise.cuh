@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(THREADS) k_apply_linear(Params P)
 {
     u64 tau_key = 0, tau_id = 0;
     if (MODE == M_PRUNE || MODE == M_FILTER) {
+        if (P.ctl->sel.onepass) return;      // the single-pass kernel has written everything
         tau_key = P.ctl->tau_key;
         tau_id = P.ctl->tau_id;
     }

@@ -345,7 +345,10 @@ __device__ __forceinline__ void block_pick(const Params &P, ScanShared &sh, bool
         if (s.above_known && src_scan && above_scan != s.n_above) s.error = 1;
         const bool sk = s.lo_key == s.hi_key;
         if (!valid) {
-            if (s.above_known) {
+            if (s.onepass) {
+                s.error = 10;       // the sampled bracket missed: outputs already written are wrong
+                s.done = 1;
+            } else if (s.above_known) {
                 s.error = 2;        // a histogram-derived bracket must hold the rank
                 s.done = 1;
             } else if (s.k <= n_above) {
@@ -484,11 +487,16 @@ __device__ __forceinline__ void final_rank(const Params &P, ScanShared &sh, u32 
     __syncthreads();
 }
 
+// Defined with the single-pass kernels: rewrites one listed unit.
+template <int SRC>
+__device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep);
+
 // First pass of a ranking call: a plain (non-cooperative) scan at full grid.
 template <int SRC>
 __global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
 {
     __shared__ ScanShared sh;
+    if (P.ctl->sel.onepass) return;          // the single-pass kernel has done this work
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
     __syncthreads();
     scan_source<SRC>(P, sh, do_list != 0, sh.sel.slot);
@@ -506,13 +514,17 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     __syncthreads();
     bool src_scan = true;
     if (!sh.sel.done) {
-        if (first_listed && threadIdx.x == 0) sh.sel.list_valid = 1;
+        if ((first_listed || sh.sel.onepass) && threadIdx.x == 0) sh.sel.list_valid = 1;
         __syncthreads();
         for (int it = 0; it < MAX_SELECT_ITERS + 2; ++it) {
             // a listing scan that overflowed the list does not count
             if (threadIdx.x == 0 && sh.sel.list_valid &&
-                __ldcg(&P.ctl->list_count[sh.sel.list_sel]) > P.cap) sh.sel.list_valid = 0;
+                __ldcg(&P.ctl->list_count[sh.sel.list_sel]) > P.cap) {
+                sh.sel.list_valid = 0;
+                if (sh.sel.onepass) { sh.sel.error = 11; sh.sel.done = 1; }
+            }
             __syncthreads();
+            if (sh.sel.done) break;
             block_pick(P, sh, src_scan, max_key);
             // clear the histogram slot that the scan after the next one will use
             if (blockIdx.x == 0) {
@@ -561,6 +573,24 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
             grid.sync();
         }
     }
+    if (SRC != SRC_ARRAY) {
+        if (sh.sel.onepass && !sh.sel.error && sh.sel.k > 0) {
+            // single-pass path: rewrite the listed units whose provisional decision was wrong
+            const u64 n_list = __ldcg(&P.ctl->list_count[0]);
+            const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
+            const u64 stride = (u64)gridDim.x * THREADS;
+            u64 fixed = 0;
+            for (u64 i = (u64)blockIdx.x * THREADS + threadIdx.x; i < n_list; i += stride) {
+                const u64 key = __ldcg(&P.list_key[i]), id = __ldcg(&P.list_id[i]);
+                const bool fin = keep_by_cutoff(key, id, tk, ti);
+                if (fin != (key >= guess)) {
+                    repair_unit<SRC>(P, i, id, fin);
+                    ++fixed;
+                }
+            }
+            if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
+        }
+    }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         Ctl *c = P.ctl;
         const Sel &s = sh.sel;
@@ -589,6 +619,7 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
             r.n_tie_kept = (long long)(s.k - s.n_gt);
             if (P.bits_key >= 63) r.tau_norm = (float)sqrt(__longlong_as_double((long long)s.lo_key));
         }
+        r.n_repaired = (long long)__ldcg(&c->n_repaired);
         c->sel = s;
         c->res = r;
     }
@@ -608,6 +639,7 @@ __global__ void __launch_bounds__(THREADS) k_init(Params P, Sel init)
         c->scan_above[0] = c->scan_above[1] = c->scan_above[2] = 0;
         c->list_count[0] = c->list_count[1] = 0;
         c->fin_count = 0;
+        c->n_repaired = 0;
     }
 }
 

@@ -60,6 +60,7 @@ __device__ __forceinline__ void store_block(const TensorDesc &d, const BlockData
 // ranked (2-D) tensors, linear items for tensors that pass through.
 __global__ void __launch_bounds__(THREADS) k_apply_block(Params P)
 {
+    if (P.ctl->sel.onepass) return;          // the single-pass kernel has written everything
     const u64 tau_key = P.ctl->tau_key, tau_id = P.ctl->tau_id;
     for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
         const int t = find_tensor(P.item_prefix, P.T, item);

@@ -47,7 +47,7 @@ class Result(C.Structure):
                 ("n_zero", C.c_int64), ("n_keep", C.c_int64), ("tau_key", C.c_uint64),
                 ("tau_id", C.c_int64), ("n_gt", C.c_int64), ("n_tie", C.c_int64),
                 ("n_tie_kept", C.c_int64), ("tau_norm", C.c_float), ("sampled", C.c_int32),
-                ("n_candidates", C.c_int64)]
+                ("n_candidates", C.c_int64), ("n_repaired", C.c_int64)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

@@ -60,6 +60,7 @@ def run_gpu(ctx, op, w, lam, s, mu, fuse, block=(4, 4), elem_offset=0, skew=0, t
 
 
 def run_oracle(op, w, lam, s, mu, fuse, block=(4, 4), theta=None):
+    fuse = tuple(f for f in fuse if f != "no_sampling")     # a path switch of the CUDA side only
     if op == "prune":
         return oracle.cstep_prune(w, lam, s, mu, fuse)
     if op == "filter":
@@ -204,6 +205,24 @@ def test_prune_configurations(ctx, cfg, scale):
     got, res, _ = check(ctx, "prune", ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
     zeros = sum(int((m == 0).sum()) for m in got["mask"])
     assert zeros == res.n_zero == math.floor(ws.sparsity * ws.numel + 0.5)
+
+
+@pytest.mark.parametrize("cfg,scale", [(1, 1.0), (2, 1.0), (4, 0.12), ("5", 0.1)])
+def test_two_pass_path_without_sampling(ctx, cfg, scale):
+    """The same configurations with the sample bracket switched off: rank first
+    (full histogram passes), then project."""
+    ws = W.config(cfg, scale=scale)
+    got, res, _ = check(ctx, ws.op, ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse + ("no_sampling",))
+    assert res.sampled == 0 and res.n_repaired == 0
+
+
+def test_single_pass_path_is_taken_and_repairs(ctx):
+    ws = W.config(1)
+    got, res, _ = check(ctx, "prune", ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
+    assert res.sampled == 1 and 0 < res.n_candidates < ws.numel // 8
+    ws = W.config("5", scale=0.2)
+    got, res, _ = check(ctx, "block", ws.w, ws.lam, ws.sparsity, ws.mu, ("fp16", "lambda", "penalty"))
+    assert res.sampled == 1 and 0 < res.n_candidates < res.n_units // 8
 
 
 # ---------------------------------------------------------------- filters
