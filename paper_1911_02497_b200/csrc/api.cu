@@ -94,7 +94,7 @@ struct Interval {
 
 // Layout of one call's workspace.
 struct Layout {
-    size_t ctl, hist, fin_key, fin_id, desc, list_key, list_id, arr_key, partial, sample, journal, total;
+    size_t ctl, hist, fin_key, fin_id, fin_idx, desc, list_key, list_id, arr_key, partial, sample, journal, total;
     size_t desc_bytes;
 };
 
@@ -104,6 +104,7 @@ struct Plan {
     long long n_items_a = 0, n_items_b = 0;
     long long S = 0, N = 0, n_seg = 0;
     u64 cap = 0;
+    std::vector<long long> edge_items;           // projection items outside the aligned fast path
 };
 
 int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s, float mu,
@@ -243,8 +244,10 @@ Layout make_layout(int T, const Plan &pl, bool ranking, bool filter, int journal
     L.hist = off; off = align_up(off + sizeof(u64) * 3 * NBINS, 256);
     L.fin_key = off; off = align_up(off + sizeof(u64) * FIN, 256);
     L.fin_id = off; off = align_up(off + sizeof(u64) * FIN, 256);
+    L.fin_idx = off; off = align_up(off + sizeof(u64) * FIN, 256);
     L.desc = off;
-    L.desc_bytes = sizeof(TensorDesc) * (size_t)T + 2 * sizeof(long long) * (size_t)(T + 1);
+    L.desc_bytes = sizeof(TensorDesc) * (size_t)T + 2 * sizeof(long long) * (size_t)(T + 1) +
+                   sizeof(long long) * pl.edge_items.size();
     off = align_up(off + L.desc_bytes, 256);
     L.list_key = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
     L.list_id = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
@@ -287,6 +290,8 @@ int upload_desc(condensa_ctx *ctx, const Plan &pl, int T, char *dst, size_t byte
     char *p = img.data();
     memcpy(p, pl.td.data(), sizeof(TensorDesc) * (size_t)T); p += sizeof(TensorDesc) * (size_t)T;
     memcpy(p, pl.prefix_a.data(), sizeof(long long) * (size_t)(T + 1)); p += sizeof(long long) * (size_t)(T + 1);
+    if (!pl.edge_items.empty()) memcpy(p, pl.edge_items.data(), sizeof(long long) * pl.edge_items.size());
+    p += sizeof(long long) * pl.edge_items.size();
     memcpy(p, pl.prefix_b.data(), sizeof(long long) * (size_t)(T + 1));
     if (ctx->last_upload_dst == dst && ctx->last_upload == img) return CONDENSA_OK;
     CU_TRY(ctx, cudaEventSynchronize(ctx->stage_ev));    // the previous upload has left the staging area
@@ -420,6 +425,13 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
                           (u64)pl.S > pl.cap && pl.S >= 8ll * N_SAMPLE;
     if (sampling && op == OP_BLOCK && pl.cap > (1ull << 20)) pl.cap = 1ull << 20;   // bounds the journal
     const int journal_floats = sampling ? (op == OP_BLOCK ? 16 : 1) : 0;
+    if (sampling) {
+        for (int t = 0; t < T; ++t)
+            for (long long j = 0; j < pl.prefix_b[t + 1] - pl.prefix_b[t]; ++j) {
+                const bool fast = op == OP_BLOCK ? block_item_is_fast(pl.td[t], j) : elem_item_is_fast(pl.td[t], j);
+                if (!fast) pl.edge_items.push_back(pl.prefix_b[t] + j);
+            }
+    }
     const Layout L = make_layout(T, pl, ranking, op == OP_FILTER, journal_floats);
     rc = ensure_workspace(ctx, L.total, stream);
     if (rc) return rc;
@@ -431,7 +443,8 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     memset(&P, 0, sizeof(P));
     P.td = (const TensorDesc *)(ws + L.desc);
     const long long *pa = (const long long *)(ws + L.desc + sizeof(TensorDesc) * (size_t)T);
-    const long long *pb = pa + (T + 1);
+    const long long *pe = pa + (T + 1);                      // edge item list
+    const long long *pb = pe + pl.edge_items.size();         // projection prefix, right behind it
     P.T = T;
     P.mu = mu;
     P.fuse = fuse & 7u;
@@ -441,6 +454,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     P.hist = (u64 *)(ws + L.hist);
     P.fin_key = (u64 *)(ws + L.fin_key);
     P.fin_id = (u64 *)(ws + L.fin_id);
+    P.fin_idx = (u64 *)(ws + L.fin_idx);
+    P.edge_items = pe;
+    P.n_edge_items = (long long)pl.edge_items.size();
     P.list_key = (u64 *)(ws + L.list_key);
     P.list_id = (u64 *)(ws + L.list_id);
     P.cap = pl.cap;
@@ -490,13 +506,17 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             prof_end(ctx, pi_, stream);
             pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : "k_fused_block", stream);
             const int gridf = stream_grid(ctx, pl.n_items_b, 4);
-            if (op == OP_PRUNE) {
-                if (need_h) k_fused_elem<true><<<gridf, THREADS, 0, stream>>>(Pf);
-                else k_fused_elem<false><<<gridf, THREADS, 0, stream>>>(Pf);
-            } else {
-                if (need_h) k_fused_block<true><<<gridf, THREADS, 0, stream>>>(Pf);
-                else k_fused_block<false><<<gridf, THREADS, 0, stream>>>(Pf);
-            }
+            const bool need_g = (fuse & CONDENSA_FUSE_PENALTY) != 0;
+#define CS_LAUNCH_FUSED(KERNEL, GRID)                                                          \
+    do {                                                                                       \
+        if (need_h && need_g) KERNEL<true, true><<<GRID, THREADS, 0, stream>>>(Pf);            \
+        else if (need_h) KERNEL<true, false><<<GRID, THREADS, 0, stream>>>(Pf);                \
+        else if (need_g) KERNEL<false, true><<<GRID, THREADS, 0, stream>>>(Pf);                \
+        else KERNEL<false, false><<<GRID, THREADS, 0, stream>>>(Pf);                           \
+    } while (0)
+            if (op == OP_PRUNE) CS_LAUNCH_FUSED(k_fused_elem, gridf);
+            else CS_LAUNCH_FUSED(k_fused_block, gridf);
+#undef CS_LAUNCH_FUSED
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
         } else {
@@ -723,6 +743,11 @@ int condensa_get_result(condensa_ctx *ctx, condensa_result *out)
     CU_TRY(ctx, cudaSetDevice(ctx->device));
     CU_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
     CU_TRY(ctx, cudaMemcpy(out, &ctx->ctl->res, sizeof(*out), cudaMemcpyDeviceToHost));
+    {
+        u64 rep = 0;
+        CU_TRY(ctx, cudaMemcpy(&rep, &ctx->ctl->n_repaired, sizeof(rep), cudaMemcpyDeviceToHost));
+        out->n_repaired = (int64_t)rep;
+    }
     if (out->status != 0) {
         int code = 0;
         cudaMemcpy(&code, &ctx->ctl->sel.error, sizeof(int), cudaMemcpyDeviceToHost);
@@ -847,6 +872,7 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
     P.hist = (u64 *)(ws + L.hist);
     P.fin_key = (u64 *)(ws + L.fin_key);
     P.fin_id = (u64 *)(ws + L.fin_id);
+    P.fin_idx = (u64 *)(ws + L.fin_idx);
     P.list_key = (u64 *)(ws + L.list_key);
     P.list_id = (u64 *)(ws + L.list_id);
     P.cap = pl.cap;

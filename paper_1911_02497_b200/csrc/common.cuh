@@ -114,7 +114,24 @@ struct Params {
                                     // (1 float per element, 16 per block)
     u64 onepass_cap;                // candidates the one-pass path accepts (<= cap)
     u64 seed;                       // sample positions
+    const long long *edge_items;    // projection work items the aligned fast kernel skips
+    long long n_edge_items;
+    u64 *fin_idx;                   // [FIN] list position of each entry of the final buffer
 };
+
+// Which projection work items the fast single-pass kernels take (host and device
+// must agree: the host lists the others for the edge kernel).
+__host__ __device__ inline bool elem_item_is_fast(const TensorDesc &d, long long local)
+{
+    const long long e_first = 4 * (local * GROUPS_PER_ITEM) - d.pad;
+    return d.vec_ok && e_first >= 0 && e_first + 4 * GROUPS_PER_ITEM <= d.numel;
+}
+
+__host__ __device__ inline bool block_item_is_fast(const TensorDesc &d, long long local)
+{
+    const long long full_blocks = (d.d0 >> 2) * d.nbc;         // blocks in complete block rows
+    return d.ranked && d.blk_vec_ok && d.numel < 0xFFFFFFFFll && (local + 1) * BLOCKS_PER_ITEM <= full_blocks;
+}
 
 // ---------------------------------------------------------------- arithmetic
 // u = w - lambda / mu as two IEEE fp32 operations.

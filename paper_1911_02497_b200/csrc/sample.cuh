@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         P.hist[i] = 0;
     const int j = blockIdx.x * SAMPLE_THREADS + threadIdx.x;
     if (j < P.n_sample) {
-        const u64 unit = mix64(P.seed + (u64)j) % (u64)P.S;
+        const u64 unit = __umul64hi(mix64(P.seed + (u64)j), (u64)P.S);   // uniform on [0, S)
         P.sample_key[j] = unit_key<SRC>(P, unit);
     }
     __threadfence();

@@ -216,10 +216,19 @@ __device__ __forceinline__ void load_block(const TensorDesc &d, long long b, Blo
 
 __device__ __forceinline__ u64 block_key(const BlockData &bd, float mu, bool has_lam, float *u)
 {
+    u32 nz = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) nz |= __float_as_uint(bd.l[i]);
+    if (has_lam && nz) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) u[i] = __fsub_rn(bd.w[i], __fdiv_rn(bd.l[i], mu));
+    } else {                           // every lambda is +0: w - (+0) is w, bit for bit
+#pragma unroll
+        for (int i = 0; i < 16; ++i) u[i] = bd.w[i];
+    }
     double acc = 0.0;
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-        u[i] = form_u(bd.w[i], bd.l[i], mu, has_lam);
         const double x = (double)u[i];
         acc = __fma_rn(x, x, acc);     // x*x is exact in fp64, so this is (acc + x*x) rounded once
     }
@@ -491,12 +500,30 @@ __device__ __forceinline__ void final_rank(const Params &P, ScanShared &sh, u32 
 template <int SRC>
 __device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep);
 
+// Defined with the single-pass kernels: the projection items the aligned fast
+// kernel leaves out (tensor heads and tails, unaligned or ragged tensors).
+struct FusedShared {
+    u32 hist[NBINS];
+    u32 cnt[2];
+    u64 base[2];
+    u64 red[WARPS];
+};
+static_assert(sizeof(FusedShared) <= sizeof(ScanShared), "the edge items reuse the scan's shared memory");
+
+template <int SRC>
+__device__ void fused_edge_items(const Params &P, FusedShared &sh);
+
 // First pass of a ranking call: a plain (non-cooperative) scan at full grid.
+// When the single-pass path is active there is nothing left to scan, and the
+// launch does that path's edge items instead.
 template <int SRC>
 __global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
 {
     __shared__ ScanShared sh;
-    if (P.ctl->sel.onepass) return;          // the single-pass kernel has done this work
+    if (P.ctl->sel.onepass) {
+        if (SRC != SRC_ARRAY) fused_edge_items<SRC>(P, reinterpret_cast<FusedShared &>(sh));
+        return;
+    }
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
     __syncthreads();
     scan_source<SRC>(P, sh, do_list != 0, sh.sel.slot);
@@ -513,6 +540,8 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
     __syncthreads();
     bool src_scan = true;
+    bool gathered = false;      // the list has been walked once with early repairs
+    u64 fixed = 0;
     if (!sh.sel.done) {
         if ((first_listed || sh.sel.onepass) && threadIdx.x == 0) sh.sel.list_valid = 1;
         __syncthreads();
@@ -545,9 +574,16 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
                     const bool below = key < s.lo_key || (sk && key == s.lo_key && id > s.hi_id);
                     if (!above && !below) {
                         const u32 pos = atomicAdd(&P.ctl->fin_count, 1u);
-                        if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; }
+                        if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; P.fin_idx[pos] = i; }
+                    } else if (SRC != SRC_ARRAY && s.onepass) {
+                        // outside the narrowed bracket the final decision is already known
+                        if (above != (key >= s.guess)) {
+                            repair_unit<SRC>(P, i, id, above);
+                            ++fixed;
+                        }
                     }
                 }
+                gathered = true;
                 grid.sync();
                 const u32 n = __ldcg(&P.ctl->fin_count);
                 if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
@@ -576,20 +612,33 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     if (SRC != SRC_ARRAY) {
         if (sh.sel.onepass && !sh.sel.error && sh.sel.k > 0) {
             // single-pass path: rewrite the listed units whose provisional decision was wrong
-            const u64 n_list = __ldcg(&P.ctl->list_count[0]);
             const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
             const u64 stride = (u64)gridDim.x * THREADS;
-            u64 fixed = 0;
-            for (u64 i = (u64)blockIdx.x * THREADS + threadIdx.x; i < n_list; i += stride) {
-                const u64 key = __ldcg(&P.list_key[i]), id = __ldcg(&P.list_id[i]);
-                const bool fin = keep_by_cutoff(key, id, tk, ti);
-                if (fin != (key >= guess)) {
-                    repair_unit<SRC>(P, i, id, fin);
-                    ++fixed;
+            if (gathered) {
+                // only the members of the final buffer are still open
+                u32 n = __ldcg(&P.ctl->fin_count);
+                if (n > FIN) n = FIN;
+                for (u64 j = (u64)blockIdx.x * THREADS + threadIdx.x; j < n; j += stride) {
+                    const u64 key = __ldcg(&P.fin_key[j]), id = __ldcg(&P.fin_id[j]);
+                    const bool fin = keep_by_cutoff(key, id, tk, ti);
+                    if (fin != (key >= guess)) {
+                        repair_unit<SRC>(P, __ldcg(&P.fin_idx[j]), id, fin);
+                        ++fixed;
+                    }
+                }
+            } else {
+                const u64 n_list = __ldcg(&P.ctl->list_count[0]);
+                for (u64 i = (u64)blockIdx.x * THREADS + threadIdx.x; i < n_list; i += stride) {
+                    const u64 key = __ldcg(&P.list_key[i]), id = __ldcg(&P.list_id[i]);
+                    const bool fin = keep_by_cutoff(key, id, tk, ti);
+                    if (fin != (key >= guess)) {
+                        repair_unit<SRC>(P, i, id, fin);
+                        ++fixed;
+                    }
                 }
             }
-            if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
         }
+        if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         Ctl *c = P.ctl;
@@ -619,7 +668,7 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
             r.n_tie_kept = (long long)(s.k - s.n_gt);
             if (P.bits_key >= 63) r.tau_norm = (float)sqrt(__longlong_as_double((long long)s.lo_key));
         }
-        r.n_repaired = (long long)__ldcg(&c->n_repaired);
+        r.n_repaired = 0;      // filled in by the host from the counter once the stream is idle
         c->sel = s;
         c->res = r;
     }
