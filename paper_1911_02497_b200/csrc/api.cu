@@ -15,6 +15,7 @@
 #include "select.cuh"
 #include "structured.cuh"
 #include "fused.cuh"
+#include "fused_fast.cuh"
 #include "sample.cuh"
 
 using namespace cs;
@@ -505,7 +506,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
             pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : "k_fused_block", stream);
-            const int gridf = stream_grid(ctx, pl.n_items_b, 4);
+            const int gridf = stream_grid(ctx, pl.n_items_b, op == OP_BLOCK ? 2 : 3);
             const bool need_g = (fuse & CONDENSA_FUSE_PENALTY) != 0;
 #define CS_LAUNCH_FUSED(KERNEL, GRID)                                                          \
     do {                                                                                       \

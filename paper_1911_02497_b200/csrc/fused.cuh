@@ -141,144 +141,6 @@ __device__ __forceinline__ void fused_block_item_generic(const Params &P, const 
     }
 }
 
-// Fast item: every block of the item lies in complete block rows of a tensor
-// whose arrays are 16-byte aligned with C % 4 == 0 and fewer than 2^32 elements.
-// Four lanes share a block (one row each, one 128-bit load per array and lane);
-// the fp64 sum runs through the four lanes in row order, so it is the same
-// sequential sum as with one thread per block. 64 blocks per CTA and iteration,
-// two iterations per round (BLOCKS_PER_ITEM / 128 rounds).
-template <bool H, bool G>
-__device__ __forceinline__ void fused_block_item_fast(const Params &P, const TensorDesc &d, long long local,
-                                                      FusedShared &sh, const Bracket &br, int &par,
-                                                      u64 &n_above, bool fp16)
-{
-    constexpr int BPI = THREADS / 4;                 // blocks per iteration
-    constexpr int ROUNDS = BLOCKS_PER_ITEM / (2 * BPI);
-    const u32 C = (u32)d.d1, nbc = (u32)d.nbc;
-    const u32 b0 = (u32)(local * BLOCKS_PER_ITEM);
-    const u32 q = threadIdx.x >> 2, r = threadIdx.x & 3;
-    const int qbase = (threadIdx.x & 31) & ~3;
-    u32 brow = b0 / nbc;
-    u32 bcol = b0 - brow * nbc + q;
-    while (bcol >= nbc) { bcol -= nbc; ++brow; }
-    const bool has_lam = d.lam != nullptr;
-    const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
-    const float mu = P.mu;
-#pragma unroll 1
-    for (int round = 0; round < ROUNDS; ++round, par ^= 1) {
-        float w[2][4], l[2][4], u[2][4];
-        u32 off[2];
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            off[i] = (4u * brow + r) * C + 4u * bcol;
-            const float4 a = ld4_ro(d.w + off[i]);
-            w[i][0] = a.x; w[i][1] = a.y; w[i][2] = a.z; w[i][3] = a.w;
-            if (has_lam) {
-                const float4 c = ld4(d.lam + off[i]);
-                l[i][0] = c.x; l[i][1] = c.y; l[i][2] = c.z; l[i][3] = c.w;
-            } else {
-                l[i][0] = l[i][1] = l[i][2] = l[i][3] = 0.0f;
-            }
-            bcol += BPI;
-            while (bcol >= nbc) { bcol -= nbc; ++brow; }
-        }
-        u64 key[2];
-        bool cand[2];
-        u32 my[2] = {0, 0};
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            form_u4(w[i], l[i], mu, has_lam, u[i]);
-            double acc = 0.0;
-#pragma unroll
-            for (int s = 0; s < 4; ++s) {
-                double a = acc;
-                if (r == (u32)s) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const double x = (double)u[i][j];
-                        a = __fma_rn(x, x, a);
-                    }
-                }
-                acc = __shfl_sync(0xffffffffu, a, qbase + s);
-            }
-            key[i] = (u64)__double_as_longlong(acc);
-            const bool above = key[i] > br.hi;
-            cand[i] = !above && key[i] >= br.lo;
-            if (r == 0) {
-                n_above += above ? 1 : 0;
-                if (cand[i]) {
-                    const u64 id = (u64)d.unit_prefix + b0 + (u32)((2 * round + i) * BPI) + q;
-                    my[i] = atomicAdd(&sh.cnt[par], 1u);
-                    atomicAdd(&sh.hist[bracket_bin(br, key[i], id)], 1u);
-                }
-            }
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const u32 c = sh.cnt[par];
-            if (c) sh.base[par] = atomicAdd(&P.ctl->list_count[0], (u64)c);
-            sh.cnt[par ^ 1] = 0;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            if (__any_sync(0xffffffffu, cand[i])) {
-                const u32 m0 = __shfl_sync(0xffffffffu, my[i], qbase);
-                if (cand[i]) {
-                    const u64 pos = sh.base[par] + m0;
-                    if (pos < P.cap) {
-                        if (r == 0) {
-                            P.list_key[pos] = key[i];
-                            P.list_id[pos] = (u64)d.unit_prefix + b0 + (u32)((2 * round + i) * BPI) + q;
-                        }
-                        if (has_lam)
-                            *reinterpret_cast<float4 *>(P.jr_lam + pos * 16 + 4 * r) =
-                                make_float4(l[i][0], l[i][1], l[i][2], l[i][3]);
-                    }
-                }
-            }
-            const bool keep = key[i] >= br.guess;
-            Out o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) o[j] = finish_lean<H>(w[i][j], l[i][j], u[i][j], keep, mu, fp16, upd);
-            *reinterpret_cast<float4 *>(d.theta + off[i]) = make_float4(o[0].theta, o[1].theta, o[2].theta, o[3].theta);
-            if (d.mask) *reinterpret_cast<u32 *>(d.mask + off[i]) = keep ? 0x01010101u : 0u;
-            if (H && d.theta_h) {
-                uint2 hh;
-                hh.x = (u32)o[0].th | ((u32)o[1].th << 16);
-                hh.y = (u32)o[2].th | ((u32)o[3].th << 16);
-                *reinterpret_cast<uint2 *>(d.theta_h + off[i]) = hh;
-            }
-            if (upd) *reinterpret_cast<float4 *>(d.lam + off[i]) = make_float4(o[0].lam, o[1].lam, o[2].lam, o[3].lam);
-            if (G && d.grad) *reinterpret_cast<float4 *>(d.grad + off[i]) = make_float4(o[0].grad, o[1].grad, o[2].grad, o[3].grad);
-        }
-    }
-}
-
-// Aligned interior items of block pruning (work items of the projection
-// decomposition; the others are done by fused_edge_items).
-template <bool H, bool G>
-__global__ void __launch_bounds__(THREADS, 4) k_fused_block(Params P)
-{
-    __shared__ FusedShared sh;
-    if (!P.ctl->sel.onepass) return;
-    const Bracket br = load_bracket(P.ctl->sel);
-    for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
-    if (threadIdx.x < 2) sh.cnt[threadIdx.x] = 0;
-    __syncthreads();
-    const bool fp16 = (P.fuse & FUSE_FP16) != 0;
-    u64 n_above = 0;
-    int par = 0;
-    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-        const int t = find_tensor(P.item_prefix, P.T, item);
-        const TensorDesc d = P.td[t];
-        const long long local = item - P.item_prefix[t];
-        if (!block_item_is_fast(d, local)) continue;
-        fused_block_item_fast<H, G>(P, d, local, sh, br, par, n_above, fp16);
-    }
-    fused_finish(P, sh, n_above);
-}
-
 // ---------------------------------------------------------------- unstructured
 // Generic item: per-lane validity, scalar accesses where needed.
 template <bool H>
@@ -419,140 +281,6 @@ __device__ __forceinline__ void fused_elem_item_generic(const Params &P, const T
             }
         }
     }
-}
-
-// Fast item: all 1024 groups exist and are 16-byte aligned in every array.
-template <bool H, bool G>
-__device__ __forceinline__ void fused_elem_item_fast(const Params &P, const TensorDesc &d, long long local,
-                                                     FusedShared &sh, const Bracket &br, int par,
-                                                     u64 &n_above, bool fp16)
-{
-    const u32 lo = (u32)br.lo, hi = (u32)br.hi, guess = (u32)br.guess;
-    const long long e_base = 4 * (local * GROUPS_PER_ITEM) - d.pad;
-    const bool has_lam = d.lam != nullptr;
-    const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
-    const float mu = P.mu;
-    const float4 *wp = reinterpret_cast<const float4 *>(d.w + e_base) + threadIdx.x;
-    float w[LIN_UNROLL][4], l[LIN_UNROLL][4], u[LIN_UNROLL][4];
-#pragma unroll
-    for (int it = 0; it < LIN_UNROLL; ++it) {
-        const float4 a = __ldg(wp + it * THREADS);
-        w[it][0] = a.x; w[it][1] = a.y; w[it][2] = a.z; w[it][3] = a.w;
-    }
-    if (has_lam) {
-        const float4 *lp = reinterpret_cast<const float4 *>(d.lam + e_base) + threadIdx.x;
-#pragma unroll
-        for (int it = 0; it < LIN_UNROLL; ++it) {
-            const float4 b = lp[it * THREADS];
-            l[it][0] = b.x; l[it][1] = b.y; l[it][2] = b.z; l[it][3] = b.w;
-        }
-    } else {
-#pragma unroll
-        for (int it = 0; it < LIN_UNROLL; ++it) l[it][0] = l[it][1] = l[it][2] = l[it][3] = 0.0f;
-    }
-    u32 candm = 0, keepm = 0, na = 0;
-#pragma unroll
-    for (int it = 0; it < LIN_UNROLL; ++it) {
-        form_u4(w[it], l[it], mu, has_lam, u[it]);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const u32 key = __float_as_uint(u[it][j]) & 0x7FFFFFFFu;
-            na += key > hi ? 1u : 0u;
-            candm |= ((key >= lo && key <= hi) ? 1u : 0u) << (4 * it + j);
-            keepm |= (key >= guess ? 1u : 0u) << (4 * it + j);
-        }
-    }
-    n_above += na;
-    u32 my = 0;
-    if (candm) {
-        my = atomicAdd(&sh.cnt[par], (u32)__popc(candm));
-        u32 mm = candm;
-        while (mm) {
-            const int q = __ffs(mm) - 1;
-            mm &= mm - 1;
-            float uu = 0.0f;
-#pragma unroll
-            for (int a = 0; a < LIN_UNROLL; ++a)
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (q == 4 * a + c) uu = u[a][c];
-            const u64 id = (u64)(d.elem_prefix + e_base) + 4u * ((u32)(q >> 2) * THREADS + threadIdx.x) + (u32)(q & 3);
-            atomicAdd(&sh.hist[bracket_bin(br, (u64)(__float_as_uint(uu) & 0x7FFFFFFFu), id)], 1u);
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const u32 c = sh.cnt[par];
-        if (c) sh.base[par] = atomicAdd(&P.ctl->list_count[0], (u64)c);
-        sh.cnt[par ^ 1] = 0;
-    }
-    __syncthreads();
-    if (candm) {
-        u64 pos = sh.base[par] + my;
-        u32 mm = candm;
-        while (mm) {
-            const int q = __ffs(mm) - 1;
-            mm &= mm - 1;
-            if (pos < P.cap) {
-                float uu = 0.0f, ll = 0.0f;
-#pragma unroll
-                for (int a = 0; a < LIN_UNROLL; ++a)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if (q == 4 * a + c) { uu = u[a][c]; ll = l[a][c]; }
-                P.list_key[pos] = (u64)(__float_as_uint(uu) & 0x7FFFFFFFu);
-                P.list_id[pos] = (u64)(d.elem_prefix + e_base) + 4u * ((u32)(q >> 2) * THREADS + threadIdx.x) + (u32)(q & 3);
-                if (has_lam) P.jr_lam[pos] = ll;
-            }
-            ++pos;
-        }
-    }
-    float4 *tp = reinterpret_cast<float4 *>(d.theta + e_base) + threadIdx.x;
-#pragma unroll
-    for (int it = 0; it < LIN_UNROLL; ++it) {
-        Out o[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            o[j] = finish_lean<H>(w[it][j], l[it][j], u[it][j], (keepm >> (4 * it + j)) & 1u, mu, fp16, upd);
-        tp[it * THREADS] = make_float4(o[0].theta, o[1].theta, o[2].theta, o[3].theta);
-        if (d.mask) {
-            const u32 k4 = (keepm >> (4 * it)) & 0xFu;      // spread 4 bits to 4 bytes
-            reinterpret_cast<u32 *>(d.mask + e_base)[it * THREADS + threadIdx.x] = (k4 * 0x00204081u) & 0x01010101u;
-        }
-        if (H && d.theta_h) {
-            uint2 hh;
-            hh.x = (u32)o[0].th | ((u32)o[1].th << 16);
-            hh.y = (u32)o[2].th | ((u32)o[3].th << 16);
-            reinterpret_cast<uint2 *>(d.theta_h + e_base)[it * THREADS + threadIdx.x] = hh;
-        }
-        if (upd) reinterpret_cast<float4 *>(d.lam + e_base)[it * THREADS + threadIdx.x] =
-            make_float4(o[0].lam, o[1].lam, o[2].lam, o[3].lam);
-        if (G && d.grad) reinterpret_cast<float4 *>(d.grad + e_base)[it * THREADS + threadIdx.x] =
-            make_float4(o[0].grad, o[1].grad, o[2].grad, o[3].grad);
-    }
-}
-
-template <bool H, bool G>
-__global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
-{
-    __shared__ FusedShared sh;
-    if (!P.ctl->sel.onepass) return;
-    const Bracket br = load_bracket(P.ctl->sel);
-    for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
-    if (threadIdx.x < 2) sh.cnt[threadIdx.x] = 0;
-    __syncthreads();
-    const bool fp16 = (P.fuse & FUSE_FP16) != 0;
-    u64 n_above = 0;
-    int par = 0;
-    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-        const int t = find_tensor(P.item_prefix, P.T, item);
-        const TensorDesc d = P.td[t];
-        const long long local = item - P.item_prefix[t];
-        if (!elem_item_is_fast(d, local)) continue;
-        fused_elem_item_fast<H, G>(P, d, local, sh, br, par, n_above, fp16);
-        par ^= 1;
-    }
-    fused_finish(P, sh, n_above);
 }
 
 // The remaining projection items, listed by the host in P.edge_items. Runs inside

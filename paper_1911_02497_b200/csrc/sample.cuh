@@ -67,6 +67,13 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
 {
     __shared__ SampleShared sh;
     Ctl *ctl = P.ctl;
+#ifdef CONDENSA_DEBUG_TIME
+    unsigned long long ts[6]; int ns = 0;
+#define SSTAMP() do { if (threadIdx.x == 0 && ns < 6) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); ts[ns++] = t_; } } while (0)
+#else
+#define SSTAMP() do {} while (0)
+#endif
+    SSTAMP();
     // what the plain start kernel does: clear histograms (all CTAs share the work)
     for (int i = blockIdx.x * SAMPLE_THREADS + threadIdx.x; i < 3 * NBINS; i += gridDim.x * SAMPLE_THREADS)
         P.hist[i] = 0;
@@ -75,6 +82,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         const u64 unit = __umul64hi(mix64(P.seed + (u64)j), (u64)P.S);   // uniform on [0, S)
         P.sample_key[j] = unit_key<SRC>(P, unit);
     }
+    SSTAMP();
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -108,6 +116,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
     }
     __syncthreads();
 
+    SSTAMP();
     const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
     const double p = (double)init.k / (double)init.S;
     const double mp = (double)m * p;
@@ -175,6 +184,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         hi = e_hi;
         lo = e_lo;
     }
+    SSTAMP();
     if (open_top) hi0 = max_key;
     if (open_bot) lo0 = 0;
     if (guess < lo0) guess = lo0;
@@ -217,6 +227,12 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         ctl->fin_count = 0;
         ctl->n_repaired = 0;
         ctl->sample_done = 0;
+#ifdef CONDENSA_DEBUG_TIME
+        SSTAMP();
+        printf("k_sample phases (us):");
+        for (int i = 1; i < ns; ++i) printf(" %.1f", (double)(ts[i] - ts[i - 1]) * 1e-3);
+        printf("\n");
+#endif
     }
 }
 

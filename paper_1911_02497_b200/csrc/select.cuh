@@ -539,6 +539,13 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
     __syncthreads();
+#ifdef CONDENSA_DEBUG_TIME
+    unsigned long long tq[8]; int nq = 0;
+#define TSTAMP() do { if (blockIdx.x == 0 && threadIdx.x == 0 && nq < 8) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); tq[nq++] = t_; } } while (0)
+#else
+#define TSTAMP() do {} while (0)
+#endif
+    TSTAMP();
     bool src_scan = true;
     bool gathered = false;      // the list has been walked once with early repairs
     u64 fixed = 0;
@@ -555,6 +562,7 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
             __syncthreads();
             if (sh.sel.done) break;
             block_pick(P, sh, src_scan, max_key);
+            TSTAMP();
             // clear the histogram slot that the scan after the next one will use
             if (blockIdx.x == 0) {
                 const int z = (sh.sel.slot + 2) % 3;
@@ -584,11 +592,14 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
                     }
                 }
                 gathered = true;
+                TSTAMP();
                 grid.sync();
+                TSTAMP();
                 const u32 n = __ldcg(&P.ctl->fin_count);
                 if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
                 __syncthreads();
                 final_rank(P, sh, n);
+                TSTAMP();
                 break;
             }
             // next scan
@@ -640,6 +651,14 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
         }
         if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
     }
+    TSTAMP();
+#ifdef CONDENSA_DEBUG_TIME
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        printf("k_select phases (us):");
+        for (int i = 1; i < nq; ++i) printf(" %.1f", (double)(tq[i] - tq[i - 1]) * 1e-3);
+        printf("  fixed(cta0,t0)=%llu pop=%llu\n", fixed, sh.sel.pop);
+    }
+#endif
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         Ctl *c = P.ctl;
         const Sel &s = sh.sel;
