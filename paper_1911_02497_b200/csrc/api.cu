@@ -235,6 +235,7 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl)
 }
 
 constexpr int N_SAMPLE = SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD;
+constexpr int SAMPLE_CTAS = 64;
 
 // journal_floats: floats of original lambda kept per listed unit (0: no single-pass path)
 Layout make_layout(int T, const Plan &pl, bool ranking, bool filter, int journal_floats = 0)
@@ -499,14 +500,15 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         Params Pf = P;                      // single-pass kernel runs on the projection decomposition
         Pf.item_prefix = pb;
         Pf.n_items = pl.n_items_b;
+        if (sampling && op == OP_BLOCK) Pa.n_edge_items = 0;     // the block kernel does its edge items itself
         if (sampling && !init.done) {
             int pi_ = prof_begin(ctx, "k_sample", stream);
-            if (op == OP_PRUNE) k_sample<SRC_ELEM><<<N_SAMPLE / SAMPLE_THREADS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
-            else k_sample<SRC_BLOCK><<<N_SAMPLE / SAMPLE_THREADS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            if (op == OP_PRUNE) k_sample<SRC_ELEM><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            else k_sample<SRC_BLOCK><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
             pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : "k_fused_block", stream);
-            const int gridf = stream_grid(ctx, pl.n_items_b, op == OP_BLOCK ? 2 : 3);
+            const int gridf = stream_grid(ctx, pl.n_items_b, op == OP_BLOCK ? CS_BLOCK_MINB : 3);
             const bool need_g = (fuse & CONDENSA_FUSE_PENALTY) != 0;
 #define CS_LAUNCH_FUSED(KERNEL, GRID)                                                          \
     do {                                                                                       \
@@ -531,7 +533,8 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             if (op == OP_PRUNE) {
                 k_scan<SRC_ELEM><<<stream_grid(ctx, pl.n_items_a, 4), THREADS, 0, stream>>>(Pa, do_list0);
             } else if (op == OP_BLOCK) {
-                k_scan<SRC_BLOCK><<<stream_grid(ctx, pl.n_items_a, 4), THREADS, 0, stream>>>(Pa, do_list0);
+                // with the single-pass path this launch only runs when the sample advised against it
+                k_scan<SRC_BLOCK><<<stream_grid(ctx, pl.n_items_a, sampling ? 1 : 4), THREADS, 0, stream>>>(Pa, do_list0);
             } else {
                 k_scan<SRC_ARRAY><<<stream_grid(ctx, (pl.S + THREADS - 1) / THREADS, 4), THREADS, 0, stream>>>(Pa, do_list0);
             }

@@ -81,11 +81,18 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
     const u32 lo = (u32)br.lo, range = (u32)br.hi - (u32)br.lo, guess = (u32)br.guess;
     const float mu = P.mu;
     const int warp = threadIdx.x >> 5;
-    u64 n_above = 0;
+    u32 n_above = 0;
+    long long t_first = 0, t_end = -1;
+    TensorDesc d;
+    d.numel = 0; d.pad = 0; d.vec_ok = 0;
     for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-        const int t = find_tensor(P.item_prefix, P.T, item);
-        const TensorDesc d = P.td[t];
-        const long long local = item - P.item_prefix[t];
+        if (item >= t_end) {        // look the tensor up only when the items leave it
+            const int t = find_tensor(P.item_prefix, P.T, item);
+            d = P.td[t];
+            t_first = P.item_prefix[t];
+            t_end = P.item_prefix[t + 1];
+        }
+        const long long local = item - t_first;
         if (!elem_item_is_fast(d, local)) continue;
         const long long e_base = 4 * (local * GROUPS_PER_ITEM) - d.pad;
         const bool has_lam = d.lam != nullptr;
@@ -102,22 +109,21 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
 #pragma unroll
             for (int it = 0; it < LIN_UNROLL; ++it) lv[it] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        u32 nkeep = 0, ncandkeep = 0;
+        u32 nkeep = 0, candm = 0;       // candm bit 4*it+j: element lies in the bracket
 #pragma unroll
         for (int it = 0; it < LIN_UNROLL; ++it) {
             const float w[4] = {wv[it].x, wv[it].y, wv[it].z, wv[it].w};
             const float l[4] = {lv[it].x, lv[it].y, lv[it].z, lv[it].w};
             float u[4], th[4], ln[4], g[4];
             form_u4(w, l, mu, has_lam, u);
-            u32 key[4];
-            u32 m = 0, anyc = 0;
+            u32 m = 0;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                key[j] = __float_as_uint(u[j]) & 0x7FFFFFFFu;
-                const bool keep = key[j] >= guess;
+                const u32 key = __float_as_uint(u[j]) & 0x7FFFFFFFu;
+                const bool keep = key >= guess;
                 th[j] = keep ? u[j] : 0.0f;
                 m |= keep ? (1u << (8 * j)) : 0u;
-                anyc |= (key[j] - lo <= range) ? 1u : 0u;
+                candm |= (key - lo <= range) ? (1u << (4 * it + j)) : 0u;
             }
             nkeep += __popc(m);
             unsigned short h[4];
@@ -131,29 +137,6 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
                 ln[j] = upd ? __fsub_rn(l[j], p) : l[j];
                 g[j] = __fsub_rn(p, ln[j]);
             }
-            if (anyc) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (key[j] - lo <= range) {
-                        const u64 id = (u64)(d.elem_prefix + e_base) + 4u * (u32)(it * THREADS + threadIdx.x) + (u32)j;
-                        ncandkeep += key[j] >= guess ? 1u : 0u;
-                        atomicAdd(&sh.hist[bracket_bin(br, (u64)key[j], id)], 1u);
-                        const u32 slot = atomicAdd(&sh.wcount[warp], 1u);
-                        if (slot < ESTG) {
-                            sh.key[warp][slot] = key[j];
-                            sh.id[warp][slot] = id;
-                            sh.lam[warp][slot] = l[j];
-                        } else {
-                            const u64 pos = atomicAdd(&P.ctl->list_count[0], 1ull);
-                            if (pos < P.cap) {
-                                P.list_key[pos] = (u64)key[j];
-                                P.list_id[pos] = id;
-                                if (has_lam) P.jr_lam[pos] = l[j];
-                            }
-                        }
-                    }
-                }
-            }
             const long long go = it * THREADS + threadIdx.x;      // group offset inside the item
             reinterpret_cast<float4 *>(d.theta + e_base)[go] = make_float4(th[0], th[1], th[2], th[3]);
             if (d.mask) reinterpret_cast<u32 *>(d.mask + e_base)[go] = m;
@@ -162,14 +145,50 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
             if (upd) reinterpret_cast<float4 *>(d.lam + e_base)[go] = make_float4(ln[0], ln[1], ln[2], ln[3]);
             if (G && d.grad) reinterpret_cast<float4 *>(d.grad + e_base)[go] = make_float4(g[0], g[1], g[2], g[3]);
         }
+        // the few elements inside the bracket: once per item, from the lambda still in registers
+        u32 ncandkeep = 0;
+        while (candm) {
+            const int qb = __ffs(candm) - 1;
+            candm &= candm - 1;
+            float ll = 0.0f;
+#pragma unroll
+            for (int a = 0; a < LIN_UNROLL; ++a) {
+                if ((qb >> 2) == a) {
+                    const float4 v = lv[a];
+                    ll = (qb & 3) == 0 ? v.x : (qb & 3) == 1 ? v.y : (qb & 3) == 2 ? v.z : v.w;
+                }
+            }
+            const u32 eo = 4u * (u32)((qb >> 2) * THREADS + threadIdx.x) + (u32)(qb & 3);
+            const float ww = __ldg(d.w + e_base + eo);
+            // same operations as above: the key comes out bit-identical
+            const float uu = (has_lam && __float_as_uint(ll) != 0u) ? __fsub_rn(ww, __fdiv_rn(ll, mu)) : ww;
+            const u32 key = __float_as_uint(uu) & 0x7FFFFFFFu;
+            const u64 id = (u64)(d.elem_prefix + e_base) + eo;
+            ncandkeep += key >= guess ? 1u : 0u;
+            atomicAdd(&sh.hist[bracket_bin(br, (u64)key, id)], 1u);
+            const u32 slot = atomicAdd(&sh.wcount[warp], 1u);
+            if (slot < ESTG) {
+                sh.key[warp][slot] = key;
+                sh.id[warp][slot] = id;
+                sh.lam[warp][slot] = ll;
+            } else {
+                const u64 pos = atomicAdd(&P.ctl->list_count[0], 1ull);
+                if (pos < P.cap) {
+                    P.list_key[pos] = (u64)key;
+                    P.list_id[pos] = id;
+                    if (has_lam) P.jr_lam[pos] = ll;
+                }
+            }
+        }
         n_above += nkeep - ncandkeep;      // keeps that are not candidates lie above the bracket
         elem_flush(P, sh, has_lam, ESTG / 2);
     }
     elem_flush(P, sh, true, 0);
     __syncthreads();
     // totals of this CTA
-    for (int o = 16; o > 0; o >>= 1) n_above += __shfl_xor_sync(0xffffffffu, n_above, o);
-    if ((threadIdx.x & 31) == 0) sh.red[warp] = n_above;
+    u64 na = n_above;
+    for (int o = 16; o > 0; o >>= 1) na += __shfl_xor_sync(0xffffffffu, na, o);
+    if ((threadIdx.x & 31) == 0) sh.red[warp] = na;
     __syncthreads();
     if (threadIdx.x == 0) {
         u64 tot = 0;
@@ -183,12 +202,17 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
 }
 
 // ---------------------------------------------------------------- 4x4 blocks
+#ifndef CS_BLOCK_MINB
+#define CS_BLOCK_MINB 2          // resident CTAs per SM the block kernel is compiled for
+#endif
 constexpr int BSTG = 48;        // staged candidate blocks per warp (a warp adds at most 32 per iteration)
 
 struct BlockFastShared {
-    u32 hist[NBINS];
-    u32 wcount[WARPS];
+    u32 hist[NBINS];            // the first four members mirror FusedShared (edge items reuse them)
+    u32 cnt[2];
+    u64 base[2];
     u64 red[WARPS];
+    u32 wcount[WARPS];
     u64 key[WARPS][BSTG];
     u64 id[WARPS][BSTG];
     float4 lam[WARPS][BSTG][4];
@@ -226,7 +250,7 @@ __device__ __forceinline__ void block_flush(const Params &P, BlockFastShared &sh
 // contiguous bytes of each of the four rows), the fp64 sum of squares in
 // row-major order, one decision, four rows of outputs.
 template <bool H, bool G>
-__global__ void __launch_bounds__(THREADS, 2) k_fused_block(Params P)
+__global__ void __launch_bounds__(THREADS, CS_BLOCK_MINB) k_fused_block(Params P)
 {
     __shared__ BlockFastShared sh;
     if (!P.ctl->sel.onepass) return;
@@ -341,6 +365,23 @@ __global__ void __launch_bounds__(THREADS, 2) k_fused_block(Params P)
     block_flush(P, sh, 0);
     __syncthreads();
     u64 na = n_above;
+    // the items outside the aligned fast path (tensor tails, ragged or unaligned
+    // tensors, tensors that pass through), listed by the host
+    if (P.n_edge_items > 0) {
+        FusedShared &fs = reinterpret_cast<FusedShared &>(sh);
+        if (threadIdx.x < 2) fs.cnt[threadIdx.x] = 0;
+        __syncthreads();
+        int par = 0;
+        for (long long i = blockIdx.x; i < P.n_edge_items; i += gridDim.x) {
+            const long long item = P.edge_items[i];
+            const int t = find_tensor(P.item_prefix, P.T, item);
+            const TensorDesc g = P.td[t];
+            const long long local = item - P.item_prefix[t];
+            if (!g.ranked) process_linear_item<M_KEEPALL>(P, g, local, 0, 0);
+            else fused_block_item_generic<H>(P, g, local, fs, br, par, na, fp16);
+        }
+        __syncthreads();
+    }
     for (int o = 16; o > 0; o >>= 1) na += __shfl_xor_sync(0xffffffffu, na, o);
     if ((threadIdx.x & 31) == 0) sh.red[warp] = na;
     __syncthreads();

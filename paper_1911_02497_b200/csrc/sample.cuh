@@ -77,8 +77,11 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
     // what the plain start kernel does: clear histograms (all CTAs share the work)
     for (int i = blockIdx.x * SAMPLE_THREADS + threadIdx.x; i < 3 * NBINS; i += gridDim.x * SAMPLE_THREADS)
         P.hist[i] = 0;
-    const int j = blockIdx.x * SAMPLE_THREADS + threadIdx.x;
-    if (j < P.n_sample) {
+    // the sampling itself is spread over many CTAs (few threads each) so that the
+    // random reads of one SM do not queue behind each other
+    const int per_cta = (P.n_sample + gridDim.x - 1) / gridDim.x;
+    const int j = blockIdx.x * per_cta + threadIdx.x;
+    if (threadIdx.x < per_cta && j < P.n_sample) {
         const u64 unit = __umul64hi(mix64(P.seed + (u64)j), (u64)P.S);   // uniform on [0, S)
         P.sample_key[j] = unit_key<SRC>(P, unit);
     }

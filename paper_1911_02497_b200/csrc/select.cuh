@@ -270,7 +270,7 @@ __device__ __forceinline__ void scan_source_array(const Params &P, ScanShared &s
 }
 
 template <int SRC>
-__device__ __forceinline__ void scan_source(const Params &P, ScanShared &sh, bool do_list, int slot)
+__device__ __noinline__ void scan_source(const Params &P, ScanShared &sh, bool do_list, int slot)
 {
     ScanCtx c;
     scan_begin(sh, c, do_list);
@@ -280,7 +280,7 @@ __device__ __forceinline__ void scan_source(const Params &P, ScanShared &sh, boo
     scan_end(P, sh, c, slot);
 }
 
-__device__ __forceinline__ void scan_list(const Params &P, ScanShared &sh, int slot, u64 n_list)
+__device__ __noinline__ void scan_list(const Params &P, ScanShared &sh, int slot, u64 n_list)
 {
     ScanCtx c;
     scan_begin(sh, c, false);
@@ -294,6 +294,12 @@ __device__ __forceinline__ void scan_list(const Params &P, ScanShared &sh, int s
 }
 
 // ---------------------------------------------------------------- pick
+#ifdef CONDENSA_DEBUG_TIME
+__device__ unsigned long long g_dbg[16];
+#define DSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_dbg[i] = t_; } } while (0)
+#else
+#define DSTAMP(i) do {} while (0)
+#endif
 __device__ __forceinline__ void set_shift(Sel &s)
 {
     const u64 range = (s.lo_key == s.hi_key) ? (s.hi_id - s.lo_id) : (s.hi_key - s.lo_key);
@@ -304,9 +310,10 @@ __device__ __forceinline__ void set_shift(Sel &s)
 // All threads of the CTA; every CTA computes the same new state from the same
 // global histogram. `src_scan`: the scan that filled the histogram visited the
 // whole source (its count of units above the bracket is then complete).
-__device__ __forceinline__ void block_pick(const Params &P, ScanShared &sh, bool src_scan, u64 max_key)
+__device__ __noinline__ void block_pick(const Params &P, ScanShared &sh, bool src_scan, u64 max_key)
 {
     Sel &s = sh.sel;
+    DSTAMP(0);
     const u64 *gh = P.hist + (size_t)s.slot * NBINS;
     constexpr int PER = NBINS / THREADS;
     u64 cnt[PER];
@@ -325,7 +332,9 @@ __device__ __forceinline__ void block_pick(const Params &P, ScanShared &sh, bool
     }
     if (lane == 31) sh.red[warp] = inc;
     if (threadIdx.x == 0) sh.pick_bin = -1;
+    DSTAMP(1);
     __syncthreads();
+    DSTAMP(2);
     u64 wbase = 0, total = 0;
     for (int i = 0; i < WARPS; ++i) {
         if (i < warp) wbase += sh.red[i];
@@ -349,6 +358,7 @@ __device__ __forceinline__ void block_pick(const Params &P, ScanShared &sh, bool
         }
     }
     __syncthreads();
+    DSTAMP(3);
     if (threadIdx.x == 0) {
         s.passes += 1;
         if (s.above_known && src_scan && above_scan != s.n_above) s.error = 1;
@@ -419,11 +429,13 @@ __device__ __forceinline__ void block_pick(const Params &P, ScanShared &sh, bool
         set_shift(s);
         if (s.passes >= MAX_SELECT_ITERS && !s.done) { s.error = 7; s.done = 1; }
     }
+    DSTAMP(4);
     __syncthreads();
+    DSTAMP(5);
 }
 
 // Rank the (at most FIN) bracket members directly. Entries are in fin_key/fin_id.
-__device__ __forceinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
+__device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
 {
     Sel &s = sh.sel;
     u64 *k = &sh.stg_key[0][0];       // FIN <= WARPS * WSTG
@@ -436,6 +448,16 @@ __device__ __forceinline__ void final_rank(const Params &P, ScanShared &sh, u32 
     if (threadIdx.x == 0) sh.fin_hit = -1;
     __syncthreads();
     const u64 r = s.k - s.n_above;     // 1-based rank inside the bracket
+    if (n <= 512) {
+        // few survivors: count, for each, how many rank before it
+        for (u32 i = threadIdx.x; i < n; i += THREADS) {
+            const u64 ki = k[i], di = d[i];
+            u32 before = 0;
+            for (u32 j = 0; j < n; ++j) before += (k[j] > ki || (k[j] == ki && d[j] < di)) ? 1u : 0u;
+            if ((u64)before + 1 == r) sh.fin_hit = (int)i;
+        }
+        __syncthreads();
+    } else {
     // bitonic sort of the padded array into ranking order (first = strongest)
     u32 n2 = 1;
     while (n2 < n) n2 <<= 1;
@@ -460,6 +482,7 @@ __device__ __forceinline__ void final_rank(const Params &P, ScanShared &sh, u32 
     }
     if (threadIdx.x == 0 && r >= 1 && r <= (u64)n) sh.fin_hit = (int)(r - 1);
     __syncthreads();
+    }
     if (sh.fin_hit >= 0) {
         const u64 tk = k[sh.fin_hit];
         u64 gt = 0, eq = 0;
@@ -521,7 +544,7 @@ __global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
 {
     __shared__ ScanShared sh;
     if (P.ctl->sel.onepass) {
-        if (SRC != SRC_ARRAY) fused_edge_items<SRC>(P, reinterpret_cast<FusedShared &>(sh));
+        if (SRC != SRC_ARRAY && P.n_edge_items > 0) fused_edge_items<SRC>(P, reinterpret_cast<FusedShared &>(sh));
         return;
     }
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
@@ -547,7 +570,6 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
 #endif
     TSTAMP();
     bool src_scan = true;
-    bool gathered = false;      // the list has been walked once with early repairs
     u64 fixed = 0;
     if (!sh.sel.done) {
         if ((first_listed || sh.sel.onepass) && threadIdx.x == 0) sh.sel.list_valid = 1;
@@ -583,15 +605,8 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
                     if (!above && !below) {
                         const u32 pos = atomicAdd(&P.ctl->fin_count, 1u);
                         if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; P.fin_idx[pos] = i; }
-                    } else if (SRC != SRC_ARRAY && s.onepass) {
-                        // outside the narrowed bracket the final decision is already known
-                        if (above != (key >= s.guess)) {
-                            repair_unit<SRC>(P, i, id, above);
-                            ++fixed;
-                        }
                     }
                 }
-                gathered = true;
                 TSTAMP();
                 grid.sync();
                 TSTAMP();
@@ -625,19 +640,7 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
             // single-pass path: rewrite the listed units whose provisional decision was wrong
             const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
             const u64 stride = (u64)gridDim.x * THREADS;
-            if (gathered) {
-                // only the members of the final buffer are still open
-                u32 n = __ldcg(&P.ctl->fin_count);
-                if (n > FIN) n = FIN;
-                for (u64 j = (u64)blockIdx.x * THREADS + threadIdx.x; j < n; j += stride) {
-                    const u64 key = __ldcg(&P.fin_key[j]), id = __ldcg(&P.fin_id[j]);
-                    const bool fin = keep_by_cutoff(key, id, tk, ti);
-                    if (fin != (key >= guess)) {
-                        repair_unit<SRC>(P, __ldcg(&P.fin_idx[j]), id, fin);
-                        ++fixed;
-                    }
-                }
-            } else {
+            {
                 const u64 n_list = __ldcg(&P.ctl->list_count[0]);
                 for (u64 i = (u64)blockIdx.x * THREADS + threadIdx.x; i < n_list; i += stride) {
                     const u64 key = __ldcg(&P.list_key[i]), id = __ldcg(&P.list_id[i]);
@@ -656,7 +659,9 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         printf("k_select phases (us):");
         for (int i = 1; i < nq; ++i) printf(" %.1f", (double)(tq[i] - tq[i - 1]) * 1e-3);
-        printf("  fixed(cta0,t0)=%llu pop=%llu\n", fixed, sh.sel.pop);
+        printf("  fixed(cta0,t0)=%llu pop=%llu | pick: start+%.1f", fixed, sh.sel.pop, (double)(g_dbg[0] - tq[0]) * 1e-3);
+        for (int i = 1; i < 6; ++i) printf(" %.1f", (double)(g_dbg[i] - g_dbg[i - 1]) * 1e-3);
+        printf("\n");
     }
 #endif
     if (blockIdx.x == 0 && threadIdx.x == 0) {
