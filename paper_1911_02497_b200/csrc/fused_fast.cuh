@@ -82,18 +82,24 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
     const float mu = P.mu;
     const int warp = threadIdx.x >> 5;
     u32 n_above = 0;
-    long long t_first = 0, t_end = -1;
-    TensorDesc d;
-    d.numel = 0; d.pad = 0; d.vec_ok = 0;
+    long long t_first = 0, t_end = -1, fast_lo = 0, fast_hi = 0;
+    struct { const float *w; float *lam, *theta, *grad; uint8_t *mask; uint16_t *theta_h; long long elem_prefix; int pad; } d;
+    d.w = nullptr; d.lam = d.theta = d.grad = nullptr; d.mask = nullptr; d.theta_h = nullptr;
+    d.elem_prefix = 0; d.pad = 0;
     for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
         if (item >= t_end) {        // look the tensor up only when the items leave it
             const int t = find_tensor(P.item_prefix, P.T, item);
-            d = P.td[t];
+            const TensorDesc &g = P.td[t];
             t_first = P.item_prefix[t];
             t_end = P.item_prefix[t + 1];
+            // fast items form a range of local indices (same rule as elem_item_is_fast)
+            fast_lo = g.pad ? 1 : 0;
+            fast_hi = g.vec_ok ? (g.numel + g.pad) / (4 * GROUPS_PER_ITEM) : 0;
+            d.w = g.w; d.lam = g.lam; d.theta = g.theta; d.grad = g.grad; d.mask = g.mask; d.theta_h = g.theta_h;
+            d.elem_prefix = g.elem_prefix; d.pad = g.pad;
         }
         const long long local = item - t_first;
-        if (!elem_item_is_fast(d, local)) continue;
+        if (local < fast_lo || local >= fast_hi) continue;
         const long long e_base = 4 * (local * GROUPS_PER_ITEM) - d.pad;
         const bool has_lam = d.lam != nullptr;
         const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
@@ -152,11 +158,11 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
             candm &= candm - 1;
             float ll = 0.0f;
 #pragma unroll
-            for (int a = 0; a < LIN_UNROLL; ++a) {
-                if ((qb >> 2) == a) {
-                    const float4 v = lv[a];
-                    ll = (qb & 3) == 0 ? v.x : (qb & 3) == 1 ? v.y : (qb & 3) == 2 ? v.z : v.w;
-                }
+            for (int a = 0; a < LIN_UNROLL; ++a) {      // select without indexing the registers
+                if (qb == 4 * a + 0) ll = lv[a].x;
+                if (qb == 4 * a + 1) ll = lv[a].y;
+                if (qb == 4 * a + 2) ll = lv[a].z;
+                if (qb == 4 * a + 3) ll = lv[a].w;
             }
             const u32 eo = 4u * (u32)((qb >> 2) * THREADS + threadIdx.x) + (u32)(qb & 3);
             const float ww = __ldg(d.w + e_base + eo);
