@@ -26,6 +26,13 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the projection kernel, from the ncu captures
+# summarised under profiles/ (taken on smaller cases; the traffic grows in proportion to the parameters).
+# Keyed by (kernel, fuse); set an entry to None when the kernel changes after its capture.
+NCU_TRAFFIC_PER_PARAM = {
+    ("k_fused_block", ("lambda",)): 15.60,
+    ("k_fused_elem", ("fp16", "lambda", "penalty")): 18.86,
+}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -233,12 +240,17 @@ def run_ours(args):
         ctx.profile_enable(False)
         peak, peak_src = measured_peak()
         kernels = {k: {"launches": n, "avg_us": 1e3 * ms / n} for k, (n, ms) in prof.items()}
-        dom = max(prof.items(), key=lambda kv: kv[1][1])
+        # the kernel that does the projection (reads w, lambda; writes theta, mask, lambda):
+        # its algorithmic bytes are the step's
+        movers = {k: v for k, v in prof.items() if k.startswith(("k_fused", "k_apply", "k_quantize", "k_lagrange"))}
+        dom = max(movers.items(), key=lambda kv: kv[1][1])
         dom_name, (dom_n, dom_ms) = dom
-        # the dominant kernel does the whole projection: its algorithmic bytes are the step's
         achieved = (N * bpp) / (dom_ms / dom_n * 1e-3) / 1e9
+        traffic = None
+        if args.scale == 1.0 and (dom_name, ws.fuse) in NCU_TRAFFIC_PER_PARAM:
+            traffic = NCU_TRAFFIC_PER_PARAM[(dom_name, ws.fuse)] * N
         roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak,
-                    "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                    "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                     "peak_source": peak_src, "algorithmic_bytes_per_launch": N * bpp,
                     "step_achieved": (N * bpp) / (ms_per_step * 1e-3) / 1e9,
                     "step_frac": (N * bpp) / (ms_per_step * 1e-3) / 1e9 / peak,
