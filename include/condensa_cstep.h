@@ -85,8 +85,16 @@ enum {
     CONDENSA_FUSE_FP16 = 1,     /* theta = fp16 round-to-nearest-even of kept u, widened back  */
     CONDENSA_FUSE_LAMBDA = 2,   /* update lambda in place                                     */
     CONDENSA_FUSE_PENALTY = 4,  /* write g to grad                                            */
-    CONDENSA_NO_SAMPLING = 64   /* do not bracket the threshold from a sample first: rank with
-                                   full histogram passes only (slower; same results)           */
+    CONDENSA_NO_SAMPLING = 64   /* rank with full histogram passes, then project (two passes over
+                                   w and lambda; same results). Default for large inputs is ONE
+                                   pass: the threshold is first bracketed from 16384 hashed sample
+                                   positions, the pass decides everything outside the bracket for
+                                   good and lists the rest, and the exact selection runs on that
+                                   list. The bracket is checked exactly afterwards; should it ever
+                                   miss (probability < 1e-18 for positions independent of the
+                                   data) the outputs of that call are invalid, lambda has been
+                                   updated, and condensa_get_result() returns
+                                   CONDENSA_ERR_INTERNAL - it is never silent.                    */
 };
 
 /* return codes */

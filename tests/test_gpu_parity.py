@@ -225,6 +225,26 @@ def test_single_pass_path_is_taken_and_repairs(ctx):
     assert res.sampled == 1 and 0 < res.n_candidates < res.n_units // 8
 
 
+def test_sample_bracket_miss_is_reported_not_silent(ctx):
+    """The single-pass path trusts a bracket taken from 16384 hashed positions and checks it
+    exactly afterwards. Here the input is built against that hash (tiny values exactly at the
+    sampled positions), so the bracket misses: the call must say so through the result status
+    instead of returning a wrong projection, and the context must stay usable."""
+    from paper_1911_02497_b200 import cstep
+    n, m, seed = 1 << 20, 16384, 0x9E3779B97F4A7C15
+    w = W.draw(n, "normal", 1.0, 77, 0, 0)
+    pos = [(W._mix64_scalar((seed + j) & ((1 << 64) - 1)) * n) >> 64 for j in range(m)]
+    w[np.array(pos)] = (W.draw(m, "normal", 1e-4, 78, 0, 0))
+    from paper_1911_02497_b200.device_set import DeviceSet
+    ds = DeviceSet([w], [np.zeros_like(w)])
+    ds.run(ctx, "prune", 0.9, 1e-3, ("lambda",))
+    with pytest.raises(cstep.CondensaError) as e:
+        ctx.get_result()
+    assert e.value.code == cstep.ERR_INTERNAL
+    # the same input without the sample bracket is projected correctly
+    check(ctx, "prune", [w], [np.zeros_like(w)], 0.9, 1e-3, ("lambda", "no_sampling"))
+
+
 # ---------------------------------------------------------------- filters
 def test_filter_small_and_ties(ctx):
     ws = W.random_set([(7, 3, 3, 3), (10, 12), (9, 7, 1, 1), (6, 300, 3, 3), (3,)], seed=2,
