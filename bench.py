@@ -115,6 +115,25 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
+def dist_max(value: float, world: int, device=None) -> float:
+    """Largest `value` over the ranks of the default process group (identity for one rank)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(total_ms_local: float, steps: int, n_params: int, world: int, device=None):
+    """Whole-job params/s of `world` independent replicas: what all ranks processed over the
+    slowest rank's time. Returns (value, ms_per_step)."""
+    total_ms = dist_max(total_ms_local, world, device)
+    ms_per_step = total_ms / steps
+    return world * n_params / (ms_per_step * 1e-3), ms_per_step
+
+
 def workload_name(ws) -> str:
     return "%s: %s s=%.2f fuse=%s, %d tensors, %d params" % (
         ws.name, ws.op, ws.sparsity, "+".join(ws.fuse) or "none", len(ws.w), ws.numel)
@@ -219,13 +238,7 @@ def run_ours(args):
         barrier()
     launches = ctx.launch_count() - launches0
     per_step_ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = float(sum(per_step_ms))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=ds.device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
-    value = world * N / (ms_per_step * 1e-3)
+    value, ms_per_step = replica_throughput(float(sum(per_step_ms)), args.steps, N, world, ds.device)
 
     line = None
     if rank == 0:
