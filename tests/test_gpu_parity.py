@@ -127,6 +127,35 @@ def test_quantize_special_values_and_skewed_alignment(ctx):
     check(ctx, "quantize", ws.w, ws.lam, mu=ws.mu, fuse=("penalty",), elem_offset=1, skew=2)
 
 
+def test_quantize_every_fp32_bit_pattern(ctx):
+    """All 2^32 binary32 patterns through the quantise entry point against the oracle's
+    explicit-bit conversion (binary16 bits and the widened theta)."""
+    import torch
+    from paper_1911_02497_b200 import cstep
+    chunk = 1 << 27
+    dev = torch.device("cuda:0")
+    w = torch.empty(chunk, dtype=torch.int32, device=dev)
+    theta = torch.empty(chunk, dtype=torch.float32, device=dev)
+    th = torch.empty(chunk, dtype=torch.int16, device=dev)
+    base = torch.arange(chunk, dtype=torch.int64, device=dev)
+    tab = cstep.tensor_table([w], None, [theta], None, None, [th], shapes=[(chunk,)])
+    for c in range((1 << 32) // chunk):
+        first = c * chunk
+        w.copy_(((base + first) & 0xFFFFFFFF).to(torch.int64).sub_((base + first >= (1 << 31)).to(torch.int64) << 32).to(torch.int32))
+        ctx.cstep_quantize(tab, 1, 1.0)
+        got_h = th.cpu().numpy().view(np.uint16)
+        exp_h = oracle.f32_to_f16_range(first, chunk)
+        assert np.array_equal(got_h, exp_h), "chunk %d" % c
+        # theta is the exact widening of those 16 bits (NaN: quiet, sign kept)
+        wide = torch.from_numpy(exp_h.view(np.int16)).to(dev).view(torch.float16).to(torch.float32)
+        tb, wb = theta.view(torch.int32), wide.view(torch.int32)
+        nan = torch.isnan(wide)
+        assert bool(torch.equal(tb[~nan], wb[~nan]))
+        neg = torch.from_numpy((exp_h >> 15).astype(np.bool_)).to(dev)
+        assert bool(torch.isnan(theta[nan]).all()) and bool(torch.equal(tb[nan] < 0, neg[nan]))    # sign kept
+    torch.cuda.synchronize()
+
+
 @pytest.mark.parametrize("fuse", [("lambda",), ("penalty",), ("lambda", "penalty")])
 def test_lagrange_update(ctx, fuse):
     ws = W.random_set([(33, 17), (4096,), (5, 3, 3, 3), (1,)], seed=8, kind="normal", scale=0.1,
