@@ -195,12 +195,18 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     ws = W.config(args.config, scale=args.scale)
+    if args.op:      # a standalone operation on the configuration's weight set (not the headline)
+        ws.op = args.op
+        ws.fuse = ("lambda", "penalty") if args.op == "lagrange" else ("lambda",)
+        args.skip_cpu = True
     fuse = ws.fuse + (("no_sampling",) if args.no_sampling else ())
     with_grad = "penalty" in ws.fuse
     ds = DeviceSet(ws.w, ws.lam, device="cuda:%d" % local, with_grad=with_grad, with_theta_h=False)
     ctx = cstep.Context(local)
     N = ws.numel
     bpp = algorithmic_bytes_per_param(ws.fuse)
+    if args.op == "lagrange":
+        bpp = 4 + 4 + 4 + 4 + 4          # read w, theta, lambda; write lambda, g
     stream = torch.cuda.current_stream()
 
     def step():
@@ -242,7 +248,7 @@ def run_ours(args):
 
     line = None
     if rank == 0:
-        res = ctx.get_result()
+        res = ctx.get_result() if ws.op in ("prune", "filter", "block") else None
         # second pass over the same call with an event pair around every kernel
         ctx.profile_enable(True)
         for _ in range(args.steps):
@@ -276,7 +282,8 @@ def run_ours(args):
         hm = [torch.empty(a.shape, dtype=torch.uint8).pin_memory() for a in hw]
         hg = [torch.empty_like(a).pin_memory() for a in hw] if with_grad else None
         tab = cstep.tensor_table(hw, hl, ht, hm, hg, None, shapes=ws.shapes)
-        opn = {"prune": cstep.OP_PRUNE, "filter": cstep.OP_FILTER, "block": cstep.OP_BLOCK}[ws.op]
+        opn = {"prune": cstep.OP_PRUNE, "filter": cstep.OP_FILTER, "block": cstep.OP_BLOCK,
+               "quantize": cstep.OP_QUANTIZE, "lagrange": cstep.OP_LAGRANGE}[ws.op]
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
         lam0 = [torch.from_numpy(a.copy()) for a in ws.lam]
 
@@ -324,8 +331,9 @@ def run_ours(args):
                 "hbm_gbs": (N * bpp) / (ms_per_step * 1e-3) / 1e9,
                 "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu,
-                "result": {"passes": res.passes, "sampled": res.sampled,
-                           "n_candidates": res.n_candidates, "n_units": res.n_units}}
+                "result": None if res is None else {"passes": res.passes, "sampled": res.sampled,
+                                                     "n_candidates": res.n_candidates, "n_units": res.n_units,
+                                                     "n_repaired": res.n_repaired}}
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -342,6 +350,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="5", help="1..5 or 5t; 5 (the largest) is the headline")
     ap.add_argument("--no-sampling", action="store_true")
+    ap.add_argument("--op", default=None, choices=["quantize", "lagrange"],
+                    help="time a standalone operation on the configuration's weights instead of its C-step")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-max-params", type=int, default=200_000_000)

@@ -476,7 +476,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     ctx->ctl = P.ctl;
     ctx->last_stream = stream;
 
-    if (!ctx->occ_stream) ctx->occ_stream = 4;
+    if (!ctx->occ_stream) ctx->occ_stream = 3;
 
     if (ranking) {
         const long long Z = (long long)std::min<double>((double)pl.S, std::max(0.0, std::floor(sparsity * (double)pl.S + 0.5)));
@@ -556,11 +556,17 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         static const char *apply_names[5] = {"k_apply_prune", "k_apply_filter", "k_apply_block", "k_quantize", "k_lagrange"};
         const int pa_ = prof_begin(ctx, apply_names[op], stream);
         switch (op) {
-        case OP_PRUNE: k_apply_linear<M_PRUNE><<<grid, THREADS, 0, stream>>>(Pb); break;
-        case OP_FILTER: k_apply_linear<M_FILTER><<<grid, THREADS, 0, stream>>>(Pb); break;
+        case OP_PRUNE:
+            if (need_h) k_apply_linear<M_PRUNE, true><<<grid, THREADS, 0, stream>>>(Pb);
+            else k_apply_linear<M_PRUNE, false><<<grid, THREADS, 0, stream>>>(Pb);
+            break;
+        case OP_FILTER:
+            if (need_h) k_apply_linear<M_FILTER, true><<<grid, THREADS, 0, stream>>>(Pb);
+            else k_apply_linear<M_FILTER, false><<<grid, THREADS, 0, stream>>>(Pb);
+            break;
         case OP_BLOCK: k_apply_block<<<grid, THREADS, 0, stream>>>(Pb); break;
-        case OP_QUANTIZE: k_apply_linear<M_KEEPALL><<<grid, THREADS, 0, stream>>>(Pb); break;
-        default: k_apply_linear<M_LAGRANGE><<<grid, THREADS, 0, stream>>>(Pb); break;
+        case OP_QUANTIZE: k_apply_linear<M_KEEPALL, true><<<grid, THREADS, 0, stream>>>(Pb); break;
+        default: k_apply_linear<M_LAGRANGE, false><<<grid, THREADS, 0, stream>>>(Pb); break;
         }
         LAUNCH_CHECK(ctx);
         prof_end(ctx, pa_, stream);
@@ -907,7 +913,7 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
         if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     }
     if (pl.n_items_b > 0) {
-        k_apply_linear<M_PRUNE><<<grid_for(pl.n_items_b, 4), THREADS, 0, stream>>>(P);
+        k_apply_linear<M_PRUNE, true><<<grid_for(pl.n_items_b, 3), THREADS, 0, stream>>>(P);
         if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     }
     return CONDENSA_OK;

@@ -219,6 +219,30 @@ __device__ __forceinline__ void form_u4(const float *w, const float *l, float mu
     }
 }
 
+// binary16 bits of four values with the plain hardware conversion; the rare
+// NaN (whose sign must be kept) is patched on a side path.
+__device__ __forceinline__ void half4(const float *x, unsigned short *h)
+{
+#pragma unroll
+    for (int j = 0; j < 4; ++j) h[j] = __half_as_ushort(__float2half_rn(x[j]));
+    const float s = (x[0] + x[1]) + (x[2] + x[3]);
+    if (s != s) {        // a NaN among them (or inf - inf): take the exact route
+#pragma unroll
+        for (int j = 0; j < 4; ++j) h[j] = f32_to_f16_bits(x[j]);
+    }
+}
+
+__device__ __forceinline__ void widen4(const unsigned short *h, const float *x, float *o)
+{
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = __half2float(__ushort_as_half(h[j]));
+    const float s = (x[0] + x[1]) + (x[2] + x[3]);
+    if (s != s) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[j] = f16_bits_to_f32(h[j]);
+    }
+}
+
 // splitmix64 output function: position hash of the sampler.
 __device__ __forceinline__ u64 mix64(u64 z)
 {

@@ -146,9 +146,106 @@ __device__ __forceinline__ void process_linear_item(const Params &P, const Tenso
     }
 }
 
-// Persistent CTAs stride over the linear work items of the whole list.
-template <int MODE>
-__global__ void __launch_bounds__(THREADS) k_apply_linear(Params P)
+// Lean form of the same work for items whose 1024 groups all exist and are 16-byte
+// aligned in every array (elem_item_is_fast): 32-bit indexing inside the item,
+// no per-lane validity, outputs stored group by group.
+template <int MODE, bool H>
+__device__ __forceinline__ void process_linear_item_fast(const Params &P, const TensorDesc &d, long long local,
+                                                         u64 tau_key, u64 tau_id)
+{
+    const long long e_base = 4 * (local * GROUPS_PER_ITEM) - d.pad;
+    const bool has_lam = d.lam != nullptr;
+    const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
+    const bool wr_grad = (P.fuse & FUSE_PENALTY) && d.grad != nullptr;
+    const bool fp16 = (P.fuse & FUSE_FP16) != 0;
+    const float mu = P.mu;
+    const u32 tau32 = tau_key > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)tau_key;     // KEY_NONE keeps nothing
+    const float4 *wp = reinterpret_cast<const float4 *>(d.w + e_base) + threadIdx.x;
+    float4 wv[LIN_UNROLL], lv[LIN_UNROLL], tv[LIN_UNROLL];
+#pragma unroll
+    for (int it = 0; it < LIN_UNROLL; ++it) wv[it] = __ldg(wp + it * THREADS);
+    if (has_lam) {
+        const float4 *lp = reinterpret_cast<const float4 *>(d.lam + e_base) + threadIdx.x;
+#pragma unroll
+        for (int it = 0; it < LIN_UNROLL; ++it) lv[it] = lp[it * THREADS];
+    } else {
+#pragma unroll
+        for (int it = 0; it < LIN_UNROLL; ++it) lv[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (MODE == M_LAGRANGE) {
+        const float4 *tp = reinterpret_cast<const float4 *>(d.theta + e_base) + threadIdx.x;
+#pragma unroll
+        for (int it = 0; it < LIN_UNROLL; ++it) tv[it] = tp[it * THREADS];
+    }
+#pragma unroll
+    for (int it = 0; it < LIN_UNROLL; ++it) {
+        const float w[4] = {wv[it].x, wv[it].y, wv[it].z, wv[it].w};
+        const float l[4] = {lv[it].x, lv[it].y, lv[it].z, lv[it].w};
+        float th[4], ln[4], g[4];
+        u32 m = 0x01010101u;
+        unsigned short h[4] = {0, 0, 0, 0};
+        const u32 eo = 4u * (u32)(it * THREADS + threadIdx.x);        // element offset inside the item
+        if (MODE == M_LAGRANGE) {
+            th[0] = tv[it].x; th[1] = tv[it].y; th[2] = tv[it].z; th[3] = tv[it].w;
+        } else {
+            float u[4];
+            form_u4(w, l, mu, has_lam, u);
+            bool keep[4] = {true, true, true, true};
+            if (MODE == M_PRUNE) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const u32 key = __float_as_uint(u[j]) & 0x7FFFFFFFu;
+                    keep[j] = key > tau32;
+                    if (key == tau32 && tau_key <= 0x7FFFFFFFull)       // tie with the threshold: the index decides
+                        keep[j] = (u64)(d.elem_prefix + e_base) + eo + j <= tau_id;
+                }
+            } else if (MODE == M_FILTER) {
+                if (d.ranked) {
+                    const long long e0 = e_base + eo;
+                    long long f = (d.numel < 0x7FFFFFFFll) ? (long long)((u32)e0 / (u32)d.d1) : e0 / d.d1;
+                    long long r = e0 - f * d.d1;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (r >= d.d1) { r -= d.d1; ++f; while (r >= d.d1) { r -= d.d1; ++f; } }
+                        const u64 sid = (u64)(d.unit_prefix + f);
+                        keep[j] = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
+                        ++r;
+                    }
+                }
+            }
+            m = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                th[j] = keep[j] ? u[j] : 0.0f;
+                m |= keep[j] ? (1u << (8 * j)) : 0u;
+            }
+            if (H) {
+                half4(th, h);
+                if (fp16) widen4(h, th, th);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float p = __fmul_rn(mu, __fsub_rn(w[j], th[j]));
+            ln[j] = upd ? __fsub_rn(l[j], p) : l[j];
+            g[j] = __fsub_rn(p, ln[j]);
+        }
+        const long long go = it * THREADS + threadIdx.x;
+        if (MODE != M_LAGRANGE) {
+            reinterpret_cast<float4 *>(d.theta + e_base)[go] = make_float4(th[0], th[1], th[2], th[3]);
+            if (d.mask) reinterpret_cast<u32 *>(d.mask + e_base)[go] = m;
+            if (H && d.theta_h) reinterpret_cast<uint2 *>(d.theta_h + e_base)[go] =
+                make_uint2((u32)h[0] | ((u32)h[1] << 16), (u32)h[2] | ((u32)h[3] << 16));
+        }
+        if (upd) reinterpret_cast<float4 *>(d.lam + e_base)[go] = make_float4(ln[0], ln[1], ln[2], ln[3]);
+        if (wr_grad) reinterpret_cast<float4 *>(d.grad + e_base)[go] = make_float4(g[0], g[1], g[2], g[3]);
+    }
+}
+
+// Persistent CTAs stride over the linear work items of the whole list. H: the
+// binary16 bits are needed (fp16 fuse or a theta_h output).
+template <int MODE, bool H>
+__global__ void __launch_bounds__(THREADS, 3) k_apply_linear(Params P)
 {
     u64 tau_key = 0, tau_id = 0;
     if (MODE == M_PRUNE || MODE == M_FILTER) {
@@ -156,10 +253,19 @@ __global__ void __launch_bounds__(THREADS) k_apply_linear(Params P)
         tau_key = P.ctl->tau_key;
         tau_id = P.ctl->tau_id;
     }
+    long long t_first = 0, t_end = -1;
+    TensorDesc d;
+    d.numel = 0; d.pad = 0; d.vec_ok = 0;
     for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-        const int t = find_tensor(P.item_prefix, P.T, item);
-        const TensorDesc d = P.td[t];
-        process_linear_item<MODE>(P, d, item - P.item_prefix[t], tau_key, tau_id);
+        if (item >= t_end) {
+            const int t = find_tensor(P.item_prefix, P.T, item);
+            d = P.td[t];
+            t_first = P.item_prefix[t];
+            t_end = P.item_prefix[t + 1];
+        }
+        const long long local = item - t_first;
+        if (elem_item_is_fast(d, local)) process_linear_item_fast<MODE, H>(P, d, local, tau_key, tau_id);
+        else process_linear_item<MODE>(P, d, local, tau_key, tau_id);
     }
 }
 
