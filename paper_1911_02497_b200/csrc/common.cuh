@@ -137,7 +137,10 @@ __host__ __device__ inline bool block_item_is_fast(const TensorDesc &d, long lon
 // u = w - lambda / mu as two IEEE fp32 operations.
 __device__ __forceinline__ float form_u(float w, float lam, float mu, bool has_lam)
 {
-    return has_lam ? __fsub_rn(w, __fdiv_rn(lam, mu)) : w;
+    // lambda == +0 gives u = w bit for bit (w - (+0) is w for every w, -0 included); taking
+    // that branch also keeps the IEEE division off its slow path for a zero numerator
+    if (!has_lam || __float_as_uint(lam) == 0u) return w;
+    return __fsub_rn(w, __fdiv_rn(lam, mu));
 }
 
 // binary32 -> binary16 bits, round to nearest even; NaN -> quiet NaN, sign kept.

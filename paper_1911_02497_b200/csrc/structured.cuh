@@ -86,9 +86,11 @@ __global__ void __launch_bounds__(THREADS) k_apply_block(Params P)
 }
 
 // Filter norms, step 1: one warp per segment of SEG elements of one filter.
-// Lane l adds elements l, l+32, ... of the segment in that order, then the 32
-// lane sums are combined by a fixed butterfly; the value depends only on the
-// segment's contents and length, never on where the filter sits.
+// Lane l adds the elements of the 4-element groups l, l+32, l+64, ... of the
+// segment, each group in index order, then the 32 lane sums are combined by a
+// fixed butterfly; the value depends only on the segment's contents and length,
+// never on where the filter sits or how it is aligned (the 128-bit and the
+// scalar path add in the same order).
 // Work items: (filter, segment) pairs of ranked tensors, WARPS per CTA step.
 __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
 {
@@ -104,27 +106,60 @@ __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
         const long long f = local / nseg, sgm = local - f * nseg;
         const long long j0 = sgm * SEG;
         const long long j1 = (j0 + SEG < d.d1) ? j0 + SEG : d.d1;
-        const float *__restrict__ wp = d.w + f * d.d1;
-        const float *lp = d.lam ? d.lam + f * d.d1 : nullptr;
+        const float *__restrict__ wp = d.w + f * d.d1 + j0;
+        const float *lp = d.lam ? d.lam + f * d.d1 + j0 : nullptr;
         const bool has_lam = lp != nullptr;
+        const int n = (int)(j1 - j0);                    // elements in this segment
+        const bool vec = ((uintptr_t)wp % 16 == 0) && (!has_lam || (uintptr_t)lp % 16 == 0);
         double acc = 0.0;
-        long long j = j0 + lane;
-        for (; j + 7 * 32 < j1; j += 8 * 32) {
-            float wv[8], lv[8];
+        const int ngroups = n >> 2;                      // full groups of four
+        if (vec) {
+            int gidx = lane;
+            for (; gidx + 3 * 32 < ngroups; gidx += 4 * 32) {
+                float4 wv[4], lv[4];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                wv[q] = __ldg(wp + j + q * 32);
-                lv[q] = has_lam ? lp[j + q * 32] : 0.0f;
+                for (int q = 0; q < 4; ++q) {
+                    wv[q] = __ldg(reinterpret_cast<const float4 *>(wp) + gidx + q * 32);
+                    lv[q] = has_lam ? reinterpret_cast<const float4 *>(lp)[gidx + q * 32] : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float w4[4] = {wv[q].x, wv[q].y, wv[q].z, wv[q].w};
+                    const float l4[4] = {lv[q].x, lv[q].y, lv[q].z, lv[q].w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const double x = (double)form_u(w4[c], l4[c], P.mu, has_lam);
+                        acc = __fma_rn(x, x, acc);
+                    }
+                }
             }
+            for (; gidx < ngroups; gidx += 32) {
+                const float4 a = __ldg(reinterpret_cast<const float4 *>(wp) + gidx);
+                const float4 b = has_lam ? reinterpret_cast<const float4 *>(lp)[gidx] : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float w4[4] = {a.x, a.y, a.z, a.w};
+                const float l4[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const double x = (double)form_u(wv[q], lv[q], P.mu, has_lam);
-                acc = __fma_rn(x, x, acc);
+                for (int c = 0; c < 4; ++c) {
+                    const double x = (double)form_u(w4[c], l4[c], P.mu, has_lam);
+                    acc = __fma_rn(x, x, acc);
+                }
+            }
+        } else {
+            for (int gidx = lane; gidx < ngroups; gidx += 32) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int j = 4 * gidx + c;
+                    const double x = (double)form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam);
+                    acc = __fma_rn(x, x, acc);
+                }
             }
         }
-        for (; j < j1; j += 32) {
-            const double x = (double)form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam);
-            acc = __fma_rn(x, x, acc);
+        // the last, incomplete group belongs to the lane whose turn it is
+        if ((n & 3) && lane == (ngroups & 31)) {
+            for (int j = 4 * ngroups; j < n; ++j) {
+                const double x = (double)form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam);
+                acc = __fma_rn(x, x, acc);
+            }
         }
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (lane == 0) P.partial[item] = acc;
