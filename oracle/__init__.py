@@ -52,6 +52,17 @@ class _Result(C.Structure):
                 ("n_tie", C.c_int64), ("n_tie_kept", C.c_int64), ("tau_norm", C.c_float)]
 
 
+class _OptTensor(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("theta", C.c_void_p), ("lam", C.c_void_p), ("grad", C.c_void_p),
+                ("buf1", C.c_void_p), ("buf2", C.c_void_p), ("numel", C.c_int64)]
+
+
+class _Opt(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("lr", C.c_float), ("momentum", C.c_float),
+                ("weight_decay", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
+                ("eps", C.c_float), ("step", C.c_int64)]
+
+
 _lib = None
 
 
@@ -82,6 +93,8 @@ def lib():
                                       C.c_int, C.c_uint, C.c_void_p]
         L.orc_cstep_quantize.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint]
         L.orc_lagrange_update.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint]
+        assert L.orc_sizeof_opt_tensor() == C.sizeof(_OptTensor) and L.orc_sizeof_opt() == C.sizeof(_Opt)
+        L.orc_lstep_update.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_void_p]
         if not L.orc_denormals_ok():
             raise RuntimeError("subnormal fp32 arithmetic is flushed in this process; "
                                "the oracle's results would not be IEEE")
@@ -258,3 +271,29 @@ def run_config(ws) -> Outputs:
     if ws.op == "block":
         return cstep_block(ws.w, ws.lam, ws.sparsity, ws.mu, ws.block, ws.fuse)
     raise ValueError(ws.op)
+
+
+def lstep_update(ws, thetas, lams, grads, buf1, buf2, mu: float, kind: str = "sgd", lr: float = 0.1,
+                 momentum: float = 0.9, weight_decay: float = 0.0, beta1: float = 0.9,
+                 beta2: float = 0.999, eps: float = 1e-8, step: int = 1):
+    """One optimizer step with the penalty gradient folded in. Returns new (w, buf1, buf2) lists;
+    the inputs are left untouched. ``buf1``/``buf2`` entries may be None where unused."""
+    T = len(ws)
+    tab = (_OptTensor * max(T, 1))()
+    keep, w_out, b1_out, b2_out = [], [], [], []
+    for t in range(T):
+        w = np.ascontiguousarray(ws[t], dtype=np.float32).copy()
+        th = np.ascontiguousarray(thetas[t], dtype=np.float32)
+        lam = None if lams is None or lams[t] is None else np.ascontiguousarray(lams[t], dtype=np.float32)
+        g = np.ascontiguousarray(grads[t], dtype=np.float32)
+        b1 = None if buf1 is None or buf1[t] is None else np.ascontiguousarray(buf1[t], dtype=np.float32).copy()
+        b2 = None if buf2 is None or buf2[t] is None else np.ascontiguousarray(buf2[t], dtype=np.float32).copy()
+        keep += [th, lam, g]
+        e = tab[t]
+        e.w, e.theta, e.lam, e.grad, e.buf1, e.buf2 = _ptr(w), _ptr(th), _ptr(lam), _ptr(g), _ptr(b1), _ptr(b2)
+        e.numel = w.size
+        w_out.append(w); b1_out.append(b1); b2_out.append(b2)
+    o = _Opt({"sgd": 0, "adam": 1}[kind], lr, momentum, weight_decay, beta1, beta2, eps, step)
+    rc = lib().orc_lstep_update(tab, T, C.c_float(mu), C.byref(o))
+    assert rc == 0
+    return w_out, b1_out, b2_out

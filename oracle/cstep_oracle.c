@@ -418,6 +418,86 @@ int orc_lagrange_update(const orc_tensor *ts, int32_t T, float mu, unsigned fuse
     return 0;
 }
 
+/* ---- L step: penalty gradient folded into the optimizer update ------------
+ * The L step trains w on the loss plus the quadratic penalty (Section 3.3, "a
+ * learning (L) step which trains the uncompressed model but with a quadratic
+ * regularization term"), with SGD momentum 0.9 for the CNNs and Adam for the
+ * LSTM (Evaluation, L-C optimizer settings). Every minibatch adds the penalty
+ * gradient mu (w - theta) - lambda to the loss gradient and takes one
+ * optimizer step; written here one fp32 operation at a time:
+ *   d = w - theta; p = mu d; g1 = p - lambda; g = grad + g1; [g = g + wd w]
+ *   SGD : b' = momentum b + g;  w' = w - lr b'
+ *   Adam: m' = beta1 m + (1-beta1) g;  v' = beta2 v + (1-beta2) g g;
+ *         w' = w - (lr / (1-beta1^t)) * m' / (sqrt(v') / sqrt(1-beta2^t) + eps)
+ * (the usual SGD-with-momentum and Adam recurrences, bias correction included). */
+typedef struct {
+    float *w;              /* in/out */
+    const float *theta;
+    const float *lambda;   /* may be NULL */
+    const float *grad;     /* loss gradient */
+    float *buf1;           /* SGD momentum buffer / Adam first moment, in/out   */
+    float *buf2;           /* Adam second moment, in/out                         */
+    int64_t numel;
+} orc_opt_tensor;
+
+typedef struct {
+    int32_t kind;          /* 0 = SGD with momentum, 1 = Adam */
+    float lr, momentum, weight_decay, beta1, beta2, eps;
+    int64_t step;          /* Adam: 1-based step number t */
+} orc_opt;
+
+int orc_lstep_update(const orc_opt_tensor *ts, int32_t T, float mu, const orc_opt *o)
+{
+    volatile float c1 = 1.0f - o->beta1, c2 = 1.0f - o->beta2;
+    double bc1 = 1.0 - pow((double)o->beta1, (double)o->step);
+    double bc2 = 1.0 - pow((double)o->beta2, (double)o->step);
+    float step_size = (float)((double)o->lr / bc1);
+    float sqrt_bc2 = (float)sqrt(bc2);
+    for (int32_t t = 0; t < T; ++t) {
+        const orc_opt_tensor *x = &ts[t];
+        for (int64_t i = 0; i < x->numel; ++i) {
+            volatile float d = x->w[i] - x->theta[i];
+            volatile float p = mu * d;
+            volatile float g1 = x->lambda ? p - x->lambda[i] : p;
+            volatile float g = x->grad[i] + g1;
+            if (o->weight_decay != 0.0f) {
+                volatile float wd = o->weight_decay * x->w[i];
+                g = g + wd;
+            }
+            if (o->kind == 0) {
+                volatile float b = g;
+                if (x->buf1) {
+                    volatile float a = o->momentum * x->buf1[i];
+                    b = a + g;
+                    x->buf1[i] = b;
+                }
+                volatile float s = o->lr * b;
+                x->w[i] = x->w[i] - s;
+            } else {
+                volatile float a = o->beta1 * x->buf1[i];
+                volatile float b = c1 * g;
+                volatile float m = a + b;
+                volatile float a2 = o->beta2 * x->buf2[i];
+                volatile float gg = g * g;
+                volatile float b2 = c2 * gg;
+                volatile float v = a2 + b2;
+                x->buf1[i] = m;
+                x->buf2[i] = v;
+                volatile float sq = sqrtf(v);
+                volatile float dn = sq / sqrt_bc2;
+                dn = dn + o->eps;
+                volatile float q = m / dn;
+                volatile float s = step_size * q;
+                x->w[i] = x->w[i] - s;
+            }
+        }
+    }
+    return 0;
+}
+
+unsigned orc_sizeof_opt_tensor(void) { return (unsigned)sizeof(orc_opt_tensor); }
+unsigned orc_sizeof_opt(void) { return (unsigned)sizeof(orc_opt); }
+
 /* 1 when subnormal fp32 arithmetic is intact in this process (no flush to
  * zero, no denormals-are-zero), which every function above relies on. */
 int orc_denormals_ok(void)

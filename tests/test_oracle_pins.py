@@ -421,3 +421,63 @@ def test_configuration_shapes():
     assert sum(int(np.prod(s)) for s in W.lstm_lm_shapes(tied=True)) == 85941000
     nb = sum(-(-s[0] // 4) * -(-s[1] // 4) for s in W.lstm_lm_shapes() if len(s) == 2)
     assert nb == 8490000
+
+
+# ---------------------------------------------------------------- L-step update
+def test_lstep_sgd_hand_case_and_torch_sgd():
+    import torch
+    # exactly representable numbers: mu (w - theta) - lambda = 0.5*(1-0.25) - 0.125 = 0.25; g = 1 + 0.25
+    w, th, lam, g, b = (np.array([v], np.float32) for v in (1.0, 0.25, 0.125, 1.0, 2.0))
+    wn, b1, _ = oracle.lstep_update([w], [th], [lam], [g], [b], None, 0.5, "sgd", lr=0.5, momentum=0.5)
+    assert b1[0].tolist() == [2.25] and wn[0].tolist() == [-0.125]
+    # against torch.optim.SGD fed with the same total gradient (an independent implementation)
+    rng = np.random.default_rng(3)
+    n = 5000
+    w = rng.standard_normal(n).astype(np.float32); th = np.where(np.abs(w) > 1, w, 0).astype(np.float32)
+    lam = (rng.standard_normal(n) * 0.01).astype(np.float32); g = rng.standard_normal(n).astype(np.float32)
+    b = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    mu = 1e-2
+    wn, b1, _ = oracle.lstep_update([w], [th], [lam], [g], [b], None, mu, "sgd", lr=0.1, momentum=0.9,
+                                    weight_decay=1e-4)
+    p = torch.nn.Parameter(torch.from_numpy(w.copy()))
+    opt = torch.optim.SGD([p], lr=0.1, momentum=0.9, weight_decay=1e-4)
+    opt.state[p]["momentum_buffer"] = torch.from_numpy(b.copy())
+    p.grad = torch.from_numpy(g) + (np.float32(mu) * (torch.from_numpy(w) - torch.from_numpy(th)) - torch.from_numpy(lam))
+    opt.step()
+    assert np.allclose(wn[0], p.detach().numpy(), rtol=2e-6, atol=1e-7)
+    assert np.allclose(b1[0], opt.state[p]["momentum_buffer"].numpy(), rtol=2e-6, atol=1e-7)
+    # theta == w and lambda == 0: the penalty vanishes and the step is plain SGD
+    wn2, _, _ = oracle.lstep_update([w], [w.copy()], [np.zeros_like(w)], [g], [np.zeros_like(w)], None, mu, "sgd",
+                                    lr=0.1, momentum=0.9)
+    assert np.array_equal(wn2[0].view(np.uint32), (w - np.float32(0.1) * g).astype(np.float32).view(np.uint32))
+
+
+def test_lstep_adam_against_torch_adam():
+    import torch
+    rng = np.random.default_rng(4)
+    n = 5000
+    w = rng.standard_normal(n).astype(np.float32); th = np.where(np.abs(w) > 1, w, 0).astype(np.float32)
+    lam = (rng.standard_normal(n) * 0.01).astype(np.float32); g = rng.standard_normal(n).astype(np.float32)
+    m = (rng.standard_normal(n) * 0.1).astype(np.float32); v = (rng.random(n) * 0.1).astype(np.float32)
+    mu, step = 1e-3, 7
+    wn, m1, v1 = oracle.lstep_update([w], [th], [lam], [g], [m], [v], mu, "adam", lr=1e-4, beta1=0.9,
+                                     beta2=0.999, eps=1e-8, step=step)
+    p = torch.nn.Parameter(torch.from_numpy(w.copy()))
+    # torch keeps its hyper-parameters in double: hand it the float values the oracle works with
+    f32 = lambda x: float(np.float32(x))
+    opt = torch.optim.Adam([p], lr=f32(1e-4), betas=(f32(0.9), f32(0.999)), eps=f32(1e-8))
+    opt.state[p]["step"] = torch.tensor(float(step - 1))
+    opt.state[p]["exp_avg"] = torch.from_numpy(m.copy())
+    opt.state[p]["exp_avg_sq"] = torch.from_numpy(v.copy())
+    p.grad = torch.from_numpy(g) + (np.float32(mu) * (torch.from_numpy(w) - torch.from_numpy(th)) - torch.from_numpy(lam))
+    opt.step()
+    # torch forms the first moment as m + (1-b1)(g - m): same value, other rounding (operands are O(1))
+    assert np.allclose(m1[0], opt.state[p]["exp_avg"].numpy(), rtol=2e-6, atol=3e-7)
+    assert np.allclose(v1[0], opt.state[p]["exp_avg_sq"].numpy(), rtol=2e-6, atol=3e-8)
+    assert np.allclose(wn[0], p.detach().numpy(), rtol=1e-6, atol=1e-7)
+    assert 1e-5 < np.abs(wn[0] - w).max() < 1e-3        # moved by about lr
+    # closed form at step 1 from zero moments: m_hat = g, v_hat = g^2, so w moves by lr * sign(g) (eps aside)
+    z = np.zeros(n, np.float32)
+    wn, _, _ = oracle.lstep_update([w], [w.copy()], [z], [g], [z], [z], mu, "adam", lr=1e-3, step=1)
+    big = np.abs(g) > 1e-3
+    assert np.allclose((w - wn[0])[big], 1e-3 * np.sign(g[big]), rtol=1e-4)
