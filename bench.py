@@ -178,6 +178,47 @@ def run_reference(args):
     return 0
 
 
+def run_lstep(args, ws, ctx, local, world):
+    """Standalone timing of the fused penalty-gradient + optimizer step (not the headline)."""
+    import torch
+    from paper_1911_02497_b200 import cstep
+    dev = torch.device("cuda", local)
+    adam = args.op == "lstep_adam"
+    mk = lambda a: torch.from_numpy(np.ascontiguousarray(a).reshape(-1)).to(dev)
+    w = [mk(a) for a in ws.w]
+    th = [torch.where(t.abs() > 0.05, t, torch.zeros_like(t)) for t in w]
+    lam = [mk(a) for a in ws.lam]
+    grad = [torch.randn_like(t) for t in w]
+    b1 = [torch.zeros_like(t) for t in w]
+    b2 = [torch.zeros_like(t) for t in w] if adam else None
+    tab = cstep.opt_table(w, th, lam, grad, b1, b2)
+    N = ws.numel
+    bpp = 36 if adam else 28             # read w, theta, lambda, grad, moments; write w, moments
+    kw = dict(kind="adam", lr=1e-4, step=3) if adam else dict(kind="sgd", lr=0.1, momentum=0.9)
+    for _ in range(max(args.warmup, 3)):
+        ctx.lstep_update(tab, len(w), ws.mu, **kw)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = ctx.launch_count()
+    a.record()
+    for _ in range(args.steps):
+        ctx.lstep_update(tab, len(w), ws.mu, **kw)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    peak, src = measured_peak()
+    gbs = N * bpp / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "lstep_params_per_s", "value": N / (ms * 1e-3), "unit": "params/s", "n_gpus": world,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": "%s on %s" % (args.op, workload_name(ws))},
+                      "gpu_launches": ctx.launch_count() - l0,
+                      "roofline": {"bound": "hbm", "kernel": "k_" + args.op, "achieved": gbs, "peak": peak,
+                                   "unit": "GB/s", "frac": gbs / peak, "traffic": None, "peak_source": src,
+                                   "algorithmic_bytes_per_launch": N * bpp}}))
+    return 0
+
+
 # --------------------------------------------------------------------------- CUDA arm
 def run_ours(args):
     import torch
@@ -207,6 +248,8 @@ def run_ours(args):
     bpp = algorithmic_bytes_per_param(ws.fuse)
     if args.op == "lagrange":
         bpp = 4 + 4 + 4 + 4 + 4          # read w, theta, lambda; write lambda, g
+    if args.op in ("lstep_sgd", "lstep_adam"):
+        return run_lstep(args, ws, ctx, local, world)
     stream = torch.cuda.current_stream()
 
     def step():
@@ -350,7 +393,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="5", help="1..5 or 5t; 5 (the largest) is the headline")
     ap.add_argument("--no-sampling", action="store_true")
-    ap.add_argument("--op", default=None, choices=["quantize", "lagrange"],
+    ap.add_argument("--op", default=None, choices=["quantize", "lagrange", "lstep_sgd", "lstep_adam"],
                     help="time a standalone operation on the configuration's weights instead of its C-step")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)

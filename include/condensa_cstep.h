@@ -170,6 +170,40 @@ CONDENSA_API int condensa_cstep_quantize(condensa_ctx *ctx, const condensa_tenso
 CONDENSA_API int condensa_cstep_lagrange_update(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
                                    float mu, unsigned fuse, void *stream);
 
+/* L step helper: the penalty gradient folded into one optimizer step, in a
+ * single pass over the list (Section 3.3: the L step trains w "with a quadratic
+ * regularization term"; Evaluation, L-C optimizer settings: SGD with momentum
+ * 0.9 for the CNNs, Adam for the LSTM; it runs on every minibatch). With `grad`
+ * the loss gradient of the minibatch, per element and in this order of single
+ * fp32 operations:
+ *     d = w - theta;  p = mu*d;  g1 = p - lambda;  g = grad + g1;  [g = g + weight_decay*w]
+ *   SGD :  b' = momentum*b + g;                     w' = w - lr*b'
+ *   Adam:  m' = beta1*m + (1-beta1)*g;  v' = beta2*v + (1-beta2)*(g*g);
+ *          w' = w - (lr/(1-beta1^step)) * ( m' / ( sqrt(v')/sqrt(1-beta2^step) + eps ) )
+ * (1-beta in fp32; the two bias corrections in double, rounded once to fp32.)
+ * w, buf1 (b or m) and buf2 (v) are updated in place; theta, lambda (NULL: 0) and
+ * grad are read. buf1 may be NULL for SGD with momentum == 0. All DEVICE pointers. */
+typedef struct {
+    float *w;
+    const float *theta;
+    const float *lambda;
+    const float *grad;
+    float *buf1;
+    float *buf2;
+    int64_t numel;
+} condensa_opt_tensor;
+
+enum { CONDENSA_OPT_SGD = 0, CONDENSA_OPT_ADAM = 1 };
+
+typedef struct {
+    int32_t kind;          /* CONDENSA_OPT_SGD or CONDENSA_OPT_ADAM */
+    float lr, momentum, weight_decay, beta1, beta2, eps;
+    int64_t step;          /* Adam: 1-based step number */
+} condensa_opt;
+
+CONDENSA_API int condensa_lstep_update(condensa_ctx *ctx, const condensa_opt_tensor *tensors, int T,
+                                       float mu, const condensa_opt *opt, void *stream);
+
 /* Operation selector for condensa_cstep_host(). */
 enum { CONDENSA_OP_PRUNE = 0, CONDENSA_OP_FILTER = 1, CONDENSA_OP_BLOCK = 2,
        CONDENSA_OP_QUANTIZE = 3, CONDENSA_OP_LAGRANGE = 4 };

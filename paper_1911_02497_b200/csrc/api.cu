@@ -17,6 +17,7 @@
 #include "fused.cuh"
 #include "fused_fast.cuh"
 #include "sample.cuh"
+#include "lstep.cuh"
 
 using namespace cs;
 
@@ -271,6 +272,8 @@ int ensure_workspace(condensa_ctx *ctx, size_t bytes, cudaStream_t stream)
     ctx->ws_bytes = 0;
     ctx->last_upload.clear();
     ctx->last_upload_dst = nullptr;
+    ctx->has_result = false;       // the record of an earlier call lived in the old workspace
+    ctx->ctl = nullptr;
     const size_t want = align_up(bytes + bytes / 4, 1 << 20);
     cudaError_t e = cudaMalloc((void **)&ctx->ws, want);
     if (e != cudaSuccess) {
@@ -286,6 +289,8 @@ int ensure_workspace(condensa_ctx *ctx, size_t bytes, cudaStream_t stream)
 
 // Copies the descriptor table and both prefix arrays to the workspace unless
 // the device already holds exactly these bytes.
+int upload_image(condensa_ctx *ctx, std::vector<char> &img, char *dst, cudaStream_t stream);
+
 int upload_desc(condensa_ctx *ctx, const Plan &pl, int T, char *dst, size_t bytes, cudaStream_t stream)
 {
     std::vector<char> img(bytes);
@@ -295,6 +300,13 @@ int upload_desc(condensa_ctx *ctx, const Plan &pl, int T, char *dst, size_t byte
     if (!pl.edge_items.empty()) memcpy(p, pl.edge_items.data(), sizeof(long long) * pl.edge_items.size());
     p += sizeof(long long) * pl.edge_items.size();
     memcpy(p, pl.prefix_b.data(), sizeof(long long) * (size_t)(T + 1));
+    return upload_image(ctx, img, dst, stream);
+}
+
+// Copies `img` to `dst` through the pinned staging area unless the device already holds these bytes there.
+int upload_image(condensa_ctx *ctx, std::vector<char> &img, char *dst, cudaStream_t stream)
+{
+    const size_t bytes = img.size();
     if (ctx->last_upload_dst == dst && ctx->last_upload == img) return CONDENSA_OK;
     CU_TRY(ctx, cudaEventSynchronize(ctx->stage_ev));    // the previous upload has left the staging area
     if (bytes > ctx->h_stage_bytes) {
@@ -669,6 +681,105 @@ int condensa_cstep_lagrange_update(condensa_ctx *ctx, const condensa_tensor *ten
     if (!(fuse & (CONDENSA_FUSE_LAMBDA | CONDENSA_FUSE_PENALTY)))
         return fail(ctx, CONDENSA_ERR_INVALID_ARG, "nothing to do: set FUSE_LAMBDA and/or FUSE_PENALTY");
     return run_op(ctx, OP_LAGRANGE, tensors, T, 0.0, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_lstep_update(condensa_ctx *ctx, const condensa_opt_tensor *ts, int T, float mu,
+                          const condensa_opt *opt, void *stream_)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!ts || T <= 0 || T > (1 << 20) || !opt) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor list or optimizer is NULL");
+    if (!(mu >= 0.0f) || !std::isfinite(mu)) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "mu must be finite and >= 0");
+    if (opt->kind != CONDENSA_OPT_SGD && opt->kind != CONDENSA_OPT_ADAM) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "unknown optimizer kind");
+    if (!std::isfinite(opt->lr) || !std::isfinite(opt->momentum) || !std::isfinite(opt->weight_decay))
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "optimizer parameters must be finite");
+    if (opt->kind == CONDENSA_OPT_ADAM &&
+        (!(opt->beta1 >= 0.0f && opt->beta1 < 1.0f) || !(opt->beta2 >= 0.0f && opt->beta2 < 1.0f) || opt->step < 1 || !(opt->eps >= 0.0f)))
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "Adam needs 0 <= beta < 1, eps >= 0 and step >= 1");
+    std::vector<Interval> iv;
+    std::vector<OptDesc> td(T);
+    std::vector<long long> prefix(T + 1, 0);
+    for (int t = 0; t < T; ++t) {
+        const condensa_opt_tensor &x = ts[t];
+        if (x.numel < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: numel < 0", t);
+        OptDesc d;
+        memset(&d, 0, sizeof(d));
+        d.numel = x.numel;
+        if (x.numel > 0) {
+            if (!x.w || !x.theta || !x.grad) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: w, theta and grad must not be NULL", t);
+            const bool need_b1 = opt->kind == CONDENSA_OPT_ADAM || opt->momentum != 0.0f;
+            if (need_b1 && !x.buf1) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: buf1 is NULL", t);
+            if (opt->kind == CONDENSA_OPT_ADAM && !x.buf2) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: buf2 is NULL", t);
+            const uintptr_t ptrs[6] = {(uintptr_t)x.w, (uintptr_t)x.theta, (uintptr_t)x.lambda, (uintptr_t)x.grad,
+                                       (uintptr_t)(need_b1 ? x.buf1 : nullptr), (uintptr_t)(opt->kind == CONDENSA_OPT_ADAM ? x.buf2 : nullptr)};
+            bool ok = true;
+            for (int i = 0; i < 6; ++i) {
+                if (ptrs[i] % 4) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor %d: pointer not 4-byte aligned", t);
+                if (ptrs[i] && ptrs[i] % 16 != ptrs[0] % 16) ok = false;
+            }
+            const size_t n4 = 4 * (size_t)x.numel;
+            iv.push_back({ptrs[0], ptrs[0] + n4, true});
+            iv.push_back({ptrs[1], ptrs[1] + n4, false});
+            if (ptrs[2]) iv.push_back({ptrs[2], ptrs[2] + n4, false});
+            iv.push_back({ptrs[3], ptrs[3] + n4, false});
+            if (ptrs[4]) iv.push_back({ptrs[4], ptrs[4] + n4, true});
+            if (ptrs[5]) iv.push_back({ptrs[5], ptrs[5] + n4, true});
+            d.w = x.w; d.theta = x.theta; d.lam = x.lambda; d.grad = x.grad;
+            d.buf1 = need_b1 ? x.buf1 : nullptr;
+            d.buf2 = opt->kind == CONDENSA_OPT_ADAM ? x.buf2 : nullptr;
+            d.vec_ok = ok ? 1 : 0;
+            d.pad = ok ? (int)((ptrs[0] % 16) / 4) : 0;
+        }
+        td[t] = d;
+        const long long groups = (x.numel + d.pad + 3) / 4;
+        prefix[t + 1] = prefix[t] + (groups + GROUPS_PER_ITEM - 1) / GROUPS_PER_ITEM;
+    }
+    std::sort(iv.begin(), iv.end(), [](const Interval &a, const Interval &b) { return a.lo < b.lo; });
+    uintptr_t reach = 0, reach_out = 0;
+    for (size_t i = 0; i < iv.size(); ++i) {
+        if (iv[i].lo < reach_out || (iv[i].out && iv[i].lo < reach))
+            return fail(ctx, CONDENSA_ERR_INVALID_ARG, "an in/out buffer overlaps another buffer of the call");
+        reach = std::max(reach, iv[i].hi);
+        if (iv[i].out) reach_out = std::max(reach_out, iv[i].hi);
+    }
+    if (prefix[T] == 0) return CONDENSA_OK;
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    // descriptor image in the same workspace slot the C-step calls use
+    Plan none;
+    none.cap = 1;
+    const Layout L = make_layout(0, none, false, false);
+    const size_t bytes = sizeof(OptDesc) * (size_t)T + sizeof(long long) * (size_t)(T + 1);
+    int rc = ensure_workspace(ctx, L.desc + align_up(bytes, 256), stream);
+    if (rc) return rc;
+    std::vector<char> img(bytes);
+    memcpy(img.data(), td.data(), sizeof(OptDesc) * (size_t)T);
+    memcpy(img.data() + sizeof(OptDesc) * (size_t)T, prefix.data(), sizeof(long long) * (size_t)(T + 1));
+    rc = upload_image(ctx, img, ctx->ws + L.desc, stream);
+    if (rc) return rc;
+    OptParams P;
+    memset(&P, 0, sizeof(P));
+    P.td = (const OptDesc *)(ctx->ws + L.desc);
+    P.item_prefix = (const long long *)(ctx->ws + L.desc + sizeof(OptDesc) * (size_t)T);
+    P.T = T;
+    P.n_items = prefix[T];
+    P.mu = mu; P.lr = opt->lr; P.momentum = opt->momentum; P.wd = opt->weight_decay;
+    P.beta1 = opt->beta1; P.beta2 = opt->beta2; P.eps = opt->eps;
+    if (opt->kind == CONDENSA_OPT_ADAM) {
+        volatile float c1 = 1.0f - opt->beta1, c2 = 1.0f - opt->beta2;
+        P.c1 = c1; P.c2 = c2;
+        const double bc1 = 1.0 - std::pow((double)opt->beta1, (double)opt->step);
+        const double bc2 = 1.0 - std::pow((double)opt->beta2, (double)opt->step);
+        P.step_size = (float)((double)opt->lr / bc1);
+        P.sqrt_bc2 = (float)std::sqrt(bc2);
+    }
+    ctx->last_stream = stream;
+    const int grid = stream_grid(ctx, P.n_items, 3);
+    const int pa_ = prof_begin(ctx, opt->kind == CONDENSA_OPT_ADAM ? "k_lstep_adam" : "k_lstep_sgd", stream);
+    if (opt->kind == CONDENSA_OPT_ADAM) k_lstep<OPT_ADAM><<<grid, THREADS, 0, stream>>>(P);
+    else k_lstep<OPT_SGD><<<grid, THREADS, 0, stream>>>(P);
+    LAUNCH_CHECK(ctx);
+    prof_end(ctx, pa_, stream);
+    return CONDENSA_OK;
 }
 
 int condensa_cstep_host(condensa_ctx *ctx, int op, const condensa_tensor *tensors, int T,

@@ -25,7 +25,7 @@ EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "conde
            "condensa_cstep_block", "condensa_cstep_quantize", "condensa_cstep_lagrange_update",
            "condensa_cstep_host", "condensa_get_result", "condensa_launch_count",
            "condensa_last_error", "condensa_profile_enable", "condensa_profile_read",
-           "condensa_cstep_prune_noalloc"]
+           "condensa_cstep_prune_noalloc", "condensa_lstep_update"]
 
 
 class CondensaError(RuntimeError):
@@ -51,6 +51,22 @@ class Result(C.Structure):
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class OptTensor(C.Structure):
+    """Mirror of ``condensa_opt_tensor``."""
+    _fields_ = [("w", C.c_void_p), ("theta", C.c_void_p), ("lam", C.c_void_p), ("grad", C.c_void_p),
+                ("buf1", C.c_void_p), ("buf2", C.c_void_p), ("numel", C.c_int64)]
+
+
+class Opt(C.Structure):
+    """Mirror of ``condensa_opt``."""
+    _fields_ = [("kind", C.c_int32), ("lr", C.c_float), ("momentum", C.c_float),
+                ("weight_decay", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
+                ("eps", C.c_float), ("step", C.c_int64)]
+
+
+OPT_SGD, OPT_ADAM = 0, 1
 
 
 class KernelTime(C.Structure):
@@ -82,6 +98,7 @@ def load():
     L.condensa_profile_enable.argtypes = [vp, i32]
     L.condensa_profile_read.argtypes = [vp, C.POINTER(KernelTime), i32, C.POINTER(i32)]
     L.condensa_cstep_prune_noalloc.argtypes = [vp, f64, f32, u32, vp]
+    L.condensa_lstep_update.argtypes = [vp, vp, i32, f32, C.POINTER(Opt), vp]
     L.condensa_launch_count.argtypes = [vp]
     L.condensa_launch_count.restype = C.c_int64
     L.condensa_last_error.argtypes = [vp]
@@ -137,6 +154,20 @@ def tensor_table(w: Sequence, lam: Optional[Sequence] = None, theta: Optional[Se
         e.numel, e.ndim = n, len(shp)
         for d in range(4):
             e.shape[d] = int(shp[d]) if d < len(shp) else 1
+    return tab
+
+
+def opt_table(w, theta, lam, grad, buf1=None, buf2=None):
+    """``condensa_opt_tensor[T]`` from per-tensor device buffers (entries of lam/buf1/buf2 may be None)."""
+    T = len(w)
+    tab = (OptTensor * max(T, 1))()
+    for t in range(T):
+        e = tab[t]
+        e.w, e.theta, e.grad = _addr(w[t]), _addr(theta[t]), _addr(grad[t])
+        e.lam = _addr(lam[t]) if lam is not None else None
+        e.buf1 = _addr(buf1[t]) if buf1 is not None else None
+        e.buf2 = _addr(buf2[t]) if buf2 is not None else None
+        e.numel = int(w[t].numel()) if hasattr(w[t], "numel") else int(w[t].size)
     return tab
 
 
@@ -212,6 +243,12 @@ class Context:
         self._check(self._lib.condensa_cstep_host(self._h, int(op), tab, T, float(sparsity),
                                                   float(mu), int(bh), int(bw), fuse_bits(fuse),
                                                   _stream_handle(stream)))
+
+    def lstep_update(self, tab, T, mu, kind="sgd", lr=0.1, momentum=0.9, weight_decay=0.0, beta1=0.9,
+                     beta2=0.999, eps=1e-8, step=1, stream=None):
+        o = Opt({"sgd": OPT_SGD, "adam": OPT_ADAM}[kind], lr, momentum, weight_decay, beta1, beta2, eps, step)
+        self._check(self._lib.condensa_lstep_update(self._h, tab, T, float(mu), C.byref(o),
+                                                    _stream_handle(stream)))
 
     def get_result(self) -> Result:
         r = Result()
