@@ -150,6 +150,18 @@ CONDENSA_API int condensa_cstep_prune(condensa_ctx *ctx, const condensa_tensor *
 CONDENSA_API int condensa_cstep_filter(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
                           double sparsity, float mu, unsigned fuse, void *stream);
 
+/* NeuronPrune / StructurePrune (Table 1: neurons are "1D blocks"; StructurePrune
+ * "combines neuron and filter pruning"). `kinds` selects the leading-index slices
+ * that are ranked together, by the fp64 sum of u^2 like filters:
+ *   CONDENSA_STRUCT_FILTER  [f, :, :, :] of every 4-D tensor,
+ *   CONDENSA_STRUCT_NEURON  rows [r, :] of every 2-D tensor,
+ * or both. Every other tensor passes through. condensa_cstep_filter() is this
+ * call with CONDENSA_STRUCT_FILTER. */
+enum { CONDENSA_STRUCT_FILTER = 1, CONDENSA_STRUCT_NEURON = 2 };
+CONDENSA_API int condensa_cstep_structure(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
+                                          double sparsity, float mu, int kinds, unsigned fuse,
+                                          void *stream);
+
 /* BlockPrune - every 2-D tensor is cut into bh x bw blocks (row-major numbering,
  * blocks that stick out over an edge hold fewer elements) ranked on the fp64 sum
  * of u^2 taken row by row inside the block (Table 1, "n-D blocks of size bs").

@@ -89,6 +89,8 @@ def lib():
         L.orc_cstep_prune.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_float, C.c_uint,
                                       C.c_void_p]
         L.orc_cstep_filter.argtypes = list(L.orc_cstep_prune.argtypes)
+        L.orc_cstep_structure.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_float, C.c_int, C.c_uint,
+                                          C.c_void_p]
         L.orc_cstep_block.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_float, C.c_int,
                                       C.c_int, C.c_uint, C.c_void_p]
         L.orc_cstep_quantize.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint]
@@ -213,10 +215,11 @@ def f16_bits_to_f32(h: np.ndarray) -> np.ndarray:
 def structure_norms(ws, lams, mu: float, kind: str, block=(4, 4)) -> np.ndarray:
     """fp64 nu of every ranked structure, in global structure order."""
     tab, _, keep = _table(ws, lams)
-    k = {"filter": 0, "block": 1}[kind]
-    S = lib().orc_structure_norms(tab, len(ws), C.c_float(mu), k, block[0], block[1], None)
+    k = {"filter": 0, "neuron": 0, "structure": 0, "block": 1}[kind]
+    bh = {"filter": 1, "neuron": 2, "structure": 3}.get(kind, block[0])
+    S = lib().orc_structure_norms(tab, len(ws), C.c_float(mu), k, bh, block[1], None)
     nu = np.empty(S, np.float64)
-    lib().orc_structure_norms(tab, len(ws), C.c_float(mu), k, block[0], block[1], _ptr(nu))
+    lib().orc_structure_norms(tab, len(ws), C.c_float(mu), k, bh, block[1], _ptr(nu))
     return nu
 
 
@@ -233,6 +236,18 @@ def cstep_filter(ws, lams, s: float, mu: float, fuse: Sequence[str] = ()) -> Out
     tab, out, keep = _table(ws, lams)
     r = _Result()
     rc = lib().orc_cstep_filter(tab, len(ws), float(s), C.c_float(mu), fuse_bits(fuse), C.byref(r))
+    assert rc == 0
+    out.result = _result(r)
+    return out
+
+
+def cstep_structure(ws, lams, s: float, mu: float, kinds: Sequence[str] = ("filter", "neuron"),
+                    fuse: Sequence[str] = ()) -> Outputs:
+    """Rank leading-index slices: 'filter' (4-D tensors) and/or 'neuron' (rows of 2-D tensors)."""
+    tab, out, keep = _table(ws, lams)
+    r = _Result()
+    mask = sum({"filter": 1, "neuron": 2}[k] for k in set(kinds))
+    rc = lib().orc_cstep_structure(tab, len(ws), float(s), C.c_float(mu), mask, fuse_bits(fuse), C.byref(r))
     assert rc == 0
     out.result = _result(r)
     return out

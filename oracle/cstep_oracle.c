@@ -277,12 +277,21 @@ int orc_cstep_prune(const orc_tensor *ts, int32_t T, double s, float mu, unsigne
 }
 
 /* nu of each structure of one tensor, fp64, accumulated in index order.
- * kind 0: filters = slices [f, :, :, :] of a 4-D tensor.
+ * kind 0: leading-index slices: filters [f, :, :, :] of a 4-D tensor (Table 1,
+ *         FilterPrune, "3D blocks") and/or neurons = rows [r, :] of a 2-D tensor
+ *         (NeuronPrune, "1D blocks"); for this kind `bh` carries the mask of
+ *         which of the two are ranked (1 = filters, 2 = neurons, 3 = both:
+ *         StructurePrune "combines neuron and filter pruning").
  * kind 1: bh x bw blocks of a 2-D tensor, numbered row-major; a block that
  *         sticks out over the edge only sums the elements that exist. */
 static int64_t structure_count(const orc_tensor *t, int kind, int bh, int bw)
 {
-    if (kind == 0) return (t->ndim == 4) ? t->shape[0] : 0;
+    if (kind == 0) {
+        if (t->numel == 0) return 0;
+        if (t->ndim == 4 && (bh & 1)) return t->shape[0];
+        if (t->ndim == 2 && (bh & 2)) return t->shape[0];
+        return 0;
+    }
     if (t->ndim != 2) return 0;
     int64_t nbr = (t->shape[0] + bh - 1) / bh, nbc = (t->shape[1] + bw - 1) / bw;
     return nbr * nbc;
@@ -291,7 +300,7 @@ static int64_t structure_count(const orc_tensor *t, int kind, int bh, int bw)
 static int64_t structure_of(const orc_tensor *t, int kind, int bh, int bw, int64_t i)
 {
     if (kind == 0) {
-        int64_t len = t->shape[1] * t->shape[2] * t->shape[3];
+        int64_t len = t->numel / t->shape[0];
         return i / len;
     }
     int64_t C = t->shape[1];
@@ -304,7 +313,7 @@ static void structure_norms(const orc_tensor *t, const float *u, int kind, int b
                             double *nu)
 {
     if (kind == 0) {
-        int64_t len = t->shape[1] * t->shape[2] * t->shape[3];
+        int64_t len = t->numel / t->shape[0];
         for (int64_t f = 0; f < t->shape[0]; ++f) {
             double acc = 0.0;
             for (int64_t j = 0; j < len; ++j) {
@@ -382,7 +391,16 @@ static int cstep_structured(const orc_tensor *ts, int32_t T, double s, float mu,
 int orc_cstep_filter(const orc_tensor *ts, int32_t T, double s, float mu, unsigned fuse,
                      orc_result *res)
 {
-    return cstep_structured(ts, T, s, mu, fuse, 0, 0, 0, res);
+    return cstep_structured(ts, T, s, mu, fuse, 0, 1, 0, res);
+}
+
+/* NeuronPrune / FilterPrune / StructurePrune in one call: `kinds` is the mask
+ * 1 = filters of 4-D tensors, 2 = neurons (rows) of 2-D tensors. */
+int orc_cstep_structure(const orc_tensor *ts, int32_t T, double s, float mu, int kinds, unsigned fuse,
+                        orc_result *res)
+{
+    if (kinds < 1 || kinds > 3) return -2;
+    return cstep_structured(ts, T, s, mu, fuse, 0, kinds, 0, res);
 }
 
 /* Block pruning (Table 1, BlockPrune): 2-D tensors are ranked by bh x bw

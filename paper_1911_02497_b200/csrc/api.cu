@@ -158,7 +158,8 @@ int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double
     return CONDENSA_OK;
 }
 
-void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl)
+// kinds: for OP_FILTER, which leading-index slices are ranked (1 = filters of 4-D tensors, 2 = rows of 2-D tensors)
+void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, int kinds = 1)
 {
     pl.td.resize(T);
     pl.prefix_a.assign(T + 1, 0);
@@ -191,10 +192,10 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl)
             d.n_units = x.numel;
             items_a = lin_items;
         } else if (op == OP_FILTER) {
-            d.ranked = (x.ndim == 4 && x.numel > 0) ? 1 : 0;
+            d.ranked = (x.numel > 0 && ((x.ndim == 4 && (kinds & 1)) || (x.ndim == 2 && (kinds & 2)))) ? 1 : 0;
             if (d.ranked) {
                 d.d0 = x.shape[0];
-                d.d1 = x.shape[1] * x.shape[2] * x.shape[3];
+                d.d1 = x.numel / x.shape[0];
                 d.n_units = d.d0;
                 items_a = d.d0 * ((d.d1 + SEG - 1) / SEG);
             }
@@ -426,13 +427,13 @@ Sel initial_state(long long S, long long k, int bits_key)
 }
 
 int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double sparsity, float mu,
-           unsigned fuse, cudaStream_t stream)
+           unsigned fuse, cudaStream_t stream, int kinds = 1)
 {
     int rc = validate(ctx, op, ts, T, sparsity, mu, fuse);
     if (rc) return rc;
     CU_TRY(ctx, cudaSetDevice(ctx->device));
     Plan pl;
-    build_plan(op, ts, T, pl);
+    build_plan(op, ts, T, pl, kinds);
     const bool ranking = op <= OP_BLOCK;
     // single-pass path: unstructured and block pruning of lists too large to list whole
     const bool sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) &&
@@ -655,6 +656,15 @@ int condensa_cstep_filter(condensa_ctx *ctx, const condensa_tensor *tensors, int
                           float mu, unsigned fuse, void *stream)
 {
     return run_op(ctx, OP_FILTER, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_cstep_structure(condensa_ctx *ctx, const condensa_tensor *tensors, int T, double sparsity,
+                             float mu, int kinds, unsigned fuse, void *stream)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    if (kinds < 1 || kinds > (CONDENSA_STRUCT_FILTER | CONDENSA_STRUCT_NEURON))
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "kinds must be CONDENSA_STRUCT_FILTER and/or CONDENSA_STRUCT_NEURON");
+    return run_op(ctx, OP_FILTER, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, kinds);
 }
 
 int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T, double sparsity,

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcondensa_cstep.so")
 FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, NO_SAMPLING = 1, 2, 4, 64
 OP_PRUNE, OP_FILTER, OP_BLOCK, OP_QUANTIZE, OP_LAGRANGE = 0, 1, 2, 3, 4
 DTYPE_FP16 = 1
+STRUCT_FILTER, STRUCT_NEURON = 1, 2
 OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_UNSUPPORTED, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
 ERR_TOO_LARGE = -6
 NOALLOC_MAX_NUMEL = 1048576
@@ -25,7 +26,8 @@ EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "conde
            "condensa_cstep_block", "condensa_cstep_quantize", "condensa_cstep_lagrange_update",
            "condensa_cstep_host", "condensa_get_result", "condensa_launch_count",
            "condensa_last_error", "condensa_profile_enable", "condensa_profile_read",
-           "condensa_cstep_prune_noalloc", "condensa_lstep_update"]
+           "condensa_cstep_prune_noalloc", "condensa_lstep_update",
+           "condensa_cstep_structure"]
 
 
 class CondensaError(RuntimeError):
@@ -91,6 +93,7 @@ def load():
     L.condensa_cstep_prune.argtypes = [vp, vp, i32, f64, f32, u32, vp]
     L.condensa_cstep_filter.argtypes = [vp, vp, i32, f64, f32, u32, vp]
     L.condensa_cstep_block.argtypes = [vp, vp, i32, f64, f32, i32, i32, u32, vp]
+    L.condensa_cstep_structure.argtypes = [vp, vp, i32, f64, f32, i32, u32, vp]
     L.condensa_cstep_quantize.argtypes = [vp, vp, i32, f32, i32, u32, vp]
     L.condensa_cstep_lagrange_update.argtypes = [vp, vp, i32, f32, u32, vp]
     L.condensa_cstep_host.argtypes = [vp, i32, vp, i32, f64, f32, i32, i32, u32, vp]
@@ -225,6 +228,11 @@ class Context:
     def cstep_filter(self, tab, T, sparsity, mu, fuse=(), stream=None):
         self._check(self._lib.condensa_cstep_filter(self._h, tab, T, float(sparsity), float(mu),
                                                     fuse_bits(fuse), _stream_handle(stream)))
+
+    def cstep_structure(self, tab, T, sparsity, mu, kinds=("filter", "neuron"), fuse=(), stream=None):
+        mask = sum({"filter": STRUCT_FILTER, "neuron": STRUCT_NEURON}[k] for k in set(kinds))
+        self._check(self._lib.condensa_cstep_structure(self._h, tab, T, float(sparsity), float(mu), mask,
+                                                       fuse_bits(fuse), _stream_handle(stream)))
 
     def cstep_block(self, tab, T, sparsity, mu, bh=4, bw=4, fuse=(), stream=None):
         self._check(self._lib.condensa_cstep_block(self._h, tab, T, float(sparsity), float(mu),

@@ -82,6 +82,9 @@ class DeviceSet:
             ctx.cstep_prune(self.table, self.T, sparsity, mu, fuse, stream)
         elif op == "filter":
             ctx.cstep_filter(self.table, self.T, sparsity, mu, fuse, stream)
+        elif op in ("neuron", "structure"):
+            kinds = ("neuron",) if op == "neuron" else ("filter", "neuron")
+            ctx.cstep_structure(self.table, self.T, sparsity, mu, kinds, fuse, stream)
         elif op == "block":
             ctx.cstep_block(self.table, self.T, sparsity, mu, block[0], block[1], fuse, stream)
         elif op == "quantize":

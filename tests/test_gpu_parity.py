@@ -55,7 +55,7 @@ def run_gpu(ctx, op, w, lam, s, mu, fuse, block=(4, 4), elem_offset=0, skew=0, t
     ds.poison_outputs() if theta is None else None
     ds.run(ctx, op, s, mu, fuse, block)
     out = ds.fetch()
-    res = ctx.get_result() if op in ("prune", "filter", "block") else None
+    res = ctx.get_result() if op in ("prune", "filter", "block", "neuron", "structure") else None
     return out, res
 
 
@@ -65,6 +65,8 @@ def run_oracle(op, w, lam, s, mu, fuse, block=(4, 4), theta=None):
         return oracle.cstep_prune(w, lam, s, mu, fuse)
     if op == "filter":
         return oracle.cstep_filter(w, lam, s, mu, fuse)
+    if op in ("neuron", "structure"):
+        return oracle.cstep_structure(w, lam, s, mu, ("neuron",) if op == "neuron" else ("filter", "neuron"), fuse)
     if op == "block":
         return oracle.cstep_block(w, lam, s, mu, block, fuse)
     if op == "quantize":
@@ -288,6 +290,20 @@ def test_filter_small_and_ties(ctx):
     ints = np.round(W.draw(8 * 3000, "normal", 3.0, 6, 0, 0)).reshape(8, 3000, 1, 1).astype(np.float32)
     check(ctx, "filter", [ints, ints[::-1].copy()], None, 0.5, 1.0, ())   # integer data: sums exact
     check(ctx, "filter", [np.ones((4, 5), np.float32)], None, 0.5, 1.0, ())   # nothing to rank
+
+
+@pytest.mark.parametrize("op", ["neuron", "structure"])
+def test_neuron_and_structure_pruning(ctx, op):
+    """Rows of 2-D tensors (NeuronPrune) and rows + filters in one ranking (StructurePrune)."""
+    ws = W.random_set([(300, 257), (7, 3, 3, 3), (64,), (40, 1024), (12, 20, 3, 3), (1, 9)], seed=44,
+                      kind="normal", scale=0.3, lam_sigma=1e-2, mu=1e-2)
+    for s in (0.0, 0.35, 0.8, 1.0):
+        check(ctx, op, ws.w, ws.lam, s, ws.mu, ("lambda", "penalty"), exact_key=False)
+    check(ctx, op, ws.w, ws.lam, 0.5, ws.mu, ("fp16", "lambda"), elem_offset=3, exact_key=False)
+    # LSTM-shaped set: rows of the big matrices
+    ws = W.config("5t", scale=0.1)
+    got, res, _ = check(ctx, op, ws.w, ws.lam, 0.6, ws.mu, ("lambda",), exact_key=False)
+    assert res.n_units == sum(a.shape[0] for a in ws.w if a.ndim == 2)
 
 
 @pytest.mark.parametrize("scale", [0.25, 1.0])

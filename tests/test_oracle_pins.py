@@ -481,3 +481,30 @@ def test_lstep_adam_against_torch_adam():
     wn, _, _ = oracle.lstep_update([w], [w.copy()], [z], [g], [z], [z], mu, "adam", lr=1e-3, step=1)
     big = np.abs(g) > 1e-3
     assert np.allclose((w - wn[0])[big], 1e-3 * np.sign(g[big]), rtol=1e-4)
+
+
+# ---------------------------------------------------------------- neurons / structures
+def test_neuron_and_structure_pruning():
+    rng = np.random.default_rng(8)
+    fc = rng.standard_normal((9, 7)).astype(np.float32)
+    conv = (rng.standard_normal((4, 2, 3, 3)) * 0.5).astype(np.float32)
+    bias = rng.standard_normal(5).astype(np.float32)
+    # neurons only: rows of the 2-D tensor, everything else passes through
+    nu = oracle.structure_norms([fc, conv, bias], [None] * 3, 1.0, "neuron")
+    assert np.allclose(nu, (fc.astype(np.float64) ** 2).sum(1), rtol=1e-14) and nu.size == 9
+    out = oracle.cstep_structure([fc, conv, bias], [None] * 3, 4 / 9, 1.0, ("neuron",))
+    keep = brute_keep(nu.view(np.uint64), 5)
+    assert np.array_equal(out.mask[0], np.repeat(keep, 7).reshape(9, 7))
+    assert out.mask[1].all() and out.mask[2].all() and out.result.n_units == 9
+    # both kinds in one ranking, numbered tensor by tensor (rows of fc first, then the filters)
+    nu = oracle.structure_norms([fc, conv, bias], [None] * 3, 1.0, "structure")
+    ref = np.concatenate([(fc.astype(np.float64) ** 2).sum(1), (conv.astype(np.float64).reshape(4, -1) ** 2).sum(1)])
+    assert np.allclose(nu, ref, rtol=1e-14)
+    out = oracle.cstep_structure([fc, conv, bias], [None] * 3, 0.5, 1.0, ("neuron", "filter"))
+    keep = brute_keep(nu.view(np.uint64), 13 - 7)            # Z = floor(6.5 + 0.5) = 7
+    assert np.array_equal(out.mask[0][:, 0], keep[:9]) and np.array_equal(out.mask[1][:, 0, 0, 0], keep[9:])
+    assert int(out.mask[0][:, 0].sum() + out.mask[1][:, 0, 0, 0].sum()) == 6
+    # the filter scheme is the same call with only the filter kind
+    a = oracle.cstep_filter([fc, conv], [None, None], 0.5, 1.0)
+    b = oracle.cstep_structure([fc, conv], [None, None], 0.5, 1.0, ("filter",))
+    assert all(np.array_equal(x, y) for x, y in zip(a.mask, b.mask))
