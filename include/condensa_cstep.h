@@ -165,8 +165,10 @@ CONDENSA_API int condensa_cstep_structure(condensa_ctx *ctx, const condensa_tens
 /* BlockPrune - every 2-D tensor is cut into bh x bw blocks (row-major numbering,
  * blocks that stick out over an edge hold fewer elements) ranked on the fp64 sum
  * of u^2 taken row by row inside the block (Table 1, "n-D blocks of size bs").
- * Only bh = bw = 4 is built; anything else returns CONDENSA_ERR_UNSUPPORTED.
- * Tensors with ndim != 2 pass through. */
+ * bh = bw = 4 takes the single-pass kernels; every other shape with sides up to 4096
+ * (the paper's LSTM run uses bs = 5) is ranked in three steps - norms per block,
+ * selection on the norm array, elementwise projection - with the same results
+ * contract. Tensors with ndim != 2 pass through. */
 CONDENSA_API int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
                          double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream);
 

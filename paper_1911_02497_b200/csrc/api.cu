@@ -159,7 +159,7 @@ int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double
 }
 
 // kinds: for OP_FILTER, which leading-index slices are ranked (1 = filters of 4-D tensors, 2 = rows of 2-D tensors)
-void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, int kinds = 1)
+void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, int kinds = 1, int bh = 4, int bw = 4)
 {
     pl.td.resize(T);
     pl.prefix_a.assign(T + 1, 0);
@@ -198,6 +198,17 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, int kinds = 
                 d.d1 = x.numel / x.shape[0];
                 d.n_units = d.d0;
                 items_a = d.d0 * ((d.d1 + SEG - 1) / SEG);
+            }
+        } else if (op == OP_BLOCKGEN) {
+            d.ranked = (x.ndim == 2 && x.numel > 0) ? 1 : 0;
+            if (d.ranked) {
+                d.d0 = x.shape[0];
+                d.d1 = x.shape[1];
+                d.bh = bh;
+                d.bw = bw;
+                d.nbc = (d.d1 + bw - 1) / bw;
+                d.n_units = ((d.d0 + bh - 1) / bh) * d.nbc;
+                items_a = (d.n_units + BLOCKS_PER_ITEM - 1) / BLOCKS_PER_ITEM;
             }
         } else if (op == OP_BLOCK) {
             d.ranked = (x.ndim == 2 && x.numel > 0) ? 1 : 0;
@@ -427,14 +438,14 @@ Sel initial_state(long long S, long long k, int bits_key)
 }
 
 int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double sparsity, float mu,
-           unsigned fuse, cudaStream_t stream, int kinds = 1)
+           unsigned fuse, cudaStream_t stream, int kinds = 1, int bh = 4, int bw = 4)
 {
-    int rc = validate(ctx, op, ts, T, sparsity, mu, fuse);
+    int rc = validate(ctx, op == OP_BLOCKGEN ? OP_BLOCK : op, ts, T, sparsity, mu, fuse);
     if (rc) return rc;
     CU_TRY(ctx, cudaSetDevice(ctx->device));
     Plan pl;
-    build_plan(op, ts, T, pl, kinds);
-    const bool ranking = op <= OP_BLOCK;
+    build_plan(op, ts, T, pl, kinds, bh, bw);
+    const bool ranking = op <= OP_BLOCK || op == OP_BLOCKGEN;
     // single-pass path: unstructured and block pruning of lists too large to list whole
     const bool sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) &&
                           (u64)pl.S > pl.cap && pl.S >= 8ll * N_SAMPLE;
@@ -447,7 +458,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
                 if (!fast) pl.edge_items.push_back(pl.prefix_b[t] + j);
             }
     }
-    const Layout L = make_layout(T, pl, ranking, op == OP_FILTER, journal_floats);
+    const Layout L = make_layout(T, pl, ranking, op == OP_FILTER || op == OP_BLOCKGEN, journal_floats);
     rc = ensure_workspace(ctx, L.total, stream);
     if (rc) return rc;
     char *ws = ctx->ws;
@@ -500,6 +511,12 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         Params Pa = P;
         Pa.item_prefix = pa;
         Pa.n_items = pl.n_items_a;
+        if (op == OP_BLOCKGEN && pl.S > 0) {
+            const int pa_ = prof_begin(ctx, "k_blockgen_norms", stream);
+            k_blockgen_norms<<<stream_grid(ctx, pl.n_items_a, 8), THREADS, 0, stream>>>(Pa);
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, pa_, stream);
+        }
         if (op == OP_FILTER && pl.S > 0) {
             int pa_ = prof_begin(ctx, "k_filter_partial", stream);
             k_filter_partial<<<stream_grid(ctx, (pl.n_items_a + WARPS - 1) / WARPS, 8), THREADS, 0, stream>>>(Pa);
@@ -566,7 +583,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     Pb.n_items = pl.n_items_b;
     if (pl.n_items_b > 0) {
         const int grid = stream_grid(ctx, pl.n_items_b, ctx->occ_stream);
-        static const char *apply_names[5] = {"k_apply_prune", "k_apply_filter", "k_apply_block", "k_quantize", "k_lagrange"};
+        static const char *apply_names[6] = {"k_apply_prune", "k_apply_filter", "k_apply_block", "k_quantize", "k_lagrange", "k_apply_blockgen"};
         const int pa_ = prof_begin(ctx, apply_names[op], stream);
         switch (op) {
         case OP_PRUNE:
@@ -578,6 +595,10 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             else k_apply_linear<M_FILTER, false><<<grid, THREADS, 0, stream>>>(Pb);
             break;
         case OP_BLOCK: k_apply_block<<<grid, THREADS, 0, stream>>>(Pb); break;
+        case OP_BLOCKGEN:
+            if (need_h) k_apply_linear<M_BLOCKGEN, true><<<grid, THREADS, 0, stream>>>(Pb);
+            else k_apply_linear<M_BLOCKGEN, false><<<grid, THREADS, 0, stream>>>(Pb);
+            break;
         case OP_QUANTIZE: k_apply_linear<M_KEEPALL, true><<<grid, THREADS, 0, stream>>>(Pb); break;
         default: k_apply_linear<M_LAGRANGE, false><<<grid, THREADS, 0, stream>>>(Pb); break;
         }
@@ -672,7 +693,9 @@ int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int 
 {
     if (!ctx) return CONDENSA_ERR_INVALID_ARG;
     if (bh < 1 || bw < 1) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "block shape must be positive");
-    if (bh != 4 || bw != 4) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "only 4x4 blocks are built");
+    if (bh > 4096 || bw > 4096) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "block sides above 4096 are not built");
+    if (bh != 4 || bw != 4)      // general shapes: norms per block, selection on the norm array, elementwise projection
+        return run_op(ctx, OP_BLOCKGEN, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, 1, bh, bw);
     return run_op(ctx, OP_BLOCK, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream);
 }
 

@@ -22,7 +22,7 @@ constexpr int WSTG = 256;                // staged list entries per warp
 constexpr int MAX_SELECT_ITERS = 24;
 constexpr u64 KEY_NONE = ~0ull;          // cut-off key that keeps nothing
 
-enum { OP_PRUNE = 0, OP_FILTER = 1, OP_BLOCK = 2, OP_QUANTIZE = 3, OP_LAGRANGE = 4 };
+enum { OP_PRUNE = 0, OP_FILTER = 1, OP_BLOCK = 2, OP_QUANTIZE = 3, OP_LAGRANGE = 4, OP_BLOCKGEN = 5 };
 enum { FUSE_FP16 = 1, FUSE_LAMBDA = 2, FUSE_PENALTY = 4, NO_SAMPLING = 64 };
 enum { SRC_ELEM = 0, SRC_BLOCK = 1, SRC_ARRAY = 2 };
 
@@ -44,6 +44,7 @@ struct TensorDesc {
     int vec_ok;              // linear path may use 128-bit accesses
     int blk_vec_ok;          // block path may use 128-bit accesses
     int ranked;              // takes part in the ranking of the current call
+    int bh, bw;              // general block pruning: block height and width
 };
 
 // Device-resident record of one ranking call.

@@ -7,7 +7,22 @@
 
 namespace cs {
 
-enum { M_KEEPALL = 0, M_PRUNE = 1, M_FILTER = 2, M_LAGRANGE = 3 };
+enum { M_KEEPALL = 0, M_PRUNE = 1, M_FILTER = 2, M_LAGRANGE = 3, M_BLOCKGEN = 4 };
+
+// Structure id of element e of a 2-D tensor cut into bh x bw blocks (row-major block numbering).
+__device__ __forceinline__ u64 blockgen_sid(const TensorDesc &d, long long e)
+{
+    long long r, c;
+    if (d.numel < 0x7FFFFFFFll) {
+        const u32 rr = (u32)e / (u32)d.d1;
+        r = rr;
+        c = (u32)e - rr * (u32)d.d1;
+        return (u64)d.unit_prefix + (u64)((u32)r / (u32)d.bh) * (u64)d.nbc + (u32)c / (u32)d.bw;
+    }
+    r = e / d.d1;
+    c = e - r * d.d1;
+    return (u64)d.unit_prefix + (u64)(r / d.bh) * (u64)d.nbc + (u64)(c / d.bw);
+}
 
 constexpr int LIN_UNROLL = GROUPS_PER_ITEM / THREADS;   // 4 groups per thread per item
 
@@ -98,6 +113,11 @@ __device__ __forceinline__ void process_linear_item(const Params &P, const Tenso
                         long long f = f0, r = r0 + (e - (e0 < 0 ? 0 : e0));
                         while (r >= d.d1) { r -= d.d1; ++f; }
                         const u64 sid = (u64)(d.unit_prefix + f);
+                        keep = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
+                    }
+                } else if (MODE == M_BLOCKGEN) {
+                    if (d.ranked && e >= 0 && e < d.numel) {
+                        const u64 sid = blockgen_sid(d, e);
                         keep = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
                     }
                 }
@@ -213,6 +233,15 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
                     }
                 }
             }
+            else if (MODE == M_BLOCKGEN) {
+                if (d.ranked) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const u64 sid = blockgen_sid(d, e_base + eo + j);
+                        keep[j] = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
+                    }
+                }
+            }
             m = 0;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -248,7 +277,7 @@ template <int MODE, bool H>
 __global__ void __launch_bounds__(THREADS, 3) k_apply_linear(Params P)
 {
     u64 tau_key = 0, tau_id = 0;
-    if (MODE == M_PRUNE || MODE == M_FILTER) {
+    if (MODE == M_PRUNE || MODE == M_FILTER || MODE == M_BLOCKGEN) {
         if (P.ctl->sel.onepass) return;      // the single-pass kernel has written everything
         tau_key = P.ctl->tau_key;
         tau_id = P.ctl->tau_id;

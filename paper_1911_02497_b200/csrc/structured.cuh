@@ -166,6 +166,34 @@ __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
     }
 }
 
+// General bh x bw blocks: one thread per block adds the squares of the elements
+// that exist, row by row, in fp64 (the same order as the plain definition).
+// Work items: BLOCKS_PER_ITEM blocks of a ranked tensor.
+__global__ void __launch_bounds__(THREADS) k_blockgen_norms(Params P)
+{
+    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        const long long local = item - P.item_prefix[t];
+        const bool has_lam = d.lam != nullptr;
+        for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it) {
+            const long long b = local * BLOCKS_PER_ITEM + it * THREADS + threadIdx.x;
+            if (b >= d.n_units) continue;
+            const long long br = b / d.nbc, bc = b - br * d.nbc;
+            const long long r1 = (br + 1) * d.bh < d.d0 ? (br + 1) * d.bh : d.d0;
+            const long long c1 = (bc + 1) * d.bw < d.d1 ? (bc + 1) * d.bw : d.d1;
+            double acc = 0.0;
+            for (long long r = br * d.bh; r < r1; ++r)
+                for (long long c = bc * d.bw; c < c1; ++c) {
+                    const long long e = r * d.d1 + c;
+                    const double x = (double)form_u(d.w[e], has_lam ? d.lam[e] : 0.0f, P.mu, has_lam);
+                    acc = __fma_rn(x, x, acc);
+                }
+            P.arr_key[d.unit_prefix + b] = (u64)__double_as_longlong(acc);
+        }
+    }
+}
+
 // Filter norms, step 2: nu_f = partial sums added in segment order.
 __global__ void __launch_bounds__(THREADS) k_filter_combine(Params P)
 {

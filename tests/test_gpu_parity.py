@@ -328,6 +328,25 @@ def test_block_shapes(ctx, shape):
     check(ctx, "block", ws.w, ws.lam, 0.7, ws.mu, ("lambda",), skew=1)
 
 
+@pytest.mark.parametrize("block", [(5, 5), (1, 8), (3, 2), (8, 1), (16, 16), (2, 4)])
+def test_block_general_shapes(ctx, block):
+    """Block sizes other than 4x4 (the paper's LSTM experiment uses bs = 5)."""
+    ws = W.random_set([(33, 28), (11,), (130, 257), (5, 5), (64, 1500)], seed=sum(block), kind="uniform",
+                      scale=0.1, lam_sigma=1e-3, mu=1e-2)
+    for s in (0.0, 0.6, 1.0):
+        check(ctx, "block", ws.w, ws.lam, s, ws.mu, ("lambda", "penalty"), block=block)
+    check(ctx, "block", ws.w, ws.lam, 0.9, ws.mu, ("fp16", "lambda"), block=block, elem_offset=1)
+    blk = np.arange(block[0] * block[1], dtype=np.float32).reshape(block)
+    got, res, _ = check(ctx, "block", [np.tile(blk, (3, 4))], None, 0.5, 1.0, (), block=block)   # 12 equal blocks
+    assert (res.n_tie, res.n_tie_kept) == (12, 6)
+
+
+def test_block_size_five_on_the_lstm_shapes(ctx):
+    ws = W.config("5", scale=0.1)
+    got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.6, ws.mu, ("lambda",), block=(5, 5))
+    assert res.n_units == sum(-(-a.shape[0] // 5) * -(-a.shape[1] // 5) for a in ws.w if a.ndim == 2)
+
+
 def test_block_ties(ctx):
     blk = np.arange(16, dtype=np.float32).reshape(4, 4)
     got, res, _ = check(ctx, "block", [np.tile(blk, (2, 3))], None, 0.5, 1.0, ())
@@ -367,8 +386,11 @@ def test_argument_errors_leave_buffers_untouched(ctx):
             f()
         assert e.value.code == cstep.ERR_INVALID_ARG
     with pytest.raises(cstep.CondensaError) as e:
-        ds.run(ctx, "block", 0.5, 1e-3, block=(5, 5))
+        ds.run(ctx, "block", 0.5, 1e-3, block=(5000, 4))
     assert e.value.code == cstep.ERR_UNSUPPORTED
+    with pytest.raises(cstep.CondensaError) as e:
+        ds.run(ctx, "block", 0.5, 1e-3, block=(0, 4))
+    assert e.value.code == cstep.ERR_INVALID_ARG
     with pytest.raises(cstep.CondensaError) as e:
         ctx.cstep_quantize(ds.table, ds.T, 1e-3, dtype=2)
     assert e.value.code == cstep.ERR_UNSUPPORTED
