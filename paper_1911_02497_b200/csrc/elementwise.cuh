@@ -234,7 +234,21 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
                 }
             }
             else if (MODE == M_BLOCKGEN) {
-                if (d.ranked) {
+                if (d.ranked && d.numel < 0x7FFFFFFFll) {
+                    // row, column and block coordinates once per group, then walked element by element
+                    const u32 C = (u32)d.d1, bh = (u32)d.bh, bw = (u32)d.bw;
+                    const u32 e0 = (u32)(e_base + eo);
+                    u32 r = e0 / C, c = e0 - r * C;
+                    u32 br = r / bh, cb = c / bw, cm = c - cb * bw;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (c >= C) { c = 0; ++r; br = r / bh; cb = 0; cm = 0; }
+                        const u64 sid = (u64)d.unit_prefix + (u64)br * (u64)d.nbc + cb;
+                        keep[j] = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
+                        ++c;
+                        if (++cm == bw) { cm = 0; ++cb; }
+                    }
+                } else if (d.ranked) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const u64 sid = blockgen_sid(d, e_base + eo + j);
