@@ -85,6 +85,8 @@ enum {
     CONDENSA_FUSE_FP16 = 1,     /* theta = fp16 round-to-nearest-even of kept u, widened back  */
     CONDENSA_FUSE_LAMBDA = 2,   /* update lambda in place                                     */
     CONDENSA_FUSE_PENALTY = 4,  /* write g to grad                                            */
+    CONDENSA_FUSE_BF16 = 8,     /* like FUSE_FP16 with bfloat16 (not together with it); theta_h
+                                   then holds bfloat16 bits                                     */
     CONDENSA_NO_SAMPLING = 64   /* rank with full histogram passes, then project (two passes over
                                    w and lambda; same results). Default for large inputs is ONE
                                    pass: the threshold is first bracketed from 16384 hashed sample
@@ -109,7 +111,7 @@ enum {
     CONDENSA_ERR_TOO_LARGE = -6      /* input larger than a fixed built-in limit               */
 };
 
-enum { CONDENSA_DTYPE_FP16 = 1 };
+enum { CONDENSA_DTYPE_FP16 = 1, CONDENSA_DTYPE_BF16 = 2 };
 
 /* Record of the last ranking call, filled on the device. */
 typedef struct {
@@ -172,9 +174,12 @@ CONDENSA_API int condensa_cstep_structure(condensa_ctx *ctx, const condensa_tens
 CONDENSA_API int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
                          double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream);
 
-/* Quantize(dtype) - theta = fp16 round-to-nearest-even of u for every element,
- * mask = 1 (Table 1; Section 2 "low-precision approximation"). Overflow goes to
- * infinity, underflow is gradual, NaN becomes a quiet NaN with the same sign. */
+/* Quantize(dtype) - theta = round-to-nearest-even of u in `dtype` for every element,
+ * mask = 1 (Table 1; Section 2 "low-precision approximation"). dtype is
+ * CONDENSA_DTYPE_FP16 (IEEE binary16) or CONDENSA_DTYPE_BF16 (bfloat16: the upper
+ * half of a binary32); theta_h receives the 16 bits. Overflow goes to infinity,
+ * underflow is gradual, NaN becomes a quiet NaN with the same sign. `fuse` may
+ * carry FUSE_LAMBDA / FUSE_PENALTY only. */
 CONDENSA_API int condensa_cstep_quantize(condensa_ctx *ctx, const condensa_tensor *tensors, int T, float mu,
                             int dtype, unsigned fuse, void *stream);
 

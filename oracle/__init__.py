@@ -22,7 +22,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cstep_oracle.c")
 _LIB = os.path.join(_HERE, "libcstep_oracle.so")
 
-FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY = 1, 2, 4
+FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, FUSE_BF16 = 1, 2, 4, 8
 
 CFLAGS = ["-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
           "-fno-unsafe-math-optimizations", "-Wall"]
@@ -79,6 +79,8 @@ def lib():
         L.orc_f16_to_f32.restype = C.c_uint32
         L.orc_f16_to_f32.argtypes = [C.c_uint16]
         L.orc_f32_to_f16_array.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+        L.orc_f32_to_bf16_array.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+        L.orc_f32_to_bf16_range.argtypes = [C.c_uint32, C.c_int64, C.c_void_p]
         L.orc_f32_to_f16_range.argtypes = [C.c_uint32, C.c_int64, C.c_void_p]
         L.orc_form_u.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int64, C.c_void_p]
         L.orc_lagrange.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_uint,
@@ -128,7 +130,7 @@ class Outputs:
 
 
 def fuse_bits(fuse: Sequence[str]) -> int:
-    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY}
+    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY, "bf16": FUSE_BF16}
     b = 0
     for f in fuse:
         b |= table[f]
@@ -193,6 +195,22 @@ def f32_to_f16_bits(x: np.ndarray) -> np.ndarray:
     assert b.dtype == np.uint32
     out = np.empty(b.shape, np.uint16)
     lib().orc_f32_to_f16_array(_ptr(b), b.size, _ptr(out))
+    return out
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    b = np.ascontiguousarray(x)
+    if b.dtype == np.float32:
+        b = b.view(np.uint32)
+    assert b.dtype == np.uint32
+    out = np.empty(b.shape, np.uint16)
+    lib().orc_f32_to_bf16_array(_ptr(b), b.size, _ptr(out))
+    return out
+
+
+def f32_to_bf16_range(first: int, n: int) -> np.ndarray:
+    out = np.empty(n, np.uint16)
+    lib().orc_f32_to_bf16_range(C.c_uint32(first), n, _ptr(out))
     return out
 
 

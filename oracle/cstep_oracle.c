@@ -47,6 +47,7 @@
 #define ORC_FUSE_FP16    1u
 #define ORC_FUSE_LAMBDA  2u
 #define ORC_FUSE_PENALTY 4u
+#define ORC_FUSE_BF16    8u
 
 typedef struct {
     const float *w;        /* weights, never written                          */
@@ -139,6 +140,27 @@ uint32_t orc_f16_to_f32(uint16_t h)
     return sign | ((e - 15 + 127) << 23) | (m << 13);
 }
 
+/* binary32 -> bfloat16 (1 sign, 8 exponent, 7 fraction bits: the upper half of a
+ * binary32), round to nearest even; NaN -> quiet NaN with the sign kept. A carry
+ * out of the fraction moves to the exponent, up to infinity, as IEEE rounding wants. */
+uint16_t orc_f32_to_bf16(uint32_t b)
+{
+    if ((b & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)(((b >> 16) & 0x8000u) | 0x7FC0u);
+    uint32_t lower = b & 0xFFFFu, q = b >> 16;
+    if (lower > 0x8000u || (lower == 0x8000u && (q & 1u))) q += 1u;
+    return (uint16_t)q;
+}
+
+void orc_f32_to_bf16_array(const uint32_t *bits, int64_t n, uint16_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_bf16(bits[i]);
+}
+
+void orc_f32_to_bf16_range(uint32_t first, int64_t n, uint16_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_bf16(first + (uint32_t)i);
+}
+
 void orc_f32_to_f16_array(const uint32_t *bits, int64_t n, uint16_t *out)
 {
     for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_f16(bits[i]);
@@ -196,7 +218,10 @@ static void finish_tensor(const orc_tensor *t, const float *u, const uint8_t *ke
         uint32_t tb = 0u;
         uint16_t hb = 0u;
         if (keep[i]) {
-            if (fuse & ORC_FUSE_FP16) {
+            if (fuse & ORC_FUSE_BF16) {
+                hb = orc_f32_to_bf16(f32_bits(u[i]));
+                tb = (uint32_t)hb << 16;              /* exact widening */
+            } else if (fuse & ORC_FUSE_FP16) {
                 hb = orc_f32_to_f16(f32_bits(u[i]));
                 tb = orc_f16_to_f32(hb);
             } else {
@@ -412,7 +437,8 @@ int orc_cstep_block(const orc_tensor *ts, int32_t T, double s, float mu, int bh,
     return cstep_structured(ts, T, s, mu, fuse, 1, bh, bw, res);
 }
 
-/* Quantisation only (Table 1, Quantize(float16)): theta = Q(u), mask = 1. */
+/* Quantisation only (Table 1, Quantize(dtype)): theta = Q(u), mask = 1. The type is
+ * binary16 unless `fuse` carries ORC_FUSE_BF16. */
 int orc_cstep_quantize(const orc_tensor *ts, int32_t T, float mu, unsigned fuse)
 {
     for (int32_t t = 0; t < T; ++t) {
@@ -421,7 +447,7 @@ int orc_cstep_quantize(const orc_tensor *ts, int32_t T, float mu, unsigned fuse)
         uint8_t *keep = (uint8_t *)malloc((size_t)(n ? n : 1));
         orc_form_u(ts[t].w, ts[t].lambda, mu, n, u);
         memset(keep, 1, (size_t)n);
-        finish_tensor(&ts[t], u, keep, mu, fuse | ORC_FUSE_FP16);
+        finish_tensor(&ts[t], u, keep, mu, (fuse & ORC_FUSE_BF16) ? fuse : (fuse | ORC_FUSE_FP16));
         free(u); free(keep);
     }
     return 0;

@@ -117,8 +117,11 @@ int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double
     if (!(mu > 0.0f) || !std::isfinite(mu)) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "mu must be finite and > 0");
     if (op <= CONDENSA_OP_BLOCK && !(s >= 0.0 && s <= 1.0))
         return fail(ctx, CONDENSA_ERR_INVALID_ARG, "sparsity must lie in [0, 1]");
-    const unsigned known = CONDENSA_FUSE_FP16 | CONDENSA_FUSE_LAMBDA | CONDENSA_FUSE_PENALTY | CONDENSA_NO_SAMPLING;
+    const unsigned known = CONDENSA_FUSE_FP16 | CONDENSA_FUSE_LAMBDA | CONDENSA_FUSE_PENALTY | CONDENSA_FUSE_BF16 |
+                           CONDENSA_NO_SAMPLING;
     if (fuse & ~known) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "unknown fuse bits");
+    if ((fuse & CONDENSA_FUSE_FP16) && (fuse & CONDENSA_FUSE_BF16))
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "FUSE_FP16 and FUSE_BF16 exclude each other");
     std::vector<Interval> iv;
     iv.reserve((size_t)T * 6);
     for (int t = 0; t < T; ++t) {
@@ -473,9 +476,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     const long long *pb = pe + pl.edge_items.size();         // projection prefix, right behind it
     P.T = T;
     P.mu = mu;
-    P.fuse = fuse & 7u;
-    if (op == OP_QUANTIZE) P.fuse |= FUSE_FP16;
-    if (op == OP_LAGRANGE) P.fuse &= ~(unsigned)FUSE_FP16;
+    P.fuse = fuse & 15u;
+    if (op == OP_QUANTIZE && !(P.fuse & FUSE_BF16)) P.fuse |= FUSE_FP16;
+    if (op == OP_LAGRANGE) P.fuse &= ~(unsigned)(FUSE_FP16 | FUSE_BF16);
     P.ctl = (Ctl *)(ws + L.ctl);
     P.hist = (u64 *)(ws + L.hist);
     P.fin_key = (u64 *)(ws + L.fin_key);
@@ -495,7 +498,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     P.jr_lam = (float *)(ws + L.journal);
     P.onepass_cap = pl.cap;
     P.seed = 0x9E3779B97F4A7C15ull;
-    bool need_h = (fuse & CONDENSA_FUSE_FP16) != 0;
+    bool need_h = (fuse & (CONDENSA_FUSE_FP16 | CONDENSA_FUSE_BF16)) != 0;
     for (int t = 0; t < T; ++t) need_h = need_h || ts[t].theta_h != nullptr;
     ctx->ctl = P.ctl;
     ctx->last_stream = stream;
@@ -703,7 +706,11 @@ int condensa_cstep_quantize(condensa_ctx *ctx, const condensa_tensor *tensors, i
                             int dtype, unsigned fuse, void *stream)
 {
     if (!ctx) return CONDENSA_ERR_INVALID_ARG;
-    if (dtype != CONDENSA_DTYPE_FP16) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "only fp16 is built");
+    if (dtype != CONDENSA_DTYPE_FP16 && dtype != CONDENSA_DTYPE_BF16)
+        return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "only fp16 and bf16 are built");
+    if (fuse & (CONDENSA_FUSE_FP16 | CONDENSA_FUSE_BF16))
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "the type is given by dtype, not by fuse bits");
+    if (dtype == CONDENSA_DTYPE_BF16) fuse |= CONDENSA_FUSE_BF16;
     return run_op(ctx, OP_QUANTIZE, tensors, T, 0.0, mu, fuse, (cudaStream_t)stream);
 }
 
@@ -1021,7 +1028,7 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
     long long *prefix = (long long *)(ws + L.desc + sizeof(TensorDesc));
     P.T = 1;
     P.mu = mu;
-    P.fuse = fuse & 7u;
+    P.fuse = fuse & 15u;
     P.ctl = (Ctl *)(ws + L.ctl);
     P.hist = (u64 *)(ws + L.hist);
     P.fin_key = (u64 *)(ws + L.fin_key);

@@ -23,7 +23,7 @@ constexpr int MAX_SELECT_ITERS = 24;
 constexpr u64 KEY_NONE = ~0ull;          // cut-off key that keeps nothing
 
 enum { OP_PRUNE = 0, OP_FILTER = 1, OP_BLOCK = 2, OP_QUANTIZE = 3, OP_LAGRANGE = 4, OP_BLOCKGEN = 5 };
-enum { FUSE_FP16 = 1, FUSE_LAMBDA = 2, FUSE_PENALTY = 4, NO_SAMPLING = 64 };
+enum { FUSE_FP16 = 1, FUSE_LAMBDA = 2, FUSE_PENALTY = 4, FUSE_BF16 = 8, NO_SAMPLING = 64 };
 enum { SRC_ELEM = 0, SRC_BLOCK = 1, SRC_ARRAY = 2 };
 
 // One tensor of the list as the kernels see it.
@@ -161,6 +161,16 @@ __device__ __forceinline__ float f16_bits_to_f32(unsigned short h)
     return f;
 }
 
+// binary32 -> bfloat16 bits, round to nearest even; NaN -> quiet NaN, sign kept.
+__device__ __forceinline__ unsigned short f32_to_bf16_bits(float x)
+{
+    const u32 b = __float_as_uint(x);
+    if ((b & 0x7FFFFFFFu) > 0x7F800000u) return (unsigned short)(((b >> 16) & 0x8000u) | 0x7FC0u);
+    return (unsigned short)((b + 0x7FFFu + ((b >> 16) & 1u)) >> 16);
+}
+
+__device__ __forceinline__ float bf16_bits_to_f32(unsigned short h) { return __uint_as_float((u32)h << 16); }
+
 struct Out {
     float theta, lam, grad;
     unsigned short th;
@@ -172,8 +182,9 @@ __device__ __forceinline__ Out finish(float w, float lam, float u, bool keep, fl
                                       unsigned fuse, bool has_lam)
 {
     Out o;
-    unsigned short hb = keep ? f32_to_f16_bits(u) : (unsigned short)0;
-    float th = keep ? ((fuse & FUSE_FP16) ? f16_bits_to_f32(hb) : u) : 0.0f;
+    const bool bf = (fuse & FUSE_BF16) != 0;
+    unsigned short hb = keep ? (bf ? f32_to_bf16_bits(u) : f32_to_f16_bits(u)) : (unsigned short)0;
+    float th = keep ? (bf ? bf16_bits_to_f32(hb) : (fuse & FUSE_FP16) ? f16_bits_to_f32(hb) : u) : 0.0f;
     float d = __fsub_rn(w, th);
     float p = __fmul_rn(mu, d);
     float lu = has_lam ? lam : 0.0f;
@@ -188,17 +199,19 @@ __device__ __forceinline__ Out finish(float w, float lam, float u, bool keep, fl
 
 // Lean form for the hot kernels: H = the binary16 bits are needed (fp16 fuse or
 // a theta_h output); `fp16`, `upd` (update lambda) are warp-uniform flags.
+// `q` is the quantisation of theta: 0 none, 1 binary16, 2 bfloat16 (theta_h then holds that type).
 template <bool H>
 __device__ __forceinline__ Out finish_lean(float w, float lam, float u, bool keep, float mu,
-                                           bool fp16, bool upd)
+                                           int q, bool upd)
 {
     Out o;
     float th = keep ? u : 0.0f;
     o.th = 0;
     if (H) {
-        const unsigned short hb = keep ? f32_to_f16_bits(u) : (unsigned short)0;
+        const unsigned short hb = keep ? (q == 2 ? f32_to_bf16_bits(u) : f32_to_f16_bits(u)) : (unsigned short)0;
         o.th = hb;
-        if (fp16) th = keep ? f16_bits_to_f32(hb) : 0.0f;
+        if (q == 1) th = keep ? f16_bits_to_f32(hb) : 0.0f;
+        if (q == 2) th = keep ? bf16_bits_to_f32(hb) : 0.0f;
     }
     const float p = __fmul_rn(mu, __fsub_rn(w, th));
     const float lu = upd ? __fsub_rn(lam, p) : lam;
@@ -225,8 +238,13 @@ __device__ __forceinline__ void form_u4(const float *w, const float *l, float mu
 
 // binary16 bits of four values with the plain hardware conversion; the rare
 // NaN (whose sign must be kept) is patched on a side path.
-__device__ __forceinline__ void half4(const float *x, unsigned short *h)
+__device__ __forceinline__ void half4(const float *x, unsigned short *h, int q = 1)
 {
+    if (q == 2) {        // bfloat16: integer rounding, NaN included
+#pragma unroll
+        for (int j = 0; j < 4; ++j) h[j] = f32_to_bf16_bits(x[j]);
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < 4; ++j) h[j] = __half_as_ushort(__float2half_rn(x[j]));
     const float s = (x[0] + x[1]) + (x[2] + x[3]);
@@ -236,8 +254,13 @@ __device__ __forceinline__ void half4(const float *x, unsigned short *h)
     }
 }
 
-__device__ __forceinline__ void widen4(const unsigned short *h, const float *x, float *o)
+__device__ __forceinline__ void widen4(const unsigned short *h, const float *x, float *o, int q = 1)
 {
+    if (q == 2) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[j] = bf16_bits_to_f32(h[j]);
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < 4; ++j) o[j] = __half2float(__ushort_as_half(h[j]));
     const float s = (x[0] + x[1]) + (x[2] + x[3]);

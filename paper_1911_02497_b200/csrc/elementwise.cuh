@@ -177,7 +177,7 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
     const bool has_lam = d.lam != nullptr;
     const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
     const bool wr_grad = (P.fuse & FUSE_PENALTY) && d.grad != nullptr;
-    const bool fp16 = (P.fuse & FUSE_FP16) != 0;
+    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
     const float mu = P.mu;
     const u32 tau32 = tau_key > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)tau_key;     // KEY_NONE keeps nothing
     const float4 *wp = reinterpret_cast<const float4 *>(d.w + e_base) + threadIdx.x;
@@ -263,8 +263,8 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
                 m |= keep[j] ? (1u << (8 * j)) : 0u;
             }
             if (H) {
-                half4(th, h);
-                if (fp16) widen4(h, th, th);
+                half4(th, h, fp16 ? fp16 : 1);
+                if (fp16) widen4(h, th, th, fp16);
             }
         }
 #pragma unroll

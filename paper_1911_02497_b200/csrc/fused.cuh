@@ -53,7 +53,7 @@ __device__ __forceinline__ void fused_finish(const Params &P, FusedShared &sh, u
 // Final write of one 4x4 block, lean form.
 template <bool H>
 __device__ __forceinline__ void store_block_lean(const TensorDesc &d, const BlockData &bd, const float *u,
-                                                 bool keep, float mu, bool fp16, bool upd, bool wr_grad)
+                                                 bool keep, float mu, int fp16, bool upd, bool wr_grad)
 {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -92,7 +92,7 @@ __device__ __forceinline__ void store_block_lean(const TensorDesc &d, const Bloc
 template <bool H>
 __device__ __forceinline__ void fused_block_item_generic(const Params &P, const TensorDesc &d, long long local,
                                                          FusedShared &sh, const Bracket &br, int &par,
-                                                         u64 &n_above, bool fp16)
+                                                         u64 &n_above, int fp16)
 {
     const bool has_lam = d.lam != nullptr;
     const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
@@ -146,7 +146,7 @@ __device__ __forceinline__ void fused_block_item_generic(const Params &P, const 
 template <bool H>
 __device__ __forceinline__ void fused_elem_item_generic(const Params &P, const TensorDesc &d, long long local,
                                                         FusedShared &sh, const Bracket &br, int par,
-                                                        u64 &n_above, bool fp16)
+                                                        u64 &n_above, int fp16)
 {
     const u32 lo = (u32)br.lo, hi = (u32)br.hi, guess = (u32)br.guess;
     const long long ng = (d.numel + d.pad + 3) >> 2;
@@ -294,7 +294,7 @@ __device__ __noinline__ void fused_edge_items(const Params &P, FusedShared &sh)
     for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
     if (threadIdx.x < 2) sh.cnt[threadIdx.x] = 0;
     __syncthreads();
-    const bool fp16 = (P.fuse & FUSE_FP16) != 0;
+    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
     const long long *prefix_b = P.edge_items + P.n_edge_items;      // [T+1]
     u64 n_above = 0;
     int par = 0;

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
     for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
     if (threadIdx.x < WARPS) sh.wcount[threadIdx.x] = 0;
     __syncthreads();
-    const bool fp16 = (P.fuse & FUSE_FP16) != 0;
+    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
     const u32 lo = (u32)br.lo, range = (u32)br.hi - (u32)br.lo, guess = (u32)br.guess;
     const float mu = P.mu;
     const int warp = threadIdx.x >> 5;
@@ -110,8 +110,8 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
             nkeep += __popc(m);
             unsigned short h[4];
             if (H) {
-                half4(th, h);                 // binary16 of theta (zeroed entries give +0)
-                if (fp16) widen4(h, th, th);
+                half4(th, h, fp16 ? fp16 : 1);     // 16-bit code of theta (zeroed entries give +0)
+                if (fp16) widen4(h, th, th, fp16);
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(THREADS, CS_BLOCK_MINB) k_fused_block(Params P
     for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
     if (threadIdx.x < WARPS) sh.wcount[threadIdx.x] = 0;
     __syncthreads();
-    const bool fp16 = (P.fuse & FUSE_FP16) != 0;
+    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
     const float mu = P.mu;
     const int warp = threadIdx.x >> 5;
     u32 n_above = 0;
@@ -321,8 +321,8 @@ __global__ void __launch_bounds__(THREADS, CS_BLOCK_MINB) k_fused_block(Params P
                 for (int j = 0; j < 4; ++j) th[j] = keep ? u[4 * i + j] : 0.0f;
                 unsigned short h[4];
                 if (H) {
-                    half4(th, h);
-                    if (fp16) widen4(h, th, th);
+                    half4(th, h, fp16 ? fp16 : 1);
+                    if (fp16) widen4(h, th, th, fp16);
                 }
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {

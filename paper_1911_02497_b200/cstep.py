@@ -16,7 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libcondensa_cstep.so")
 
 FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, NO_SAMPLING = 1, 2, 4, 64
 OP_PRUNE, OP_FILTER, OP_BLOCK, OP_QUANTIZE, OP_LAGRANGE = 0, 1, 2, 3, 4
-DTYPE_FP16 = 1
+DTYPE_FP16, DTYPE_BF16 = 1, 2
+FUSE_BF16 = 8
 STRUCT_FILTER, STRUCT_NEURON = 1, 2
 OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_UNSUPPORTED, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
 ERR_TOO_LARGE = -6
@@ -115,7 +116,7 @@ def load():
 def fuse_bits(fuse) -> int:
     if isinstance(fuse, int):
         return fuse
-    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY,
+    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY, "bf16": FUSE_BF16,
              "no_sampling": NO_SAMPLING}
     b = 0
     for f in fuse:

@@ -87,8 +87,9 @@ class DeviceSet:
             ctx.cstep_structure(self.table, self.T, sparsity, mu, kinds, fuse, stream)
         elif op == "block":
             ctx.cstep_block(self.table, self.T, sparsity, mu, block[0], block[1], fuse, stream)
-        elif op == "quantize":
-            ctx.cstep_quantize(self.table, self.T, mu, cstep.DTYPE_FP16, fuse, stream)
+        elif op in ("quantize", "quantize_bf16"):
+            dt = cstep.DTYPE_BF16 if op == "quantize_bf16" else cstep.DTYPE_FP16
+            ctx.cstep_quantize(self.table, self.T, mu, dt, fuse, stream)
         elif op == "lagrange":
             ctx.cstep_lagrange_update(self.table, self.T, mu, fuse, stream)
         else:

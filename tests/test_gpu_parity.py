@@ -71,6 +71,8 @@ def run_oracle(op, w, lam, s, mu, fuse, block=(4, 4), theta=None):
         return oracle.cstep_block(w, lam, s, mu, block, fuse)
     if op == "quantize":
         return oracle.cstep_quantize(w, lam, mu, fuse)
+    if op == "quantize_bf16":
+        return oracle.cstep_quantize(w, lam, mu, tuple(fuse) + ("bf16",))
     return oracle.lagrange_update(w, theta, lam, mu, fuse)
 
 
@@ -129,9 +131,33 @@ def test_quantize_special_values_and_skewed_alignment(ctx):
     check(ctx, "quantize", ws.w, ws.lam, mu=ws.mu, fuse=("penalty",), elem_offset=1, skew=2)
 
 
-def test_quantize_every_fp32_bit_pattern(ctx):
+def test_bf16_quantize_and_fused_paths(ctx):
+    sp = np.array([0.0, -0.0, np.inf, -np.inf, np.nan, -np.nan, 1.0, 1.00390625, 1.01171875, 3.3895314e38,
+                   3.38e38, 1e-40, -1e-45, 0.1, 65504.0], np.float32)
+    got, _, exp = check(ctx, "quantize_bf16", [np.tile(sp, 300)], [None], mu=1.0, fuse=())
+    assert np.array_equal(got["theta_h"][0], exp.theta_h[0])
+    for n, off in ((5, 0), (4099, 1), (100003, 3)):
+        ws = W.random_set([(n,)], seed=n, kind="normal", scale=3.0, lam_sigma=1e-2, mu=1e-2)
+        check(ctx, "quantize_bf16", ws.w, ws.lam, mu=ws.mu, fuse=("lambda", "penalty"), elem_offset=off)
+    ws = W.config(4, scale=0.1)                               # single-pass path with bfloat16
+    check(ctx, "prune", ws.w, ws.lam, ws.sparsity, ws.mu, ("bf16", "lambda", "penalty"))
+    check(ctx, "prune", ws.w, ws.lam, ws.sparsity, ws.mu, ("bf16", "lambda", "no_sampling"))
+    ws = W.config("5", scale=0.12)
+    check(ctx, "block", ws.w, ws.lam, ws.sparsity, ws.mu, ("bf16", "lambda"))
+    check(ctx, "block", ws.w, ws.lam, ws.sparsity, ws.mu, ("bf16", "lambda"), block=(5, 5))
+    ws = W.config(3, scale=0.2)
+    check(ctx, "filter", ws.w, ws.lam, ws.sparsity, ws.mu, ("bf16", "lambda"), exact_key=False)
+    from paper_1911_02497_b200 import cstep
+    from paper_1911_02497_b200.device_set import DeviceSet
+    ds = DeviceSet(ws.w, ws.lam)
+    with pytest.raises(cstep.CondensaError):
+        ds.run(ctx, "prune", 0.5, 1e-3, ("fp16", "bf16"))
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_quantize_every_fp32_bit_pattern(ctx, dtype):
     """All 2^32 binary32 patterns through the quantise entry point against the oracle's
-    explicit-bit conversion (binary16 bits and the widened theta)."""
+    explicit-bit conversion (16-bit code and the widened theta)."""
     import torch
     from paper_1911_02497_b200 import cstep
     chunk = 1 << 27
@@ -144,12 +170,13 @@ def test_quantize_every_fp32_bit_pattern(ctx):
     for c in range((1 << 32) // chunk):
         first = c * chunk
         w.copy_(((base + first) & 0xFFFFFFFF).to(torch.int64).sub_((base + first >= (1 << 31)).to(torch.int64) << 32).to(torch.int32))
-        ctx.cstep_quantize(tab, 1, 1.0)
+        ctx.cstep_quantize(tab, 1, 1.0, dtype=cstep.DTYPE_FP16 if dtype == "fp16" else cstep.DTYPE_BF16)
         got_h = th.cpu().numpy().view(np.uint16)
-        exp_h = oracle.f32_to_f16_range(first, chunk)
+        exp_h = (oracle.f32_to_f16_range if dtype == "fp16" else oracle.f32_to_bf16_range)(first, chunk)
         assert np.array_equal(got_h, exp_h), "chunk %d" % c
         # theta is the exact widening of those 16 bits (NaN: quiet, sign kept)
-        wide = torch.from_numpy(exp_h.view(np.int16)).to(dev).view(torch.float16).to(torch.float32)
+        wide = torch.from_numpy(exp_h.view(np.int16)).to(dev).view(
+            torch.float16 if dtype == "fp16" else torch.bfloat16).to(torch.float32)
         tb, wb = theta.view(torch.int32), wide.view(torch.int32)
         nan = torch.isnan(wide)
         assert bool(torch.equal(tb[~nan], wb[~nan]))
@@ -379,7 +406,7 @@ def test_argument_errors_leave_buffers_untouched(ctx):
     ds.poison_outputs()
     bad = [lambda: ds.run(ctx, "prune", 1.5, 1e-3), lambda: ds.run(ctx, "prune", float("nan"), 1e-3),
            lambda: ds.run(ctx, "prune", 0.5, 0.0), lambda: ds.run(ctx, "prune", 0.5, float("inf")),
-           lambda: ds.run(ctx, "prune", 0.5, -1.0), lambda: ds.run(ctx, "prune", 0.5, 1e-3, fuse=8),
+           lambda: ds.run(ctx, "prune", 0.5, -1.0), lambda: ds.run(ctx, "prune", 0.5, 1e-3, fuse=16),
            lambda: ds.run(ctx, "lagrange", 0.0, 1e-3, fuse=())]
     for f in bad:
         with pytest.raises(cstep.CondensaError) as e:
@@ -392,7 +419,7 @@ def test_argument_errors_leave_buffers_untouched(ctx):
         ds.run(ctx, "block", 0.5, 1e-3, block=(0, 4))
     assert e.value.code == cstep.ERR_INVALID_ARG
     with pytest.raises(cstep.CondensaError) as e:
-        ctx.cstep_quantize(ds.table, ds.T, 1e-3, dtype=2)
+        ctx.cstep_quantize(ds.table, ds.T, 1e-3, dtype=3)
     assert e.value.code == cstep.ERR_UNSUPPORTED
     # aliasing: theta on top of w; the same lambda twice
     tab = cstep.tensor_table(ds.w, ds.lam, ds.w, shapes=ds.shapes)

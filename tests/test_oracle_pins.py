@@ -508,3 +508,40 @@ def test_neuron_and_structure_pruning():
     a = oracle.cstep_filter([fc, conv], [None, None], 0.5, 1.0)
     b = oracle.cstep_structure([fc, conv], [None, None], 0.5, 1.0, ("filter",))
     assert all(np.array_equal(x, y) for x, y in zip(a.mask, b.mask))
+
+
+# ---------------------------------------------------------------- bfloat16
+def test_bf16_hand_values_and_torch():
+    import torch
+    hand = {0x3F800000: 0x3F80,      # 1
+            0x3F808000: 0x3F80,      # 1 + 2^-8 is the tie between 0x3F80 and 0x3F81: even
+            0x3F818000: 0x3F82,      # 1 + 3*2^-8 ties up to the even 0x3F82
+            0x3F808001: 0x3F81,      # just above the tie
+            0x7F7F8000: 0x7F80,      # the tie above the largest bfloat16 goes to infinity
+            0x7F7F7FFF: 0x7F7F,      # just below it stays finite
+            0x80000000: 0x8000, 0x00000001: 0x0000, 0x00008000: 0x0000, 0x00008001: 0x0001,
+            0x00018000: 0x0002,      # subnormal tie to even
+            0x7F800000: 0x7F80, 0xFF800000: 0xFF80, 0x7FC00000: 0x7FC0, 0xFF800001: 0xFFC0,
+            0x3DCCCCCD: 0x3DCD}      # 0.1f rounds up
+    for fb, hb in hand.items():
+        assert int(oracle.lib().orc_f32_to_bf16(fb)) == hb, hex(fb)
+    rng = np.random.default_rng(5)
+    pats = [rng.integers(0, 1 << 32, size=1 << 20, dtype=np.uint64).astype(np.uint32)]
+    hi = np.arange(0, 1 << 16, dtype=np.uint32)[:, None] << 16           # every bfloat16 with the critical tails
+    lo = np.array([0, 1, 0x7FFF, 0x8000, 0x8001, 0xFFFF], np.uint32)[None, :]
+    pats.append((hi | lo).reshape(-1))
+    p = np.concatenate(pats)
+    got = oracle.f32_to_bf16_bits(p)
+    ref = torch.from_numpy(p.view(np.int32)).view(torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    nan = np.isnan(p.view(np.float32))
+    assert np.array_equal(got[~nan], ref[~nan])
+    assert np.all((got[nan] & 0x7FFF) == 0x7FC0) and np.array_equal(got[nan] >> 15, (p[nan] >> 31).astype(np.uint16))
+    # scheme level: prune then quantise to bfloat16
+    ws = W.config(1, scale=1 / 64)
+    out = oracle.cstep_prune(ws.w, ws.lam, 0.9, ws.mu, ("bf16", "lambda"))
+    plain = oracle.cstep_prune(ws.w, ws.lam, 0.9, ws.mu, ())
+    u = oracle.form_u(ws.w[0], ws.lam[0], ws.mu)
+    q = torch.from_numpy(u).to(torch.bfloat16)
+    exp = np.where(plain.mask[0] == 1, q.to(torch.float32).numpy(), np.float32(0))
+    assert np.array_equal(out.mask[0], plain.mask[0]) and np.array_equal(bits(out.theta[0]), bits(exp))
+    assert np.array_equal(out.theta_h[0], np.where(plain.mask[0] == 1, q.view(torch.int16).numpy().view(np.uint16), 0))
