@@ -288,7 +288,7 @@ __device__ __forceinline__ void fused_elem_item_generic(const Params &P, const T
 // the scan decomposition there, so the projection decomposition is passed in
 // P.edge_* with its own prefix array right behind the item list.
 template <int SRC>
-__device__ __noinline__ void fused_edge_items(const Params &P, FusedShared &sh)
+__device__ void fused_edge_items(const Params &P, FusedShared &sh)
 {
     const Bracket br = load_bracket(P.ctl->sel);
     for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
@@ -317,13 +317,15 @@ __device__ __noinline__ void fused_edge_items(const Params &P, FusedShared &sh)
 
 // Rewrite one listed unit whose provisional decision was wrong. Called from the
 // selection kernel after the cut-off is known. `idx` is the list position.
+// `pre_s`, when given, holds the tensors' first unit numbers in shared memory
+// (the search for the owning tensor is then free of global loads).
 template <int SRC>
-__device__ __noinline__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep)
+__device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, const long long *pre_s)
 {
     int lo = 0, hi = P.T - 1;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
-        const long long pre = (SRC == SRC_ELEM) ? P.td[mid].elem_prefix : P.td[mid].unit_prefix;
+        const long long pre = pre_s ? pre_s[mid] : (SRC == SRC_ELEM) ? P.td[mid].elem_prefix : P.td[mid].unit_prefix;
         if ((u64)pre <= id) lo = mid; else hi = mid - 1;
     }
     const TensorDesc d = P.td[lo];

@@ -453,7 +453,11 @@ __device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
         for (u32 i = threadIdx.x; i < n; i += THREADS) {
             const u64 ki = k[i], di = d[i];
             u32 before = 0;
-            for (u32 j = 0; j < n; ++j) before += (k[j] > ki || (k[j] == ki && d[j] < di)) ? 1u : 0u;
+#pragma unroll 8
+            for (u32 j = 0; j < n; ++j) {
+                const u64 kj = k[j], dj = d[j];          // branch-free: both loads always issue
+                before += (u32)(kj > ki) | ((u32)(kj == ki) & (u32)(dj < di));
+            }
             if ((u64)before + 1 == r) sh.fin_hit = (int)i;
         }
         __syncthreads();
@@ -519,9 +523,43 @@ __device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
     __syncthreads();
 }
 
+// Cut-off and record of the call, from the final selection state (one thread).
+__device__ __forceinline__ void write_result(const Params &P, const Sel &s)
+{
+    Ctl *c = P.ctl;
+    Result r;
+    r.status = s.error ? -5 : 0;
+    r.passes = s.passes;
+    r.n_units = (long long)s.S;
+    r.n_keep = (long long)s.k;
+    r.n_zero = (long long)(s.S - s.k);
+    r.sampled = s.sampled;
+    r.n_candidates = (long long)(c->list_count[0] + c->list_count[1]);
+    r.tau_norm = 0.0f;
+    if (s.k == 0 || s.S == 0 || s.error) {
+        c->tau_key = KEY_NONE;
+        c->tau_id = 0;
+        r.tau_key = (P.bits_key >= 63) ? 0x7FF0000000000000ull : 0x7F800000ull;
+        r.tau_id = -1;
+        r.n_gt = r.n_tie = r.n_tie_kept = 0;
+    } else {
+        c->tau_key = s.lo_key;
+        c->tau_id = s.lo_id;
+        r.tau_key = s.lo_key;
+        r.tau_id = (long long)s.lo_id;
+        r.n_gt = (long long)s.n_gt;
+        r.n_tie = (long long)s.n_tie;
+        r.n_tie_kept = (long long)(s.k - s.n_gt);
+        if (P.bits_key >= 63) r.tau_norm = (float)sqrt(__longlong_as_double((long long)s.lo_key));
+    }
+    r.n_repaired = 0;      // filled in by the host from the counter once the stream is idle
+    c->sel = s;
+    c->res = r;
+}
+
 // Defined with the single-pass kernels: rewrites one listed unit.
 template <int SRC>
-__device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep);
+__device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, const long long *pre_s);
 
 // Defined with the single-pass kernels: the projection items the aligned fast
 // kernel leaves out (tensor heads and tails, unaligned or ragged tensors).
@@ -535,6 +573,92 @@ static_assert(sizeof(FusedShared) <= sizeof(ScanShared), "the edge items reuse t
 
 template <int SRC>
 __device__ void fused_edge_items(const Params &P, FusedShared &sh);
+
+// One walk over the list of the single-pass path by the whole grid. A listed unit
+// whose final decision is known and differs from the provisional one is rewritten;
+// with `rank`, the units still inside the bracket are copied to the final buffer
+// instead. A rewrite is a chain of dependent memory accesses and only a few per
+// cent of the entries need one, so each CTA first queues them in shared memory
+// and then rewrites them one per thread. The caller may have fetched this
+// CTA's first chunk already (`pre`). Returns this thread's rewrite count.
+constexpr int LIST_ROUNDS = 8;                 // list entries per thread and chunk
+static_assert(LIST_ROUNDS * THREADS <= WARPS * WSTG, "the queue reuses the staging arrays");
+
+struct ListChunk {
+    u64 key[LIST_ROUNDS], id[LIST_ROUNDS];
+};
+
+__device__ __forceinline__ void load_list_chunk(const Params &P, u64 base, u64 n_list, ListChunk &ch)
+{
+#pragma unroll
+    for (int r = 0; r < LIST_ROUNDS; ++r) {
+        const u64 i = base + (u64)r * THREADS + threadIdx.x;
+        ch.key[r] = i < n_list ? __ldcg(&P.list_key[i]) : 0;
+        ch.id[r] = i < n_list ? __ldcg(&P.list_id[i]) : 0;
+    }
+}
+
+template <int SRC>
+__device__ __forceinline__ u64 list_repair_pass(const Params &P, ScanShared &sh, bool rank, u64 n_list, const ListChunk *pre)
+{
+    __shared__ u32 s_qn;
+    u64 *q_idx = &sh.stg_key[0][0];
+    u64 *q_id = &sh.stg_id[0][0];
+    // first unit number of every tensor, for the owner search of the rewrites
+    long long *pre_s = reinterpret_cast<long long *>(sh.hist);
+    const bool pre_ok = P.T <= NBINS / 2;
+    __syncthreads();
+    if (pre_ok)
+        for (int t = threadIdx.x; t < P.T; t += THREADS)
+            pre_s[t] = (SRC == SRC_ELEM) ? P.td[t].elem_prefix : P.td[t].unit_prefix;
+    Ctl *c = P.ctl;
+    const Sel &s = sh.sel;
+    const bool sk = s.lo_key == s.hi_key;
+    const u64 chunk = (u64)LIST_ROUNDS * THREADS;
+    u64 fixed = 0;
+    bool first = true;
+    for (u64 base = (u64)blockIdx.x * chunk; base < n_list; base += (u64)gridDim.x * chunk) {
+        if (threadIdx.x == 0) s_qn = 0;
+        __syncthreads();
+        ListChunk ch;
+        if (first && pre) ch = *pre;
+        else load_list_chunk(P, base, n_list, ch);
+        first = false;
+#pragma unroll
+        for (int r = 0; r < LIST_ROUNDS; ++r) {
+            const u64 i = base + (u64)r * THREADS + threadIdx.x;
+            if (i >= n_list) continue;
+            const u64 key = ch.key[r], id = ch.id[r];
+            bool fin;
+            if (rank) {
+                const bool above = key > s.hi_key || (sk && key == s.hi_key && id < s.lo_id);
+                const bool below = key < s.lo_key || (sk && key == s.lo_key && id > s.hi_id);
+                if (!above && !below) {
+                    const u32 pos = atomicAdd(&c->fin_count, 1u);
+                    if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; P.fin_idx[pos] = i; }
+                    continue;
+                }
+                fin = above;
+            } else {
+                fin = keep_by_cutoff(key, id, s.lo_key, s.lo_id);
+            }
+            if (fin != (key >= s.guess)) {
+                const u32 pos = atomicAdd(&s_qn, 1u);
+                q_idx[pos] = i;
+                q_id[pos] = id | (fin ? (1ull << 63) : 0ull);
+            }
+        }
+        __syncthreads();
+        const u32 qn = s_qn;
+        for (u32 j = threadIdx.x; j < qn; j += THREADS) {
+            const u64 packed = q_id[j];
+            repair_unit<SRC>(P, q_idx[j], packed & ~(1ull << 63), (packed >> 63) != 0, pre_ok ? pre_s : nullptr);
+            ++fixed;
+        }
+        __syncthreads();
+    }
+    return fixed;
+}
 
 // First pass of a ranking call: a plain (non-cooperative) scan at full grid.
 // When the single-pass path is active there is nothing left to scan, and the
@@ -560,6 +684,26 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     __shared__ ScanShared sh;
     cg::grid_group grid = cg::this_grid();
     const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
+    if (P.ctl->resolved) {
+        // The resolve kernel has produced cut-off and record. What is left are the
+        // units it ranked directly: spread thinly over the grid, since each rewrite
+        // is a chain of dependent memory accesses.
+        if (SRC != SRC_ARRAY) {
+            const u32 nf = __ldcg(&P.ctl->fin_count);
+            const u32 n = nf < (u32)FIN ? nf : (u32)FIN;
+            const u32 j = threadIdx.x * gridDim.x + blockIdx.x;
+            if (j < n && !P.ctl->sel.error) {
+                const u64 tk = P.ctl->sel.lo_key, ti = P.ctl->sel.lo_id, guess = P.ctl->sel.guess;
+                const u64 key = __ldcg(&P.fin_key[j]), id = __ldcg(&P.fin_id[j]);
+                const bool fin = keep_by_cutoff(key, id, tk, ti);
+                if (fin != (key >= guess)) {
+                    repair_unit<SRC>(P, __ldcg(&P.fin_idx[j]), id, fin, nullptr);
+                    atomicAdd(&P.ctl->n_repaired, 1ull);
+                }
+            }
+        }
+        return;
+    }
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
     __syncthreads();
 #ifdef CONDENSA_DEBUG_TIME
@@ -638,19 +782,8 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     if (SRC != SRC_ARRAY) {
         if (sh.sel.onepass && !sh.sel.error && sh.sel.k > 0) {
             // single-pass path: rewrite the listed units whose provisional decision was wrong
-            const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
-            const u64 stride = (u64)gridDim.x * THREADS;
-            {
-                const u64 n_list = __ldcg(&P.ctl->list_count[0]);
-                for (u64 i = (u64)blockIdx.x * THREADS + threadIdx.x; i < n_list; i += stride) {
-                    const u64 key = __ldcg(&P.list_key[i]), id = __ldcg(&P.list_id[i]);
-                    const bool fin = keep_by_cutoff(key, id, tk, ti);
-                    if (fin != (key >= guess)) {
-                        repair_unit<SRC>(P, i, id, fin);
-                        ++fixed;
-                    }
-                }
-            }
+            __syncthreads();
+            fixed = list_repair_pass<SRC>(P, sh, false, __ldcg(&P.ctl->list_count[0]), nullptr);
         }
         if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
     }
@@ -664,37 +797,60 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
         printf("\n");
     }
 #endif
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        Ctl *c = P.ctl;
-        const Sel &s = sh.sel;
-        Result r;
-        r.status = s.error ? -5 : 0;
-        r.passes = s.passes;
-        r.n_units = (long long)s.S;
-        r.n_keep = (long long)s.k;
-        r.n_zero = (long long)(s.S - s.k);
-        r.sampled = s.sampled;
-        r.n_candidates = (long long)(c->list_count[0] + c->list_count[1]);
-        r.tau_norm = 0.0f;
-        if (s.k == 0 || s.S == 0 || s.error) {
-            c->tau_key = KEY_NONE;
-            c->tau_id = 0;
-            r.tau_key = (P.bits_key >= 63) ? 0x7FF0000000000000ull : 0x7F800000ull;
-            r.tau_id = -1;
-            r.n_gt = r.n_tie = r.n_tie_kept = 0;
-        } else {
-            c->tau_key = s.lo_key;
-            c->tau_id = s.lo_id;
-            r.tau_key = s.lo_key;
-            r.tau_id = (long long)s.lo_id;
-            r.n_gt = (long long)s.n_gt;
-            r.n_tie = (long long)s.n_tie;
-            r.n_tie_kept = (long long)(s.k - s.n_gt);
-            if (P.bits_key >= 63) r.tau_norm = (float)sqrt(__longlong_as_double((long long)s.lo_key));
-        }
-        r.n_repaired = 0;      // filled in by the host from the counter once the stream is idle
-        c->sel = s;
-        c->res = r;
+    if (blockIdx.x == 0 && threadIdx.x == 0) write_result(P, sh.sel);
+}
+
+// Common end of the single-pass path, without a grid barrier. Every CTA makes the
+// first pick from the complete histogram (all arrive at the same state); if that
+// leaves at most FIN listed units open, every CTA walks its share of the list:
+// entries outside the narrowed bracket are final (and rewritten if their
+// provisional decision was wrong), the others go to the final buffer. The CTA that
+// finishes last (threadfence + counter, nobody waits) ranks the final buffer and
+// writes the record; the members of that buffer are rewritten at the start of
+// k_select, which is launched next in any case. In every other case (more
+// survivors, a failed check) this kernel changes nothing and k_select does the
+// whole job from the same histogram.
+template <int SRC>
+__global__ void __launch_bounds__(THREADS) k_resolve(Params P)
+{
+    __shared__ ScanShared sh;
+    __shared__ u32 s_last;
+    Ctl *c = P.ctl;
+    const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
+    if (threadIdx.x == 0) sh.sel = c->sel;
+    // this CTA's first chunk of the list is fetched while the pick is made
+    const u64 n_all = __ldcg(&c->list_count[0]);
+    const u64 n_list = n_all < P.cap ? n_all : P.cap;
+    ListChunk pre;
+    load_list_chunk(P, (u64)blockIdx.x * LIST_ROUNDS * THREADS, n_list, pre);
+    __syncthreads();
+    if (!sh.sel.onepass || sh.sel.done || sh.sel.error || sh.sel.k == 0 || n_all > P.cap) return;
+    if (threadIdx.x == 0) sh.sel.list_valid = 1;
+    __syncthreads();
+    block_pick(P, sh, true, max_key);
+    if (sh.sel.error) return;
+    const bool need_rank = !sh.sel.done;
+    if (need_rank && sh.sel.pop > FIN) return;
+    {
+        const u64 fixed = list_repair_pass<SRC>(P, sh, need_rank, n_list, &pre);
+        if (fixed) atomicAdd(&c->n_repaired, fixed);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&c->resolve_done, 1u) == gridDim.x - 1 ? 1u : 0u;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (need_rank) {
+        const u32 n = __ldcg(&c->fin_count);
+        if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
+        __syncthreads();
+        final_rank(P, sh, n);      // its members are rewritten by the next launch
+    }
+    if (threadIdx.x == 0) {
+        write_result(P, sh.sel);
+        c->resolved = 1;
+        c->resolve_done = 0;
     }
 }
 
@@ -713,6 +869,8 @@ __global__ void __launch_bounds__(THREADS) k_init(Params P, Sel init)
         c->list_count[0] = c->list_count[1] = 0;
         c->fin_count = 0;
         c->n_repaired = 0;
+        c->resolve_done = 0;
+        c->resolved = 0;
     }
 }
 
