@@ -309,6 +309,9 @@ def run_ours(args):
         # its algorithmic bytes are the step's
         movers = {k: v for k, v in prof.items() if k.startswith(("k_fused", "k_apply", "k_quantize", "k_lagrange"))
                   and v[1] / v[0] > 0.02}          # launches that return at once do not count
+        if not movers:                             # small sets: every launch is short
+            movers = {k: v for k, v in prof.items()
+                      if k.startswith(("k_fused", "k_apply", "k_quantize", "k_lagrange"))}
         dom = max(movers.items(), key=lambda kv: kv[1][1])
         dom_name, (dom_n, dom_ms) = dom
         achieved = (N * bpp) / (dom_ms / dom_n * 1e-3) / 1e9
