@@ -219,6 +219,56 @@ def run_lstep(args, ws, ctx, local, world):
     return 0
 
 
+def run_thin(args, ws, ctx, local, world):
+    """Standalone timing of thinning after filter pruning (not the headline): zero-filter flags,
+    compaction along the chain of conv layers, and the non-zero count of the whole list."""
+    import torch
+    from paper_1911_02497_b200.device_set import DeviceSet
+    ds = DeviceSet(ws.w, ws.lam, device="cuda:%d" % local)
+    ds.run(ctx, "filter", ws.sparsity, ws.mu, ("lambda",), ws.block)
+    convs = [t for t in range(len(ws.w)) if len(ws.shapes[t]) == 4]
+    keep = [torch.empty(ws.shapes[t][0], dtype=torch.uint8, device=ds.device) for t in convs]
+    dst = [torch.empty(int(np.prod(ws.shapes[t])), dtype=torch.float32, device=ds.device) for t in convs]
+    dims = [torch.zeros(2, dtype=torch.int64, device=ds.device) for t in convs]
+    counts = torch.zeros(len(ws.w) + 1, dtype=torch.int64, device=ds.device)
+    flush = torch.empty(2 * L2_BYTES // 4, dtype=torch.float32, device=ds.device)
+
+    def step():
+        for i, t in enumerate(convs):
+            Fo, Ci, kh, kw = ws.shapes[t]
+            ctx.thin_flags(ds.theta[t], Fo, Ci, kh * kw, 0, keep[i])
+            ctx.thin_compact(ds.theta[t], Fo, Ci, kh * kw, keep[i], keep[i - 1] if i else None, dst[i], dims[i])
+        ctx.count_nonzero(ds.theta, counts)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    l0 = ctx.launch_count()
+    for a, b in ev:
+        flush.fill_(1.0)
+        a.record()
+        step()
+        b.record()
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
+    N = sum(int(np.prod(ws.shapes[t])) for t in convs)
+    kept = sum(int(d[0]) * int(d[1]) * ws.shapes[t][2] * ws.shapes[t][3] for d, t in zip(dims, convs))
+    algo = 4 * N + 8 * kept + 4 * ws.numel        # flags read theta; compaction reads and writes the kept part; count reads
+    peak, src = measured_peak()
+    gbs = algo / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "thin_params_per_s", "value": ws.numel / (ms * 1e-3), "unit": "params/s",
+                      "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": "thin (flags + chain compaction + non-zero count) on %s" % workload_name(ws),
+                                 "l2": "L2 flushed between steps by writing a 252 MB buffer"},
+                      "gpu_launches": ctx.launch_count() - l0, "kept_params": kept, "nonzero": int(counts[-1]),
+                      "roofline": {"bound": "hbm", "kernel": "thin step", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                                   "frac": gbs / peak, "traffic": None, "peak_source": src,
+                                   "algorithmic_bytes_per_launch": algo}}))
+    return 0
+
+
 # --------------------------------------------------------------------------- CUDA arm
 def run_ours(args):
     import torch
@@ -253,6 +303,8 @@ def run_ours(args):
         bpp = 4 + 4 + 4 + 4 + 4          # read w, theta, lambda; write lambda, g
     if args.op in ("lstep_sgd", "lstep_adam"):
         return run_lstep(args, ws, ctx, local, world)
+    if args.op == "thin":
+        return run_thin(args, ws, ctx, local, world)
     stream = torch.cuda.current_stream()
 
     def step():
@@ -400,7 +452,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="5", help="1..5 or 5t; 5 (the largest) is the headline")
     ap.add_argument("--no-sampling", action="store_true")
-    ap.add_argument("--op", default=None, choices=["quantize", "lagrange", "lstep_sgd", "lstep_adam"],
+    ap.add_argument("--op", default=None, choices=["quantize", "lagrange", "lstep_sgd", "lstep_adam", "thin"],
                     help="time a standalone operation on the configuration's weights instead of its C-step")
     ap.add_argument("--block-size", type=int, default=0, help="block side for the block configs (default 4)")
     ap.add_argument("--skip-cpu", action="store_true")

@@ -256,6 +256,47 @@ CONDENSA_API int condensa_profile_read(condensa_ctx *ctx, condensa_kernel_time *
 /* Number of kernels this context has launched so far. */
 CONDENSA_API int64_t condensa_launch_count(const condensa_ctx *ctx);
 
+/* ---- Network thinning (paper, Implementation, "Network Thinning") and the
+ * non-zero count of the memory-footprint objective (Evaluation, Objective 1).
+ *
+ * Structure pruning leaves zero structures (filters, neurons, channels that
+ * are zero throughout); thinning finds and removes them so that the tensors
+ * become smaller dense ones. The paper's three phases are: build a graph of
+ * the network, derive a thinning strategy from the dependencies between
+ * nodes, apply it. The first two are host work on the caller's side; these
+ * calls are the third phase's device work on one tensor at a time. A tensor
+ * is seen as the row-major 3-D view [d0][d1][inner]: a conv weight
+ * F x C x kh x kw has d0 = F, d1 = C, inner = kh*kw; a matrix R x C has
+ * d0 = R, d1 = C, inner = 1; a bias has d0 = n, d1 = inner = 1.
+ * All pointers are DEVICE pointers unless stated; calls are asynchronous on
+ * `stream`; a value is zero when it is +0 or -0. */
+
+/* keep[i] = 1 if the slice i along `axis` (0: [i][:][:], 1: [:][i][:]) holds a
+ * non-zero value, else 0. `keep` has d0 (axis 0) or d1 (axis 1) bytes and is
+ * overwritten. Extents may be 0. */
+CONDENSA_API int condensa_thin_flags(condensa_ctx *ctx, const float *theta, int64_t d0, int64_t d1,
+                                     int64_t inner, int axis, uint8_t *keep, void *stream);
+
+/* dst = src with the slices removed whose flag is 0: dst is the dense row-major
+ * [d0'][d1'][inner] tensor of the entries src[i][j][:] with keep0[i] != 0 and
+ * keep1[j] != 0, in their original order. A NULL flag array keeps the whole
+ * axis. dims_out (device, two int64) receives d0' and d1'. dst must hold
+ * d0' * d1' * inner floats (d0 * d1 * inner always suffices) and must not
+ * overlap src. d0, d1 and d1 * inner must be below 2^31. The caller's
+ * strategy supplies the flags: e.g. keep0 of a conv layer from its own
+ * filters, keep1 from the flags of the layer that feeds it. */
+CONDENSA_API int condensa_thin_compact(condensa_ctx *ctx, const float *src, int64_t d0, int64_t d1,
+                                       int64_t inner, const uint8_t *keep0, const uint8_t *keep1,
+                                       float *dst, int64_t *dims_out, void *stream);
+
+/* counts[t] = number of non-zero values of arrays[t] (numel[t] floats each),
+ * counts[T] = their sum; the memory footprint is that count times the bytes of
+ * a stored value. `arrays` and `numel` are HOST arrays of T entries (the
+ * pointers in `arrays` are device pointers); `counts` is a DEVICE array of
+ * T + 1 int64, overwritten. */
+CONDENSA_API int condensa_count_nonzero(condensa_ctx *ctx, const float *const *arrays, const int64_t *numel,
+                                        int T, int64_t *counts, void *stream);
+
 /* condensa_cstep_prune() for callers that must not allocate device memory.
  * (An addition of this library: the paper has no counterpart.)
  *

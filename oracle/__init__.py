@@ -330,3 +330,43 @@ def lstep_update(ws, thetas, lams, grads, buf1, buf2, mu: float, kind: str = "sg
     rc = lib().orc_lstep_update(tab, T, C.c_float(mu), C.byref(o))
     assert rc == 0
     return w_out, b1_out, b2_out
+
+
+# ---------------------------------------------------------------- thinning
+# Paper, Implementation ("Network Thinning"): zero structures are found and
+# removed. Evaluation, Objective 1: the footprint counts non-zero parameters.
+def thin_flags(theta3: np.ndarray, axis: int) -> np.ndarray:
+    """theta3: array of shape [d0, d1, inner]. keep[i] = 1 iff slice i along
+    ``axis`` (0 or 1) holds a value that is not zero (+0 and -0 are zero)."""
+    x = np.asarray(theta3)
+    assert x.ndim == 3 and axis in (0, 1)
+    d = x.shape[axis]
+    keep = np.zeros(d, dtype=np.uint8)
+    for i in range(d):
+        sl = x[i, :, :] if axis == 0 else x[:, i, :]
+        keep[i] = 1 if np.any(sl != 0) else 0
+    return keep
+
+
+def thin_compact(src3: np.ndarray, keep0: Optional[np.ndarray], keep1: Optional[np.ndarray]) -> np.ndarray:
+    """The dense tensor of the entries src3[i, j, :] whose flags keep0[i] and
+    keep1[j] are non-zero, original order kept (None keeps the whole axis)."""
+    x = np.asarray(src3)
+    rows = [i for i in range(x.shape[0]) if keep0 is None or keep0[i] != 0]
+    cols = [j for j in range(x.shape[1]) if keep1 is None or keep1[j] != 0]
+    out = np.empty((len(rows), len(cols), x.shape[2]), dtype=x.dtype)
+    for a, i in enumerate(rows):
+        for b, j in enumerate(cols):
+            out[a, b, :] = x[i, j, :]
+    return out
+
+
+def count_nonzero(arrays) -> np.ndarray:
+    """Non-zero values per array, then their total (length T + 1, int64)."""
+    c = [int(np.sum(np.asarray(a).reshape(-1) != 0)) for a in arrays]
+    return np.array(c + [sum(c)], dtype=np.int64)
+
+
+def footprint_bytes(arrays, bytes_per_value: int) -> int:
+    """Bytes taken by the non-zero parameters (Objective 1)."""
+    return int(count_nonzero(arrays)[-1]) * int(bytes_per_value)

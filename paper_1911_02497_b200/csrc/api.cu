@@ -18,6 +18,7 @@
 #include "fused_fast.cuh"
 #include "sample.cuh"
 #include "lstep.cuh"
+#include "thin.cuh"
 
 using namespace cs;
 
@@ -836,6 +837,120 @@ int condensa_lstep_update(condensa_ctx *ctx, const condensa_opt_tensor *ts, int 
     const int pa_ = prof_begin(ctx, opt->kind == CONDENSA_OPT_ADAM ? "k_lstep_adam" : "k_lstep_sgd", stream);
     if (opt->kind == CONDENSA_OPT_ADAM) k_lstep<OPT_ADAM><<<grid, THREADS, 0, stream>>>(P);
     else k_lstep<OPT_SGD><<<grid, THREADS, 0, stream>>>(P);
+    LAUNCH_CHECK(ctx);
+    prof_end(ctx, pa_, stream);
+    return CONDENSA_OK;
+}
+
+// ---------------------------------------------------------------- thinning
+int condensa_thin_flags(condensa_ctx *ctx, const float *theta, int64_t d0, int64_t d1, int64_t inner, int axis,
+                        uint8_t *keep, void *stream_)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (d0 < 0 || d1 < 0 || inner < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "negative extent");
+    if (axis != 0 && axis != 1) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "axis must be 0 or 1");
+    const long long d = axis ? d1 : d0;
+    if (d == 0) return CONDENSA_OK;
+    if (!keep) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "keep is NULL");
+    if ((double)d0 * (double)d1 * (double)inner > 9.0e18) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "tensor too large");
+    const long long n = d0 * d1 * inner;
+    if (n > 0 && !theta) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "theta is NULL");
+    if ((uintptr_t)theta % 4) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "theta is not 4-byte aligned");
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    CU_TRY(ctx, cudaMemsetAsync(keep, 0, (size_t)d, stream));
+    ctx->last_stream = stream;
+    if (n == 0) return CONDENSA_OK;
+    const int pa_ = prof_begin(ctx, "k_thin_flags", stream);
+    k_thin_flags<<<stream_grid(ctx, (n + THIN_ITEM - 1) / THIN_ITEM, 8), THREADS, 0, stream>>>(theta, d0, d1, inner, axis, keep);
+    LAUNCH_CHECK(ctx);
+    prof_end(ctx, pa_, stream);
+    return CONDENSA_OK;
+}
+
+int condensa_thin_compact(condensa_ctx *ctx, const float *src, int64_t d0, int64_t d1, int64_t inner,
+                          const uint8_t *keep0, const uint8_t *keep1, float *dst, int64_t *dims_out, void *stream_)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (d0 < 0 || d1 < 0 || inner < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "negative extent");
+    if (!dims_out) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "dims_out is NULL");
+    if (d0 > 0x7FFFFFFFll || d1 > 0x7FFFFFFFll || (double)d1 * (double)inner >= 2147483648.0)
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "d0, d1 and d1 * inner must be below 2^31");
+    const long long n = d0 * d1 * inner;
+    if (n > 0 && (!src || !dst)) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "src or dst is NULL");
+    if ((uintptr_t)src % 4 || (uintptr_t)dst % 4 || (uintptr_t)dims_out % 8)
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "misaligned pointer");
+    if (n > 0) {
+        const uintptr_t a = (uintptr_t)src, b = (uintptr_t)dst, bytes = (uintptr_t)n * 4;
+        if (a < b + bytes && b < a + bytes) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "src and dst overlap");
+    }
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    // index lists live in the descriptor area of the workspace
+    Plan none;
+    none.cap = 1;
+    const Layout L = make_layout(0, none, false, false);
+    const size_t bytes = align_up(sizeof(int) * (size_t)d0, 256) + align_up(sizeof(int) * (size_t)d1, 256);
+    int rc = ensure_workspace(ctx, L.desc + bytes, stream);
+    if (rc) return rc;
+    ctx->last_upload.clear();           // a kernel overwrites the area: nothing is cached there any more
+    ctx->last_upload_dst = nullptr;
+    int *idx0 = (int *)(ctx->ws + L.desc);
+    int *idx1 = (int *)(ctx->ws + L.desc + align_up(sizeof(int) * (size_t)d0, 256));
+    ctx->last_stream = stream;
+    int pa_ = prof_begin(ctx, "k_thin_index", stream);
+    k_thin_index<<<1, THIN_INDEX_THREADS, 0, stream>>>(keep0, keep1, d0, d1, idx0, idx1, (long long *)dims_out);
+    LAUNCH_CHECK(ctx);
+    prof_end(ctx, pa_, stream);
+    if (n == 0) return CONDENSA_OK;
+    const long long L_in = d1 * inner;
+    const long long tiles = d0 * ((L_in + 1023) / 1024);
+    const bool vec = !keep1 && L_in % 4 == 0 && (uintptr_t)src % 16 == 0 && (uintptr_t)dst % 16 == 0;
+    const int grid = stream_grid(ctx, tiles, 8);
+    pa_ = prof_begin(ctx, "k_thin_gather", stream);
+    if (vec) k_thin_gather<true><<<grid, THREADS, 0, stream>>>(src, dst, d1, inner, keep0 ? idx0 : nullptr, nullptr, (const long long *)dims_out);
+    else k_thin_gather<false><<<grid, THREADS, 0, stream>>>(src, dst, d1, inner, keep0 ? idx0 : nullptr, keep1 ? idx1 : nullptr, (const long long *)dims_out);
+    LAUNCH_CHECK(ctx);
+    prof_end(ctx, pa_, stream);
+    return CONDENSA_OK;
+}
+
+int condensa_count_nonzero(condensa_ctx *ctx, const float *const *arrays, const int64_t *numel, int T,
+                           int64_t *counts, void *stream_)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!arrays || !numel || T <= 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "array list is empty or NULL");
+    if (!counts || (uintptr_t)counts % 8) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "counts is NULL or misaligned");
+    std::vector<CountDesc> td((size_t)T);
+    std::vector<long long> prefix((size_t)T + 1, 0);
+    for (int t = 0; t < T; ++t) {
+        if (numel[t] < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "array %d: negative numel", t);
+        if (numel[t] > 0 && !arrays[t]) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "array %d is NULL", t);
+        if ((uintptr_t)arrays[t] % 4) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "array %d is not 4-byte aligned", t);
+        td[t].x = arrays[t];
+        td[t].numel = numel[t];
+        prefix[t + 1] = prefix[t] + (numel[t] + THIN_ITEM - 1) / THIN_ITEM;
+    }
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    Plan none;
+    none.cap = 1;
+    const Layout L = make_layout(0, none, false, false);
+    const size_t bytes = sizeof(CountDesc) * (size_t)T + sizeof(long long) * (size_t)(T + 1);
+    int rc = ensure_workspace(ctx, L.desc + align_up(bytes, 256), stream);
+    if (rc) return rc;
+    std::vector<char> img(bytes);
+    memcpy(img.data(), td.data(), sizeof(CountDesc) * (size_t)T);
+    memcpy(img.data() + sizeof(CountDesc) * (size_t)T, prefix.data(), sizeof(long long) * (size_t)(T + 1));
+    rc = upload_image(ctx, img, ctx->ws + L.desc, stream);
+    if (rc) return rc;
+    CU_TRY(ctx, cudaMemsetAsync(counts, 0, sizeof(int64_t) * (size_t)(T + 1), stream));
+    ctx->last_stream = stream;
+    if (prefix[T] == 0) return CONDENSA_OK;
+    const int pa_ = prof_begin(ctx, "k_count_nonzero", stream);
+    k_count_nonzero<<<stream_grid(ctx, prefix[T], 8), THREADS, 0, stream>>>(
+        (const CountDesc *)(ctx->ws + L.desc), (const long long *)(ctx->ws + L.desc + sizeof(CountDesc) * (size_t)T), T,
+        prefix[T], (unsigned long long *)counts);
     LAUNCH_CHECK(ctx);
     prof_end(ctx, pa_, stream);
     return CONDENSA_OK;

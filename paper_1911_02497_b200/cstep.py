@@ -28,7 +28,8 @@ EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "conde
            "condensa_cstep_host", "condensa_get_result", "condensa_launch_count",
            "condensa_last_error", "condensa_profile_enable", "condensa_profile_read",
            "condensa_cstep_prune_noalloc", "condensa_lstep_update",
-           "condensa_cstep_structure"]
+           "condensa_cstep_structure", "condensa_thin_flags", "condensa_thin_compact",
+           "condensa_count_nonzero"]
 
 
 class CondensaError(RuntimeError):
@@ -103,6 +104,10 @@ def load():
     L.condensa_profile_read.argtypes = [vp, C.POINTER(KernelTime), i32, C.POINTER(i32)]
     L.condensa_cstep_prune_noalloc.argtypes = [vp, f64, f32, u32, vp]
     L.condensa_lstep_update.argtypes = [vp, vp, i32, f32, C.POINTER(Opt), vp]
+    i64 = C.c_int64
+    L.condensa_thin_flags.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp]
+    L.condensa_thin_compact.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp, vp]
+    L.condensa_count_nonzero.argtypes = [vp, C.POINTER(vp), C.POINTER(i64), i32, vp, vp]
     L.condensa_launch_count.argtypes = [vp]
     L.condensa_launch_count.restype = C.c_int64
     L.condensa_last_error.argtypes = [vp]
@@ -258,6 +263,23 @@ class Context:
         o = Opt({"sgd": OPT_SGD, "adam": OPT_ADAM}[kind], lr, momentum, weight_decay, beta1, beta2, eps, step)
         self._check(self._lib.condensa_lstep_update(self._h, tab, T, float(mu), C.byref(o),
                                                     _stream_handle(stream)))
+
+    def thin_flags(self, theta, d0, d1, inner, axis, keep, stream=None):
+        self._check(self._lib.condensa_thin_flags(self._h, _addr(theta), int(d0), int(d1), int(inner), int(axis),
+                                                  _addr(keep), _stream_handle(stream)))
+
+    def thin_compact(self, src, d0, d1, inner, keep0, keep1, dst, dims_out, stream=None):
+        self._check(self._lib.condensa_thin_compact(self._h, _addr(src), int(d0), int(d1), int(inner),
+                                                    _addr(keep0), _addr(keep1), _addr(dst), _addr(dims_out),
+                                                    _stream_handle(stream)))
+
+    def count_nonzero(self, arrays, counts, stream=None):
+        """``arrays``: device float32 tensors; ``counts``: device int64 tensor of len(arrays) + 1."""
+        T = len(arrays)
+        ptrs = (C.c_void_p * max(T, 1))(*[_addr(a) for a in arrays])
+        numel = (C.c_int64 * max(T, 1))(*[int(a.numel()) for a in arrays])
+        self._check(self._lib.condensa_count_nonzero(self._h, ptrs, numel, T, _addr(counts),
+                                                     _stream_handle(stream)))
 
     def get_result(self) -> Result:
         r = Result()
