@@ -88,7 +88,10 @@ enum {
     CONDENSA_FUSE_BF16 = 8,     /* like FUSE_FP16 with bfloat16 (not together with it); theta_h
                                    then holds bfloat16 bits                                     */
     CONDENSA_NO_SAMPLING = 64   /* rank with full histogram passes, then project (two passes over
-                                   w and lambda; same results). Default for large inputs is ONE
+                                   w and lambda; same results). It also sends rankings of at most
+                                   16384 structures (filters, rows, general blocks), which by
+                                   default are settled by one CTA in shared memory, through the
+                                   grid-wide selection. Default for large inputs is ONE
                                    pass: the threshold is first bracketed from 16384 hashed sample
                                    positions, the pass decides everything outside the bracket for
                                    good and lists the rest, and the exact selection runs on that

@@ -19,6 +19,7 @@
 #include "sample.cuh"
 #include "lstep.cuh"
 #include "thin.cuh"
+#include "small_select.cuh"
 
 using namespace cs;
 
@@ -57,6 +58,7 @@ struct condensa_ctx {
     Ctl *ctl = nullptr;
     int occ_select[3] = {0, 0, 0};
     int occ_stream = 0;
+    bool small_smem_set = false;    // dynamic shared memory limit of k_select_small raised on this device
     DeviceMirror mirror;
     // optional per-kernel timing (event pair around every launch)
     bool prof_on = false;
@@ -511,6 +513,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         const long long k = pl.S - Z;
         Sel init = initial_state(pl.S, k, P.bits_key);
         const int do_list0 = (u64)pl.S <= pl.cap ? 1 : 0;
+        // rankings of a short key array (filters, rows, general blocks) skip the grid-wide selection
+        const bool small = (op == OP_FILTER || op == OP_BLOCKGEN) && pl.S <= SMALL_S_MAX &&
+                           !(fuse & CONDENSA_NO_SAMPLING);
 
         Params Pa = P;
         Pa.item_prefix = pa;
@@ -556,13 +561,24 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
 #undef CS_LAUNCH_FUSED
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
+        } else if (small) {
+            // a few thousand structures: the whole selection in one CTA
+            if (!ctx->small_smem_set) {
+                CU_TRY(ctx, cudaFuncSetAttribute(k_select_small, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)(sizeof(u64) * SMALL_S_MAX)));
+                ctx->small_smem_set = true;
+            }
+            const int pi_ = prof_begin(ctx, "k_select_small", stream);
+            k_select_small<<<1, SMALL_THREADS, sizeof(u64) * (size_t)pl.S, stream>>>(Pa, init);
+            LAUNCH_CHECK(ctx);
+            prof_end(ctx, pi_, stream);
         } else {
             int pi_ = prof_begin(ctx, "k_init", stream);
             k_init<<<8, THREADS, 0, stream>>>(P, init);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
         }
-        if (!init.done) {
+        if (!init.done && !small) {
             const int ps_ = prof_begin(ctx, op == OP_PRUNE ? "k_scan_elem" : op == OP_BLOCK ? "k_scan_block" : "k_scan_array", stream);
             if (op == OP_PRUNE) {
                 k_scan<SRC_ELEM><<<stream_grid(ctx, pl.n_items_a, 4), THREADS, 0, stream>>>(Pa, do_list0);
@@ -594,7 +610,8 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pr_, stream);
         }
-        if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, stream);
+        if (small) rc = CONDENSA_OK;
+        else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, stream);
         else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, stream);
         else rc = launch_select<SRC_ARRAY>(ctx, Pa, do_list0, stream);
         if (rc) return rc;

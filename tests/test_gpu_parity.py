@@ -333,6 +333,28 @@ def test_neuron_and_structure_pruning(ctx, op):
     assert res.n_units == sum(a.shape[0] for a in ws.w if a.ndim == 2)
 
 
+@pytest.mark.parametrize("extra", [(), ("no_sampling",)])
+def test_short_rankings_one_cta_and_general_selection_agree(ctx, extra):
+    """Rankings of at most 16384 structures run in one CTA; `no_sampling` forces the
+    grid-wide selection. Both must give the oracle's result: many equal norms (ties
+    settled by index), every rank from the first to the last, k = 0 and k = S, and a
+    ranking just below and just above the one-CTA limit."""
+    rng = np.random.default_rng(9)
+    vals = rng.integers(1, 6, size=700).astype(np.float32)        # few distinct norms: long ties
+    rows = np.repeat(vals[:, None], 8, axis=1) * np.where(rng.random((700, 8)) < 0.5, -1, 1).astype(np.float32)
+    for s in (0.0, 1 / 700, 0.31, 0.5, 0.77, 1 - 1 / 700, 1.0):
+        got, res, exp = check(ctx, "neuron", [rows], None, s, 1.0, tuple(extra))
+    assert res.n_units == 700
+    # blocks of a general shape: 5 x 5 blocks of a 200 x 300 matrix (2400 units), with lambda
+    ws = W.random_set([(200, 300), (64,)], seed=12, kind="normal", scale=0.2, lam_sigma=1e-2, mu=1e-2)
+    check(ctx, "block", ws.w, ws.lam, 0.6, ws.mu, ("lambda",) + tuple(extra), block=(5, 5))
+    # around the limit: 16384 and 16385 rows
+    for n in (16384, 16385):
+        m = W.draw(n * 4, "normal", 1.0, 13, 0, 0).reshape(n, 4)
+        got, res, _ = check(ctx, "neuron", [m], None, 0.9, 1.0, tuple(extra), exact_key=False)
+        assert res.n_units == n
+
+
 @pytest.mark.parametrize("scale", [0.25, 1.0])
 def test_filter_configuration(ctx, scale):
     ws = W.config(3, scale=scale)
