@@ -531,10 +531,12 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             k_filter_partial<<<stream_grid(ctx, (pl.n_items_a + WARPS - 1) / WARPS, 8), THREADS, 0, stream>>>(Pa);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pa_, stream);
-            pa_ = prof_begin(ctx, "k_filter_combine", stream);
-            k_filter_combine<<<stream_grid(ctx, (pl.S + THREADS - 1) / THREADS, 8), THREADS, 0, stream>>>(Pa);
-            LAUNCH_CHECK(ctx);
-            prof_end(ctx, pa_, stream);
+            if (!small) {           // the one-CTA selection forms the norms itself
+                pa_ = prof_begin(ctx, "k_filter_combine", stream);
+                k_filter_combine<<<stream_grid(ctx, (pl.S + THREADS - 1) / THREADS, 8), THREADS, 0, stream>>>(Pa);
+                LAUNCH_CHECK(ctx);
+                prof_end(ctx, pa_, stream);
+            }
         }
         Params Pf = P;                      // single-pass kernel runs on the projection decomposition
         Pf.item_prefix = pb;
@@ -569,7 +571,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
                 ctx->small_smem_set = true;
             }
             const int pi_ = prof_begin(ctx, "k_select_small", stream);
-            k_select_small<<<1, SMALL_THREADS, sizeof(u64) * (size_t)pl.S, stream>>>(Pa, init);
+            k_select_small<<<1, SMALL_THREADS, sizeof(u64) * (size_t)pl.S, stream>>>(Pa, init, op == OP_FILTER ? 1 : 0);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
         } else {

@@ -11,13 +11,19 @@
 #pragma once
 #include "common.cuh"
 #include "select.cuh"
+#include "structured.cuh"
 
 namespace cs {
 
 constexpr int SMALL_THREADS = 1024;
 constexpr int SMALL_S_MAX = 16384;       // keys held in shared memory (128 KB)
 
+constexpr int SMALL_T_CACHE = 512;       // tensors whose ranges are cached in shared memory
+
 struct SmallShared {
+    long long t_units[SMALL_T_CACHE + 1];  // first structure of every tensor (+ total)
+    long long t_items[SMALL_T_CACHE];      // first partial sum of every tensor
+    int t_nseg[SMALL_T_CACHE];             // partial sums per filter
     u32 hist[NBINS];
     u32 wsum[SMALL_THREADS / 32];
     u32 pick_bin, pick_before, pick_count;
@@ -43,13 +49,48 @@ __device__ __forceinline__ u32 small_excl_scan(u32 v, u32 *wsum)
     return base + inc - v;
 }
 
-__global__ void __launch_bounds__(SMALL_THREADS) k_select_small(Params P, Sel init)
+// `combine`: the keys are first formed from the filter partial sums (and stored
+// to the key array, which the projection reads).
+__global__ void __launch_bounds__(SMALL_THREADS) k_select_small(Params P, Sel init, int combine)
 {
     extern __shared__ __align__(16) u64 skey[];        // [S]
     __shared__ SmallShared sh;
     Ctl *c = P.ctl;
     const u32 S = (u32)init.S;
-    for (u32 i = threadIdx.x; i < S; i += SMALL_THREADS) skey[i] = P.arr_key[i];
+    if (combine && P.T <= SMALL_T_CACHE) {
+        // tensor ranges first (one round trip), then every key needs only its partial sums
+        for (int t = threadIdx.x; t < P.T; t += SMALL_THREADS) {
+            const TensorDesc &d = P.td[t];
+            sh.t_units[t] = d.unit_prefix;
+            sh.t_items[t] = P.item_prefix[t];
+            sh.t_nseg[t] = (int)((d.d1 + SEG - 1) / SEG);
+        }
+        if (threadIdx.x == 0) sh.t_units[P.T] = (long long)S;
+        __syncthreads();
+        for (u32 i = threadIdx.x; i < S; i += SMALL_THREADS) {
+            int lo = 0, hi = P.T - 1;          // the tensor with t_units[t] <= i < t_units[t + 1]
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (sh.t_units[mid] <= (long long)i) lo = mid; else hi = mid - 1;
+            }
+            while (lo > 0 && sh.t_units[lo + 1] == sh.t_units[lo]) --lo;      // tensors without ranked structures
+            const int nseg = sh.t_nseg[lo];
+            const double *p = P.partial + sh.t_items[lo] + ((long long)i - sh.t_units[lo]) * nseg;
+            double acc = 0.0;
+            for (int sgm = 0; sgm < nseg; ++sgm) acc = __dadd_rn(acc, p[sgm]);      // segment order, as k_filter_combine
+            const u64 key = (u64)__double_as_longlong(acc);
+            P.arr_key[i] = key;
+            skey[i] = key;
+        }
+    } else if (combine) {
+        for (u32 i = threadIdx.x; i < S; i += SMALL_THREADS) {
+            const u64 key = filter_norm_key(P, (long long)i);
+            P.arr_key[i] = key;
+            skey[i] = key;
+        }
+    } else {
+        for (u32 i = threadIdx.x; i < S; i += SMALL_THREADS) skey[i] = P.arr_key[i];
+    }
     if (threadIdx.x == 0) {
         // what the start kernel of the general path does
         c->tau_key = KEY_NONE;

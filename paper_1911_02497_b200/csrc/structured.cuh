@@ -194,28 +194,32 @@ __global__ void __launch_bounds__(THREADS) k_blockgen_norms(Params P)
     }
 }
 
-// Filter norms, step 2: nu_f = partial sums added in segment order.
+// Filter norms, step 2: nu_f = partial sums added in segment order (fp64 bits).
+__device__ __forceinline__ u64 filter_norm_key(const Params &P, long long sid)
+{
+    // tensor that owns structure sid
+    int lo = 0, hi = P.T - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (P.td[mid].unit_prefix <= sid) lo = mid; else hi = mid - 1;
+    }
+    // skip tensors without ranked structures that share the same prefix
+    int t = lo;
+    while (t > 0 && P.td[t].n_units == 0) --t;
+    const TensorDesc &d = P.td[t];
+    const long long f = sid - d.unit_prefix;
+    const long long nseg = (d.d1 + SEG - 1) / SEG;
+    const double *p = P.partial + P.item_prefix[t] + f * nseg;
+    double acc = 0.0;
+    for (long long sgm = 0; sgm < nseg; ++sgm) acc = __dadd_rn(acc, p[sgm]);
+    return (u64)__double_as_longlong(acc);
+}
+
 __global__ void __launch_bounds__(THREADS) k_filter_combine(Params P)
 {
     const long long stride = (long long)gridDim.x * THREADS;
-    for (long long sid = (long long)blockIdx.x * THREADS + threadIdx.x; sid < P.S; sid += stride) {
-        // tensor that owns structure sid
-        int lo = 0, hi = P.T - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (P.td[mid].unit_prefix <= sid) lo = mid; else hi = mid - 1;
-        }
-        // skip tensors without ranked structures that share the same prefix
-        int t = lo;
-        while (t > 0 && P.td[t].n_units == 0) --t;
-        const TensorDesc d = P.td[t];
-        const long long f = sid - d.unit_prefix;
-        const long long nseg = (d.d1 + SEG - 1) / SEG;
-        const double *p = P.partial + P.item_prefix[t] + f * nseg;
-        double acc = 0.0;
-        for (long long sgm = 0; sgm < nseg; ++sgm) acc = __dadd_rn(acc, p[sgm]);
-        P.arr_key[sid] = (u64)__double_as_longlong(acc);
-    }
+    for (long long sid = (long long)blockIdx.x * THREADS + threadIdx.x; sid < P.S; sid += stride)
+        P.arr_key[sid] = filter_norm_key(P, sid);
 }
 
 }  // namespace cs
