@@ -541,7 +541,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         Params Pf = P;                      // single-pass kernel runs on the projection decomposition
         Pf.item_prefix = pb;
         Pf.n_items = pl.n_items_b;
-        if (sampling && op == OP_BLOCK) Pa.n_edge_items = 0;     // the block kernel does its edge items itself
+        if (sampling) Pa.n_edge_items = 0;     // the single-pass kernels do their edge items themselves
         if (sampling && !init.done) {
             int pi_ = prof_begin(ctx, "k_sample", stream);
             if (op == OP_PRUNE) k_sample<SRC_ELEM><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);

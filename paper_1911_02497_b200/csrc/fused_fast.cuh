@@ -12,9 +12,11 @@ namespace cs {
 constexpr int ESTG = 64;        // staged candidates per warp
 
 struct ElemFastShared {
-    u32 hist[NBINS];
-    u32 wcount[WARPS];
+    u32 hist[NBINS];            // the first four members mirror FusedShared (edge items reuse them)
+    u32 cnt[2];
+    u64 base[2];
     u64 red[WARPS];
+    u32 wcount[WARPS];
     u64 id[WARPS][ESTG];
     u32 key[WARPS][ESTG];
     float lam[WARPS][ESTG];
@@ -167,8 +169,25 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
     }
     elem_flush(P, sh, true, 0);
     __syncthreads();
-    // totals of this CTA
     u64 na = n_above;
+    // the items outside the aligned fast path (tensor heads and tails, unaligned
+    // tensors), listed by the host
+    if (P.n_edge_items > 0) {
+        FusedShared &fs = reinterpret_cast<FusedShared &>(sh);
+        if (threadIdx.x < 2) fs.cnt[threadIdx.x] = 0;
+        __syncthreads();
+        const long long *prefix_b = P.edge_items + P.n_edge_items;      // [T+1] projection items per tensor
+        int par = 0;
+        for (long long i = blockIdx.x; i < P.n_edge_items; i += gridDim.x) {
+            const long long item = P.edge_items[i];
+            const int t = find_tensor(prefix_b, P.T, item);
+            const TensorDesc g = P.td[t];
+            fused_elem_item_generic<H>(P, g, item - prefix_b[t], fs, br, par, na, fp16);
+            par ^= 1;
+        }
+        __syncthreads();
+    }
+    // totals of this CTA
     for (int o = 16; o > 0; o >>= 1) na += __shfl_xor_sync(0xffffffffu, na, o);
     if ((threadIdx.x & 31) == 0) sh.red[warp] = na;
     __syncthreads();
