@@ -284,11 +284,21 @@ __device__ __noinline__ void scan_list(const Params &P, ScanShared &sh, int slot
 {
     ScanCtx c;
     scan_begin(sh, c, false);
-    const u64 stride = (u64)gridDim.x * THREADS;
-    for (u64 base = (u64)blockIdx.x * THREADS; base < n_list; base += stride) {
-        const u64 i = base + threadIdx.x;
-        const bool ok = i < n_list;
-        scan_emit(P, sh, c, ok ? __ldcg(&P.list_key[i]) : 0, ok ? __ldcg(&P.list_id[i]) : 0, ok);
+    // several entries per thread are fetched before the first is used: the walk is
+    // a few rounds per thread and would otherwise pay one memory round trip per entry
+    constexpr int R = 8;
+    const u64 chunk = (u64)R * THREADS;
+    for (u64 base = (u64)blockIdx.x * chunk; base < n_list; base += (u64)gridDim.x * chunk) {
+        u64 key[R], id[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const u64 i = base + (u64)r * THREADS + threadIdx.x;
+            key[r] = i < n_list ? __ldcg(&P.list_key[i]) : 0;
+            id[r] = i < n_list ? __ldcg(&P.list_id[i]) : 0;
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            scan_emit(P, sh, c, key[r], id[r], base + (u64)r * THREADS + threadIdx.x < n_list);
     }
     scan_end(P, sh, c, slot);
 }
@@ -741,14 +751,27 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
                 const u64 n_list = __ldcg(&P.ctl->list_count[sh.sel.list_sel]);
                 const Sel &s = sh.sel;
                 const bool sk = s.lo_key == s.hi_key;
-                const u64 stride = (u64)gridDim.x * THREADS;
-                for (u64 i = (u64)blockIdx.x * THREADS + threadIdx.x; i < n_list; i += stride) {
-                    const u64 key = __ldcg(&P.list_key[i]), id = __ldcg(&P.list_id[i]);
-                    const bool above = key > s.hi_key || (sk && key == s.hi_key && id < s.lo_id);
-                    const bool below = key < s.lo_key || (sk && key == s.lo_key && id > s.hi_id);
-                    if (!above && !below) {
-                        const u32 pos = atomicAdd(&P.ctl->fin_count, 1u);
-                        if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; P.fin_idx[pos] = i; }
+                constexpr int R = 8;                 // entries fetched per thread before the first is used
+                const u64 chunk = (u64)R * THREADS;
+                for (u64 base = (u64)blockIdx.x * chunk; base < n_list; base += (u64)gridDim.x * chunk) {
+                    u64 kk[R], dd[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const u64 i = base + (u64)r * THREADS + threadIdx.x;
+                        kk[r] = i < n_list ? __ldcg(&P.list_key[i]) : 0;
+                        dd[r] = i < n_list ? __ldcg(&P.list_id[i]) : 0;
+                    }
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const u64 i = base + (u64)r * THREADS + threadIdx.x;
+                        if (i >= n_list) continue;
+                        const u64 key = kk[r], id = dd[r];
+                        const bool above = key > s.hi_key || (sk && key == s.hi_key && id < s.lo_id);
+                        const bool below = key < s.lo_key || (sk && key == s.lo_key && id > s.hi_id);
+                        if (!above && !below) {
+                            const u32 pos = atomicAdd(&P.ctl->fin_count, 1u);
+                            if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; P.fin_idx[pos] = i; }
+                        }
                     }
                 }
                 TSTAMP();
