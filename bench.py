@@ -419,8 +419,13 @@ def run_ours(args):
             if not small:
                 got_mask = [m.cpu().numpy().reshape(s) for m, s in zip(hm, ws.shapes)]
                 cpu["parity_mask_equal"] = bool(all(np.array_equal(a, b) for a, b in zip(got_mask, out.mask)))
-                cpu["parity_tau_equal"] = bool(res.tau_key == out.result.tau_key and
-                                               res.tau_id == out.result.tau_id)
+                key_ok = res.tau_key == out.result.tau_key
+                if ws.op == "filter" and not key_ok:
+                    # filter norms: the fp64 summation order differs from the oracle's sequential one
+                    a, b = (np.array([k], np.uint64).view(np.float64)[0] for k in (res.tau_key, out.result.tau_key))
+                    key_ok = bool(abs(a - b) <= 1e-12 * abs(b))
+                    cpu["tau_key_rel_err"] = float(abs(a - b) / abs(b)) if b else 0.0
+                cpu["parity_tau_equal"] = bool(key_ok and res.tau_id == out.result.tau_id)
         line = {"metric": "cstep_params_per_s", "value": value, "unit": "params/s", "n_gpus": world,
                 "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
