@@ -31,7 +31,7 @@ L2_BYTES = 126 * 1024 * 1024
 # Keyed by (kernel, fuse); set an entry to None when the kernel changes after its capture.
 NCU_TRAFFIC_PER_PARAM = {
     ("k_fused_block", ("lambda",)): 15.60,
-    ("k_fused_elem", ("fp16", "lambda", "penalty")): 18.86,
+    ("k_fused_elem", ("fp16", "lambda", "penalty")): 18.94,
 }
 FALLBACK_HBM_GBS = 6650.0
 
