@@ -413,12 +413,12 @@ void prof_collect(condensa_ctx *ctx)
     } while (0)
 
 template <int SRC>
-int launch_select(condensa_ctx *ctx, Params &P, int first_listed, cudaStream_t stream)
+int launch_select(condensa_ctx *ctx, Params &P, int first_listed, int pre_scan, cudaStream_t stream)
 {
     if (!ctx->occ_select[SRC]) ctx->occ_select[SRC] = occupancy(k_select<SRC>);
     const int per_sm = std::min(ctx->occ_select[SRC], 2);
     dim3 grid((unsigned)(ctx->num_sms * per_sm)), block(THREADS);
-    void *args[] = {(void *)&P, (void *)&first_listed};
+    void *args[] = {(void *)&P, (void *)&first_listed, (void *)&pre_scan};
     const int pa_ = prof_begin(ctx, "k_select", stream);
     CU_TRY(ctx, cudaLaunchCooperativeKernel((const void *)k_select<SRC>, grid, block, args, 0, stream));
     ctx->launches += 1;
@@ -580,7 +580,8 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
         }
-        if (!init.done && !small) {
+        // with the single-pass path the fallback scan, if it is needed at all, runs inside k_select
+        if (!init.done && !small && !sampling) {
             const int ps_ = prof_begin(ctx, op == OP_PRUNE ? "k_scan_elem" : op == OP_BLOCK ? "k_scan_block" : "k_scan_array", stream);
             if (op == OP_PRUNE) {
                 k_scan<SRC_ELEM><<<stream_grid(ctx, pl.n_items_a, 4), THREADS, 0, stream>>>(Pa, do_list0);
@@ -613,9 +614,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             prof_end(ctx, pr_, stream);
         }
         if (small) rc = CONDENSA_OK;
-        else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, stream);
-        else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, stream);
-        else rc = launch_select<SRC_ARRAY>(ctx, Pa, do_list0, stream);
+        else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, sampling ? 1 : 0, stream);
+        else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, sampling ? 1 : 0, stream);
+        else rc = launch_select<SRC_ARRAY>(ctx, Pa, do_list0, 0, stream);
         if (rc) return rc;
         ctx->has_result = true;
     }
@@ -1212,7 +1213,8 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
     if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     {
         dim3 grid((unsigned)(sms * std::min(g_noalloc_occ[dev], 2))), block(THREADS);
-        void *args[] = {(void *)&P, (void *)&do_list0};
+        int pre_scan = 0;        // the scan kernel above has run
+        void *args[] = {(void *)&P, (void *)&do_list0, (void *)&pre_scan};
         e = cudaLaunchCooperativeKernel((const void *)k_select<SRC_ELEM>, grid, block, args, 0, stream);
         if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     }

@@ -688,8 +688,11 @@ __global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
 
 // Cooperative driver: picks, further scans, direct ranking of the last few,
 // result record. Entered with the histogram of the first scan in slot 0.
+// `pre_scan`: no scan kernel ran before this launch (the call went for the single
+// pass); if the sample advised against it, the first full histogram pass is
+// made here.
 template <int SRC>
-__global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
+__global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, int pre_scan)
 {
     __shared__ ScanShared sh;
     cg::grid_group grid = cg::this_grid();
@@ -716,6 +719,10 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed)
     }
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
     __syncthreads();
+    if (pre_scan && !sh.sel.onepass && !sh.sel.done) {
+        scan_source<SRC>(P, sh, first_listed != 0, sh.sel.slot);
+        grid.sync();
+    }
 #ifdef CONDENSA_DEBUG_TIME
     unsigned long long tq[8]; int nq = 0;
 #define TSTAMP() do { if (blockIdx.x == 0 && threadIdx.x == 0 && nq < 8) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); tq[nq++] = t_; } } while (0)
