@@ -413,12 +413,14 @@ void prof_collect(condensa_ctx *ctx)
     } while (0)
 
 template <int SRC>
-int launch_select(condensa_ctx *ctx, Params &P, int first_listed, int pre_scan, cudaStream_t stream)
+int launch_select(condensa_ctx *ctx, Params &P, int first_listed, int pre_scan, cudaStream_t stream,
+                  const long long *prefix_b = nullptr, long long n_items_b = 0, int post_apply = 0)
 {
     if (!ctx->occ_select[SRC]) ctx->occ_select[SRC] = occupancy(k_select<SRC>);
     const int per_sm = std::min(ctx->occ_select[SRC], 2);
     dim3 grid((unsigned)(ctx->num_sms * per_sm)), block(THREADS);
-    void *args[] = {(void *)&P, (void *)&first_listed, (void *)&pre_scan};
+    void *args[] = {(void *)&P, (void *)&first_listed, (void *)&pre_scan, (void *)&prefix_b, (void *)&n_items_b,
+                    (void *)&post_apply};
     const int pa_ = prof_begin(ctx, "k_select", stream);
     CU_TRY(ctx, cudaLaunchCooperativeKernel((const void *)k_select<SRC>, grid, block, args, 0, stream));
     ctx->launches += 1;
@@ -508,6 +510,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
 
     if (!ctx->occ_stream) ctx->occ_stream = 3;
 
+    bool applied_in_select = false;
     if (ranking) {
         const long long Z = (long long)std::min<double>((double)pl.S, std::max(0.0, std::floor(sparsity * (double)pl.S + 0.5)));
         const long long k = pl.S - Z;
@@ -613,9 +616,12 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pr_, stream);
         }
+        // a call that went for the single pass needs no projection launch: after a fall-back k_select projects itself
+        const int post_apply = sampling && !init.done ? (need_h ? 2 : 1) : 0;
+        applied_in_select = post_apply != 0;
         if (small) rc = CONDENSA_OK;
-        else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, sampling ? 1 : 0, stream);
-        else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, sampling ? 1 : 0, stream);
+        else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, sampling ? 1 : 0, stream, pb, pl.n_items_b, post_apply);
+        else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, sampling ? 1 : 0, stream, pb, pl.n_items_b, post_apply);
         else rc = launch_select<SRC_ARRAY>(ctx, Pa, do_list0, 0, stream);
         if (rc) return rc;
         ctx->has_result = true;
@@ -624,7 +630,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     Params Pb = P;
     Pb.item_prefix = pb;
     Pb.n_items = pl.n_items_b;
-    if (pl.n_items_b > 0) {
+    if (pl.n_items_b > 0 && !applied_in_select) {
         const int grid = stream_grid(ctx, pl.n_items_b, ctx->occ_stream);
         static const char *apply_names[6] = {"k_apply_prune", "k_apply_filter", "k_apply_block", "k_quantize", "k_lagrange", "k_apply_blockgen"};
         const int pa_ = prof_begin(ctx, apply_names[op], stream);
@@ -1213,8 +1219,11 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
     if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     {
         dim3 grid((unsigned)(sms * std::min(g_noalloc_occ[dev], 2))), block(THREADS);
-        int pre_scan = 0;        // the scan kernel above has run
-        void *args[] = {(void *)&P, (void *)&do_list0, (void *)&pre_scan};
+        int pre_scan = 0, post_apply = 0;        // the scan kernel above has run; the projection kernel follows
+        const long long *no_prefix = nullptr;
+        long long no_items = 0;
+        void *args[] = {(void *)&P, (void *)&do_list0, (void *)&pre_scan, (void *)&no_prefix, (void *)&no_items,
+                        (void *)&post_apply};
         e = cudaLaunchCooperativeKernel((const void *)k_select<SRC_ELEM>, grid, block, args, 0, stream);
         if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     }

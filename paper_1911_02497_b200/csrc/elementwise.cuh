@@ -285,17 +285,10 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
     }
 }
 
-// Persistent CTAs stride over the linear work items of the whole list. H: the
-// binary16 bits are needed (fp16 fuse or a theta_h output).
+// The linear work items of the whole list, strided over the CTAs of the grid.
 template <int MODE, bool H>
-__global__ void __launch_bounds__(THREADS, 3) k_apply_linear(Params P)
+__device__ __forceinline__ void apply_linear_items(const Params &P, u64 tau_key, u64 tau_id)
 {
-    u64 tau_key = 0, tau_id = 0;
-    if (MODE == M_PRUNE || MODE == M_FILTER || MODE == M_BLOCKGEN) {
-        if (P.ctl->sel.onepass) return;      // the single-pass kernel has written everything
-        tau_key = P.ctl->tau_key;
-        tau_id = P.ctl->tau_id;
-    }
     long long t_first = 0, t_end = -1;
     TensorDesc d;
     d.numel = 0; d.pad = 0; d.vec_ok = 0;
@@ -310,6 +303,20 @@ __global__ void __launch_bounds__(THREADS, 3) k_apply_linear(Params P)
         if (elem_item_is_fast(d, local)) process_linear_item_fast<MODE, H>(P, d, local, tau_key, tau_id);
         else process_linear_item<MODE>(P, d, local, tau_key, tau_id);
     }
+}
+
+// Persistent CTAs stride over the linear work items of the whole list. H: the
+// binary16 bits are needed (fp16 fuse or a theta_h output).
+template <int MODE, bool H>
+__global__ void __launch_bounds__(THREADS, 3) k_apply_linear(Params P)
+{
+    u64 tau_key = 0, tau_id = 0;
+    if (MODE == M_PRUNE || MODE == M_FILTER || MODE == M_BLOCKGEN) {
+        if (P.ctl->sel.onepass) return;      // the single-pass kernel has written everything
+        tau_key = P.ctl->tau_key;
+        tau_id = P.ctl->tau_id;
+    }
+    apply_linear_items<MODE, H>(P, tau_key, tau_id);
 }
 
 }  // namespace cs

@@ -567,6 +567,10 @@ __device__ __forceinline__ void write_result(const Params &P, const Sel &s)
     c->res = r;
 }
 
+// Defined with the projection kernels: the final write with the exact cut-off.
+template <int SRC>
+__device__ void apply_after_select(const Params &P, int need_h);
+
 // Defined with the single-pass kernels: rewrites one listed unit.
 template <int SRC>
 __device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, const long long *pre_s);
@@ -690,9 +694,12 @@ __global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
 // result record. Entered with the histogram of the first scan in slot 0.
 // `pre_scan`: no scan kernel ran before this launch (the call went for the single
 // pass); if the sample advised against it, the first full histogram pass is
-// made here.
+// made here. `post_apply` (1, or 2 when the 16-bit codes are needed): no
+// projection kernel follows this launch; after such a fall-back the final write
+// is made here too, on the projection work items `prefix_b` / `n_items_b`.
 template <int SRC>
-__global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, int pre_scan)
+__global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, int pre_scan,
+                                                    const long long *prefix_b, long long n_items_b, int post_apply)
 {
     __shared__ ScanShared sh;
     cg::grid_group grid = cg::this_grid();
@@ -828,6 +835,16 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
     }
 #endif
     if (blockIdx.x == 0 && threadIdx.x == 0) write_result(P, sh.sel);
+    if constexpr (SRC != SRC_ARRAY) {
+        if (post_apply && !sh.sel.onepass) {       // the same on every CTA: the sampler's verdict never changes
+            __threadfence();
+            grid.sync();
+            Params Pb = P;
+            Pb.item_prefix = prefix_b;
+            Pb.n_items = n_items_b;
+            apply_after_select<SRC>(Pb, post_apply == 2);
+        }
+    }
 }
 
 // Common end of the single-pass path, without a grid barrier. Every CTA makes the

@@ -58,10 +58,8 @@ __device__ __forceinline__ void store_block(const TensorDesc &d, const BlockData
 
 // Projection pass of block pruning. Work items: BLOCKS_PER_ITEM blocks for
 // ranked (2-D) tensors, linear items for tensors that pass through.
-__global__ void __launch_bounds__(THREADS) k_apply_block(Params P)
+__device__ __forceinline__ void apply_block_items(const Params &P, u64 tau_key, u64 tau_id)
 {
-    if (P.ctl->sel.onepass) return;          // the single-pass kernel has written everything
-    const u64 tau_key = P.ctl->tau_key, tau_id = P.ctl->tau_id;
     for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
         const int t = find_tensor(P.item_prefix, P.T, item);
         const TensorDesc d = P.td[t];
@@ -82,6 +80,27 @@ __global__ void __launch_bounds__(THREADS) k_apply_block(Params P)
             const bool keep = keep_by_cutoff(key, (u64)(d.unit_prefix + b), tau_key, tau_id);
             store_block(d, bd, u, keep, P.mu, P.fuse);
         }
+    }
+}
+
+__global__ void __launch_bounds__(THREADS) k_apply_block(Params P)
+{
+    if (P.ctl->sel.onepass) return;          // the single-pass kernel has written everything
+    apply_block_items(P, P.ctl->tau_key, P.ctl->tau_id);
+}
+
+// Projection with the exact cut-off at the end of the selection kernel (declared
+// there): used when a call that went for the single pass had to fall back.
+template <int SRC>
+__device__ __noinline__ void apply_after_select(const Params &P, int need_h)
+{
+    // the cut-off was written by another CTA of this launch: read it past the L1
+    const u64 tau_key = __ldcg(&P.ctl->tau_key), tau_id = __ldcg(&P.ctl->tau_id);
+    if (SRC == SRC_ELEM) {
+        if (need_h) apply_linear_items<M_PRUNE, true>(P, tau_key, tau_id);
+        else apply_linear_items<M_PRUNE, false>(P, tau_key, tau_id);
+    } else if (SRC == SRC_BLOCK) {
+        apply_block_items(P, tau_key, tau_id);
     }
 }
 
