@@ -462,11 +462,15 @@ __device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
         // few survivors: count, for each, how many rank before it
         for (u32 i = threadIdx.x; i < n; i += THREADS) {
             const u64 ki = k[i], di = d[i];
-            u32 before = 0;
+            u32 before = 0, same = 0;
 #pragma unroll 8
             for (u32 j = 0; j < n; ++j) {
-                const u64 kj = k[j], dj = d[j];          // branch-free: both loads always issue
-                before += (u32)(kj > ki) | ((u32)(kj == ki) & (u32)(dj < di));
+                const u64 kj = k[j];                     // keys only: equal keys are rare
+                before += (u32)(kj > ki);
+                same += (u32)(kj == ki);
+            }
+            if (same > 1) {                              // ties beside itself: the lower id ranks first
+                for (u32 j = 0; j < n; ++j) before += (u32)(k[j] == ki) & (u32)(d[j] < di);
             }
             if ((u64)before + 1 == r) sh.fin_hit = (int)i;
         }
@@ -864,6 +868,13 @@ __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
     __shared__ u32 s_last;
     Ctl *c = P.ctl;
     const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
+#ifdef CONDENSA_DEBUG_TIME
+    unsigned long long tr[8]; int nr = 0;
+#define RSTAMP() do { if (threadIdx.x == 0 && nr < 8) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); tr[nr++] = t_; } } while (0)
+#else
+#define RSTAMP() do {} while (0)
+#endif
+    RSTAMP();
     if (threadIdx.x == 0) sh.sel = c->sel;
     // this CTA's first chunk of the list is fetched while the pick is made
     const u64 n_all = __ldcg(&c->list_count[0]);
@@ -875,6 +886,7 @@ __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
     if (threadIdx.x == 0) sh.sel.list_valid = 1;
     __syncthreads();
     block_pick(P, sh, true, max_key);
+    RSTAMP();
     if (sh.sel.error) return;
     const bool need_rank = !sh.sel.done;
     if (need_rank && sh.sel.pop > FIN) return;
@@ -882,22 +894,31 @@ __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
         const u64 fixed = list_repair_pass<SRC>(P, sh, need_rank, n_list, &pre);
         if (fixed) atomicAdd(&c->n_repaired, fixed);
     }
+    RSTAMP();
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) s_last = atomicAdd(&c->resolve_done, 1u) == gridDim.x - 1 ? 1u : 0u;
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    RSTAMP();
     if (need_rank) {
         const u32 n = __ldcg(&c->fin_count);
         if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
         __syncthreads();
         final_rank(P, sh, n);      // its members are rewritten by the next launch
     }
+    RSTAMP();
     if (threadIdx.x == 0) {
         write_result(P, sh.sel);
         c->resolved = 1;
         c->resolve_done = 0;
+#ifdef CONDENSA_DEBUG_TIME
+        RSTAMP();
+        printf("k_resolve last CTA %d phases (us):", (int)blockIdx.x);
+        for (int i = 1; i < nr; ++i) printf(" %.1f", (double)(tr[i] - tr[i - 1]) * 1e-3);
+        printf("\n");
+#endif
     }
 }
 
