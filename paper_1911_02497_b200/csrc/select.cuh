@@ -573,7 +573,7 @@ __device__ __forceinline__ void write_result(const Params &P, const Sel &s)
 
 // Defined with the projection kernels: the final write with the exact cut-off.
 template <int SRC>
-__device__ void apply_after_select(const Params &P, int need_h);
+__device__ __noinline__ void apply_after_select(const Params &P, int need_h);
 
 // Defined with the single-pass kernels: rewrites one listed unit.
 template <int SRC>
