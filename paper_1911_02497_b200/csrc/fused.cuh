@@ -283,38 +283,6 @@ __device__ __forceinline__ void fused_elem_item_generic(const Params &P, const T
     }
 }
 
-// The remaining projection items, listed by the host in P.edge_items. Runs inside
-// the first-pass launch when the single-pass path is active. P.item_prefix is
-// the scan decomposition there, so the projection decomposition is passed in
-// P.edge_* with its own prefix array right behind the item list.
-template <int SRC>
-__device__ void fused_edge_items(const Params &P, FusedShared &sh)
-{
-    const Bracket br = load_bracket(P.ctl->sel);
-    for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
-    if (threadIdx.x < 2) sh.cnt[threadIdx.x] = 0;
-    __syncthreads();
-    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
-    const long long *prefix_b = P.edge_items + P.n_edge_items;      // [T+1]
-    u64 n_above = 0;
-    int par = 0;
-    for (long long i = blockIdx.x; i < P.n_edge_items; i += gridDim.x) {
-        const long long item = P.edge_items[i];
-        const int t = find_tensor(prefix_b, P.T, item);
-        const TensorDesc d = P.td[t];
-        const long long local = item - prefix_b[t];
-        if (SRC == SRC_ELEM) {
-            fused_elem_item_generic<true>(P, d, local, sh, br, par, n_above, fp16);
-            par ^= 1;
-        } else if (!d.ranked) {
-            process_linear_item<M_KEEPALL>(P, d, local, 0, 0);
-        } else {
-            fused_block_item_generic<true>(P, d, local, sh, br, par, n_above, fp16);
-        }
-    }
-    fused_finish(P, sh, n_above);
-}
-
 // Rewrite one listed unit whose provisional decision was wrong. Called from the
 // selection kernel after the cut-off is known. `idx` is the list position.
 // `pre_s`, when given, holds the tensors' first unit numbers in shared memory

@@ -579,18 +579,15 @@ __device__ __noinline__ void apply_after_select(const Params &P, int need_h);
 template <int SRC>
 __device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, const long long *pre_s);
 
-// Defined with the single-pass kernels: the projection items the aligned fast
-// kernel leaves out (tensor heads and tails, unaligned or ragged tensors).
+// Shared memory of the generic (edge) items of the single-pass kernels: the
+// projection items the aligned fast code leaves out (tensor heads and tails,
+// unaligned or ragged tensors).
 struct FusedShared {
     u32 hist[NBINS];
     u32 cnt[2];
     u64 base[2];
     u64 red[WARPS];
 };
-static_assert(sizeof(FusedShared) <= sizeof(ScanShared), "the edge items reuse the scan's shared memory");
-
-template <int SRC>
-__device__ void fused_edge_items(const Params &P, FusedShared &sh);
 
 // One walk over the list of the single-pass path by the whole grid. A listed unit
 // whose final decision is known and differs from the provisional one is rewritten;
@@ -678,17 +675,12 @@ __device__ __forceinline__ u64 list_repair_pass(const Params &P, ScanShared &sh,
     return fixed;
 }
 
-// First pass of a ranking call: a plain (non-cooperative) scan at full grid.
-// When the single-pass path is active there is nothing left to scan, and the
-// launch does that path's edge items instead.
+// First pass of a ranking call that does not go for the single pass: a plain
+// (non-cooperative) scan at full grid.
 template <int SRC>
 __global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
 {
     __shared__ ScanShared sh;
-    if (P.ctl->sel.onepass) {
-        if (SRC != SRC_ARRAY && P.n_edge_items > 0) fused_edge_items<SRC>(P, reinterpret_cast<FusedShared &>(sh));
-        return;
-    }
     if (threadIdx.x == 0) sh.sel = P.ctl->sel;
     __syncthreads();
     scan_source<SRC>(P, sh, do_list != 0, sh.sel.slot);
