@@ -235,6 +235,26 @@ def test_prune_ties_and_degenerate_inputs(ctx):
     check(ctx, "prune", [q], None, 0.9, 1.0, ("lambda",))
 
 
+def test_edge_sparsities_at_single_pass_sizes(ctx):
+    """Sizes that go for the single pass, with the sparsities at which it must step aside or
+    work at the very ends of the ranking: nothing pruned, everything pruned, one unit pruned,
+    one unit kept. With 16-bit output, so that the projection a fall-back makes inside the
+    selection kernel writes the codes too."""
+    n = 400000
+    w = W.draw(n, "normal", 0.05, 71, 0, 0)
+    lam = W.draw(n, "normal", 0.01, 71, 1, 0)
+    for s in (0.0, 1.0, 1.0 / n, 1.0 - 1.0 / n):
+        check(ctx, "prune", [w[:150000], w[150000:]], [lam[:150000], lam[150000:]], s, 1e-2, ("fp16", "lambda", "penalty"))
+    m = W.draw(600 * 1000, "uniform", 0.1, 72, 0, 0).reshape(600, 1000)        # 37500 blocks
+    big = W.draw(2400 * 1000, "uniform", 0.1, 73, 0, 0).reshape(2400, 1000)    # 150000 blocks: together a single-pass size
+    nb = 150000 + 37500
+    for s in (0.0, 1.0, 1.0 / nb, 1.0 - 1.0 / nb):
+        check(ctx, "block", [big, m, np.ones(7, np.float32)], None, s, 1e-3, ("bf16", "lambda"))
+    # a tie group far larger than the candidate list: the sample advises against the single pass
+    ties = np.where(np.arange(n) % 2 == 0, 0.25, -0.25).astype(np.float32)
+    check(ctx, "prune", [ties], None, 0.5, 1.0, ("fp16", "lambda"))
+
+
 def test_prune_k_zero_keep_all_and_empty_tensors(ctx):
     ws = W.random_set([(1000,), (0,), (37,)], seed=1, kind="normal", scale=1.0)
     for s in (0.0, 1.0, 1e-9, 1 - 1e-9):
