@@ -272,6 +272,90 @@ def test_structured_ties_use_structure_index():
     assert out.result.n_tie == 6 and out.result.n_tie_kept == 3 and out.result.tau_id == 2
 
 
+@pytest.mark.parametrize("block", [(5, 5), (3, 2), (1, 8), (8, 1), (2, 7)])
+def test_general_block_shapes_kept_set_mask_and_theta_bruteforce(block):
+    """BlockPrune with any block shape (Table 1; the LSTM run of the Evaluation uses
+    bs = 5): norms from numpy slices, kept set from the O(n^2) rank definition, the
+    element mask by np.kron of the block grid - non-square and ragged on purpose, so
+    that exchanging block height and width anywhere in the oracle fails here."""
+    bh, bw = block
+    shapes, s = [(11, 13), (6,), (33, 28)], 0.55
+    ws = W.random_set(shapes, seed=31, kind="normal", scale=0.2, lam_sigma=1e-2, mu=1e-2)
+    out = oracle.cstep_block(ws.w, ws.lam, s, ws.mu, block, fuse=("lambda",))
+    nu_ref = []
+    for t, shp in enumerate(shapes):
+        if len(shp) != 2:
+            continue
+        u = oracle.form_u(ws.w[t], ws.lam[t], ws.mu).astype(np.float64)
+        for br in range(-(-shp[0] // bh)):
+            for bc in range(-(-shp[1] // bw)):
+                blk = u[bh * br:bh * br + bh, bw * bc:bw * bc + bw]
+                acc = 0.0
+                for x in blk.reshape(-1):          # row by row inside the block
+                    acc = acc + x * x
+                nu_ref.append(acc)
+    nu_ref = np.array(nu_ref, np.float64)
+    nu = oracle.structure_norms(ws.w, ws.lam, ws.mu, "block", block)
+    assert np.array_equal(nu.view(np.uint64), nu_ref.view(np.uint64))
+    S = nu_ref.size
+    z = int(math.floor(s * S + 0.5))
+    keep_s = brute_keep(nu_ref.view(np.uint64), S - z)
+    assert out.result.n_units == S and out.result.n_zero == z and int(keep_s.sum()) == S - z
+    sid = 0
+    for t, shp in enumerate(shapes):
+        u = oracle.form_u(ws.w[t], ws.lam[t], ws.mu)
+        if len(shp) != 2:
+            assert out.mask[t].all() and np.array_equal(bits(out.theta[t]), bits(u))
+            continue
+        nbr, nbc = -(-shp[0] // bh), -(-shp[1] // bw)
+        grid = keep_s[sid:sid + nbr * nbc].reshape(nbr, nbc)
+        exp = np.kron(grid, np.ones((bh, bw), np.uint8))[:shp[0], :shp[1]]
+        sid += nbr * nbc
+        assert np.array_equal(out.mask[t], exp)
+        assert np.array_equal(bits(out.theta[t]), np.where(exp == 1, bits(u), 0))
+        # multiplier update on top of that theta: lambda' = lambda - mu (w - theta)
+        th = np.where(exp == 1, u, np.float32(0))
+        lam_ref = ws.lam[t] - np.float32(ws.mu) * (ws.w[t] - th)
+        assert np.array_equal(bits(out.lam[t]), bits(lam_ref.astype(np.float32)))
+    assert sid == S
+    kept_ids = np.flatnonzero(keep_s)
+    weakest = kept_ids[np.lexsort((-kept_ids, nu_ref[kept_ids]))[0]]
+    assert out.result.tau_id == weakest
+
+
+def test_general_block_ties_use_block_index():
+    blk = np.arange(6, dtype=np.float32).reshape(3, 2) + 1
+    w = np.tile(blk, (2, 4))                                   # 2 x 4 identical 3x2 blocks
+    out = oracle.cstep_block([w], [None], 0.5, 1.0, (3, 2))
+    assert out.mask[0][::3, ::2].tolist() == [[1, 1, 1, 1], [0, 0, 0, 0]]
+    assert out.result.n_tie == 8 and out.result.n_tie_kept == 4 and out.result.tau_id == 3
+    out = oracle.cstep_block([w.T.copy()], [None], 0.25, 1.0, (2, 3))     # 4 x 2 blocks of 2x3
+    assert out.mask[0][::2, ::3].tolist() == [[1, 1], [1, 1], [1, 1], [0, 0]]
+
+
+def test_filter_and_neuron_ties_use_structure_index():
+    """Bit-identical filters tie: the lower global structure id is kept, within a
+    tensor and across tensors, for FilterPrune and for the mixed StructurePrune list."""
+    rng = np.random.default_rng(17)
+    f = rng.standard_normal((1, 3, 3, 3)).astype(np.float32)
+    a = np.repeat(f, 4, axis=0)                                # four identical filters
+    b = np.repeat(f, 3, axis=0)
+    out = oracle.cstep_filter([a, b], [None, None], 3 / 7, 1.0)   # Z = 3 of 7, all tied
+    assert out.result.n_tie == 7 and out.result.n_tie_kept == 4 and out.result.tau_id == 3
+    assert out.mask[0].all() and not out.mask[1].any()
+    strong = (2 * f).astype(np.float32)
+    c = np.concatenate([f, strong, f, f], axis=0)              # ids 0..3, id 1 is the strongest
+    out = oracle.cstep_filter([c], [None], 0.5, 1.0)           # keep 2: id 1, then the lowest tied id 0
+    assert out.mask[0].reshape(4, -1)[:, 0].tolist() == [1, 1, 0, 0]
+    assert out.result.n_gt == 1 and out.result.n_tie == 3 and out.result.n_tie_kept == 1 and out.result.tau_id == 0
+    # rows of a matrix that equal a filter, ranked together with it
+    row = f.reshape(1, 27)
+    m = np.concatenate([row, row], axis=0)
+    out = oracle.cstep_structure([m, a], [None, None], 0.5, 1.0, ("filter", "neuron"))   # 6 tied, keep ids 0..2
+    assert out.mask[0].all() and out.mask[1].reshape(4, -1)[:, 0].tolist() == [1, 0, 0, 0]
+    assert out.result.tau_id == 2 and out.result.n_tie == 6
+
+
 # ---------------------------------------------------------------- binary16
 def _golden_f16():
     rows = []
