@@ -28,8 +28,9 @@
  *    need only their natural alignment (4 bytes for fp32): 16-byte alignment is
  *    faster but not required.
  *  - Calls are asynchronous and ordered on the `stream` argument (a cudaStream_t
- *    passed as void*; NULL is the legacy default stream). A context may be used
- *    by one stream at a time. The library allocates device memory only in
+ *    passed as void*; NULL is the legacy default stream). A context's workspace is
+ *    shared by its calls: a call on another stream than the previous one first
+ *    waits (on the device) for that call's kernels. The library allocates device memory only in
  *    condensa_create() and when a call needs a larger workspace than any call
  *    before it on that context (this synchronises the device once); steady-state
  *    calls allocate nothing and do not synchronise.
@@ -93,13 +94,18 @@ enum {
                                    default are settled by one CTA in shared memory, through the
                                    grid-wide selection. Default for large inputs is ONE
                                    pass: the threshold is first bracketed from 16384 hashed sample
-                                   positions, the pass decides everything outside the bracket for
-                                   good and lists the rest, and the exact selection runs on that
-                                   list. The bracket is checked exactly afterwards; should it ever
-                                   miss (probability < 1e-18 for positions independent of the
-                                   data) the outputs of that call are invalid, lambda has been
-                                   updated, and condensa_get_result() returns
-                                   CONDENSA_ERR_INTERNAL - it is never silent.                    */
+                                   positions (seed: condensa_set_seed), the pass decides everything
+                                   outside the bracket for good and lists the rest, and the exact
+                                   selection runs on that list. The bracket is checked exactly
+                                   afterwards. Should it miss (probability < 1e-18 for positions
+                                   independent of the data), the call falls back to the two-pass
+                                   route by itself and returns the exact result whenever the first
+                                   pass has not destroyed an input, i.e. unless FUSE_LAMBDA is set
+                                   and a tensor has a lambda buffer. In that one case the outputs
+                                   of the call are invalid, lambda has been overwritten, and
+                                   condensa_get_result() returns CONDENSA_ERR_INTERNAL (CONDENSA_OK
+                                   from the call itself is provisional until then) - never silent.
+                                   Callers that cannot accept this set CONDENSA_NO_SAMPLING.      */
 };
 
 /* return codes */
@@ -135,12 +141,19 @@ typedef struct {
     int64_t n_candidates;  /* units that had to be listed for the exact selection             */
     int64_t n_repaired;    /* single-pass path: listed units whose provisional decision was
                               wrong and were rewritten                                        */
+    uint64_t seed;         /* seed of the sample positions the call used (condensa_set_seed)  */
 } condensa_result;
 
 /* Create a context on CUDA device `device`. workspace_bytes = 0 sizes the
  * workspace on demand; otherwise that much is reserved up front. */
 CONDENSA_API int condensa_create(condensa_ctx **out, int device, size_t workspace_bytes);
 CONDENSA_API int condensa_destroy(condensa_ctx *ctx);
+
+/* Seed of the hashed sample positions of the single-pass path. Every context draws
+ * its own at creation, so that no fixed input can be built against the positions;
+ * setting it makes a run reproducible. It never changes a result, only how many
+ * units the exact selection has to look at (see CONDENSA_NO_SAMPLING). */
+CONDENSA_API int condensa_set_seed(condensa_ctx *ctx, uint64_t seed);
 
 /* Prune() - unstructured magnitude pruning (Table 1; Section 3.3 "pruning").
  * key = bits(u) & 0x7FFFFFFF. theta = u (or fp16(u) with FUSE_FP16: Compose([Prune(),
@@ -308,23 +321,26 @@ CONDENSA_API int condensa_count_nonzero(condensa_ctx *ctx, const float *const *a
  * reserve; and latency-critical loops that cannot accept the device-wide
  * synchronisation cudaMalloc/cudaFree imply. The context-based calls allocate
  * a workspace the first time they see a problem size; this call never does:
- * no cudaMalloc, cudaFree, cudaMallocHost or other allocating routine, on any
- * call. Its scratch (selection state, histograms, candidate list: 2176 KiB) is
- * a fixed array inside the library image, so every GPU that loads the library
- * holds those bytes until the process exits.
+ * no cudaMalloc, cudaFree, cudaMallocHost or other routine that allocates device
+ * or pinned memory, on any call (ordinary host heap is used while the arguments
+ * are checked). Its scratch (selection state, histograms, candidate list:
+ * 2304 KiB) is a fixed array inside the library image, so every GPU that loads
+ * the library holds those bytes until the process exits.
  *
  * Operation: exactly condensa_cstep_prune() on a list of ONE tensor, with the
  * same arithmetic, ranking and tie rule and bit-identical theta, mask, lambda,
  * grad and theta_h. `tensor` is a HOST pointer to one condensa_tensor whose
  * buffers are DEVICE pointers on the CURRENT device (cudaGetDevice); all
- * outputs are the caller's. There is no context and no result record.
+ * outputs are the caller's. There is no context and no result record;
+ * condensa_noalloc_status() tells whether the device-side checks of the last
+ * call passed.
  *
  * Limits and rules:
  *  - tensor->numel <= CONDENSA_NOALLOC_MAX_NUMEL, else CONDENSA_ERR_TOO_LARGE
  *    and nothing is launched or written.
  *  - The first call on each device looks up the scratch's device address (once
- *    per device, with that device current). Make that first call outside any
- *    stream capture.
+ *    per device, with that device current; host threads are serialised for
+ *    it). Make that first call outside any stream capture.
  *  - All calls on a device share the one scratch array, which still holds the
  *    previous call's contents; each call clears the parts that must start at
  *    zero on `stream` before using them. Two calls that may overlap on the GPU
@@ -334,6 +350,12 @@ CONDENSA_API int condensa_count_nonzero(condensa_ctx *ctx, const float *const *a
 #define CONDENSA_NOALLOC_MAX_NUMEL 1048576
 CONDENSA_API int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
                                               float mu, unsigned fuse, void *stream);
+
+/* Waits for the stream of the last condensa_cstep_prune_noalloc() call on the
+ * current device and returns CONDENSA_OK, or CONDENSA_ERR_INTERNAL if one of its
+ * device-side consistency checks failed (the outputs are then invalid). Allocates
+ * nothing. (No counterpart in the paper.) */
+CONDENSA_API int condensa_noalloc_status(void);
 
 /* Text of the last error on this context (never NULL). ctx may be NULL to get
  * the text of a failed condensa_create() or condensa_cstep_prune_noalloc(). */

@@ -7,6 +7,10 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <ctime>
+#include <functional>
+#include <mutex>
+#include <random>
 #include <string>
 #include <vector>
 
@@ -50,6 +54,9 @@ struct condensa_ctx {
     char *h_stage = nullptr;        // pinned staging of the descriptor upload
     size_t h_stage_bytes = 0;
     cudaEvent_t stage_ev = nullptr;
+    cudaEvent_t tail_ev = nullptr;  // recorded behind the last kernel of every call
+    bool tail_recorded = false;
+    uint64_t seed = 0;              // sample positions of the single-pass path
     std::vector<char> last_upload;  // what the device descriptor area holds now
     char *last_upload_dst = nullptr;
     int64_t launches = 0;
@@ -255,6 +262,7 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, int kinds = 
 
 constexpr int N_SAMPLE = SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD;
 constexpr int SAMPLE_CTAS = 64;
+constexpr long long ONE_LAUNCH_MAX_N = 4ll << 20;    // parameters of a list that the one-launch route takes
 
 // journal_floats: floats of original lambda kept per listed unit (0: no single-pass path)
 Layout make_layout(int T, const Plan &pl, bool ranking, bool filter, int journal_floats = 0)
@@ -414,14 +422,18 @@ void prof_collect(condensa_ctx *ctx)
 
 template <int SRC>
 int launch_select(condensa_ctx *ctx, Params &P, int first_listed, int pre_scan, cudaStream_t stream,
-                  const long long *prefix_b = nullptr, long long n_items_b = 0, int post_apply = 0)
+                  const long long *prefix_b = nullptr, long long n_items_b = 0, int post_apply = 0,
+                  const Sel *init = nullptr)
 {
     if (!ctx->occ_select[SRC]) ctx->occ_select[SRC] = occupancy(k_select<SRC>);
     const int per_sm = std::min(ctx->occ_select[SRC], 2);
     dim3 grid((unsigned)(ctx->num_sms * per_sm)), block(THREADS);
+    int do_init = init ? 1 : 0;
+    Sel init_v;
+    if (init) init_v = *init; else memset(&init_v, 0, sizeof(init_v));
     void *args[] = {(void *)&P, (void *)&first_listed, (void *)&pre_scan, (void *)&prefix_b, (void *)&n_items_b,
-                    (void *)&post_apply};
-    const int pa_ = prof_begin(ctx, "k_select", stream);
+                    (void *)&post_apply, (void *)&do_init, (void *)&init_v};
+    const int pa_ = prof_begin(ctx, init ? "k_select_all" : "k_select", stream);
     CU_TRY(ctx, cudaLaunchCooperativeKernel((const void *)k_select<SRC>, grid, block, args, 0, stream));
     ctx->launches += 1;
     prof_end(ctx, pa_, stream);
@@ -502,10 +514,21 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     P.n_sample = N_SAMPLE;
     P.jr_lam = (float *)(ws + L.journal);
     P.onepass_cap = pl.cap;
-    P.seed = 0x9E3779B97F4A7C15ull;
+    P.seed = ctx->seed;
+    {
+        // a missed sample bracket can be repaired inside the call unless the first pass
+        // has overwritten multipliers in place
+        bool lam_in_place = false;
+        if (fuse & CONDENSA_FUSE_LAMBDA)
+            for (int t = 0; t < T; ++t) lam_in_place = lam_in_place || (ts[t].lambda != nullptr && ts[t].numel > 0);
+        P.miss_fallback = lam_in_place ? 0 : 1;
+    }
     bool need_h = (fuse & (CONDENSA_FUSE_FP16 | CONDENSA_FUSE_BF16)) != 0;
     for (int t = 0; t < T; ++t) need_h = need_h || ts[t].theta_h != nullptr;
     ctx->ctl = P.ctl;
+    // the workspace is shared by all calls of the context: a call on another stream
+    // first waits for the previous call's kernels
+    if (ctx->tail_recorded && ctx->last_stream != stream) CU_TRY(ctx, cudaStreamWaitEvent(stream, ctx->tail_ev, 0));
     ctx->last_stream = stream;
 
     if (!ctx->occ_stream) ctx->occ_stream = 3;
@@ -519,6 +542,10 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         // rankings of a short key array (filters, rows, general blocks) skip the grid-wide selection
         const bool small = (op == OP_FILTER || op == OP_BLOCKGEN) && pl.S <= SMALL_S_MAX &&
                            !(fuse & CONDENSA_NO_SAMPLING);
+
+        // lists that stay in the L2 between the passes: one cooperative launch does
+        // start, histogram passes, selection and projection
+        const bool one_launch = (op == OP_PRUNE || op == OP_BLOCK) && !sampling && pl.N <= ONE_LAUNCH_MAX_N;
 
         Params Pa = P;
         Pa.item_prefix = pa;
@@ -577,14 +604,14 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             k_select_small<<<1, SMALL_THREADS, sizeof(u64) * (size_t)pl.S, stream>>>(Pa, init, op == OP_FILTER ? 1 : 0);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
-        } else {
+        } else if (!one_launch) {
             int pi_ = prof_begin(ctx, "k_init", stream);
             k_init<<<8, THREADS, 0, stream>>>(P, init);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
         }
         // with the single-pass path the fallback scan, if it is needed at all, runs inside k_select
-        if (!init.done && !small && !sampling) {
+        if (!init.done && !small && !sampling && !one_launch) {
             const int ps_ = prof_begin(ctx, op == OP_PRUNE ? "k_scan_elem" : op == OP_BLOCK ? "k_scan_block" : "k_scan_array", stream);
             if (op == OP_PRUNE) {
                 k_scan<SRC_ELEM><<<stream_grid(ctx, pl.n_items_a, 4), THREADS, 0, stream>>>(Pa, do_list0);
@@ -617,11 +644,13 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             prof_end(ctx, pr_, stream);
         }
         // a call that went for the single pass needs no projection launch: after a fall-back k_select projects itself
-        const int post_apply = sampling && !init.done ? (need_h ? 2 : 1) : 0;
+        const int post_apply = ((sampling && !init.done) || one_launch) ? (need_h ? 2 : 1) : 0;
         applied_in_select = post_apply != 0;
+        const int pre_scan = (sampling || one_launch) ? 1 : 0;
+        const Sel *init_p = one_launch ? &init : nullptr;
         if (small) rc = CONDENSA_OK;
-        else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, sampling ? 1 : 0, stream, pb, pl.n_items_b, post_apply);
-        else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, sampling ? 1 : 0, stream, pb, pl.n_items_b, post_apply);
+        else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, pre_scan, stream, pb, pl.n_items_b, post_apply, init_p);
+        else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, pre_scan, stream, pb, pl.n_items_b, post_apply, init_p);
         else rc = launch_select<SRC_ARRAY>(ctx, Pa, do_list0, 0, stream);
         if (rc) return rc;
         ctx->has_result = true;
@@ -654,6 +683,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         LAUNCH_CHECK(ctx);
         prof_end(ctx, pa_, stream);
     }
+    if (cudaEventRecord(ctx->tail_ev, stream) == cudaSuccess) ctx->tail_recorded = true;
     return CONDENSA_OK;
 }
 
@@ -684,15 +714,30 @@ int condensa_create(condensa_ctx **out, int device, size_t workspace_bytes)
         delete c;
         return fail(nullptr, CONDENSA_ERR_UNSUPPORTED, "device lacks cooperative launch");
     }
-    if ((e = cudaEventCreateWithFlags(&c->stage_ev, cudaEventDisableTiming)) != cudaSuccess) {
+    if ((e = cudaEventCreateWithFlags(&c->stage_ev, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&c->tail_ev, cudaEventDisableTiming)) != cudaSuccess) {
+        if (c->stage_ev) cudaEventDestroy(c->stage_ev);
         delete c;
         return fail(nullptr, CONDENSA_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+    }
+    {
+        // sample positions differ from context to context, so that no fixed input can be
+        // built against them; condensa_set_seed() makes a run reproducible
+        uint64_t z = 0x9E3779B97F4A7C15ull;
+        try {
+            std::random_device rd;
+            z = ((uint64_t)rd() << 32) ^ (uint64_t)rd();
+        } catch (...) {
+            z ^= (uint64_t)(uintptr_t)c ^ ((uint64_t)std::hash<std::string>()(std::to_string((long long)clock())) << 1);
+        }
+        c->seed = z;
     }
     if (workspace_bytes) {
         int rc = ensure_workspace(c, workspace_bytes, nullptr);
         if (rc) {
             g_create_error = c->err;
             cudaEventDestroy(c->stage_ev);
+            cudaEventDestroy(c->tail_ev);
             delete c;
             return rc;
         }
@@ -711,8 +756,16 @@ int condensa_destroy(condensa_ctx *ctx)
     if (ctx->mirror.buf) cudaFree(ctx->mirror.buf);
     if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
     if (ctx->stage_ev) cudaEventDestroy(ctx->stage_ev);
+    if (ctx->tail_ev) cudaEventDestroy(ctx->tail_ev);
     for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
     delete ctx;
+    return CONDENSA_OK;
+}
+
+int condensa_set_seed(condensa_ctx *ctx, uint64_t seed)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    ctx->seed = seed;
     return CONDENSA_OK;
 }
 
@@ -1115,15 +1168,28 @@ int64_t condensa_launch_count(const condensa_ctx *ctx) { return ctx ? ctx->launc
 // one-tensor descriptor and a candidate list for up to
 // CONDENSA_NOALLOC_MAX_NUMEL elements. It is part of the loaded module, so
 // every GPU that loads this library holds these bytes until the process exits.
-constexpr size_t NOALLOC_SCRATCH_BYTES = 2176u * 1024u;
+constexpr size_t NOALLOC_SCRATCH_BYTES = 2304u * 1024u;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
 namespace {
 
+// Upper bound of make_layout() for one tensor of CONDENSA_NOALLOC_MAX_NUMEL elements:
+// control block, three histograms, three final-buffer arrays, descriptor area, two
+// list arrays of S / 8 entries, each rounded up to 256 bytes.
+constexpr size_t noalloc_up(size_t x) { return (x + 255) / 256 * 256; }
+constexpr size_t NOALLOC_LAYOUT_MAX =
+    noalloc_up(sizeof(Ctl)) + noalloc_up(sizeof(u64) * 3 * NBINS) + 3 * noalloc_up(sizeof(u64) * FIN) +
+    noalloc_up(sizeof(TensorDesc) + 4 * sizeof(long long)) + 2 * noalloc_up(sizeof(u64) * (CONDENSA_NOALLOC_MAX_NUMEL / 8));
+static_assert(CONDENSA_NOALLOC_MAX_NUMEL / 8 >= 65536, "the list capacity rule of build_plan is S / 8 from this size on");
+static_assert(NOALLOC_LAYOUT_MAX <= NOALLOC_SCRATCH_BYTES, "the built-in scratch must hold the largest accepted input");
+
 constexpr int NOALLOC_MAX_DEVICES = 64;
+std::mutex g_noalloc_mutex;                          // guards the once-per-device set-up and the error text
 unsigned char *g_noalloc_ptr[NOALLOC_MAX_DEVICES];   // device address of the scratch, per device
 int g_noalloc_occ[NOALLOC_MAX_DEVICES];
 int g_noalloc_sms[NOALLOC_MAX_DEVICES];
+size_t g_noalloc_ctl_off[NOALLOC_MAX_DEVICES];       // where the last call on the device put its control block
+cudaStream_t g_noalloc_stream[NOALLOC_MAX_DEVICES];
 
 // Writes the descriptor of the single tensor and its two work-item prefix
 // arrays into the scratch (the regular path copies them from pinned memory).
@@ -1138,6 +1204,7 @@ __global__ void k_noalloc_setup(TensorDesc d, long long items, TensorDesc *td, l
 
 int noalloc_fail(int code, const char *text)
 {
+    std::lock_guard<std::mutex> lk(g_noalloc_mutex);
     g_create_error = text;
     return code;
 }
@@ -1162,19 +1229,27 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return noalloc_fail(CONDENSA_ERR_UNSUPPORTED, "device index too large");
-    if (!g_noalloc_ptr[dev]) {
-        // Once per device, with that device current: the array's name is only a
-        // host-side handle here; kernels need the address the runtime maps it to.
-        unsigned char *p = nullptr;
-        e = cudaGetSymbolAddress((void **)&p, g_noalloc_scratch);
-        if (e != cudaSuccess || !p) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
-        int sms = 0, coop = 0;
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-        if (!coop || sms <= 0) return noalloc_fail(CONDENSA_ERR_UNSUPPORTED, "device lacks cooperative launch");
-        g_noalloc_occ[dev] = occupancy(k_select<SRC_ELEM>);
-        g_noalloc_sms[dev] = sms;
-        g_noalloc_ptr[dev] = p;
+    {
+        std::unique_lock<std::mutex> lk(g_noalloc_mutex);
+        if (!g_noalloc_ptr[dev]) {
+            // Once per device, with that device current: the array's name is only a
+            // host-side handle here; kernels need the address the runtime maps it to.
+            unsigned char *p = nullptr;
+            e = cudaGetSymbolAddress((void **)&p, g_noalloc_scratch);
+            int sms = 0, coop = 0;
+            if (e == cudaSuccess && p) {
+                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+                cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+            }
+            if (e != cudaSuccess || !p || !coop || sms <= 0) {
+                lk.unlock();
+                return noalloc_fail(e != cudaSuccess || !p ? CONDENSA_ERR_CUDA : CONDENSA_ERR_UNSUPPORTED,
+                                    e != cudaSuccess ? cudaGetErrorString(e) : "device lacks cooperative launch");
+            }
+            g_noalloc_occ[dev] = occupancy(k_select<SRC_ELEM>);
+            g_noalloc_sms[dev] = sms;
+            g_noalloc_ptr[dev] = p;
+        }
     }
     Plan pl;
     build_plan(OP_PRUNE, tensor, 1, pl);
@@ -1206,31 +1281,42 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
     Sel init = initial_state(pl.S, pl.S - Z, 31);
     int do_list0 = (u64)pl.S <= pl.cap ? 1 : 0;
     const int sms = g_noalloc_sms[dev];
-    auto grid_for = [&](long long items, int per_sm) {
-        long long g = (long long)sms * per_sm;
-        if (g > items) g = items;
-        return (int)(g < 1 ? 1 : g);
-    };
 
     k_noalloc_setup<<<1, 32, 0, stream>>>(pl.td[0], pl.n_items_a, (TensorDesc *)(ws + L.desc), prefix);
-    k_init<<<8, THREADS, 0, stream>>>(P, init);      // clears the histograms and counters the last call left
-    if (!init.done)
-        k_scan<SRC_ELEM><<<grid_for(pl.n_items_a, 4), THREADS, 0, stream>>>(P, do_list0);
     if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     {
+        // one cooperative launch: clears what the last call left in the scratch, ranks, projects
         dim3 grid((unsigned)(sms * std::min(g_noalloc_occ[dev], 2))), block(THREADS);
-        int pre_scan = 0, post_apply = 0;        // the scan kernel above has run; the projection kernel follows
-        const long long *no_prefix = nullptr;
-        long long no_items = 0;
-        void *args[] = {(void *)&P, (void *)&do_list0, (void *)&pre_scan, (void *)&no_prefix, (void *)&no_items,
-                        (void *)&post_apply};
+        int pre_scan = 1, post_apply = 2, do_init = 1;
+        const long long *prefix_b = prefix + 2;
+        long long items_b = pl.n_items_b;
+        void *args[] = {(void *)&P, (void *)&do_list0, (void *)&pre_scan, (void *)&prefix_b, (void *)&items_b,
+                        (void *)&post_apply, (void *)&do_init, (void *)&init};
         e = cudaLaunchCooperativeKernel((const void *)k_select<SRC_ELEM>, grid, block, args, 0, stream);
         if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
     }
-    if (pl.n_items_b > 0) {
-        k_apply_linear<M_PRUNE, true><<<grid_for(pl.n_items_b, 3), THREADS, 0, stream>>>(P);
-        if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    {
+        std::lock_guard<std::mutex> lk(g_noalloc_mutex);
+        g_noalloc_ctl_off[dev] = L.ctl;
+        g_noalloc_stream[dev] = stream;
     }
+    return CONDENSA_OK;
+}
+
+int condensa_noalloc_status(void)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES || !g_noalloc_ptr[dev])
+        return noalloc_fail(CONDENSA_ERR_INVALID_ARG, "condensa_cstep_prune_noalloc has not run on this device");
+    if ((e = cudaStreamSynchronize(g_noalloc_stream[dev])) != cudaSuccess)
+        return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    int status = 0;
+    const Ctl *ctl = (const Ctl *)(g_noalloc_ptr[dev] + g_noalloc_ctl_off[dev]);
+    if ((e = cudaMemcpy(&status, &ctl->res.status, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    if (status != 0) return noalloc_fail(CONDENSA_ERR_INTERNAL, "device-side selection check failed in the last allocation-free call");
     return CONDENSA_OK;
 }
 

@@ -17,7 +17,7 @@ constexpr int BLOCKS_PER_ITEM = 256;     // block work item = 256 4x4 blocks (on
 constexpr int SEG = 2048;                // filter norm segment (elements)
 constexpr int LOG_NBINS = 11;
 constexpr int NBINS = 1 << LOG_NBINS;    // histogram bins per selection pass
-constexpr int FIN = 1024;                // bracket population finished by direct ranking
+constexpr int FIN = 4096;                // bracket population finished by ranking in shared memory
 constexpr int WSTG = 256;                // staged list entries per warp
 constexpr int MAX_SELECT_ITERS = 24;
 constexpr u64 KEY_NONE = ~0ull;          // cut-off key that keeps nothing
@@ -57,6 +57,7 @@ struct Result {
     int sampled;
     long long n_candidates;
     long long n_repaired;
+    u64 seed;                // seed of the sample positions this call used
 };
 
 // Selection state: the bracket is the set of units whose (key, id) lies in
@@ -120,6 +121,9 @@ struct Params {
     const long long *edge_items;    // projection work items the aligned fast kernel skips
     long long n_edge_items;
     u64 *fin_idx;                   // [FIN] list position of each entry of the final buffer
+    int miss_fallback;              // a missed sample bracket may be repaired by the two-pass route inside the
+                                    // same call: nothing the first pass wrote is needed again (no multiplier
+                                    // is updated in place)
 };
 
 // Which projection work items the fast single-pass kernels take (host and device

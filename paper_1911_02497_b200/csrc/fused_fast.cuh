@@ -22,7 +22,10 @@ struct ElemFastShared {
     float lam[WARPS][ESTG];
 };
 
-__device__ __forceinline__ void elem_flush(const Params &P, ElemFastShared &sh, bool has_lam, u32 limit)
+// The journal entry is written for every staged candidate: entries staged by an
+// earlier item of this CTA may belong to another tensor (one with multipliers)
+// than the item that triggers the flush; tensors without multipliers stage 0.
+__device__ __forceinline__ void elem_flush(const Params &P, ElemFastShared &sh, u32 limit)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __syncwarp();
@@ -37,7 +40,7 @@ __device__ __forceinline__ void elem_flush(const Params &P, ElemFastShared &sh, 
             if (pos < P.cap) {
                 P.list_key[pos] = (u64)sh.key[warp][i];
                 P.list_id[pos] = sh.id[warp][i];
-                if (has_lam) P.jr_lam[pos] = sh.lam[warp][i];
+                P.jr_lam[pos] = sh.lam[warp][i];
             }
         }
         __syncwarp();
@@ -165,9 +168,9 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
             }
         }
         n_above += nkeep - ncandkeep;      // keeps that are not candidates lie above the bracket
-        elem_flush(P, sh, has_lam, ESTG / 2);
+        elem_flush(P, sh, ESTG / 2);
     }
-    elem_flush(P, sh, true, 0);
+    elem_flush(P, sh, 0);
     __syncthreads();
     u64 na = n_above;
     // the items outside the aligned fast path (tensor heads and tails, unaligned

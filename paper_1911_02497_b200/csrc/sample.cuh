@@ -67,13 +67,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
 {
     __shared__ SampleShared sh;
     Ctl *ctl = P.ctl;
-#ifdef CONDENSA_DEBUG_TIME
-    unsigned long long ts[6]; int ns = 0;
-#define SSTAMP() do { if (threadIdx.x == 0 && ns < 6) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); ts[ns++] = t_; } } while (0)
-#else
-#define SSTAMP() do {} while (0)
-#endif
-    SSTAMP();
     // what the plain start kernel does: clear histograms (all CTAs share the work)
     for (int i = blockIdx.x * SAMPLE_THREADS + threadIdx.x; i < 3 * NBINS; i += gridDim.x * SAMPLE_THREADS)
         P.hist[i] = 0;
@@ -85,7 +78,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         const u64 unit = __umul64hi(mix64(P.seed + (u64)j), (u64)P.S);   // uniform on [0, S)
         P.sample_key[j] = unit_key<SRC>(P, unit);
     }
-    SSTAMP();
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -118,8 +110,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         hi = sh.red2[i] > hi ? sh.red2[i] : hi;
     }
     __syncthreads();
-
-    SSTAMP();
     const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
     const double p = (double)init.k / (double)init.S;
     const double mp = (double)m * p;
@@ -187,7 +177,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         hi = e_hi;
         lo = e_lo;
     }
-    SSTAMP();
     if (open_top) hi0 = max_key;
     if (open_bot) lo0 = 0;
     if (guess < lo0) guess = lo0;
@@ -201,10 +190,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
     inside = cta_sum(inside, sh.red);
     if (threadIdx.x == 0) {
         const double predicted = (double)inside * ((double)init.S / (double)m);
-#ifdef CONDENSA_DEBUG_SAMPLE
-        printf("k_sample: m=%d k=%llu S=%llu ranks=%lld/%lld/%lld lo0=%llx hi0=%llx guess=%llx inside=%llu predicted=%.0f cap=%llu shift=%d\n",
-               m, init.k, init.S, r_hi, r_mid, r_lo, lo0, hi0, guess, inside, predicted, P.onepass_cap, shift);
-#endif
         // written field by field into global memory (the state starts as `init`)
         Sel *d = &ctl->sel;
         *d = init;
@@ -219,10 +204,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
             const int bl = bit_length(lo0 == hi0 ? init.hi_id - init.lo_id : hi0 - lo0);
             d->shift = bl > LOG_NBINS ? bl - LOG_NBINS : 0;
         }
-#ifdef CONDENSA_DEBUG_SAMPLE
-        printf("k_sample wrote onepass=%d sampled=%d lo=%llx guess=%llx shift=%d\n", d->onepass, d->sampled,
-               d->lo_key, d->guess, d->shift);
-#endif
         ctl->tau_key = KEY_NONE;
         ctl->tau_id = 0;
         ctl->scan_above[0] = ctl->scan_above[1] = ctl->scan_above[2] = 0;
@@ -232,12 +213,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         ctl->sample_done = 0;
         ctl->resolve_done = 0;
         ctl->resolved = 0;
-#ifdef CONDENSA_DEBUG_TIME
-        SSTAMP();
-        printf("k_sample phases (us):");
-        for (int i = 1; i < ns; ++i) printf(" %.1f", (double)(ts[i] - ts[i - 1]) * 1e-3);
-        printf("\n");
-#endif
     }
 }
 

@@ -17,15 +17,20 @@ namespace cg = cooperative_groups;
 
 struct ScanShared {
     u32 hist[NBINS];
-    u64 stg_key[WARPS][WSTG];
-    u64 stg_id[WARPS][WSTG];
+    u64 stg_key[WARPS][WSTG];      // the two staging arrays are adjacent: the direct ranking uses
+    u64 stg_id[WARPS][WSTG];       // them as one array of 2 * WARPS * WSTG values
     u64 red[WARPS];
     Sel sel;
     u64 pick_before;
     u64 pick_count;
     int pick_bin;
     int fin_hit;
+    u64 rk_value;                  // direct ranking: value found, entries before it, entries equal to it
+    u32 rk_before, rk_count;
 };
+static_assert(offsetof(ScanShared, stg_id) == offsetof(ScanShared, stg_key) + sizeof(u64) * WARPS * WSTG,
+              "staging arrays must be adjacent");
+static_assert(FIN <= 2 * WARPS * WSTG, "the direct ranking keeps FIN values in the staging arrays");
 
 struct ScanCtx {
     u64 n_above;     // per thread
@@ -304,12 +309,6 @@ __device__ __noinline__ void scan_list(const Params &P, ScanShared &sh, int slot
 }
 
 // ---------------------------------------------------------------- pick
-#ifdef CONDENSA_DEBUG_TIME
-__device__ unsigned long long g_dbg[16];
-#define DSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_dbg[i] = t_; } } while (0)
-#else
-#define DSTAMP(i) do {} while (0)
-#endif
 __device__ __forceinline__ void set_shift(Sel &s)
 {
     const u64 range = (s.lo_key == s.hi_key) ? (s.hi_id - s.lo_id) : (s.hi_key - s.lo_key);
@@ -320,10 +319,14 @@ __device__ __forceinline__ void set_shift(Sel &s)
 // All threads of the CTA; every CTA computes the same new state from the same
 // global histogram. `src_scan`: the scan that filled the histogram visited the
 // whole source (its count of units above the bracket is then complete).
-__device__ __noinline__ void block_pick(const Params &P, ScanShared &sh, bool src_scan, u64 max_key)
+// `may_fall_back`: a sampled single-pass bracket that turns out not to hold the rank
+// is replaced by the full range (the caller then runs the two-pass route) when the
+// call allows it; otherwise, and in the kernel that must not change anything, it is
+// error 10.
+__device__ __noinline__ void block_pick(const Params &P, ScanShared &sh, bool src_scan, u64 max_key,
+                                        bool may_fall_back = false)
 {
     Sel &s = sh.sel;
-    DSTAMP(0);
     const u64 *gh = P.hist + (size_t)s.slot * NBINS;
     constexpr int PER = NBINS / THREADS;
     u64 cnt[PER];
@@ -342,9 +345,7 @@ __device__ __noinline__ void block_pick(const Params &P, ScanShared &sh, bool sr
     }
     if (lane == 31) sh.red[warp] = inc;
     if (threadIdx.x == 0) sh.pick_bin = -1;
-    DSTAMP(1);
     __syncthreads();
-    DSTAMP(2);
     u64 wbase = 0, total = 0;
     for (int i = 0; i < WARPS; ++i) {
         if (i < warp) wbase += sh.red[i];
@@ -368,15 +369,25 @@ __device__ __noinline__ void block_pick(const Params &P, ScanShared &sh, bool sr
         }
     }
     __syncthreads();
-    DSTAMP(3);
     if (threadIdx.x == 0) {
         s.passes += 1;
         if (s.above_known && src_scan && above_scan != s.n_above) s.error = 1;
         const bool sk = s.lo_key == s.hi_key;
         if (!valid) {
             if (s.onepass) {
-                s.error = 10;       // the sampled bracket missed: outputs already written are wrong
-                s.done = 1;
+                if (may_fall_back && P.miss_fallback) {
+                    // the sampled bracket missed, but nothing the first pass wrote is needed
+                    // again: start over on the full key range; the projection follows the
+                    // selection and overwrites every output
+                    s.onepass = 0;
+                    s.lo_key = 0;
+                    s.hi_key = max_key;
+                    s.n_above = 0;
+                    s.pop = s.S;
+                } else {
+                    s.error = 10;   // the sampled bracket missed: outputs already written are wrong
+                    s.done = 1;
+                }
             } else if (s.above_known) {
                 s.error = 2;        // a histogram-derived bracket must hold the rank
                 s.done = 1;
@@ -439,102 +450,155 @@ __device__ __noinline__ void block_pick(const Params &P, ScanShared &sh, bool sr
         set_shift(s);
         if (s.passes >= MAX_SELECT_ITERS && !s.done) { s.error = 7; s.done = 1; }
     }
-    DSTAMP(4);
     __syncthreads();
-    DSTAMP(5);
 }
 
-// Rank the (at most FIN) bracket members directly. Entries are in fin_key/fin_id.
-__device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
+// Value of rank r (1-based) among the entries of v[0..n) that lie in [lo, hi], in
+// descending (asc = false) or ascending order, by range-partition passes in shared
+// memory (all threads of the CTA). Leaves in sh.rk_value the value, in sh.rk_before
+// how many in-range entries rank strictly before it and in sh.rk_count how many
+// equal it; sh.fin_hit is -1 if the rank does not exist. At most 7 passes: the
+// range shrinks by LOG_NBINS bits per pass.
+__device__ __noinline__ void smem_select(const u64 *v, u32 n, u64 lo, u64 hi, bool asc, u64 r, ScanShared &sh)
 {
-    Sel &s = sh.sel;
-    u64 *k = &sh.stg_key[0][0];       // FIN <= WARPS * WSTG
-    u64 *d = &sh.stg_id[0][0];
-    if (n > FIN) n = FIN;
-    for (u32 i = threadIdx.x; i < n; i += THREADS) {
-        k[i] = __ldcg(&P.fin_key[i]);
-        d[i] = __ldcg(&P.fin_id[i]);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int PER = NBINS / THREADS;
+    u32 before = 0;
+    if (threadIdx.x == 0) sh.fin_hit = 0;
+    for (int pass = 0; pass < 8; ++pass) {
+        const int bl = bit_length(hi - lo);
+        const int shift = bl > LOG_NBINS ? bl - LOG_NBINS : 0;
+        for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
+        __syncthreads();
+        for (u32 i = threadIdx.x; i < n; i += THREADS) {
+            const u64 x = v[i];
+            if (x >= lo && x <= hi) atomicAdd(&sh.hist[(u32)((asc ? x - lo : hi - x) >> shift)], 1u);
+        }
+        __syncthreads();
+        u32 cnt[PER], tsum = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) { cnt[j] = sh.hist[threadIdx.x * PER + j]; tsum += cnt[j]; }
+        u32 inc = tsum;
+        for (int o = 1; o < 32; o <<= 1) {
+            const u32 y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        if (lane == 31) sh.red[warp] = inc;
+        if (threadIdx.x == 0) sh.pick_bin = -1;
+        __syncthreads();
+        u32 wbase = 0;
+        for (int i = 0; i < warp; ++i) wbase += (u32)sh.red[i];
+        u32 run = wbase + inc - tsum;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            if (r > run && r <= (u64)run + cnt[j]) {
+                sh.pick_bin = threadIdx.x * PER + j;
+                sh.pick_before = run;
+                sh.pick_count = cnt[j];
+            }
+            run += cnt[j];
+        }
+        __syncthreads();
+        const int b = sh.pick_bin;
+        const u32 pb = (u32)sh.pick_before, pc = (u32)sh.pick_count;
+        __syncthreads();
+        if (b < 0) {                        // the rank does not exist among the entries
+            if (threadIdx.x == 0) sh.fin_hit = -1;
+            __syncthreads();
+            return;
+        }
+        before += pb;
+        r -= pb;
+        const u64 width = 1ull << shift;
+        if (asc) {
+            const u64 nl = lo + ((u64)b << shift);
+            hi = (hi - nl >= width - 1) ? nl + (width - 1) : hi;
+            lo = nl;
+        } else {
+            const u64 nh = hi - ((u64)b << shift);
+            lo = (nh - lo >= width - 1) ? nh - (width - 1) : lo;
+            hi = nh;
+        }
+        if (pc == 1 && lo != hi) {          // one entry left in the range: it is the value
+            for (u32 i = threadIdx.x; i < n; i += THREADS) {
+                const u64 x = v[i];
+                if (x >= lo && x <= hi) sh.rk_value = x;
+            }
+            if (threadIdx.x == 0) { sh.rk_before = before; sh.rk_count = 1; }
+            __syncthreads();
+            return;
+        }
+        if (lo == hi) {
+            if (threadIdx.x == 0) { sh.rk_value = lo; sh.rk_before = before; sh.rk_count = pc; }
+            __syncthreads();
+            return;
+        }
     }
     if (threadIdx.x == 0) sh.fin_hit = -1;
     __syncthreads();
-    const u64 r = s.k - s.n_above;     // 1-based rank inside the bracket
-    if (n <= 512) {
-        // few survivors: count, for each, how many rank before it
-        for (u32 i = threadIdx.x; i < n; i += THREADS) {
-            const u64 ki = k[i], di = d[i];
-            u32 before = 0, same = 0;
-#pragma unroll 8
-            for (u32 j = 0; j < n; ++j) {
-                const u64 kj = k[j];                     // keys only: equal keys are rare
-                before += (u32)(kj > ki);
-                same += (u32)(kj == ki);
-            }
-            if (same > 1) {                              // ties beside itself: the lower id ranks first
-                for (u32 j = 0; j < n; ++j) before += (u32)(k[j] == ki) & (u32)(d[j] < di);
-            }
-            if ((u64)before + 1 == r) sh.fin_hit = (int)i;
-        }
-        __syncthreads();
-    } else {
-    // bitonic sort of the padded array into ranking order (first = strongest)
-    u32 n2 = 1;
-    while (n2 < n) n2 <<= 1;
-    for (u32 i = n + threadIdx.x; i < n2; i += THREADS) { k[i] = 0; d[i] = ~0ull; }   // ranks last
+}
+
+// Rank the (at most FIN) bracket members directly. Entries are in fin_key/fin_id.
+// The keys go to shared memory and the key of the wanted rank is found there;
+// among the entries that carry this key the index decides (lower first), found the
+// same way on their indices.
+__device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
+{
+    Sel &s = sh.sel;
+    u64 *v = &sh.stg_key[0][0];
+    if (n > FIN) n = FIN;
+    for (u32 i = threadIdx.x; i < n; i += THREADS) v[i] = __ldcg(&P.fin_key[i]);
     __syncthreads();
-    for (u32 size = 2; size <= n2; size <<= 1) {
-        for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
-            for (u32 t = threadIdx.x; t < (n2 >> 1); t += THREADS) {
-                const u32 i = 2 * t - (t & (stride - 1));
-                const u32 j = i + stride;
-                const bool i_after_j = k[j] > k[i] || (k[j] == k[i] && d[j] < d[i]);
-                const bool j_after_i = k[i] > k[j] || (k[i] == k[j] && d[i] < d[j]);
-                const bool up = (i & size) == 0;
-                if (up ? i_after_j : j_after_i) {
-                    const u64 tk = k[i], td = d[i];
-                    k[i] = k[j]; d[i] = d[j];
-                    k[j] = tk; d[j] = td;
-                }
-            }
-            __syncthreads();
-        }
-    }
-    if (threadIdx.x == 0 && r >= 1 && r <= (u64)n) sh.fin_hit = (int)(r - 1);
-    __syncthreads();
-    }
-    if (sh.fin_hit >= 0) {
-        const u64 tk = k[sh.fin_hit];
-        u64 gt = 0, eq = 0;
-        for (u32 i = threadIdx.x; i < n; i += THREADS) {
-            gt += k[i] > tk ? 1 : 0;
-            eq += k[i] == tk ? 1 : 0;
-        }
-        for (int o = 16; o > 0; o >>= 1) {
-            gt += __shfl_xor_sync(0xffffffffu, gt, o);
-            eq += __shfl_xor_sync(0xffffffffu, eq, o);
-        }
+    const u64 r = s.k - s.n_above;          // 1-based rank inside the bracket
+    bool ok = s.k > s.n_above && r <= (u64)n;
+    u64 tk = 0, tid = 0;
+    u32 gt = 0, eq = 0;
+    if (ok) {
+        smem_select(v, n, s.lo_key, s.hi_key, false, r, sh);
+        ok = sh.fin_hit >= 0;
+        tk = sh.rk_value; gt = sh.rk_before; eq = sh.rk_count;
         __syncthreads();
-        if ((threadIdx.x & 31) == 0) {
-            sh.red[threadIdx.x >> 5] = gt;
-            sh.hist[threadIdx.x >> 5] = (u32)eq;
-        }
+    }
+    if (ok) {
+        // the (r - gt)-th lowest index among the entries with this key
+        for (u32 i = threadIdx.x; i < n; i += THREADS) v[i] = (v[i] == tk) ? __ldcg(&P.fin_id[i]) : ~0ull;
         __syncthreads();
-        if (threadIdx.x == 0) {
-            u64 g = 0, e = 0;
-            for (int i = 0; i < WARPS; ++i) { g += sh.red[i]; e += sh.hist[i]; }
+        smem_select(v, n, s.lo_key == s.hi_key ? s.lo_id : 0ull, s.lo_key == s.hi_key ? s.hi_id : s.S - 1, true,
+                    r - gt, sh);
+        ok = sh.fin_hit >= 0 && sh.rk_count == 1;
+        tid = sh.rk_value;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        if (ok) {
             if (!s.key_fixed) {
                 s.key_fixed = 1;
-                s.n_gt = s.n_above + g;
-                s.n_tie = e;
+                s.n_gt = s.n_above + gt;
+                s.n_tie = eq;
             }
             s.lo_key = s.hi_key = tk;
-            s.lo_id = s.hi_id = d[sh.fin_hit];
-            s.done = 1;
+            s.lo_id = s.hi_id = tid;
+        } else {
+            s.error = 8;
         }
-    } else if (threadIdx.x == 0) {
-        s.error = 8;
         s.done = 1;
     }
     __syncthreads();
+}
+
+// Control block at the start of a ranking call (one thread).
+__device__ __forceinline__ void init_ctl(Ctl *c, const Sel &init)
+{
+    c->sel = init;
+    c->tau_key = KEY_NONE;
+    c->tau_id = 0;
+    c->scan_above[0] = c->scan_above[1] = c->scan_above[2] = 0;
+    c->list_count[0] = c->list_count[1] = 0;
+    c->fin_count = 0;
+    c->n_repaired = 0;
+    c->sample_done = 0;
+    c->resolve_done = 0;
+    c->resolved = 0;
 }
 
 // Cut-off and record of the call, from the final selection state (one thread).
@@ -567,6 +631,7 @@ __device__ __forceinline__ void write_result(const Params &P, const Sel &s)
         if (P.bits_key >= 63) r.tau_norm = (float)sqrt(__longlong_as_double((long long)s.lo_key));
     }
     r.n_repaired = 0;      // filled in by the host from the counter once the stream is idle
+    r.seed = P.seed;
     c->sel = s;
     c->res = r;
 }
@@ -693,46 +758,34 @@ __global__ void __launch_bounds__(THREADS) k_scan(Params P, int do_list)
 // made here. `post_apply` (1, or 2 when the 16-bit codes are needed): no
 // projection kernel follows this launch; after such a fall-back the final write
 // is made here too, on the projection work items `prefix_b` / `n_items_b`.
+// `do_init`: nothing ran before this launch at all: the histograms and counters are
+// cleared and the initial state `init` is installed here first (the one-launch
+// route of lists small enough to stay in the L2 between the passes).
 template <int SRC>
 __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, int pre_scan,
-                                                    const long long *prefix_b, long long n_items_b, int post_apply)
+                                                    const long long *prefix_b, long long n_items_b, int post_apply,
+                                                    int do_init, Sel init)
 {
     __shared__ ScanShared sh;
+    __shared__ int s_skip_pick;
     cg::grid_group grid = cg::this_grid();
     const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
-    if (P.ctl->resolved) {
-        // The resolve kernel has produced cut-off and record. What is left are the
-        // units it ranked directly: spread thinly over the grid, since each rewrite
-        // is a chain of dependent memory accesses.
-        if (SRC != SRC_ARRAY) {
-            const u32 nf = __ldcg(&P.ctl->fin_count);
-            const u32 n = nf < (u32)FIN ? nf : (u32)FIN;
-            const u32 j = threadIdx.x * gridDim.x + blockIdx.x;
-            if (j < n && !P.ctl->sel.error) {
-                const u64 tk = P.ctl->sel.lo_key, ti = P.ctl->sel.lo_id, guess = P.ctl->sel.guess;
-                const u64 key = __ldcg(&P.fin_key[j]), id = __ldcg(&P.fin_id[j]);
-                const bool fin = keep_by_cutoff(key, id, tk, ti);
-                if (fin != (key >= guess)) {
-                    repair_unit<SRC>(P, __ldcg(&P.fin_idx[j]), id, fin, nullptr);
-                    atomicAdd(&P.ctl->n_repaired, 1ull);
-                }
-            }
-        }
-        return;
+    if (do_init) {
+        for (int i = blockIdx.x * THREADS + threadIdx.x; i < 3 * NBINS; i += gridDim.x * THREADS) P.hist[i] = 0;
+        if (blockIdx.x == 0 && threadIdx.x == 0) init_ctl(P.ctl, init);
+        __threadfence();
+        grid.sync();
+    } else if (P.ctl->resolved) {
+        return;                       // the resolve kernel has finished the call
     }
-    if (threadIdx.x == 0) sh.sel = P.ctl->sel;
+    if (threadIdx.x == 0) {
+        if (do_init) sh.sel = init; else sh.sel = P.ctl->sel;
+    }
     __syncthreads();
     if (pre_scan && !sh.sel.onepass && !sh.sel.done) {
         scan_source<SRC>(P, sh, first_listed != 0, sh.sel.slot);
         grid.sync();
     }
-#ifdef CONDENSA_DEBUG_TIME
-    unsigned long long tq[8]; int nq = 0;
-#define TSTAMP() do { if (blockIdx.x == 0 && threadIdx.x == 0 && nq < 8) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); tq[nq++] = t_; } } while (0)
-#else
-#define TSTAMP() do {} while (0)
-#endif
-    TSTAMP();
     bool src_scan = true;
     u64 fixed = 0;
     if (!sh.sel.done) {
@@ -740,20 +793,36 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
         __syncthreads();
         for (int it = 0; it < MAX_SELECT_ITERS + 2; ++it) {
             // a listing scan that overflowed the list does not count
-            if (threadIdx.x == 0 && sh.sel.list_valid &&
-                __ldcg(&P.ctl->list_count[sh.sel.list_sel]) > P.cap) {
-                sh.sel.list_valid = 0;
-                if (sh.sel.onepass) { sh.sel.error = 11; sh.sel.done = 1; }
+            if (threadIdx.x == 0) {
+                s_skip_pick = 0;
+                if (sh.sel.list_valid && __ldcg(&P.ctl->list_count[sh.sel.list_sel]) > P.cap) {
+                    sh.sel.list_valid = 0;
+                    if (sh.sel.onepass) {
+                        if (P.miss_fallback) {
+                            // more candidates than the sample predicted: like a missed bracket,
+                            // start over on the full key range with a scan of the source
+                            Sel &f = sh.sel;
+                            f.onepass = 0; f.sampled = 0;
+                            f.lo_key = 0; f.hi_key = max_key; f.lo_id = 0; f.hi_id = f.S - 1;
+                            f.n_above = 0; f.above_known = 1; f.pop = f.S;
+                            set_shift(f);
+                            s_skip_pick = 1;
+                        } else {
+                            sh.sel.error = 11; sh.sel.done = 1;
+                        }
+                    }
+                }
             }
             __syncthreads();
             if (sh.sel.done) break;
-            block_pick(P, sh, src_scan, max_key);
-            TSTAMP();
-            // clear the histogram slot that the scan after the next one will use
-            if (blockIdx.x == 0) {
-                const int z = (sh.sel.slot + 2) % 3;
-                for (int i = threadIdx.x; i < NBINS; i += THREADS) P.hist[(size_t)z * NBINS + i] = 0;
-                if (threadIdx.x == 0) P.ctl->scan_above[z] = 0;
+            if (!s_skip_pick) {
+                block_pick(P, sh, src_scan, max_key, true);
+                // clear the histogram slot that the scan after the next one will use
+                if (blockIdx.x == 0) {
+                    const int z = (sh.sel.slot + 2) % 3;
+                    for (int i = threadIdx.x; i < NBINS; i += THREADS) P.hist[(size_t)z * NBINS + i] = 0;
+                    if (threadIdx.x == 0) P.ctl->scan_above[z] = 0;
+                }
             }
             if (sh.sel.done) break;
             if (sh.sel.list_valid && sh.sel.pop <= FIN) {
@@ -784,14 +853,11 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
                         }
                     }
                 }
-                TSTAMP();
                 grid.sync();
-                TSTAMP();
                 const u32 n = __ldcg(&P.ctl->fin_count);
                 if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
                 __syncthreads();
                 final_rank(P, sh, n);
-                TSTAMP();
                 break;
             }
             // next scan
@@ -820,16 +886,6 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
         }
         if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
     }
-    TSTAMP();
-#ifdef CONDENSA_DEBUG_TIME
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        printf("k_select phases (us):");
-        for (int i = 1; i < nq; ++i) printf(" %.1f", (double)(tq[i] - tq[i - 1]) * 1e-3);
-        printf("  fixed(cta0,t0)=%llu pop=%llu | pick: start+%.1f", fixed, sh.sel.pop, (double)(g_dbg[0] - tq[0]) * 1e-3);
-        for (int i = 1; i < 6; ++i) printf(" %.1f", (double)(g_dbg[i] - g_dbg[i - 1]) * 1e-3);
-        printf("\n");
-    }
-#endif
     if (blockIdx.x == 0 && threadIdx.x == 0) write_result(P, sh.sel);
     if constexpr (SRC != SRC_ARRAY) {
         if (post_apply && !sh.sel.onepass) {       // the same on every CTA: the sampler's verdict never changes
@@ -848,11 +904,12 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
 // leaves at most FIN listed units open, every CTA walks its share of the list:
 // entries outside the narrowed bracket are final (and rewritten if their
 // provisional decision was wrong), the others go to the final buffer. The CTA that
-// finishes last (threadfence + counter, nobody waits) ranks the final buffer and
-// writes the record; the members of that buffer are rewritten at the start of
-// k_select, which is launched next in any case. In every other case (more
-// survivors, a failed check) this kernel changes nothing and k_select does the
-// whole job from the same histogram.
+// finishes last (threadfence + counter, nobody waits) ranks the final buffer in
+// shared memory, writes cut-off and record, rewrites the members of that buffer
+// whose provisional decision was wrong and marks the call as resolved; k_select,
+// launched next in any case, then returns at once. In every other case (more
+// survivors, a failed check, a missed bracket) this kernel changes nothing and
+// k_select does the whole job from the same histogram.
 template <int SRC>
 __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
 {
@@ -860,13 +917,6 @@ __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
     __shared__ u32 s_last;
     Ctl *c = P.ctl;
     const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
-#ifdef CONDENSA_DEBUG_TIME
-    unsigned long long tr[8]; int nr = 0;
-#define RSTAMP() do { if (threadIdx.x == 0 && nr < 8) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); tr[nr++] = t_; } } while (0)
-#else
-#define RSTAMP() do {} while (0)
-#endif
-    RSTAMP();
     if (threadIdx.x == 0) sh.sel = c->sel;
     // this CTA's first chunk of the list is fetched while the pick is made
     const u64 n_all = __ldcg(&c->list_count[0]);
@@ -878,7 +928,6 @@ __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
     if (threadIdx.x == 0) sh.sel.list_valid = 1;
     __syncthreads();
     block_pick(P, sh, true, max_key);
-    RSTAMP();
     if (sh.sel.error) return;
     const bool need_rank = !sh.sel.done;
     if (need_rank && sh.sel.pop > FIN) return;
@@ -886,31 +935,46 @@ __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
         const u64 fixed = list_repair_pass<SRC>(P, sh, need_rank, n_list, &pre);
         if (fixed) atomicAdd(&c->n_repaired, fixed);
     }
-    RSTAMP();
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) s_last = atomicAdd(&c->resolve_done, 1u) == gridDim.x - 1 ? 1u : 0u;
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    RSTAMP();
+    u32 n = 0;
     if (need_rank) {
-        const u32 n = __ldcg(&c->fin_count);
+        n = __ldcg(&c->fin_count);
         if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
         __syncthreads();
-        final_rank(P, sh, n);      // its members are rewritten by the next launch
+        if (!sh.sel.error) final_rank(P, sh, n);
     }
-    RSTAMP();
+    __syncthreads();
+    if (need_rank && !sh.sel.error && SRC != SRC_ARRAY) {
+        // the members of the final buffer: their final decision is known only now
+        long long *pre_s = reinterpret_cast<long long *>(sh.hist);
+        const bool pre_ok = P.T <= NBINS / 2;
+        if (pre_ok)
+            for (int t = threadIdx.x; t < P.T; t += THREADS)
+                pre_s[t] = (SRC == SRC_ELEM) ? P.td[t].elem_prefix : P.td[t].unit_prefix;
+        __syncthreads();
+        const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
+        u64 fixed = 0;
+        for (u32 j = threadIdx.x; j < n; j += THREADS) {
+            const u64 key = __ldcg(&P.fin_key[j]), id = __ldcg(&P.fin_id[j]);
+            const bool fin = keep_by_cutoff(key, id, tk, ti);
+            if (fin != (key >= guess)) {
+                repair_unit<SRC>(P, __ldcg(&P.fin_idx[j]), id, fin, pre_ok ? pre_s : nullptr);
+                ++fixed;
+            }
+        }
+        if (fixed) atomicAdd(&c->n_repaired, fixed);
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         write_result(P, sh.sel);
-        c->resolved = 1;
         c->resolve_done = 0;
-#ifdef CONDENSA_DEBUG_TIME
-        RSTAMP();
-        printf("k_resolve last CTA %d phases (us):", (int)blockIdx.x);
-        for (int i = 1; i < nr; ++i) printf(" %.1f", (double)(tr[i] - tr[i - 1]) * 1e-3);
-        printf("\n");
-#endif
+        __threadfence();
+        c->resolved = 1;
     }
 }
 
@@ -920,18 +984,7 @@ __global__ void __launch_bounds__(THREADS) k_init(Params P, Sel init)
 {
     const int n = 3 * NBINS;
     for (int i = blockIdx.x * THREADS + threadIdx.x; i < n; i += gridDim.x * THREADS) P.hist[i] = 0;
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        Ctl *c = P.ctl;
-        c->sel = init;
-        c->tau_key = KEY_NONE;
-        c->tau_id = 0;
-        c->scan_above[0] = c->scan_above[1] = c->scan_above[2] = 0;
-        c->list_count[0] = c->list_count[1] = 0;
-        c->fin_count = 0;
-        c->n_repaired = 0;
-        c->resolve_done = 0;
-        c->resolved = 0;
-    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) init_ctl(P.ctl, init);
 }
 
 }  // namespace cs

@@ -29,7 +29,7 @@ EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "conde
            "condensa_last_error", "condensa_profile_enable", "condensa_profile_read",
            "condensa_cstep_prune_noalloc", "condensa_lstep_update",
            "condensa_cstep_structure", "condensa_thin_flags", "condensa_thin_compact",
-           "condensa_count_nonzero"]
+           "condensa_count_nonzero", "condensa_set_seed", "condensa_noalloc_status"]
 
 
 class CondensaError(RuntimeError):
@@ -51,7 +51,7 @@ class Result(C.Structure):
                 ("n_zero", C.c_int64), ("n_keep", C.c_int64), ("tau_key", C.c_uint64),
                 ("tau_id", C.c_int64), ("n_gt", C.c_int64), ("n_tie", C.c_int64),
                 ("n_tie_kept", C.c_int64), ("tau_norm", C.c_float), ("sampled", C.c_int32),
-                ("n_candidates", C.c_int64), ("n_repaired", C.c_int64)]
+                ("n_candidates", C.c_int64), ("n_repaired", C.c_int64), ("seed", C.c_uint64)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -103,6 +103,8 @@ def load():
     L.condensa_profile_enable.argtypes = [vp, i32]
     L.condensa_profile_read.argtypes = [vp, C.POINTER(KernelTime), i32, C.POINTER(i32)]
     L.condensa_cstep_prune_noalloc.argtypes = [vp, f64, f32, u32, vp]
+    L.condensa_noalloc_status.argtypes = []
+    L.condensa_set_seed.argtypes = [vp, C.c_uint64]
     L.condensa_lstep_update.argtypes = [vp, vp, i32, f32, C.POINTER(Opt), vp]
     i64 = C.c_int64
     L.condensa_thin_flags.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp]
@@ -201,6 +203,15 @@ def cstep_prune_noalloc(tab, sparsity, mu, fuse=(), stream=None):
         raise CondensaError(rc, (L.condensa_last_error(None) or b"").decode())
 
 
+def noalloc_status():
+    """``condensa_noalloc_status``: waits for the last allocation-free call on the current
+    device and raises if one of its device-side checks failed."""
+    L = load()
+    rc = L.condensa_noalloc_status()
+    if rc != OK:
+        raise CondensaError(rc, (L.condensa_last_error(None) or b"").decode())
+
+
 class Context:
     """Owns a ``condensa_ctx`` (workspace and descriptor cache of one device)."""
 
@@ -226,6 +237,9 @@ class Context:
     def _check(self, rc: int):
         if rc != OK:
             raise CondensaError(rc, (self._lib.condensa_last_error(self._h) or b"").decode())
+
+    def set_seed(self, seed: int):
+        self._check(self._lib.condensa_set_seed(self._h, int(seed) & ((1 << 64) - 1)))
 
     def cstep_prune(self, tab, T, sparsity, mu, fuse=(), stream=None):
         self._check(self._lib.condensa_cstep_prune(self._h, tab, T, float(sparsity), float(mu),

@@ -15,10 +15,14 @@ pytestmark = pytest.mark.gpu
 REL = 1e-6      # tolerance stated for fp32 norms and multiplier updates
 
 
+SEED = 0x5EEDC0FFEE      # sample positions of the module's context (reproducible runs)
+
+
 @pytest.fixture(scope="module")
 def ctx():
     from paper_1911_02497_b200 import cstep
     c = cstep.Context(0)
+    c.set_seed(SEED)
     yield c
     c.close()
 
@@ -303,24 +307,89 @@ def test_single_pass_path_is_taken_and_repairs(ctx):
     assert res.sampled == 1 and 0 < res.n_candidates < res.n_units // 8
 
 
-def test_sample_bracket_miss_is_reported_not_silent(ctx):
-    """The single-pass path trusts a bracket taken from 16384 hashed positions and checks it
-    exactly afterwards. Here the input is built against that hash (tiny values exactly at the
-    sampled positions), so the bracket misses: the call must say so through the result status
-    instead of returning a wrong projection, and the context must stay usable."""
-    from paper_1911_02497_b200 import cstep
-    n, m, seed = 1 << 20, 16384, 0x9E3779B97F4A7C15
+def _adversarial_for_seed(seed, n=1 << 20, m=16384):
+    """An input built against the sample positions of `seed`: tiny values exactly there, so that
+    the bracket taken from the sample cannot hold the threshold of the whole tensor."""
     w = W.draw(n, "normal", 1.0, 77, 0, 0)
     pos = [(W._mix64_scalar((seed + j) & ((1 << 64) - 1)) * n) >> 64 for j in range(m)]
-    w[np.array(pos)] = (W.draw(m, "normal", 1e-4, 78, 0, 0))
+    w[np.array(pos)] = W.draw(m, "normal", 1e-4, 78, 0, 0)
+    return w
+
+
+def test_sample_bracket_miss_falls_back_or_is_reported(ctx):
+    """The single-pass path trusts a bracket taken from 16384 hashed positions and checks it
+    exactly afterwards. With an input built against the positions of a known seed the bracket
+    misses. When the first pass has not overwritten multipliers the call must fall back by
+    itself and return the oracle's result; with in-place multipliers it must say so through the
+    result status instead of returning a wrong projection; with any other seed the same input
+    goes through the single pass; and the context must stay usable throughout."""
+    from paper_1911_02497_b200 import cstep
     from paper_1911_02497_b200.device_set import DeviceSet
-    ds = DeviceSet([w], [np.zeros_like(w)])
-    ds.run(ctx, "prune", 0.9, 1e-3, ("lambda",))
-    with pytest.raises(cstep.CondensaError) as e:
-        ctx.get_result()
-    assert e.value.code == cstep.ERR_INTERNAL
-    # the same input without the sample bracket is projected correctly
-    check(ctx, "prune", [w], [np.zeros_like(w)], 0.9, 1e-3, ("lambda", "no_sampling"))
+    seed = 0x9E3779B97F4A7C15
+    w = _adversarial_for_seed(seed)
+    lam = W.draw(w.size, "normal", 1e-4, 79, 1, 0)
+    try:
+        ctx.set_seed(seed)
+        # no multiplier is updated: falls back inside the call, exact result, not sampled
+        for fuse, l in ((("penalty", "fp16"), [lam]), (("lambda",), [None]), ((), [lam])):
+            got, res, _ = check(ctx, "prune", [w], l, 0.9, 1e-3, fuse)
+            assert res.sampled == 0 and res.n_repaired == 0 and res.seed == seed
+        # multipliers updated in place: reported, never silent
+        ds = DeviceSet([w], [lam])
+        ds.run(ctx, "prune", 0.9, 1e-3, ("lambda",))
+        with pytest.raises(cstep.CondensaError) as e:
+            ctx.get_result()
+        assert e.value.code == cstep.ERR_INTERNAL
+        # another seed: the same input and call succeed on the single pass
+        ctx.set_seed(seed + 12345)
+        got, res, _ = check(ctx, "prune", [w], [lam], 0.9, 1e-3, ("lambda",))
+        assert res.sampled == 1 and res.seed == seed + 12345
+        # and without the sample bracket it is projected correctly whatever the seed
+        ctx.set_seed(seed)
+        check(ctx, "prune", [w], [lam], 0.9, 1e-3, ("lambda", "no_sampling"))
+    finally:
+        ctx.set_seed(SEED)
+
+
+def test_more_candidates_than_the_list_holds_falls_back(ctx):
+    """A tie group that the sample cannot see but that overflows the candidate list: the values at
+    the sampled positions are spread out, everything else within the bracket is one value."""
+    seed = 0x1234ABCD
+    n, m = 1 << 20, 16384
+    w = np.full(n, 0.5, np.float32)
+    w[::20] = 2.0                                    # 5 % clearly above the cut of s = 0.9
+    pos = np.array([(W._mix64_scalar((seed + j) & ((1 << 64) - 1)) * n) >> 64 for j in range(m)])
+    w[pos] = W.draw(m, "uniform", 0.5 / 0.9, 80, 0, 0)   # the sample sees |u| spread evenly, 10 % above 0.5
+    try:
+        ctx.set_seed(seed)
+        for fuse in (("penalty",), ("fp16",)):
+            got, res, _ = check(ctx, "prune", [w], [np.zeros_like(w)], 0.9, 1e-3, fuse)
+            assert res.sampled == 0 and res.n_tie > 900000
+    finally:
+        ctx.set_seed(SEED)
+
+
+def test_single_pass_with_and_without_multipliers_in_one_list(ctx):
+    """Tensors with and without a lambda buffer in one sampled call: the journal of a candidate
+    must carry the multiplier of its own tensor (candidates staged by one tensor are flushed
+    while the CTA already works on the next)."""
+    shapes = [(70001,), (50000,), (123457,), (4099,), (200003,)]
+    ws = W.random_set(shapes, seed=91, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
+    lam = [ws.lam[0], None, ws.lam[2], None, ws.lam[4]]
+    for sd in (1, 2, 3):
+        ctx.set_seed(sd)
+        got, res, _ = check(ctx, "prune", ws.w, lam, 0.9, ws.mu, ("fp16", "lambda", "penalty"))
+        assert res.sampled == 1 and res.n_repaired > 0
+        got, res, _ = check(ctx, "prune", ws.w, lam, 0.9, ws.mu, ("lambda",), elem_offset=1)
+        assert res.sampled == 1
+    ctx.set_seed(SEED)
+
+
+def test_result_record_of_the_one_cta_selection(ctx):
+    """The record a short ranking leaves: passes, counts and cut-off as the oracle has them."""
+    ws = W.random_set([(300, 64)], seed=3, kind="normal", scale=1.0)
+    got, res, exp = check(ctx, "neuron", ws.w, None, 0.5, 1.0, (), exact_key=False)
+    assert res.passes >= 1 and res.n_candidates == 300 and res.sampled == 0 and res.n_repaired == 0
 
 
 # ---------------------------------------------------------------- filters

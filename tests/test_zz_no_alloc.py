@@ -59,6 +59,35 @@ def test_noalloc_prune_matches_regular_entry_point_twice_in_a_row():
         ctx.close()
 
 
+def test_noalloc_at_the_size_limit_allocates_nothing_and_reports_status():
+    """The largest accepted input (it takes the largest scratch layout), the device's free
+    memory across a steady-state call (the library must not have allocated), and the status
+    call that tells whether the device-side checks of the last call passed."""
+    import torch
+    from paper_1911_02497_b200 import cstep
+    ctx = cstep.Context(0)
+    try:
+        ws = W.random_set([(cstep.NOALLOC_MAX_NUMEL,)], seed=13, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
+        got, want = _both(ctx, ws, 0.95, ("lambda", "penalty"))
+        cstep.noalloc_status()
+        for key in ("theta", "mask", "lam", "grad"):
+            assert np.array_equal(_bits(got[key][0]), _bits(want[key][0])), key
+        from paper_1911_02497_b200.device_set import DeviceSet
+        ds = DeviceSet(ws.w, ws.lam)
+        cstep.cstep_prune_noalloc(ds.table, 0.5, ws.mu, ("lambda",))      # any first-use set-up is behind us now
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info(0)
+        ds.reset_lambda()
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info(0)
+        cstep.cstep_prune_noalloc(ds.table, 0.5, ws.mu, ("lambda",))
+        cstep.noalloc_status()
+        free2, _ = torch.cuda.mem_get_info(0)
+        assert free2 == free1, (free0, free1, free2)
+    finally:
+        ctx.close()
+
+
 def test_noalloc_rejects_what_does_not_fit():
     import torch
     from paper_1911_02497_b200 import cstep
