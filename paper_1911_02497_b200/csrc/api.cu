@@ -66,6 +66,7 @@ struct condensa_ctx {
     int occ_select[3] = {0, 0, 0};
     int occ_stream = 0;
     bool small_smem_set = false;    // dynamic shared memory limit of k_select_small raised on this device
+    bool block_smem_set = false;    // the same for the tiled block kernel
     DeviceMirror mirror;
     // optional per-kernel timing (event pair around every launch)
     bool prof_on = false;
@@ -117,6 +118,7 @@ struct Plan {
     long long S = 0, N = 0, n_seg = 0;
     u64 cap = 0;
     std::vector<long long> edge_items;           // projection items outside the aligned fast path
+    std::vector<long long> tile_prefix;          // block pruning: warp tiles of the aligned interior per tensor
 };
 
 int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s, float mu,
@@ -276,7 +278,7 @@ Layout make_layout(int T, const Plan &pl, bool ranking, bool filter, int journal
     L.fin_idx = off; off = align_up(off + sizeof(u64) * FIN, 256);
     L.desc = off;
     L.desc_bytes = sizeof(TensorDesc) * (size_t)T + 2 * sizeof(long long) * (size_t)(T + 1) +
-                   sizeof(long long) * pl.edge_items.size();
+                   sizeof(long long) * (pl.edge_items.size() + pl.tile_prefix.size());
     off = align_up(off + L.desc_bytes, 256);
     L.list_key = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
     L.list_id = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
@@ -325,7 +327,8 @@ int upload_desc(condensa_ctx *ctx, const Plan &pl, int T, char *dst, size_t byte
     memcpy(p, pl.prefix_a.data(), sizeof(long long) * (size_t)(T + 1)); p += sizeof(long long) * (size_t)(T + 1);
     if (!pl.edge_items.empty()) memcpy(p, pl.edge_items.data(), sizeof(long long) * pl.edge_items.size());
     p += sizeof(long long) * pl.edge_items.size();
-    memcpy(p, pl.prefix_b.data(), sizeof(long long) * (size_t)(T + 1));
+    memcpy(p, pl.prefix_b.data(), sizeof(long long) * (size_t)(T + 1)); p += sizeof(long long) * (size_t)(T + 1);
+    if (!pl.tile_prefix.empty()) memcpy(p, pl.tile_prefix.data(), sizeof(long long) * pl.tile_prefix.size());
     return upload_image(ctx, img, dst, stream);
 }
 
@@ -477,6 +480,14 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
                 const bool fast = op == OP_BLOCK ? block_item_is_fast(pl.td[t], j) : elem_item_is_fast(pl.td[t], j);
                 if (!fast) pl.edge_items.push_back(pl.prefix_b[t] + j);
             }
+        if (op == OP_BLOCK) {
+            pl.tile_prefix.assign((size_t)T + 1, 0);
+            for (int t = 0; t < T; ++t) {
+                const TensorDesc &d = pl.td[t];
+                const long long tiles = block_tile_count(d);
+                pl.tile_prefix[t + 1] = pl.tile_prefix[t] + tiles;
+            }
+        }
     }
     const Layout L = make_layout(T, pl, ranking, op == OP_FILTER || op == OP_BLOCKGEN, journal_floats);
     rc = ensure_workspace(ctx, L.total, stream);
@@ -503,6 +514,8 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     P.fin_idx = (u64 *)(ws + L.fin_idx);
     P.edge_items = pe;
     P.n_edge_items = (long long)pl.edge_items.size();
+    P.tile_prefix = pb + (T + 1);
+    P.n_tiles = pl.tile_prefix.empty() ? 0 : pl.tile_prefix[T];
     P.list_key = (u64 *)(ws + L.list_key);
     P.list_id = (u64 *)(ws + L.list_id);
     P.cap = pl.cap;
@@ -579,17 +592,28 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
             pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : "k_fused_block", stream);
-            const int gridf = stream_grid(ctx, pl.n_items_b, op == OP_BLOCK ? CS_BLOCK_MINB : 3);
+            // block pruning: one CTA per WARPS warp tiles at least, and enough CTAs for the edge items
+            const long long work = op == OP_BLOCK ? std::max<long long>(Pf.n_tiles, (long long)pl.edge_items.size())
+                                                  : pl.n_items_b;
+            const int gridf = stream_grid(ctx, work, op == OP_BLOCK ? 1 : 3);
             const bool need_g = (fuse & CONDENSA_FUSE_PENALTY) != 0;
-#define CS_LAUNCH_FUSED(KERNEL, GRID)                                                          \
+            if (op == OP_BLOCK && !ctx->block_smem_set) {
+                const int dyn = (int)BLOCK_FAST_DYN_SMEM;
+                CU_TRY(ctx, cudaFuncSetAttribute(k_fused_block<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+                CU_TRY(ctx, cudaFuncSetAttribute(k_fused_block<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+                CU_TRY(ctx, cudaFuncSetAttribute(k_fused_block<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+                CU_TRY(ctx, cudaFuncSetAttribute(k_fused_block<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+                ctx->block_smem_set = true;
+            }
+#define CS_LAUNCH_FUSED(KERNEL, GRID, NTHR, SMEM)                                              \
     do {                                                                                       \
-        if (need_h && need_g) KERNEL<true, true><<<GRID, THREADS, 0, stream>>>(Pf);            \
-        else if (need_h) KERNEL<true, false><<<GRID, THREADS, 0, stream>>>(Pf);                \
-        else if (need_g) KERNEL<false, true><<<GRID, THREADS, 0, stream>>>(Pf);                \
-        else KERNEL<false, false><<<GRID, THREADS, 0, stream>>>(Pf);                           \
+        if (need_h && need_g) KERNEL<true, true><<<GRID, NTHR, SMEM, stream>>>(Pf);            \
+        else if (need_h) KERNEL<true, false><<<GRID, NTHR, SMEM, stream>>>(Pf);                \
+        else if (need_g) KERNEL<false, true><<<GRID, NTHR, SMEM, stream>>>(Pf);                \
+        else KERNEL<false, false><<<GRID, NTHR, SMEM, stream>>>(Pf);                           \
     } while (0)
-            if (op == OP_PRUNE) CS_LAUNCH_FUSED(k_fused_elem, gridf);
-            else CS_LAUNCH_FUSED(k_fused_block, gridf);
+            if (op == OP_PRUNE) CS_LAUNCH_FUSED(k_fused_elem, gridf, THREADS, 0);
+            else CS_LAUNCH_FUSED(k_fused_block, gridf, BT_THREADS, BLOCK_FAST_DYN_SMEM);
 #undef CS_LAUNCH_FUSED
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);

@@ -92,6 +92,7 @@ struct Ctl {
     u64 n_repaired;           // one-pass: provisional decisions that had to be rewritten
     u32 resolve_done;         // CTAs of the resolve kernel that have finished
     int resolved;             // the resolve kernel has produced cut-off, repairs and record
+    int async_error;          // a bounded wait for a bulk copy ran out in the single-pass kernel
     Result res;
 };
 
@@ -121,6 +122,8 @@ struct Params {
     const long long *edge_items;    // projection work items the aligned fast kernel skips
     long long n_edge_items;
     u64 *fin_idx;                   // [FIN] list position of each entry of the final buffer
+    const long long *tile_prefix;   // [T+1] warp tiles per tensor of the tiled block kernel
+    long long n_tiles;
     int miss_fallback;              // a missed sample bracket may be repaired by the two-pass route inside the
                                     // same call: nothing the first pass wrote is needed again (no multiplier
                                     // is updated in place)
@@ -134,10 +137,17 @@ __host__ __device__ inline bool elem_item_is_fast(const TensorDesc &d, long long
     return d.vec_ok && e_first >= 0 && e_first + 4 * GROUPS_PER_ITEM <= d.numel;
 }
 
+// Block pruning: the blocks [0, block_fast_end) of a tensor - its complete block rows, when
+// the arrays are aligned - are done by the tiled single-pass kernel, the others by generic
+// code on the work items that reach beyond that bound (listed by the host).
+__host__ __device__ inline long long block_fast_end(const TensorDesc &d)
+{
+    return (d.ranked && d.blk_vec_ok && d.numel < 0xFFFFFFFFll) ? (d.d0 >> 2) * d.nbc : 0;
+}
+
 __host__ __device__ inline bool block_item_is_fast(const TensorDesc &d, long long local)
 {
-    const long long full_blocks = (d.d0 >> 2) * d.nbc;         // blocks in complete block rows
-    return d.ranked && d.blk_vec_ok && d.numel < 0xFFFFFFFFll && (local + 1) * BLOCKS_PER_ITEM <= full_blocks;
+    return d.ranked && (local + 1) * BLOCKS_PER_ITEM <= block_fast_end(d);
 }
 
 // ---------------------------------------------------------------- arithmetic

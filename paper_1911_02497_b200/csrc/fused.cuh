@@ -100,7 +100,7 @@ __device__ __forceinline__ void fused_block_item_generic(const Params &P, const 
 #pragma unroll 1
     for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it, par ^= 1) {
         const long long b = local * BLOCKS_PER_ITEM + it * THREADS + threadIdx.x;
-        const bool ok = b < d.n_units;
+        const bool ok = b < d.n_units && b >= block_fast_end(d);     // the tiled kernel has done the others
         BlockData bd;
         float u[16];
         u64 key = 0;

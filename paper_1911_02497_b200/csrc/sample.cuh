@@ -75,7 +75,8 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
     const int per_cta = (P.n_sample + gridDim.x - 1) / gridDim.x;
     const int j = blockIdx.x * per_cta + threadIdx.x;
     if (threadIdx.x < per_cta && j < P.n_sample) {
-        const u64 unit = __umul64hi(mix64(P.seed + (u64)j), (u64)P.S);   // uniform on [0, S)
+        // hashed twice, so that the positions of two seeds are unrelated however close the seeds are
+        const u64 unit = __umul64hi(mix64(mix64(P.seed) ^ (u64)j), (u64)P.S);   // uniform on [0, S)
         P.sample_key[j] = unit_key<SRC>(P, unit);
     }
     __threadfence();
@@ -213,6 +214,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         ctl->sample_done = 0;
         ctl->resolve_done = 0;
         ctl->resolved = 0;
+        ctl->async_error = 0;
     }
 }
 

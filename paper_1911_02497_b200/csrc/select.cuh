@@ -599,6 +599,7 @@ __device__ __forceinline__ void init_ctl(Ctl *c, const Sel &init)
     c->sample_done = 0;
     c->resolve_done = 0;
     c->resolved = 0;
+    c->async_error = 0;
 }
 
 // Cut-off and record of the call, from the final selection state (one thread).
@@ -780,6 +781,7 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
     }
     if (threadIdx.x == 0) {
         if (do_init) sh.sel = init; else sh.sel = P.ctl->sel;
+        if (!do_init && P.ctl->async_error) { sh.sel.error = 12; sh.sel.done = 1; }   // a bulk copy never arrived
     }
     __syncthreads();
     if (pre_scan && !sh.sel.onepass && !sh.sel.done) {
@@ -924,7 +926,7 @@ __global__ void __launch_bounds__(THREADS) k_resolve(Params P)
     ListChunk pre;
     load_list_chunk(P, (u64)blockIdx.x * LIST_ROUNDS * THREADS, n_list, pre);
     __syncthreads();
-    if (!sh.sel.onepass || sh.sel.done || sh.sel.error || sh.sel.k == 0 || n_all > P.cap) return;
+    if (!sh.sel.onepass || sh.sel.done || sh.sel.error || sh.sel.k == 0 || n_all > P.cap || c->async_error) return;
     if (threadIdx.x == 0) sh.sel.list_valid = 1;
     __syncthreads();
     block_pick(P, sh, true, max_key);

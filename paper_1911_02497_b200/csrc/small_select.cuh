@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(SMALL_THREADS) k_select_small(Params P, Sel in
         c->sample_done = 0;
         c->resolve_done = 0;
         c->resolved = 0;
+        c->async_error = 0;
     }
     __syncthreads();
     if (init.done) {                       // nothing to rank (k == 0 or S == 0)

@@ -311,7 +311,7 @@ def _adversarial_for_seed(seed, n=1 << 20, m=16384):
     """An input built against the sample positions of `seed`: tiny values exactly there, so that
     the bracket taken from the sample cannot hold the threshold of the whole tensor."""
     w = W.draw(n, "normal", 1.0, 77, 0, 0)
-    pos = [(W._mix64_scalar((seed + j) & ((1 << 64) - 1)) * n) >> 64 for j in range(m)]
+    pos = [(W._mix64_scalar(W._mix64_scalar(seed) ^ j) * n) >> 64 for j in range(m)]
     w[np.array(pos)] = W.draw(m, "normal", 1e-4, 78, 0, 0)
     return w
 
@@ -358,7 +358,7 @@ def test_more_candidates_than_the_list_holds_falls_back(ctx):
     n, m = 1 << 20, 16384
     w = np.full(n, 0.5, np.float32)
     w[::20] = 2.0                                    # 5 % clearly above the cut of s = 0.9
-    pos = np.array([(W._mix64_scalar((seed + j) & ((1 << 64) - 1)) * n) >> 64 for j in range(m)])
+    pos = np.array([(W._mix64_scalar(W._mix64_scalar(seed) ^ j) * n) >> 64 for j in range(m)])
     w[pos] = W.draw(m, "uniform", 0.5 / 0.9, 80, 0, 0)   # the sample sees |u| spread evenly, 10 % above 0.5
     try:
         ctx.set_seed(seed)
@@ -477,6 +477,27 @@ def test_block_general_shapes(ctx, block):
     blk = np.arange(block[0] * block[1], dtype=np.float32).reshape(block)
     got, res, _ = check(ctx, "block", [np.tile(blk, (3, 4))], None, 0.5, 1.0, (), block=block)   # 12 equal blocks
     assert (res.n_tie, res.n_tie_kept) == (12, 6)
+
+
+def test_single_pass_block_kernel_tiles_edges_and_many_tensors(ctx):
+    """The tiled single-pass block kernel at a size that takes it (more than 131072 blocks):
+    more tensors than its descriptor cache holds, block rows that are no multiple of the tile
+    width, ragged last block rows, a matrix whose width is no multiple of 4 and a vector (both
+    done by the generic code), then the same list on buffers that are not 16-byte aligned."""
+    shapes = [(130, 1000)] * 17 + [(66, 1001), (4097,), (64, 32), (4, 128)]
+    ws = W.random_set(shapes, seed=77, kind="uniform", scale=0.1, lam_sigma=1e-3, mu=1e-2)
+    for sd in (5, 6):
+        ctx.set_seed(sd)
+        got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.9, ws.mu, ("lambda", "penalty"))
+        assert res.sampled == 1 and res.n_units > 131072 and res.n_candidates > 0
+    got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.5, ws.mu, ("fp16", "lambda"))
+    assert res.sampled == 1
+    lam = [l if t % 3 else None for t, l in enumerate(ws.lam)]
+    got, res, _ = check(ctx, "block", ws.w, lam, 0.8, ws.mu, ("bf16", "lambda", "penalty"))
+    assert res.sampled == 1
+    got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.9, ws.mu, ("lambda",), elem_offset=2)
+    assert res.sampled == 1
+    ctx.set_seed(SEED)
 
 
 def test_block_size_five_on_the_lstm_shapes(ctx):
