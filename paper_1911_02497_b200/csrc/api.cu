@@ -648,25 +648,6 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             LAUNCH_CHECK(ctx);
             prof_end(ctx, ps_, stream);
         }
-        // The barrier-free end of the single pass finishes the call when one pick leaves
-        // at most FIN units open: with the bracket spread over 1024..2048 bins that is
-        // the expected case while the bracket holds fewer than about FIN * 768 units.
-        // Larger brackets go straight to k_select, which handles every case.
-        bool resolve = false;
-        if (sampling && !init.done) {
-            const double m = (double)SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD;
-            const double pk = (double)k / (double)pl.S;
-            const double width = 2.0 * (9.0 * std::sqrt(m * pk * (1.0 - pk)) + 2.0) / m;
-            resolve = width * (double)pl.S <= (double)FIN * 768.0;
-        }
-        if (resolve) {
-            const int pr_ = prof_begin(ctx, "k_resolve", stream);
-            const int gr = ctx->num_sms * 2;
-            if (op == OP_PRUNE) k_resolve<SRC_ELEM><<<gr, THREADS, 0, stream>>>(Pa);
-            else k_resolve<SRC_BLOCK><<<gr, THREADS, 0, stream>>>(Pa);
-            LAUNCH_CHECK(ctx);
-            prof_end(ctx, pr_, stream);
-        }
         // a call that went for the single pass needs no projection launch: after a fall-back k_select projects itself
         const int post_apply = ((sampling && !init.done) || one_launch) ? (need_h ? 2 : 1) : 0;
         applied_in_select = post_apply != 0;

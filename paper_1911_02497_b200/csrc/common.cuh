@@ -90,8 +90,6 @@ struct Ctl {
     u32 fin_count;
     u32 sample_done;          // CTAs of the sample kernel that have finished
     u64 n_repaired;           // one-pass: provisional decisions that had to be rewritten
-    u32 resolve_done;         // CTAs of the resolve kernel that have finished
-    int resolved;             // the resolve kernel has produced cut-off, repairs and record
     int async_error;          // a bounded wait for a bulk copy ran out in the single-pass kernel
     Result res;
 };

@@ -284,44 +284,60 @@ __device__ __forceinline__ void fused_elem_item_generic(const Params &P, const T
 }
 
 // Rewrite one listed unit whose provisional decision was wrong. Called from the
-// selection kernel after the cut-off is known. `idx` is the list position.
-// `pre_s`, when given, holds the tensors' first unit numbers in shared memory
-// (the search for the owning tensor is then free of global loads).
+// selection kernels after the cut-off is known. `idx` is the list position (the
+// journal holds the original lambda there). An element is rewritten by one thread
+// (`part` 0); a block by four, `part` being the row: u comes from the journal by the
+// same two operations as everywhere (the norm is not needed again).
 template <int SRC>
-__device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, const long long *pre_s)
+__device__ __noinline__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, int part, const long long *pre_s,
+                                         const TensorDesc *tdc)
 {
+    // One copy of this code per kernel and as few instructions as possible: it runs once per
+    // call on a few threads, right after a pass that has swept the L2, so its time is the time
+    // to fetch its instructions.
     int lo = 0, hi = P.T - 1;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
         const long long pre = pre_s ? pre_s[mid] : (SRC == SRC_ELEM) ? P.td[mid].elem_prefix : P.td[mid].unit_prefix;
         if ((u64)pre <= id) lo = mid; else hi = mid - 1;
     }
-    const TensorDesc d = P.td[lo];
+    const TensorDesc &d = tdc ? tdc[lo] : P.td[lo];
     const bool has_lam = d.lam != nullptr;
+    const bool wr_lam = (P.fuse & FUSE_LAMBDA) && has_lam;
+    const bool wr_grad = (P.fuse & FUSE_PENALTY) && d.grad != nullptr;
+    long long off;          // first element to rewrite
+    int nv;                 // how many consecutive elements
+    const float *jr;        // their original multipliers
     if (SRC == SRC_ELEM) {
-        const long long e = (long long)id - d.elem_prefix;
-        if (e < 0 || e >= d.numel) return;
-        const float w = d.w[e];
-        const float lam = has_lam ? __ldcg(&P.jr_lam[idx]) : 0.0f;
-        const float u = form_u(w, lam, P.mu, has_lam);
-        const Out o = finish(w, lam, u, keep, P.mu, P.fuse, has_lam);
-        d.theta[e] = o.theta;
-        if (d.mask) d.mask[e] = o.m;
-        if (d.theta_h) d.theta_h[e] = o.th;
-        if ((P.fuse & FUSE_LAMBDA) && has_lam) d.lam[e] = o.lam;
-        if ((P.fuse & FUSE_PENALTY) && d.grad) d.grad[e] = o.grad;
+        off = (long long)id - d.elem_prefix;
+        if (off < 0 || off >= d.numel) return;
+        nv = 1;
+        jr = P.jr_lam + idx;
     } else {
         const long long b = (long long)id - d.unit_prefix;
         if (b < 0 || b >= d.n_units) return;
-        BlockData bd;
-        float u[16];
-        load_block(d, b, bd);                       // w is intact; lambda was overwritten
-        if (has_lam) {
+        const long long br = d.n_units < 0x7FFFFFFFll ? (long long)((u32)b / (u32)d.nbc) : b / d.nbc;
+        const long long bc = b - br * d.nbc;
+        const long long r = 4 * br + part, c0 = 4 * bc;
+        if (r >= d.d0) return;
+        off = r * d.d1 + c0;
+        nv = d.d1 - c0 < 4 ? (int)(d.d1 - c0) : 4;           // columns of this row that exist
+        jr = P.jr_lam + idx * 16 + 4 * part;
+    }
+    float w[4], l[4];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) bd.l[q] = __ldcg(&P.jr_lam[idx * 16 + q]);
-        }
-        (void)block_key(bd, P.mu, has_lam, u);      // recomputes u from the original lambda
-        store_block(d, bd, u, keep, P.mu, P.fuse);
+    for (int j = 0; j < 4; ++j) {
+        w[j] = j < nv ? __ldg(d.w + off + j) : 0.0f;
+        l[j] = (j < nv && has_lam) ? __ldcg(jr + j) : 0.0f;
+    }
+#pragma unroll 1
+    for (int j = 0; j < nv; ++j) {
+        const Out o = finish(w[j], l[j], form_u(w[j], l[j], P.mu, has_lam), keep, P.mu, P.fuse, has_lam);
+        d.theta[off + j] = o.theta;
+        if (d.mask) d.mask[off + j] = o.m;
+        if (d.theta_h) d.theta_h[off + j] = o.th;
+        if (wr_lam) d.lam[off + j] = o.lam;
+        if (wr_grad) d.grad[off + j] = o.grad;
     }
 }
 

@@ -212,8 +212,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         ctl->fin_count = 0;
         ctl->n_repaired = 0;
         ctl->sample_done = 0;
-        ctl->resolve_done = 0;
-        ctl->resolved = 0;
         ctl->async_error = 0;
     }
 }

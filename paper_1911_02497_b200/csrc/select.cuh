@@ -15,6 +15,8 @@ namespace cs {
 
 namespace cg = cooperative_groups;
 
+constexpr int REPAIR_TD_CACHE = 16;
+
 struct ScanShared {
     u32 hist[NBINS];
     u64 stg_key[WARPS][WSTG];      // the two staging arrays are adjacent: the direct ranking uses
@@ -27,6 +29,7 @@ struct ScanShared {
     int fin_hit;
     u64 rk_value;                  // direct ranking: value found, entries before it, entries equal to it
     u32 rk_before, rk_count;
+    TensorDesc tdc[REPAIR_TD_CACHE];   // descriptors of short tensor lists, for the rewrites
 };
 static_assert(offsetof(ScanShared, stg_id) == offsetof(ScanShared, stg_key) + sizeof(u64) * WARPS * WSTG,
               "staging arrays must be adjacent");
@@ -553,6 +556,37 @@ __device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
     bool ok = s.k > s.n_above && r <= (u64)n;
     u64 tk = 0, tid = 0;
     u32 gt = 0, eq = 0;
+    if (ok && n <= (u32)THREADS) {
+        // few survivors: one entry per thread, which counts how many rank before it
+        u64 *ids = v + FIN / 2;
+        if (threadIdx.x < n) ids[threadIdx.x] = __ldcg(&P.fin_id[threadIdx.x]);
+        if (threadIdx.x == 0) sh.fin_hit = -1;
+        __syncthreads();
+        if (threadIdx.x < n) {
+            const u64 ki = v[threadIdx.x];
+            u32 g = 0, e = 0, lower = 0;
+#pragma unroll 8
+            for (u32 j = 0; j < n; ++j) {
+                const u64 kj = v[j];
+                g += (u32)(kj > ki);
+                e += (u32)(kj == ki);
+            }
+            if (e > 1) {                    // equal keys beside itself: the lower index ranks first
+                const u64 di = ids[threadIdx.x];
+                for (u32 j = 0; j < n; ++j) lower += (u32)(v[j] == ki && ids[j] < di);
+            }
+            if ((u64)g + lower + 1 == r) {
+                sh.fin_hit = (int)threadIdx.x;
+                sh.rk_value = ki;
+                sh.rk_before = g;
+                sh.rk_count = e;
+            }
+        }
+        __syncthreads();
+        ok = sh.fin_hit >= 0;
+        if (ok) { tk = sh.rk_value; gt = sh.rk_before; eq = sh.rk_count; tid = ids[sh.fin_hit]; }
+        __syncthreads();
+    } else {
     if (ok) {
         smem_select(v, n, s.lo_key, s.hi_key, false, r, sh);
         ok = sh.fin_hit >= 0;
@@ -568,6 +602,7 @@ __device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
         ok = sh.fin_hit >= 0 && sh.rk_count == 1;
         tid = sh.rk_value;
         __syncthreads();
+    }
     }
     if (threadIdx.x == 0) {
         if (ok) {
@@ -597,8 +632,6 @@ __device__ __forceinline__ void init_ctl(Ctl *c, const Sel &init)
     c->fin_count = 0;
     c->n_repaired = 0;
     c->sample_done = 0;
-    c->resolve_done = 0;
-    c->resolved = 0;
     c->async_error = 0;
 }
 
@@ -641,9 +674,38 @@ __device__ __forceinline__ void write_result(const Params &P, const Sel &s)
 template <int SRC>
 __device__ __noinline__ void apply_after_select(const Params &P, int need_h);
 
-// Defined with the single-pass kernels: rewrites one listed unit.
+// Defined with the single-pass kernels: rewrites one listed unit - an element, or row
+// `part` (0..3) of a 4x4 block. `pre_s` / `tdc`, when given, hold the tensors' first unit
+// numbers and descriptors in shared memory (no global loads for the owner search).
 template <int SRC>
-__device__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, const long long *pre_s);
+__device__ __noinline__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, int part, const long long *pre_s,
+                                         const TensorDesc *tdc);
+
+// Threads per rewritten unit: a block is rewritten by four threads, a row each, which keeps the
+// dependent chain of one rewrite short.
+template <int SRC>
+struct RepairLanes { static constexpr u32 value = (SRC == SRC_BLOCK) ? 4u : 1u; };
+
+// Fills the shared-memory copies used by the rewrites (all threads; a barrier must follow).
+template <int SRC>
+__device__ __forceinline__ void repair_tables(const Params &P, ScanShared &sh, const long long *&pre_s, const TensorDesc *&tdc)
+{
+    long long *ps = reinterpret_cast<long long *>(sh.hist);
+    pre_s = nullptr;
+    tdc = nullptr;
+    if (P.T <= NBINS / 2) {
+        for (int t = threadIdx.x; t < P.T; t += THREADS)
+            ps[t] = (SRC == SRC_ELEM) ? P.td[t].elem_prefix : P.td[t].unit_prefix;
+        pre_s = ps;
+    }
+    if (P.T <= REPAIR_TD_CACHE) {
+        const int words = P.T * (int)(sizeof(TensorDesc) / sizeof(u32));
+        const u32 *src = reinterpret_cast<const u32 *>(P.td);
+        u32 *dst = reinterpret_cast<u32 *>(sh.tdc);
+        for (int i = threadIdx.x; i < words; i += THREADS) dst[i] = src[i];
+        tdc = sh.tdc;
+    }
+}
 
 // Shared memory of the generic (edge) items of the single-pass kernels: the
 // projection items the aligned fast code leaves out (tensor heads and tails,
@@ -655,63 +717,91 @@ struct FusedShared {
     u64 red[WARPS];
 };
 
-// One walk over the list of the single-pass path by the whole grid. A listed unit
-// whose final decision is known and differs from the provisional one is rewritten;
-// with `rank`, the units still inside the bracket are copied to the final buffer
-// instead. A rewrite is a chain of dependent memory accesses and only a few per
-// cent of the entries need one, so each CTA first queues them in shared memory
-// and then rewrites them one per thread. The caller may have fetched this
-// CTA's first chunk already (`pre`). Returns this thread's rewrite count.
+// One walk over the candidate list by the whole grid; every CTA takes one contiguous share.
+//   gather  units inside the current bracket are copied to the final buffer (to be ranked);
+//           otherwise the bracket is one unit, the cut-off, and every entry is decided by it;
+//   repair  (single-pass path) a unit whose decision is known by now and differs from the
+//           provisional one is rewritten.
+// A rewrite is a chain of dependent memory accesses and only a few per cent of the entries
+// need one, so a CTA queues them in shared memory while it classifies its share and rewrites
+// a queue-full at a time, one unit (or block row) per thread. The caller may have fetched
+// this CTA's first chunk already (`pre`). Returns this thread's rewrite count.
 constexpr int LIST_ROUNDS = 8;                 // list entries per thread and chunk
-static_assert(LIST_ROUNDS * THREADS <= WARPS * WSTG, "the queue reuses the staging arrays");
+constexpr u32 LIST_QUEUE = WARPS * WSTG;       // queue entries (the staging arrays)
+static_assert((u32)LIST_ROUNDS * THREADS <= LIST_QUEUE, "a chunk must fit the queue");
 
 struct ListChunk {
     u64 key[LIST_ROUNDS], id[LIST_ROUNDS];
 };
 
-__device__ __forceinline__ void load_list_chunk(const Params &P, u64 base, u64 n_list, ListChunk &ch)
+// Share of the list of CTA `blockIdx.x`: [first, end).
+__device__ __forceinline__ void list_share(u64 n_list, u64 &first, u64 &end)
+{
+    u64 per = (n_list + gridDim.x - 1) / gridDim.x;
+    per = (per + THREADS - 1) / THREADS * THREADS;
+    first = (u64)blockIdx.x * per;
+    end = first + per < n_list ? first + per : n_list;
+    if (first > n_list) first = n_list;
+}
+
+__device__ __forceinline__ void load_list_chunk(const Params &P, u64 base, u64 end, ListChunk &ch)
 {
 #pragma unroll
     for (int r = 0; r < LIST_ROUNDS; ++r) {
         const u64 i = base + (u64)r * THREADS + threadIdx.x;
-        ch.key[r] = i < n_list ? __ldcg(&P.list_key[i]) : 0;
-        ch.id[r] = i < n_list ? __ldcg(&P.list_id[i]) : 0;
+        ch.key[r] = i < end ? __ldcg(&P.list_key[i]) : 0;
+        ch.id[r] = i < end ? __ldcg(&P.list_id[i]) : 0;
     }
 }
 
 template <int SRC>
-__device__ __forceinline__ u64 list_repair_pass(const Params &P, ScanShared &sh, bool rank, u64 n_list, const ListChunk *pre)
+__device__ __forceinline__ u64 repair_queue(const Params &P, const u64 *q_idx, const u64 *q_id, u32 qn,
+                                            const long long *pre_s, const TensorDesc *tdc)
+{
+    constexpr u32 LPU = RepairLanes<SRC>::value;
+    u64 fixed = 0;
+    for (u32 j = threadIdx.x; j < qn * LPU; j += THREADS) {
+        const u32 e = j / LPU;
+        const u64 packed = q_id[e];
+        repair_unit<SRC>(P, q_idx[e], packed & ~(1ull << 63), (packed >> 63) != 0, (int)(j % LPU), pre_s, tdc);
+        fixed += (j % LPU) == 0 ? 1 : 0;
+    }
+    return fixed;
+}
+
+template <int SRC>
+__device__ __noinline__ u64 list_walk(const Params &P, ScanShared &sh, bool gather, bool repair, u64 n_list,
+                                      const ListChunk *pre)
 {
     __shared__ u32 s_qn;
     u64 *q_idx = &sh.stg_key[0][0];
     u64 *q_id = &sh.stg_id[0][0];
-    // first unit number of every tensor, for the owner search of the rewrites
-    long long *pre_s = reinterpret_cast<long long *>(sh.hist);
-    const bool pre_ok = P.T <= NBINS / 2;
+    const long long *pre_s = nullptr;
+    const TensorDesc *tdc = nullptr;
     __syncthreads();
-    if (pre_ok)
-        for (int t = threadIdx.x; t < P.T; t += THREADS)
-            pre_s[t] = (SRC == SRC_ELEM) ? P.td[t].elem_prefix : P.td[t].unit_prefix;
+    if (SRC != SRC_ARRAY && repair) repair_tables<SRC>(P, sh, pre_s, tdc);
+    if (threadIdx.x == 0) s_qn = 0;
+    __syncthreads();
     Ctl *c = P.ctl;
     const Sel &s = sh.sel;
     const bool sk = s.lo_key == s.hi_key;
     const u64 chunk = (u64)LIST_ROUNDS * THREADS;
+    u64 first, end;
+    list_share(n_list, first, end);
     u64 fixed = 0;
-    bool first = true;
-    for (u64 base = (u64)blockIdx.x * chunk; base < n_list; base += (u64)gridDim.x * chunk) {
-        if (threadIdx.x == 0) s_qn = 0;
-        __syncthreads();
+    bool have_pre = pre != nullptr;
+    for (u64 base = first; base < end; base += chunk) {
         ListChunk ch;
-        if (first && pre) ch = *pre;
-        else load_list_chunk(P, base, n_list, ch);
-        first = false;
+        if (have_pre) ch = *pre;
+        else load_list_chunk(P, base, end, ch);
+        have_pre = false;
 #pragma unroll
         for (int r = 0; r < LIST_ROUNDS; ++r) {
             const u64 i = base + (u64)r * THREADS + threadIdx.x;
-            if (i >= n_list) continue;
+            if (i >= end) continue;
             const u64 key = ch.key[r], id = ch.id[r];
             bool fin;
-            if (rank) {
+            if (gather) {
                 const bool above = key > s.hi_key || (sk && key == s.hi_key && id < s.lo_id);
                 const bool below = key < s.lo_key || (sk && key == s.lo_key && id > s.hi_id);
                 if (!above && !below) {
@@ -723,20 +813,22 @@ __device__ __forceinline__ u64 list_repair_pass(const Params &P, ScanShared &sh,
             } else {
                 fin = keep_by_cutoff(key, id, s.lo_key, s.lo_id);
             }
-            if (fin != (key >= s.guess)) {
+            if (SRC != SRC_ARRAY && repair && fin != (key >= s.guess)) {
                 const u32 pos = atomicAdd(&s_qn, 1u);
                 q_idx[pos] = i;
                 q_id[pos] = id | (fin ? (1ull << 63) : 0ull);
             }
         }
-        __syncthreads();
-        const u32 qn = s_qn;
-        for (u32 j = threadIdx.x; j < qn; j += THREADS) {
-            const u64 packed = q_id[j];
-            repair_unit<SRC>(P, q_idx[j], packed & ~(1ull << 63), (packed >> 63) != 0, pre_ok ? pre_s : nullptr);
-            ++fixed;
+        if (SRC != SRC_ARRAY && repair) {
+            __syncthreads();
+            // rewrite when another chunk might not fit behind what is queued, or at the end
+            if (s_qn + (u32)chunk > LIST_QUEUE || base + chunk >= end) {
+                fixed += repair_queue<SRC>(P, q_idx, q_id, s_qn, pre_s, tdc);
+                __syncthreads();
+                if (threadIdx.x == 0) s_qn = 0;
+            }
+            __syncthreads();
         }
-        __syncthreads();
     }
     return fixed;
 }
@@ -776,8 +868,6 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
         if (blockIdx.x == 0 && threadIdx.x == 0) init_ctl(P.ctl, init);
         __threadfence();
         grid.sync();
-    } else if (P.ctl->resolved) {
-        return;                       // the resolve kernel has finished the call
     }
     if (threadIdx.x == 0) {
         if (do_init) sh.sel = init; else sh.sel = P.ctl->sel;
@@ -788,8 +878,20 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
         scan_source<SRC>(P, sh, first_listed != 0, sh.sel.slot);
         grid.sync();
     }
-    bool src_scan = true;
+    bool src_scan = true, gathered = false, have_pre = false;
     u64 fixed = 0;
+    u32 n_fin = 0;
+    ListChunk pre;
+    if (sh.sel.onepass && !sh.sel.done) {
+        // single-pass path: this CTA's first chunk of the list is fetched while the pick is made
+        const u64 n_all = __ldcg(&P.ctl->list_count[0]);
+        if (n_all <= P.cap) {
+            u64 first, end;
+            list_share(n_all, first, end);
+            load_list_chunk(P, first, end, pre);
+            have_pre = true;
+        }
+    }
     if (!sh.sel.done) {
         if ((first_listed || sh.sel.onepass) && threadIdx.x == 0) sh.sel.list_valid = 1;
         __syncthreads();
@@ -828,38 +930,18 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
             }
             if (sh.sel.done) break;
             if (sh.sel.list_valid && sh.sel.pop <= FIN) {
-                // gather the bracket members from the list and rank them
+                // gather the bracket members from the list (the single-pass path also rewrites, on
+                // this walk, the listed units outside the bracket that were decided wrongly), then rank
                 const u64 n_list = __ldcg(&P.ctl->list_count[sh.sel.list_sel]);
-                const Sel &s = sh.sel;
-                const bool sk = s.lo_key == s.hi_key;
-                constexpr int R = 8;                 // entries fetched per thread before the first is used
-                const u64 chunk = (u64)R * THREADS;
-                for (u64 base = (u64)blockIdx.x * chunk; base < n_list; base += (u64)gridDim.x * chunk) {
-                    u64 kk[R], dd[R];
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const u64 i = base + (u64)r * THREADS + threadIdx.x;
-                        kk[r] = i < n_list ? __ldcg(&P.list_key[i]) : 0;
-                        dd[r] = i < n_list ? __ldcg(&P.list_id[i]) : 0;
-                    }
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const u64 i = base + (u64)r * THREADS + threadIdx.x;
-                        if (i >= n_list) continue;
-                        const u64 key = kk[r], id = dd[r];
-                        const bool above = key > s.hi_key || (sk && key == s.hi_key && id < s.lo_id);
-                        const bool below = key < s.lo_key || (sk && key == s.lo_key && id > s.hi_id);
-                        if (!above && !below) {
-                            const u32 pos = atomicAdd(&P.ctl->fin_count, 1u);
-                            if (pos < FIN) { P.fin_key[pos] = key; P.fin_id[pos] = id; P.fin_idx[pos] = i; }
-                        }
-                    }
-                }
+                fixed += list_walk<SRC>(P, sh, true, sh.sel.onepass != 0, n_list, (it == 0 && have_pre) ? &pre : nullptr);
+                gathered = true;
+                __threadfence();
                 grid.sync();
                 const u32 n = __ldcg(&P.ctl->fin_count);
                 if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
                 __syncthreads();
-                final_rank(P, sh, n);
+                if (!sh.sel.error) final_rank(P, sh, n);
+                n_fin = n;
                 break;
             }
             // next scan
@@ -880,11 +962,32 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
             grid.sync();
         }
     }
-    if (SRC != SRC_ARRAY) {
+    if constexpr (SRC != SRC_ARRAY) {
         if (sh.sel.onepass && !sh.sel.error && sh.sel.k > 0) {
-            // single-pass path: rewrite the listed units whose provisional decision was wrong
             __syncthreads();
-            fixed = list_repair_pass<SRC>(P, sh, false, __ldcg(&P.ctl->list_count[0]), nullptr);
+            if (gathered) {
+                // the members of the final buffer: their decision is known only now; one unit
+                // (or block row) per thread of the grid
+                const long long *pre_s;
+                const TensorDesc *tdc;
+                repair_tables<SRC>(P, sh, pre_s, tdc);
+                __syncthreads();
+                const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
+                constexpr u32 LPU = RepairLanes<SRC>::value;
+                const u32 nf = n_fin < (u32)FIN ? n_fin : (u32)FIN;
+                for (u32 j = threadIdx.x * gridDim.x + blockIdx.x; j < nf * LPU; j += gridDim.x * THREADS) {
+                    const u32 e = j / LPU;
+                    const u64 key = __ldcg(&P.fin_key[e]), id = __ldcg(&P.fin_id[e]), idx = __ldcg(&P.fin_idx[e]);
+                    const bool fin = keep_by_cutoff(key, id, tk, ti);
+                    if (fin != (key >= guess)) {
+                        repair_unit<SRC>(P, idx, id, fin, (int)(j % LPU), pre_s, tdc);
+                        fixed += (j % LPU) == 0 ? 1 : 0;
+                    }
+                }
+            } else {
+                // the pick ended on a single unit: every listed unit is decided by the cut-off
+                fixed += list_walk<SRC>(P, sh, false, true, __ldcg(&P.ctl->list_count[0]), nullptr);
+            }
         }
         if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
     }
@@ -898,85 +1001,6 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
             Pb.n_items = n_items_b;
             apply_after_select<SRC>(Pb, post_apply == 2);
         }
-    }
-}
-
-// Common end of the single-pass path, without a grid barrier. Every CTA makes the
-// first pick from the complete histogram (all arrive at the same state); if that
-// leaves at most FIN listed units open, every CTA walks its share of the list:
-// entries outside the narrowed bracket are final (and rewritten if their
-// provisional decision was wrong), the others go to the final buffer. The CTA that
-// finishes last (threadfence + counter, nobody waits) ranks the final buffer in
-// shared memory, writes cut-off and record, rewrites the members of that buffer
-// whose provisional decision was wrong and marks the call as resolved; k_select,
-// launched next in any case, then returns at once. In every other case (more
-// survivors, a failed check, a missed bracket) this kernel changes nothing and
-// k_select does the whole job from the same histogram.
-template <int SRC>
-__global__ void __launch_bounds__(THREADS) k_resolve(Params P)
-{
-    __shared__ ScanShared sh;
-    __shared__ u32 s_last;
-    Ctl *c = P.ctl;
-    const u64 max_key = (P.bits_key >= 63) ? 0x7FFFFFFFFFFFFFFFull : ((1ull << P.bits_key) - 1ull);
-    if (threadIdx.x == 0) sh.sel = c->sel;
-    // this CTA's first chunk of the list is fetched while the pick is made
-    const u64 n_all = __ldcg(&c->list_count[0]);
-    const u64 n_list = n_all < P.cap ? n_all : P.cap;
-    ListChunk pre;
-    load_list_chunk(P, (u64)blockIdx.x * LIST_ROUNDS * THREADS, n_list, pre);
-    __syncthreads();
-    if (!sh.sel.onepass || sh.sel.done || sh.sel.error || sh.sel.k == 0 || n_all > P.cap || c->async_error) return;
-    if (threadIdx.x == 0) sh.sel.list_valid = 1;
-    __syncthreads();
-    block_pick(P, sh, true, max_key);
-    if (sh.sel.error) return;
-    const bool need_rank = !sh.sel.done;
-    if (need_rank && sh.sel.pop > FIN) return;
-    {
-        const u64 fixed = list_repair_pass<SRC>(P, sh, need_rank, n_list, &pre);
-        if (fixed) atomicAdd(&c->n_repaired, fixed);
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&c->resolve_done, 1u) == gridDim.x - 1 ? 1u : 0u;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    u32 n = 0;
-    if (need_rank) {
-        n = __ldcg(&c->fin_count);
-        if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
-        __syncthreads();
-        if (!sh.sel.error) final_rank(P, sh, n);
-    }
-    __syncthreads();
-    if (need_rank && !sh.sel.error && SRC != SRC_ARRAY) {
-        // the members of the final buffer: their final decision is known only now
-        long long *pre_s = reinterpret_cast<long long *>(sh.hist);
-        const bool pre_ok = P.T <= NBINS / 2;
-        if (pre_ok)
-            for (int t = threadIdx.x; t < P.T; t += THREADS)
-                pre_s[t] = (SRC == SRC_ELEM) ? P.td[t].elem_prefix : P.td[t].unit_prefix;
-        __syncthreads();
-        const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
-        u64 fixed = 0;
-        for (u32 j = threadIdx.x; j < n; j += THREADS) {
-            const u64 key = __ldcg(&P.fin_key[j]), id = __ldcg(&P.fin_id[j]);
-            const bool fin = keep_by_cutoff(key, id, tk, ti);
-            if (fin != (key >= guess)) {
-                repair_unit<SRC>(P, __ldcg(&P.fin_idx[j]), id, fin, pre_ok ? pre_s : nullptr);
-                ++fixed;
-            }
-        }
-        if (fixed) atomicAdd(&c->n_repaired, fixed);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        write_result(P, sh.sel);
-        c->resolve_done = 0;
-        __threadfence();
-        c->resolved = 1;
     }
 }
 

@@ -101,8 +101,6 @@ __global__ void __launch_bounds__(SMALL_THREADS) k_select_small(Params P, Sel in
         c->fin_count = 0;
         c->n_repaired = 0;
         c->sample_done = 0;
-        c->resolve_done = 0;
-        c->resolved = 0;
         c->async_error = 0;
     }
     __syncthreads();
