@@ -16,6 +16,8 @@ namespace cs {
 constexpr int SAMPLE_THREADS = 1024;
 constexpr int SAMPLE_KEYS_PER_THREAD = 16;          // n_sample = 16384 keys for one CTA
 
+constexpr int SAMPLE_TD_CACHE = 16;
+
 struct SampleShared {
     u32 hist[NBINS];
     u64 red[32];
@@ -23,18 +25,22 @@ struct SampleShared {
     u64 rank_before[3];
     u32 rank_bin[3];
     u32 last;
+    TensorDesc tdc[SAMPLE_TD_CACHE];
 };
 
+// Key of unit `unit`. `tdc`, when given, is a copy of the descriptor table in shared memory
+// (short tensor lists): the owner search then needs no global loads.
 template <int SRC>
-__device__ __forceinline__ u64 unit_key(const Params &P, u64 unit)
+__device__ __forceinline__ u64 unit_key(const Params &P, u64 unit, const TensorDesc *tdc)
 {
+    const TensorDesc *tab = tdc ? tdc : P.td;
     int lo = 0, hi = P.T - 1;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
-        const long long pre = (SRC == SRC_ELEM) ? P.td[mid].elem_prefix : P.td[mid].unit_prefix;
+        const long long pre = (SRC == SRC_ELEM) ? tab[mid].elem_prefix : tab[mid].unit_prefix;
         if ((u64)pre <= unit) lo = mid; else hi = mid - 1;
     }
-    const TensorDesc d = P.td[lo];
+    const TensorDesc &d = tab[lo];
     const bool has_lam = d.lam != nullptr;
     if (SRC == SRC_ELEM) {
         const long long e = (long long)unit - d.elem_prefix;
@@ -72,12 +78,21 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         P.hist[i] = 0;
     // the sampling itself is spread over many CTAs (few threads each) so that the
     // random reads of one SM do not queue behind each other
+    const TensorDesc *tdc = nullptr;
+    if (P.T <= SAMPLE_TD_CACHE) {
+        const int words = P.T * (int)(sizeof(TensorDesc) / sizeof(u32));
+        const u32 *src = reinterpret_cast<const u32 *>(P.td);
+        u32 *dst = reinterpret_cast<u32 *>(sh.tdc);
+        for (int i = threadIdx.x; i < words; i += SAMPLE_THREADS) dst[i] = src[i];
+        tdc = sh.tdc;
+        __syncthreads();
+    }
     const int per_cta = (P.n_sample + gridDim.x - 1) / gridDim.x;
     const int j = blockIdx.x * per_cta + threadIdx.x;
     if (threadIdx.x < per_cta && j < P.n_sample) {
         // hashed twice, so that the positions of two seeds are unrelated however close the seeds are
         const u64 unit = __umul64hi(mix64(mix64(P.seed) ^ (u64)j), (u64)P.S);   // uniform on [0, S)
-        P.sample_key[j] = unit_key<SRC>(P, unit);
+        P.sample_key[j] = unit_key<SRC>(P, unit, tdc);
     }
     __threadfence();
     __syncthreads();

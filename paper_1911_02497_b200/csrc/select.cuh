@@ -551,6 +551,8 @@ __device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
     u64 *v = &sh.stg_key[0][0];
     if (n > FIN) n = FIN;
     for (u32 i = threadIdx.x; i < n; i += THREADS) v[i] = __ldcg(&P.fin_key[i]);
+    if (n <= (u32)THREADS && threadIdx.x < n) v[FIN / 2 + threadIdx.x] = __ldcg(&P.fin_id[threadIdx.x]);
+    if (threadIdx.x == 0) sh.fin_hit = -1;
     __syncthreads();
     const u64 r = s.k - s.n_above;          // 1-based rank inside the bracket
     bool ok = s.k > s.n_above && r <= (u64)n;
@@ -559,9 +561,6 @@ __device__ __noinline__ void final_rank(const Params &P, ScanShared &sh, u32 n)
     if (ok && n <= (u32)THREADS) {
         // few survivors: one entry per thread, which counts how many rank before it
         u64 *ids = v + FIN / 2;
-        if (threadIdx.x < n) ids[threadIdx.x] = __ldcg(&P.fin_id[threadIdx.x]);
-        if (threadIdx.x == 0) sh.fin_hit = -1;
-        __syncthreads();
         if (threadIdx.x < n) {
             const u64 ki = v[threadIdx.x];
             u32 g = 0, e = 0, lower = 0;
@@ -717,56 +716,30 @@ struct FusedShared {
     u64 red[WARPS];
 };
 
-// One walk over the candidate list by the whole grid; every CTA takes one contiguous share.
+// One walk over the candidate list by the whole grid, in chunks strided over the CTAs.
 //   gather  units inside the current bracket are copied to the final buffer (to be ranked);
 //           otherwise the bracket is one unit, the cut-off, and every entry is decided by it;
 //   repair  (single-pass path) a unit whose decision is known by now and differs from the
 //           provisional one is rewritten.
 // A rewrite is a chain of dependent memory accesses and only a few per cent of the entries
-// need one, so a CTA queues them in shared memory while it classifies its share and rewrites
-// a queue-full at a time, one unit (or block row) per thread. The caller may have fetched
-// this CTA's first chunk already (`pre`). Returns this thread's rewrite count.
+// need one, so a CTA queues them in shared memory while it classifies a chunk and then
+// rewrites them, one unit (or block row) per thread. The caller may have fetched this CTA's
+// first chunk already (`pre`). Returns this thread's rewrite count.
 constexpr int LIST_ROUNDS = 8;                 // list entries per thread and chunk
-constexpr u32 LIST_QUEUE = WARPS * WSTG;       // queue entries (the staging arrays)
-static_assert((u32)LIST_ROUNDS * THREADS <= LIST_QUEUE, "a chunk must fit the queue");
+static_assert(LIST_ROUNDS * THREADS <= WARPS * WSTG, "the queue reuses the staging arrays");
 
 struct ListChunk {
     u64 key[LIST_ROUNDS], id[LIST_ROUNDS];
 };
 
-// Share of the list of CTA `blockIdx.x`: [first, end).
-__device__ __forceinline__ void list_share(u64 n_list, u64 &first, u64 &end)
-{
-    u64 per = (n_list + gridDim.x - 1) / gridDim.x;
-    per = (per + THREADS - 1) / THREADS * THREADS;
-    first = (u64)blockIdx.x * per;
-    end = first + per < n_list ? first + per : n_list;
-    if (first > n_list) first = n_list;
-}
-
-__device__ __forceinline__ void load_list_chunk(const Params &P, u64 base, u64 end, ListChunk &ch)
+__device__ __forceinline__ void load_list_chunk(const Params &P, u64 base, u64 n_list, ListChunk &ch)
 {
 #pragma unroll
     for (int r = 0; r < LIST_ROUNDS; ++r) {
         const u64 i = base + (u64)r * THREADS + threadIdx.x;
-        ch.key[r] = i < end ? __ldcg(&P.list_key[i]) : 0;
-        ch.id[r] = i < end ? __ldcg(&P.list_id[i]) : 0;
+        ch.key[r] = i < n_list ? __ldcg(&P.list_key[i]) : 0;
+        ch.id[r] = i < n_list ? __ldcg(&P.list_id[i]) : 0;
     }
-}
-
-template <int SRC>
-__device__ __forceinline__ u64 repair_queue(const Params &P, const u64 *q_idx, const u64 *q_id, u32 qn,
-                                            const long long *pre_s, const TensorDesc *tdc)
-{
-    constexpr u32 LPU = RepairLanes<SRC>::value;
-    u64 fixed = 0;
-    for (u32 j = threadIdx.x; j < qn * LPU; j += THREADS) {
-        const u32 e = j / LPU;
-        const u64 packed = q_id[e];
-        repair_unit<SRC>(P, q_idx[e], packed & ~(1ull << 63), (packed >> 63) != 0, (int)(j % LPU), pre_s, tdc);
-        fixed += (j % LPU) == 0 ? 1 : 0;
-    }
-    return fixed;
 }
 
 template <int SRC>
@@ -780,25 +753,24 @@ __device__ __noinline__ u64 list_walk(const Params &P, ScanShared &sh, bool gath
     const TensorDesc *tdc = nullptr;
     __syncthreads();
     if (SRC != SRC_ARRAY && repair) repair_tables<SRC>(P, sh, pre_s, tdc);
-    if (threadIdx.x == 0) s_qn = 0;
-    __syncthreads();
     Ctl *c = P.ctl;
     const Sel &s = sh.sel;
     const bool sk = s.lo_key == s.hi_key;
     const u64 chunk = (u64)LIST_ROUNDS * THREADS;
-    u64 first, end;
-    list_share(n_list, first, end);
+    constexpr u32 LPU = RepairLanes<SRC>::value;
     u64 fixed = 0;
     bool have_pre = pre != nullptr;
-    for (u64 base = first; base < end; base += chunk) {
+    for (u64 base = (u64)blockIdx.x * chunk; base < n_list; base += (u64)gridDim.x * chunk) {
+        if (threadIdx.x == 0) s_qn = 0;
+        __syncthreads();
         ListChunk ch;
         if (have_pre) ch = *pre;
-        else load_list_chunk(P, base, end, ch);
+        else load_list_chunk(P, base, n_list, ch);
         have_pre = false;
 #pragma unroll
         for (int r = 0; r < LIST_ROUNDS; ++r) {
             const u64 i = base + (u64)r * THREADS + threadIdx.x;
-            if (i >= end) continue;
+            if (i >= n_list) continue;
             const u64 key = ch.key[r], id = ch.id[r];
             bool fin;
             if (gather) {
@@ -819,16 +791,17 @@ __device__ __noinline__ u64 list_walk(const Params &P, ScanShared &sh, bool gath
                 q_id[pos] = id | (fin ? (1ull << 63) : 0ull);
             }
         }
+        __syncthreads();
         if (SRC != SRC_ARRAY && repair) {
-            __syncthreads();
-            // rewrite when another chunk might not fit behind what is queued, or at the end
-            if (s_qn + (u32)chunk > LIST_QUEUE || base + chunk >= end) {
-                fixed += repair_queue<SRC>(P, q_idx, q_id, s_qn, pre_s, tdc);
-                __syncthreads();
-                if (threadIdx.x == 0) s_qn = 0;
+            const u32 qn = s_qn;
+            for (u32 j = threadIdx.x; j < qn * LPU; j += THREADS) {
+                const u32 e = j / LPU;
+                const u64 packed = q_id[e];
+                repair_unit<SRC>(P, q_idx[e], packed & ~(1ull << 63), (packed >> 63) != 0, (int)(j % LPU), pre_s, tdc);
+                fixed += (j % LPU) == 0 ? 1 : 0;
             }
-            __syncthreads();
         }
+        __syncthreads();
     }
     return fixed;
 }
@@ -878,17 +851,14 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
         scan_source<SRC>(P, sh, first_listed != 0, sh.sel.slot);
         grid.sync();
     }
-    bool src_scan = true, gathered = false, have_pre = false;
+    bool src_scan = true, have_pre = false;
     u64 fixed = 0;
-    u32 n_fin = 0;
     ListChunk pre;
     if (sh.sel.onepass && !sh.sel.done) {
         // single-pass path: this CTA's first chunk of the list is fetched while the pick is made
         const u64 n_all = __ldcg(&P.ctl->list_count[0]);
         if (n_all <= P.cap) {
-            u64 first, end;
-            list_share(n_all, first, end);
-            load_list_chunk(P, first, end, pre);
+            load_list_chunk(P, (u64)blockIdx.x * LIST_ROUNDS * THREADS, n_all, pre);
             have_pre = true;
         }
     }
@@ -930,18 +900,15 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
             }
             if (sh.sel.done) break;
             if (sh.sel.list_valid && sh.sel.pop <= FIN) {
-                // gather the bracket members from the list (the single-pass path also rewrites, on
-                // this walk, the listed units outside the bracket that were decided wrongly), then rank
+                // gather the bracket members from the list, then rank them
                 const u64 n_list = __ldcg(&P.ctl->list_count[sh.sel.list_sel]);
-                fixed += list_walk<SRC>(P, sh, true, sh.sel.onepass != 0, n_list, (it == 0 && have_pre) ? &pre : nullptr);
-                gathered = true;
+                (void)list_walk<SRC>(P, sh, true, false, n_list, (it == 0 && have_pre) ? &pre : nullptr);
                 __threadfence();
                 grid.sync();
                 const u32 n = __ldcg(&P.ctl->fin_count);
                 if (threadIdx.x == 0 && (u64)n != sh.sel.pop) sh.sel.error = 9;
                 __syncthreads();
                 if (!sh.sel.error) final_rank(P, sh, n);
-                n_fin = n;
                 break;
             }
             // next scan
@@ -965,29 +932,11 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
     if constexpr (SRC != SRC_ARRAY) {
         if (sh.sel.onepass && !sh.sel.error && sh.sel.k > 0) {
             __syncthreads();
-            if (gathered) {
-                // the members of the final buffer: their decision is known only now; one unit
-                // (or block row) per thread of the grid
-                const long long *pre_s;
-                const TensorDesc *tdc;
-                repair_tables<SRC>(P, sh, pre_s, tdc);
-                __syncthreads();
-                const u64 tk = sh.sel.lo_key, ti = sh.sel.lo_id, guess = sh.sel.guess;
-                constexpr u32 LPU = RepairLanes<SRC>::value;
-                const u32 nf = n_fin < (u32)FIN ? n_fin : (u32)FIN;
-                for (u32 j = threadIdx.x * gridDim.x + blockIdx.x; j < nf * LPU; j += gridDim.x * THREADS) {
-                    const u32 e = j / LPU;
-                    const u64 key = __ldcg(&P.fin_key[e]), id = __ldcg(&P.fin_id[e]), idx = __ldcg(&P.fin_idx[e]);
-                    const bool fin = keep_by_cutoff(key, id, tk, ti);
-                    if (fin != (key >= guess)) {
-                        repair_unit<SRC>(P, idx, id, fin, (int)(j % LPU), pre_s, tdc);
-                        fixed += (j % LPU) == 0 ? 1 : 0;
-                    }
-                }
-            } else {
-                // the pick ended on a single unit: every listed unit is decided by the cut-off
-                fixed += list_walk<SRC>(P, sh, false, true, __ldcg(&P.ctl->list_count[0]), nullptr);
-            }
+            // The cut-off is known: every listed unit whose provisional decision was wrong is
+            // rewritten now. This comes last on purpose: the rewrites read w from DRAM, which is
+            // still busy taking the single pass's writes out of the L2 when this kernel starts;
+            // the pick, the gather and the ranking before it work out of the L2.
+            fixed += list_walk<SRC>(P, sh, false, true, __ldcg(&P.ctl->list_count[0]), nullptr);
         }
         if (fixed) atomicAdd(&P.ctl->n_repaired, fixed);
     }

@@ -238,6 +238,16 @@ def config(which, scale: float = 1.0, threads: int = 8) -> WeightSet:
     raise ValueError("unknown configuration %r" % (which,))
 
 
+def config_numel(which) -> int:
+    """Parameters of a configuration at full size, without drawing it."""
+    which = str(which)
+    if which == "1":
+        return 1048576
+    shapes = {"2": resnet56_shapes, "3": vgg19_shapes, "4": alexnet_shapes,
+              "5": lstm_lm_shapes, "5t": lambda: lstm_lm_shapes(tied=True)}[which]()
+    return int(sum(int(np.prod(s)) for s in shapes))
+
+
 def random_set(shapes: Sequence[Sequence[int]], seed: int, kind: str = "normal",
                scale: float = 1.0, lam_sigma: float = 0.0, mu: float = 1e-3,
                op: str = "prune", sparsity: float = 0.5,
