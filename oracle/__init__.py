@@ -22,7 +22,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cstep_oracle.c")
 _LIB = os.path.join(_HERE, "libcstep_oracle.so")
 
-FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, FUSE_BF16 = 1, 2, 4, 8
+FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, FUSE_BF16, FUSE_E4M3, FUSE_E5M2 = 1, 2, 4, 8, 16, 32
+CRITERIA = {"l2": 0, "l1": 1, "max": 2}
 
 CFLAGS = ["-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
           "-fno-unsafe-math-optimizations", "-Wall"]
@@ -50,6 +51,11 @@ class _Result(C.Structure):
     _fields_ = [("n_units", C.c_int64), ("n_zero", C.c_int64), ("n_keep", C.c_int64),
                 ("tau_key", C.c_uint64), ("tau_id", C.c_int64), ("n_gt", C.c_int64),
                 ("n_tie", C.c_int64), ("n_tie_kept", C.c_int64), ("tau_norm", C.c_float)]
+
+
+class _Spec(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("kinds", C.c_int32), ("nd", C.c_int32), ("crit", C.c_int32),
+                ("bs", C.c_int64 * 4)]
 
 
 class _OptTensor(C.Structure):
@@ -96,6 +102,17 @@ def lib():
         L.orc_cstep_block.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_float, C.c_int,
                                       C.c_int, C.c_uint, C.c_void_p]
         L.orc_cstep_quantize.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint]
+        assert L.orc_sizeof_spec() == C.sizeof(_Spec)
+        L.orc_structure_values.restype = C.c_int64
+        L.orc_structure_values.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_void_p, C.c_void_p]
+        L.orc_cstep_structured.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_float, C.c_void_p, C.c_uint,
+                                           C.c_void_p]
+        L.orc_f32_to_fp8.restype = C.c_uint8
+        L.orc_f32_to_fp8.argtypes = [C.c_uint32, C.c_int]
+        L.orc_fp8_to_f32.restype = C.c_uint32
+        L.orc_fp8_to_f32.argtypes = [C.c_uint8, C.c_int]
+        L.orc_f32_to_fp8_array.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p]
+        L.orc_f32_to_fp8_range.argtypes = [C.c_uint32, C.c_int64, C.c_int, C.c_void_p]
         L.orc_lagrange_update.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint]
         assert L.orc_sizeof_opt_tensor() == C.sizeof(_OptTensor) and L.orc_sizeof_opt() == C.sizeof(_Opt)
         L.orc_lstep_update.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_void_p]
@@ -130,7 +147,8 @@ class Outputs:
 
 
 def fuse_bits(fuse: Sequence[str]) -> int:
-    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY, "bf16": FUSE_BF16}
+    table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY, "bf16": FUSE_BF16,
+             "e4m3": FUSE_E4M3, "e5m2": FUSE_E5M2}
     b = 0
     for f in fuse:
         b |= table[f]
@@ -228,6 +246,70 @@ def f16_bits_to_f32(h: np.ndarray) -> np.ndarray:
     for i in range(flat_h.size):
         flat_o[i] = L.orc_f16_to_f32(int(flat_h[i]))
     return out.view(np.float32)
+
+
+FP8_FORMATS = {"e4m3": 0, "e5m2": 1}
+
+
+def f32_to_fp8_bits(x: np.ndarray, fmt: str) -> np.ndarray:
+    """8-bit code (uint8) of each fp32 value (or uint32 bit pattern) in x; fmt 'e4m3' or 'e5m2'."""
+    b = np.ascontiguousarray(x)
+    if b.dtype == np.float32:
+        b = b.view(np.uint32)
+    assert b.dtype == np.uint32
+    out = np.empty(b.shape, np.uint8)
+    lib().orc_f32_to_fp8_array(_ptr(b), b.size, FP8_FORMATS[fmt], _ptr(out))
+    return out
+
+
+def f32_to_fp8_range(first: int, n: int, fmt: str) -> np.ndarray:
+    out = np.empty(n, np.uint8)
+    lib().orc_f32_to_fp8_range(C.c_uint32(first), n, FP8_FORMATS[fmt], _ptr(out))
+    return out
+
+
+def fp8_bits_to_f32(h: np.ndarray, fmt: str) -> np.ndarray:
+    h = np.ascontiguousarray(h, dtype=np.uint8)
+    L = lib()
+    out = np.array([L.orc_fp8_to_f32(int(v), FP8_FORMATS[fmt]) for v in h.reshape(-1)], np.uint32)
+    return out.view(np.float32).reshape(h.shape)
+
+
+def _spec(kind: str, block=None, criterion: str = "l2") -> _Spec:
+    """kind: 'filter', 'neuron', 'structure' (filters and neurons) or 'block' with
+    ``block`` = the block extents, one per tensor dimension."""
+    sp = _Spec()
+    sp.crit = CRITERIA[criterion]
+    if kind == "block":
+        sp.kind, sp.nd = 1, len(block)
+        for d, b in enumerate(block):
+            sp.bs[d] = int(b)
+    else:
+        sp.kind, sp.kinds = 0, {"filter": 1, "neuron": 2, "structure": 3}[kind]
+    return sp
+
+
+def structure_values(ws, lams, mu: float, kind: str, block=None, criterion: str = "l2") -> np.ndarray:
+    """The fp64 value every ranked structure is ranked by, in global structure order."""
+    tab, _, keep = _table(ws, lams)
+    sp = _spec(kind, block, criterion)
+    S = lib().orc_structure_values(tab, len(ws), C.c_float(mu), C.byref(sp), None)
+    nu = np.empty(S, np.float64)
+    lib().orc_structure_values(tab, len(ws), C.c_float(mu), C.byref(sp), _ptr(nu))
+    return nu
+
+
+def cstep_structured(ws, lams, s: float, mu: float, kind: str, block=None, criterion: str = "l2",
+                     fuse: Sequence[str] = ()) -> Outputs:
+    """Structured pruning by a specification: leading-index slices or n-D blocks, ranked by the
+    L2, L1 or max criterion."""
+    tab, out, keep = _table(ws, lams)
+    r = _Result()
+    sp = _spec(kind, block, criterion)
+    rc = lib().orc_cstep_structured(tab, len(ws), float(s), C.c_float(mu), C.byref(sp), fuse_bits(fuse), C.byref(r))
+    assert rc == 0, rc
+    out.result = _result(r)
+    return out
 
 
 def structure_norms(ws, lams, mu: float, kind: str, block=(4, 4)) -> np.ndarray:

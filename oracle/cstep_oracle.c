@@ -48,6 +48,8 @@
 #define ORC_FUSE_LAMBDA  2u
 #define ORC_FUSE_PENALTY 4u
 #define ORC_FUSE_BF16    8u
+#define ORC_FUSE_E4M3    16u
+#define ORC_FUSE_E5M2    32u
 
 typedef struct {
     const float *w;        /* weights, never written                          */
@@ -151,6 +153,75 @@ uint16_t orc_f32_to_bf16(uint32_t b)
     return (uint16_t)q;
 }
 
+/* ---- binary32 -> 8-bit floating point (Table 1, Quantize(dtype); Conclusion: further
+ * data types for quantization) -------------------------------------------------
+ * Two formats (Micikevicius et al., "FP8 formats for deep learning", 2022):
+ *   fmt 0  E4M3: 1 sign, 4 exponent (bias 7), 3 fraction bits; no infinities, the one
+ *          NaN is S.1111.111; largest finite value 448 = S.1111.110.
+ *   fmt 1  E5M2: 1 sign, 5 exponent (bias 15), 2 fraction bits, laid out like IEEE;
+ *          largest finite value 57344 = S.11110.11.
+ * Rounding is to nearest, ties to even, with gradual underflow. Reading taken for the
+ * range: the conversion SATURATES - whatever rounds beyond the largest finite value,
+ * infinities included, becomes that value with its sign (the formats' saturating mode,
+ * and what the conversion instruction of the GPU does); an 8-bit weight format with
+ * infinities in it would be of no use as a codebook. NaN maps to S.1111111. */
+uint8_t orc_f32_to_fp8(uint32_t b, int fmt)
+{
+    const int M = fmt ? 2 : 3, bias = fmt ? 15 : 7;
+    const uint32_t maxcode = fmt ? 0x7Bu : 0x7Eu;
+    uint32_t sign = (b >> 24) & 0x80u;
+    uint32_t e = (b >> 23) & 0xFFu;
+    uint32_t m = b & 0x7FFFFFu;
+    if (e == 0xFFu) return (uint8_t)(sign | (m ? 0x7Fu : maxcode));
+    if (e == 0) return (uint8_t)sign;                      /* below 2^-126: far under the smallest code */
+    int32_t eh = (int32_t)e - 127 + bias;                  /* exponent field if the value is normal there */
+    uint32_t q;
+    if (eh >= 1) {
+        int drop = 23 - M;
+        q = ((uint32_t)eh << M) | (m >> drop);
+        uint32_t rem = m & ((1u << drop) - 1u), half = 1u << (drop - 1);
+        if (rem > half || (rem == half && (q & 1u))) q += 1u;     /* may carry into the exponent */
+        if (q > maxcode) q = maxcode;
+    } else {
+        int shift = (23 - M) + (1 - eh);                   /* the significand in units of the smallest subnormal */
+        if (shift > 25) return (uint8_t)sign;
+        uint32_t sig = m | 0x800000u;
+        q = sig >> shift;
+        uint32_t rem = sig & ((1u << shift) - 1u), half = 1u << (shift - 1);
+        if (rem > half || (rem == half && (q & 1u))) q += 1u;     /* may reach the smallest normal: still right */
+    }
+    return (uint8_t)(sign | q);
+}
+
+/* 8-bit floating point -> binary32, exact. */
+uint32_t orc_fp8_to_f32(uint8_t h, int fmt)
+{
+    const int M = fmt ? 2 : 3, E = fmt ? 5 : 4, bias = fmt ? 15 : 7;
+    uint32_t sign = ((uint32_t)h & 0x80u) << 24;
+    uint32_t e = ((uint32_t)h >> M) & ((1u << E) - 1u);
+    uint32_t m = (uint32_t)h & ((1u << M) - 1u);
+    if (fmt == 0 && e == 15u && m == 7u) return sign | 0x7FC00000u;
+    if (fmt == 1 && e == 31u) return sign | 0x7F800000u | (m ? 0x400000u : 0u);
+    if (e == 0) {
+        if (m == 0) return sign;
+        int32_t ex = 1 - bias;                             /* value = m * 2^(1 - bias - M): normalise */
+        while (!(m & (1u << M))) { m <<= 1; ex -= 1; }
+        m &= (1u << M) - 1u;
+        return sign | ((uint32_t)(ex + 127) << 23) | (m << (23 - M));
+    }
+    return sign | ((e - (uint32_t)bias + 127u) << 23) | (m << (23 - M));
+}
+
+void orc_f32_to_fp8_array(const uint32_t *bits, int64_t n, int fmt, uint8_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_fp8(bits[i], fmt);
+}
+
+void orc_f32_to_fp8_range(uint32_t first, int64_t n, int fmt, uint8_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_fp8(first + (uint32_t)i, fmt);
+}
+
 void orc_f32_to_bf16_array(const uint32_t *bits, int64_t n, uint16_t *out)
 {
     for (int64_t i = 0; i < n; ++i) out[i] = orc_f32_to_bf16(bits[i]);
@@ -218,7 +289,11 @@ static void finish_tensor(const orc_tensor *t, const float *u, const uint8_t *ke
         uint32_t tb = 0u;
         uint16_t hb = 0u;
         if (keep[i]) {
-            if (fuse & ORC_FUSE_BF16) {
+            if (fuse & (ORC_FUSE_E4M3 | ORC_FUSE_E5M2)) {
+                int fmt = (fuse & ORC_FUSE_E5M2) ? 1 : 0;
+                hb = orc_f32_to_fp8(f32_bits(u[i]), fmt);   /* the 8-bit code, in the low byte */
+                tb = orc_fp8_to_f32((uint8_t)hb, fmt);
+            } else if (fuse & ORC_FUSE_BF16) {
                 hb = orc_f32_to_bf16(f32_bits(u[i]));
                 tb = (uint32_t)hb << 16;              /* exact widening */
             } else if (fuse & ORC_FUSE_FP16) {
@@ -301,80 +376,107 @@ int orc_cstep_prune(const orc_tensor *ts, int32_t T, double s, float mu, unsigne
     return 0;
 }
 
-/* nu of each structure of one tensor, fp64, accumulated in index order.
- * kind 0: leading-index slices: filters [f, :, :, :] of a 4-D tensor (Table 1,
- *         FilterPrune, "3D blocks") and/or neurons = rows [r, :] of a 2-D tensor
- *         (NeuronPrune, "1D blocks"); for this kind `bh` carries the mask of
- *         which of the two are ranked (1 = filters, 2 = neurons, 3 = both:
- *         StructurePrune "combines neuron and filter pruning").
- * kind 1: bh x bw blocks of a 2-D tensor, numbered row-major; a block that
- *         sticks out over the edge only sums the elements that exist. */
-static int64_t structure_count(const orc_tensor *t, int kind, int bh, int bw)
+/* ---- structured pruning ---------------------------------------------------
+ * A structure specification (Table 1: NeuronPrune / FilterPrune / StructurePrune
+ * aggregate 1-D / 3-D blocks, BlockPrune(criteria, bs) aggregates n-D blocks of
+ * size bs; each prunes "based on criteria"):
+ *   kind 0  leading-index slices: filters [f, :, :, :] of 4-D tensors (kinds & 1)
+ *           and/or neurons = rows [r, :] of 2-D tensors (kinds & 2);
+ *   kind 1  n-D blocks: every tensor with ndim == nd is cut into blocks of
+ *           bs[0] x ... x bs[nd-1] elements, numbered row-major over the grid of
+ *           blocks; a block that sticks out over an edge holds only the elements
+ *           that exist.
+ * crit: the value a structure is ranked by, accumulated in fp64 over its elements
+ * in row-major order: 0 = sum of u^2 (the squared L2 norm: the argmin of Section
+ * 3.3), 1 = sum of |u| (L1 norm), 2 = max |u|. The paper names no criterion; L1 and
+ * max are the usual alternatives and are NOT the argmin. Every other tensor
+ * passes through unpruned. */
+typedef struct {
+    int32_t kind, kinds, nd, crit;
+    int64_t bs[4];
+} orc_spec;
+
+static int spec_ranks(const orc_spec *sp, const orc_tensor *t)
 {
-    if (kind == 0) {
-        if (t->numel == 0) return 0;
-        if (t->ndim == 4 && (bh & 1)) return t->shape[0];
-        if (t->ndim == 2 && (bh & 2)) return t->shape[0];
-        return 0;
-    }
-    if (t->ndim != 2) return 0;
-    int64_t nbr = (t->shape[0] + bh - 1) / bh, nbc = (t->shape[1] + bw - 1) / bw;
-    return nbr * nbc;
+    if (t->numel == 0) return 0;
+    if (sp->kind == 0) return (t->ndim == 4 && (sp->kinds & 1)) || (t->ndim == 2 && (sp->kinds & 2));
+    return t->ndim == sp->nd;
 }
 
-static int64_t structure_of(const orc_tensor *t, int kind, int bh, int bw, int64_t i)
+static int64_t structure_count(const orc_spec *sp, const orc_tensor *t)
 {
-    if (kind == 0) {
-        int64_t len = t->numel / t->shape[0];
-        return i / len;
-    }
-    int64_t C = t->shape[1];
-    int64_t nbc = (C + bw - 1) / bw;
-    int64_t r = i / C, c = i % C;
-    return (r / bh) * nbc + (c / bw);
+    if (!spec_ranks(sp, t)) return 0;
+    if (sp->kind == 0) return t->shape[0];
+    int64_t n = 1;
+    for (int d = 0; d < sp->nd; ++d) n *= (t->shape[d] + sp->bs[d] - 1) / sp->bs[d];
+    return n;
 }
 
-static void structure_norms(const orc_tensor *t, const float *u, int kind, int bh, int bw,
-                            double *nu)
+/* Structure (numbered inside its tensor) that holds element i. */
+static int64_t structure_of(const orc_spec *sp, const orc_tensor *t, int64_t i)
 {
-    if (kind == 0) {
+    if (sp->kind == 0) return i / (t->numel / t->shape[0]);
+    int64_t coord[4], rest = i;
+    for (int d = sp->nd - 1; d >= 0; --d) { coord[d] = rest % t->shape[d]; rest /= t->shape[d]; }
+    int64_t id = 0;
+    for (int d = 0; d < sp->nd; ++d)
+        id = id * ((t->shape[d] + sp->bs[d] - 1) / sp->bs[d]) + coord[d] / sp->bs[d];
+    return id;
+}
+
+static double crit_add(double acc, float u, int crit)
+{
+    double x = (double)u;
+    if (crit == 0) return acc + x * x;
+    if (crit == 1) return acc + fabs(x);
+    double a = fabs(x);
+    return (a > acc || a != a) ? a : acc;      /* a NaN element makes the value NaN (ranks first) */
+}
+
+static void structure_values(const orc_spec *sp, const orc_tensor *t, const float *u, double *nu)
+{
+    if (sp->kind == 0) {
         int64_t len = t->numel / t->shape[0];
         for (int64_t f = 0; f < t->shape[0]; ++f) {
             double acc = 0.0;
-            for (int64_t j = 0; j < len; ++j) {
-                double x = (double)u[f * len + j];
-                acc = acc + x * x;
-            }
+            for (int64_t j = 0; j < len; ++j) acc = crit_add(acc, u[f * len + j], sp->crit);
             nu[f] = acc;
         }
         return;
     }
-    int64_t R = t->shape[0], C = t->shape[1];
-    int64_t nbr = (R + bh - 1) / bh, nbc = (C + bw - 1) / bw;
-    for (int64_t br = 0; br < nbr; ++br)
-        for (int64_t bc = 0; bc < nbc; ++bc) {
-            double acc = 0.0;
-            for (int64_t r = br * bh; r < (br + 1) * bh && r < R; ++r)
-                for (int64_t c = bc * bw; c < (bc + 1) * bw && c < C; ++c) {
-                    double x = (double)u[r * C + c];
-                    acc = acc + x * x;
-                }
-            nu[br * nbc + bc] = acc;
-        }
+    int64_t nb[4] = {1, 1, 1, 1}, sh[4] = {1, 1, 1, 1}, bs[4] = {1, 1, 1, 1};
+    /* right-align to four dimensions so that one loop nest serves every nd */
+    for (int d = 0; d < sp->nd; ++d) {
+        sh[4 - sp->nd + d] = t->shape[d];
+        bs[4 - sp->nd + d] = sp->bs[d];
+    }
+    for (int d = 0; d < 4; ++d) nb[d] = (sh[d] + bs[d] - 1) / bs[d];
+    int64_t id = 0;
+    for (int64_t b0 = 0; b0 < nb[0]; ++b0)
+    for (int64_t b1 = 0; b1 < nb[1]; ++b1)
+    for (int64_t b2 = 0; b2 < nb[2]; ++b2)
+    for (int64_t b3 = 0; b3 < nb[3]; ++b3) {
+        double acc = 0.0;
+        for (int64_t i0 = b0 * bs[0]; i0 < (b0 + 1) * bs[0] && i0 < sh[0]; ++i0)
+        for (int64_t i1 = b1 * bs[1]; i1 < (b1 + 1) * bs[1] && i1 < sh[1]; ++i1)
+        for (int64_t i2 = b2 * bs[2]; i2 < (b2 + 1) * bs[2] && i2 < sh[2]; ++i2)
+        for (int64_t i3 = b3 * bs[3]; i3 < (b3 + 1) * bs[3] && i3 < sh[3]; ++i3)
+            acc = crit_add(acc, u[((i0 * sh[1] + i1) * sh[2] + i2) * sh[3] + i3], sp->crit);
+        nu[id++] = acc;
+    }
 }
 
-/* nu for every structure in the list, in global structure order; returns the
- * count. nu may be NULL to only count. */
-int64_t orc_structure_norms(const orc_tensor *ts, int32_t T, float mu, int kind, int bh, int bw,
-                            double *nu)
+/* The ranked value of every structure in the list, in global structure order; returns
+ * the count. nu may be NULL to only count. */
+int64_t orc_structure_values(const orc_tensor *ts, int32_t T, float mu, const orc_spec *sp, double *nu)
 {
     int64_t S = 0;
     for (int32_t t = 0; t < T; ++t) {
-        int64_t c = structure_count(&ts[t], kind, bh, bw);
+        int64_t c = structure_count(sp, &ts[t]);
         if (c && nu) {
             float *u = (float *)malloc(sizeof(float) * (size_t)ts[t].numel);
             orc_form_u(ts[t].w, ts[t].lambda, mu, ts[t].numel, u);
-            structure_norms(&ts[t], u, kind, bh, bw, nu + S);
+            structure_values(sp, &ts[t], u, nu + S);
             free(u);
         }
         S += c;
@@ -382,27 +484,46 @@ int64_t orc_structure_norms(const orc_tensor *ts, int32_t T, float mu, int kind,
     return S;
 }
 
-static int cstep_structured(const orc_tensor *ts, int32_t T, double s, float mu, unsigned fuse,
-                            int kind, int bh, int bw, orc_result *res)
+/* Older form of the same: kind 0 with the slice mask in `bh`, or kind 1 with 2-D
+ * bh x bw blocks; squared L2 norm. */
+int64_t orc_structure_norms(const orc_tensor *ts, int32_t T, float mu, int kind, int bh, int bw,
+                            double *nu)
 {
-    int64_t S = orc_structure_norms(ts, T, mu, kind, bh, bw, NULL);
+    orc_spec sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.kind = kind;
+    if (kind == 0) sp.kinds = bh; else { sp.nd = 2; sp.bs[0] = bh; sp.bs[1] = bw; }
+    return orc_structure_values(ts, T, mu, &sp, nu);
+}
+
+int orc_cstep_structured(const orc_tensor *ts, int32_t T, double s, float mu, const orc_spec *sp,
+                         unsigned fuse, orc_result *res)
+{
+    if (sp->kind == 0 && (sp->kinds < 1 || sp->kinds > 3)) return -2;
+    if (sp->kind == 1) {
+        if (sp->nd < 1 || sp->nd > 4) return -2;
+        for (int d = 0; d < sp->nd; ++d) if (sp->bs[d] < 1) return -2;
+    }
+    if (sp->crit < 0 || sp->crit > 2) return -2;
+    int64_t S = orc_structure_values(ts, T, mu, sp, NULL);
     double *nu = (double *)malloc(sizeof(double) * (size_t)(S ? S : 1));
     unit_t *units = (unit_t *)malloc(sizeof(unit_t) * (size_t)(S ? S : 1));
     uint8_t *keep_s = (uint8_t *)malloc((size_t)(S ? S : 1));
     if (!nu || !units || !keep_s) { free(nu); free(units); free(keep_s); return -1; }
-    orc_structure_norms(ts, T, mu, kind, bh, bw, nu);
+    orc_structure_values(ts, T, mu, sp, nu);
     for (int64_t i = 0; i < S; ++i) { units[i].key = f64_bits(nu[i]); units[i].id = i; }
     rank_units(units, S, s, keep_s, res, 0x7FF0000000000000ull);
-    if (res->n_keep > 0) res->tau_norm = (float)sqrt(nu[res->tau_id]);
+    /* reported value of the weakest kept structure: the norm for the L2 criterion, else the value itself */
+    if (res->n_keep > 0) res->tau_norm = sp->crit == 0 ? (float)sqrt(nu[res->tau_id]) : (float)nu[res->tau_id];
     int64_t sbase = 0;
     for (int32_t t = 0; t < T; ++t) {
         int64_t n = ts[t].numel;
-        int64_t c = structure_count(&ts[t], kind, bh, bw);
+        int64_t c = structure_count(sp, &ts[t]);
         float *u = (float *)malloc(sizeof(float) * (size_t)(n ? n : 1));
         uint8_t *keep = (uint8_t *)malloc((size_t)(n ? n : 1));
         orc_form_u(ts[t].w, ts[t].lambda, mu, n, u);
         for (int64_t i = 0; i < n; ++i)
-            keep[i] = c ? keep_s[sbase + structure_of(&ts[t], kind, bh, bw, i)] : 1;
+            keep[i] = c ? keep_s[sbase + structure_of(sp, &ts[t], i)] : 1;
         finish_tensor(&ts[t], u, keep, mu, fuse);
         free(u); free(keep);
         sbase += c;
@@ -416,7 +537,10 @@ static int cstep_structured(const orc_tensor *ts, int32_t T, double s, float mu,
 int orc_cstep_filter(const orc_tensor *ts, int32_t T, double s, float mu, unsigned fuse,
                      orc_result *res)
 {
-    return cstep_structured(ts, T, s, mu, fuse, 0, 1, 0, res);
+    orc_spec sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.kinds = 1;
+    return orc_cstep_structured(ts, T, s, mu, &sp, fuse, res);
 }
 
 /* NeuronPrune / FilterPrune / StructurePrune in one call: `kinds` is the mask
@@ -424,8 +548,10 @@ int orc_cstep_filter(const orc_tensor *ts, int32_t T, double s, float mu, unsign
 int orc_cstep_structure(const orc_tensor *ts, int32_t T, double s, float mu, int kinds, unsigned fuse,
                         orc_result *res)
 {
-    if (kinds < 1 || kinds > 3) return -2;
-    return cstep_structured(ts, T, s, mu, fuse, 0, kinds, 0, res);
+    orc_spec sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.kinds = kinds;
+    return orc_cstep_structured(ts, T, s, mu, &sp, fuse, res);
 }
 
 /* Block pruning (Table 1, BlockPrune): 2-D tensors are ranked by bh x bw
@@ -434,11 +560,16 @@ int orc_cstep_block(const orc_tensor *ts, int32_t T, double s, float mu, int bh,
                     unsigned fuse, orc_result *res)
 {
     if (bh < 1 || bw < 1) return -2;
-    return cstep_structured(ts, T, s, mu, fuse, 1, bh, bw, res);
+    orc_spec sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.kind = 1; sp.nd = 2; sp.bs[0] = bh; sp.bs[1] = bw;
+    return orc_cstep_structured(ts, T, s, mu, &sp, fuse, res);
 }
 
+unsigned orc_sizeof_spec(void) { return (unsigned)sizeof(orc_spec); }
+
 /* Quantisation only (Table 1, Quantize(dtype)): theta = Q(u), mask = 1. The type is
- * binary16 unless `fuse` carries ORC_FUSE_BF16. */
+ * binary16 unless `fuse` carries ORC_FUSE_BF16, ORC_FUSE_E4M3 or ORC_FUSE_E5M2. */
 int orc_cstep_quantize(const orc_tensor *ts, int32_t T, float mu, unsigned fuse)
 {
     for (int32_t t = 0; t < T; ++t) {
@@ -447,7 +578,7 @@ int orc_cstep_quantize(const orc_tensor *ts, int32_t T, float mu, unsigned fuse)
         uint8_t *keep = (uint8_t *)malloc((size_t)(n ? n : 1));
         orc_form_u(ts[t].w, ts[t].lambda, mu, n, u);
         memset(keep, 1, (size_t)n);
-        finish_tensor(&ts[t], u, keep, mu, (fuse & ORC_FUSE_BF16) ? fuse : (fuse | ORC_FUSE_FP16));
+        finish_tensor(&ts[t], u, keep, mu, (fuse & (ORC_FUSE_BF16 | ORC_FUSE_E4M3 | ORC_FUSE_E5M2)) ? fuse : (fuse | ORC_FUSE_FP16));
         free(u); free(keep);
     }
     return 0;

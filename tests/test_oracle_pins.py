@@ -629,3 +629,138 @@ def test_bf16_hand_values_and_torch():
     exp = np.where(plain.mask[0] == 1, q.to(torch.float32).numpy(), np.float32(0))
     assert np.array_equal(out.mask[0], plain.mask[0]) and np.array_equal(bits(out.theta[0]), bits(exp))
     assert np.array_equal(out.theta_h[0], np.where(plain.mask[0] == 1, q.view(torch.int16).numpy().view(np.uint16), 0))
+
+
+# ---------------------------------------------------------------- 8-bit floating point
+def test_fp8_hand_values_roundtrip_midpoints_and_torch():
+    """Quantize(dtype) with the two 8-bit formats: hand-worked values, every code widens and
+    converts back to itself, every midpoint between neighbouring codes goes to the even one,
+    and torch's independent cast agrees wherever the value is inside the format's range."""
+    import torch
+    rows = []
+    with open(os.path.join(GOLD, "fp8_hand_values.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                fmt, a, b = line.split()
+                rows.append((fmt, int(a, 16), int(b, 16)))
+    assert len(rows) >= 30
+    for fmt, fb, code in rows:
+        assert int(oracle.lib().orc_f32_to_fp8(fb, oracle.FP8_FORMATS[fmt])) == code, (fmt, hex(fb))
+    for fmt, tdt, top in (("e4m3", torch.float8_e4m3fn, 0x7E), ("e5m2", torch.float8_e5m2, 0x7B)):
+        codes = np.array([c for c in range(256) if (c & 0x7F) <= top], np.uint8)        # the finite codes
+        wide = oracle.fp8_bits_to_f32(codes, fmt)
+        ref = torch.from_numpy(codes.copy()).view(tdt).to(torch.float32).numpy()        # torch's widening: exact
+        assert np.array_equal(bits(wide), bits(ref))
+        assert np.array_equal(oracle.f32_to_fp8_bits(wide, fmt), codes)
+        # midpoints of neighbouring non-negative codes: exactly representable in fp32, go to the even code
+        pos = np.arange(0, top, dtype=np.uint8)
+        lo, hi = oracle.fp8_bits_to_f32(pos, fmt).astype(np.float64), oracle.fp8_bits_to_f32(pos + 1, fmt).astype(np.float64)
+        mid = ((lo + hi) / 2).astype(np.float32)
+        assert np.array_equal(mid.astype(np.float64), (lo + hi) / 2)
+        got = oracle.f32_to_fp8_bits(mid, fmt)
+        assert np.array_equal(got, np.where(pos % 2 == 0, pos, pos + 1))
+        assert np.array_equal(oracle.f32_to_fp8_bits(-mid, fmt), np.where(pos % 2 == 0, pos, pos + 1) | 0x80)
+        # random and rounding-critical patterns inside the range against torch
+        rng = np.random.default_rng(6)
+        p = rng.integers(0, 1 << 32, size=1 << 20, dtype=np.uint64).astype(np.uint32)
+        x = p.view(np.float32)
+        maxv = float(oracle.fp8_bits_to_f32(np.array([top], np.uint8), fmt)[0])
+        inside = np.isfinite(x) & (np.abs(x) <= maxv)
+        x = np.concatenate([x[inside], (rng.standard_normal(1 << 18) * 2).astype(np.float32),
+                            (rng.standard_normal(1 << 18) * 1e-2).astype(np.float32)])
+        ref = torch.from_numpy(x.copy()).to(tdt).view(torch.uint8).numpy()
+        assert np.array_equal(oracle.f32_to_fp8_bits(x, fmt), ref)
+    # the scheme: theta is the widened code, theta_h carries the code, prune first then quantise
+    w = np.array([0.3, -1.06, 500.0, 3e-4, 0.0], np.float32)
+    out = oracle.cstep_quantize([w], [None], 1.0, ("e4m3",))
+    assert out.theta[0].tolist() == [0.3125, -1.0, 448.0, 0.0, 0.0]
+    assert out.theta_h[0].tolist() == [0x2A, 0xB8, 0x7E, 0x00, 0x00] and out.mask[0].all()
+    out = oracle.cstep_prune([w], [None], 0.6, 1.0, ("e5m2",))
+    assert out.theta[0].tolist() == [0.0, -1.0, 512.0, 0.0, 0.0] and out.mask[0].tolist() == [0, 1, 1, 0, 0]
+
+
+# ---------------------------------------------------------------- criteria and n-D blocks
+@pytest.mark.parametrize("crit", ["l2", "l1", "max"])
+def test_structure_criteria_closed_forms_and_bruteforce(crit):
+    """FilterPrune / NeuronPrune / BlockPrune "based on criteria" (Table 1): the ranked value from
+    numpy, the kept set from the O(n^2) rank definition, for slices and for 2-D blocks."""
+    rng = np.random.default_rng(12)
+    conv = rng.standard_normal((6, 3, 3, 3)).astype(np.float32)
+    fc = rng.standard_normal((7, 10)).astype(np.float32)
+    lam = [(rng.standard_normal(a.shape) * 0.01).astype(np.float32) for a in (conv, fc)]
+    mu = 0.05
+    f = {"l2": lambda a: (a * a).sum(1), "l1": lambda a: np.abs(a).sum(1), "max": lambda a: np.abs(a).max(1)}[crit]
+    u = [oracle.form_u(a, l, mu).astype(np.float64) for a, l in zip((conv, fc), lam)]
+    nu = oracle.structure_values([conv, fc], lam, mu, "structure", criterion=crit)
+    ref = np.concatenate([f(u[0].reshape(6, -1)), f(u[1])])
+    assert np.allclose(nu, ref, rtol=1e-14, atol=0)
+    if crit == "max":
+        assert np.array_equal(nu, ref)                         # a maximum has no rounding
+    out = oracle.cstep_structured([conv, fc], lam, 0.5, mu, "structure", criterion=crit, fuse=("lambda",))
+    keep = brute_keep(nu.view(np.uint64), 13 - 7)
+    assert np.array_equal(out.mask[0][:, 0, 0, 0], keep[:6]) and np.array_equal(out.mask[1][:, 0], keep[6:])
+    assert np.array_equal(out.mask[0], np.repeat(keep[:6], 27).reshape(conv.shape))
+    if crit != "l2":
+        assert out.result.tau_norm == pytest.approx(nu[out.result.tau_id], rel=1e-6)
+    # 2-D blocks of 3 x 2 on a ragged matrix
+    m = rng.standard_normal((8, 7)).astype(np.float32)
+    nu = oracle.structure_values([m], [None], 1.0, "block", (3, 2), crit)
+    ref = np.array([f(m[3 * r:3 * r + 3, 2 * c:2 * c + 2].astype(np.float64).reshape(1, -1))[0]
+                    for r in range(3) for c in range(4)])
+    assert np.allclose(nu, ref, rtol=1e-14, atol=0)
+    out = oracle.cstep_structured([m], [None], 0.5, 1.0, "block", (3, 2), crit)
+    grid = brute_keep(nu.view(np.uint64), 6).reshape(3, 4)
+    assert np.array_equal(out.mask[0], np.kron(grid, np.ones((3, 2), np.uint8))[:8, :7])
+    # integer data: L1 sums are exact in any order
+    ints = rng.integers(-50, 51, size=(5, 40)).astype(np.float32)
+    assert oracle.structure_values([ints], [None], 1.0, "neuron", criterion="l1").tolist() == np.abs(ints).sum(1).tolist()
+    # with the L2 criterion the specification form is the older call
+    a = oracle.cstep_structured([conv, fc], lam, 0.4, mu, "filter", fuse=("lambda",))
+    b = oracle.cstep_filter([conv, fc], lam, 0.4, mu, fuse=("lambda",))
+    assert all(np.array_equal(x, y) for x, y in zip(a.mask, b.mask)) and a.result.tau_key == b.result.tau_key
+
+
+@pytest.mark.parametrize("block", [(2, 2, 2), (1, 3, 2), (2, 1, 3, 3), (4, 4), (5,), (3, 2, 1, 2)])
+def test_nd_blocks_values_kept_set_and_mask_bruteforce(block):
+    """BlockPrune with n-D blocks (Table 1: "n-D blocks of size bs"): every tensor whose rank equals
+    the number of block extents is cut into blocks; values from numpy slices in row-major order
+    inside the block, kept set by the rank definition, the mask block by block."""
+    nd = len(block)
+    shape = {1: (23,), 2: (9, 10), 3: (5, 7, 4), 4: (5, 3, 4, 5)}[nd]
+    other = {1: (4, 4), 2: (6,), 3: (6, 5), 4: (7, 2, 2)}[nd]
+    ws = W.random_set([shape, other, shape], seed=40 + nd, kind="normal", scale=0.3, lam_sigma=1e-2, mu=1e-2)
+    s = 0.45
+    out = oracle.cstep_structured(ws.w, ws.lam, s, ws.mu, "block", block, "l2", fuse=("lambda",))
+    nu = oracle.structure_values(ws.w, ws.lam, ws.mu, "block", block)
+    ref, grids = [], []
+    for t in (0, 2):
+        u = oracle.form_u(ws.w[t], ws.lam[t], ws.mu).astype(np.float64)
+        nb = [-(-shape[d] // block[d]) for d in range(nd)]
+        grids.append(nb)
+        for bidx in itertools.product(*[range(n) for n in nb]):
+            sl = tuple(slice(bidx[d] * block[d], (bidx[d] + 1) * block[d]) for d in range(nd))
+            acc = 0.0
+            for x in u[sl].reshape(-1):                # row-major inside the block
+                acc = acc + x * x
+            ref.append(acc)
+    ref = np.array(ref)
+    assert np.array_equal(nu.view(np.uint64), ref.view(np.uint64))
+    S = ref.size
+    z = int(math.floor(s * S + 0.5))
+    keep_s = brute_keep(ref.view(np.uint64), S - z)
+    assert out.result.n_units == S and out.result.n_zero == z
+    assert out.mask[1].all()                            # another rank: passes through
+    sid = 0
+    for t, nb in zip((0, 2), grids):
+        n = int(np.prod(nb))
+        grid = keep_s[sid:sid + n].reshape(nb)
+        exp = grid
+        for d in range(nd):
+            exp = np.repeat(exp, block[d], axis=d)
+        exp = exp[tuple(slice(0, shape[d]) for d in range(nd))]
+        assert np.array_equal(out.mask[t], exp)
+        u = oracle.form_u(ws.w[t], ws.lam[t], ws.mu)
+        assert np.array_equal(bits(out.theta[t]), np.where(exp == 1, bits(u), 0))
+        sid += n
+    assert sid == S
