@@ -86,8 +86,11 @@ enum {
     CONDENSA_FUSE_FP16 = 1,     /* theta = fp16 round-to-nearest-even of kept u, widened back  */
     CONDENSA_FUSE_LAMBDA = 2,   /* update lambda in place                                     */
     CONDENSA_FUSE_PENALTY = 4,  /* write g to grad                                            */
-    CONDENSA_FUSE_BF16 = 8,     /* like FUSE_FP16 with bfloat16 (not together with it); theta_h
-                                   then holds bfloat16 bits                                     */
+    CONDENSA_FUSE_BF16 = 8,     /* like FUSE_FP16 with bfloat16; theta_h then holds bfloat16 bits  */
+    CONDENSA_FUSE_E4M3 = 16,    /* like FUSE_FP16 with the 8-bit format E4M3 (see
+                                   condensa_cstep_quantize); theta_h then holds the code in its
+                                   low byte                                                     */
+    CONDENSA_FUSE_E5M2 = 32,    /* the same with E5M2. At most one of the four types per call   */
     CONDENSA_NO_SAMPLING = 64   /* rank with full histogram passes, then project (two passes over
                                    w and lambda; same results). It also sends rankings of at most
                                    16384 structures (filters, rows, general blocks), which by
@@ -120,7 +123,7 @@ enum {
     CONDENSA_ERR_TOO_LARGE = -6      /* input larger than a fixed built-in limit               */
 };
 
-enum { CONDENSA_DTYPE_FP16 = 1, CONDENSA_DTYPE_BF16 = 2 };
+enum { CONDENSA_DTYPE_FP16 = 1, CONDENSA_DTYPE_BF16 = 2, CONDENSA_DTYPE_FP8_E4M3 = 3, CONDENSA_DTYPE_FP8_E5M2 = 4 };
 
 /* Record of the last ranking call, filled on the device. */
 typedef struct {
@@ -190,12 +193,49 @@ CONDENSA_API int condensa_cstep_structure(condensa_ctx *ctx, const condensa_tens
 CONDENSA_API int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
                          double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream);
 
+/* Structured pruning by a specification (Table 1: NeuronPrune(criteria), FilterPrune(criteria),
+ * StructurePrune(criteria), BlockPrune(criteria, bs) - "prune based on criteria", blocks of
+ * 1, 3 or n dimensions "of size bs"). The calls above are special cases of this one.
+ *   kind CONDENSA_SPEC_SLICES  leading-index slices: `kinds` as in condensa_cstep_structure().
+ *   kind CONDENSA_SPEC_BLOCKS  every tensor with ndim == spec->ndim is cut into blocks of
+ *        block[0] x ... x block[ndim-1] elements, numbered row-major over the grid of blocks;
+ *        a block that sticks out over an edge holds fewer elements. Extents up to 4096; tensor
+ *        extents below 2^31.
+ *   criterion: the value a structure is ranked by, accumulated in fp64 over its elements in
+ *        row-major order - CONDENSA_CRIT_L2 the sum of u^2 (the squared L2 norm; this is the
+ *        argmin of Section 3.3), CONDENSA_CRIT_L1 the sum of |u|, CONDENSA_CRIT_MAX the largest
+ *        |u|. The paper names no criterion; L1 and MAX are the usual alternatives and are not
+ *        the projection of Section 3.3. condensa_result.tau_key holds the fp64 bits of the
+ *        weakest kept value, tau_norm its square root for L2 and the value itself otherwise.
+ * Every other tensor passes through (theta = u, mask = 1). */
+enum { CONDENSA_SPEC_SLICES = 0, CONDENSA_SPEC_BLOCKS = 1 };
+enum { CONDENSA_CRIT_L2 = 0, CONDENSA_CRIT_L1 = 1, CONDENSA_CRIT_MAX = 2 };
+typedef struct {
+    int32_t kind;         /* CONDENSA_SPEC_SLICES or CONDENSA_SPEC_BLOCKS              */
+    int32_t kinds;        /* SLICES: CONDENSA_STRUCT_FILTER and/or CONDENSA_STRUCT_NEURON */
+    int32_t criterion;    /* CONDENSA_CRIT_*                                            */
+    int32_t ndim;         /* BLOCKS: number of block extents                            */
+    int64_t block[4];     /* BLOCKS: the extents                                        */
+} condensa_structure_spec;
+CONDENSA_API int condensa_cstep_structured(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
+                                           double sparsity, float mu, const condensa_structure_spec *spec,
+                                           unsigned fuse, void *stream);
+
 /* Quantize(dtype) - theta = round-to-nearest-even of u in `dtype` for every element,
- * mask = 1 (Table 1; Section 2 "low-precision approximation"). dtype is
- * CONDENSA_DTYPE_FP16 (IEEE binary16) or CONDENSA_DTYPE_BF16 (bfloat16: the upper
- * half of a binary32); theta_h receives the 16 bits. Overflow goes to infinity,
- * underflow is gradual, NaN becomes a quiet NaN with the same sign. `fuse` may
- * carry FUSE_LAMBDA / FUSE_PENALTY only. */
+ * mask = 1 (Table 1; Section 2 "low-precision approximation"; Conclusion: further data
+ * types for quantization). dtype is
+ *   CONDENSA_DTYPE_FP16      IEEE binary16;
+ *   CONDENSA_DTYPE_BF16      bfloat16, the upper half of a binary32;
+ *   CONDENSA_DTYPE_FP8_E4M3  1 sign, 4 exponent (bias 7), 3 fraction bits, no infinity,
+ *                            NaN = S.1111.111, largest finite value 448;
+ *   CONDENSA_DTYPE_FP8_E5M2  1 sign, 5 exponent (bias 15), 2 fraction bits, largest
+ *                            finite value 57344.
+ * theta_h receives the code (16 bits; an 8-bit code in the low byte). Underflow is
+ * gradual; NaN becomes a quiet NaN with the same sign. Overflow goes to infinity for the
+ * two 16-bit types and SATURATES for the two 8-bit types: whatever rounds beyond the
+ * largest finite value, infinity included, becomes that value (an 8-bit codebook with
+ * infinities in it would be useless for weights; this is also what the conversion
+ * instruction of the GPU does). `fuse` may carry FUSE_LAMBDA / FUSE_PENALTY only. */
 CONDENSA_API int condensa_cstep_quantize(condensa_ctx *ctx, const condensa_tensor *tensors, int T, float mu,
                             int dtype, unsigned fuse, void *stream);
 
@@ -251,6 +291,15 @@ enum { CONDENSA_OP_PRUNE = 0, CONDENSA_OP_FILTER = 1, CONDENSA_OP_BLOCK = 2,
  * CONDENSA_OP_BLOCK only, sparsity for the three pruning operations. */
 CONDENSA_API int condensa_cstep_host(condensa_ctx *ctx, int op, const condensa_tensor *tensors, int T,
                         double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream);
+
+/* Workspace a context needs for calls of a given shape, so that condensa_create() can
+ * reserve it and no call allocates later: `op` is a CONDENSA_OP_* value (PRUNE, FILTER,
+ * BLOCK, QUANTIZE, LAGRANGE), `tensors` / `T` the list (only numel, ndim, shape and the
+ * alignment of the pointers are looked at), `spec` the structure specification of a
+ * structured call (NULL: filters resp. 4 x 4 blocks by the L2 norm), `fuse` as for the
+ * call. Writes the byte count to *bytes. Host only; nothing is launched. */
+CONDENSA_API int condensa_workspace_bytes(int op, const condensa_tensor *tensors, int T,
+                                          const condensa_structure_spec *spec, unsigned fuse, size_t *bytes);
 
 /* Waits for the stream of the last ranking call and copies its record. */
 CONDENSA_API int condensa_get_result(condensa_ctx *ctx, condensa_result *out);

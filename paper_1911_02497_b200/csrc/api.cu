@@ -130,10 +130,12 @@ int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double
     if (op <= CONDENSA_OP_BLOCK && !(s >= 0.0 && s <= 1.0))
         return fail(ctx, CONDENSA_ERR_INVALID_ARG, "sparsity must lie in [0, 1]");
     const unsigned known = CONDENSA_FUSE_FP16 | CONDENSA_FUSE_LAMBDA | CONDENSA_FUSE_PENALTY | CONDENSA_FUSE_BF16 |
-                           CONDENSA_NO_SAMPLING;
+                           CONDENSA_FUSE_E4M3 | CONDENSA_FUSE_E5M2 | CONDENSA_NO_SAMPLING;
     if (fuse & ~known) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "unknown fuse bits");
-    if ((fuse & CONDENSA_FUSE_FP16) && (fuse & CONDENSA_FUSE_BF16))
-        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "FUSE_FP16 and FUSE_BF16 exclude each other");
+    {
+        const unsigned qb = fuse & (CONDENSA_FUSE_FP16 | CONDENSA_FUSE_BF16 | CONDENSA_FUSE_E4M3 | CONDENSA_FUSE_E5M2);
+        if (qb & (qb - 1)) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "at most one quantisation type may be fused");
+    }
     std::vector<Interval> iv;
     iv.reserve((size_t)T * 6);
     for (int t = 0; t < T; ++t) {
@@ -173,9 +175,19 @@ int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double
     return CONDENSA_OK;
 }
 
-// kinds: for OP_FILTER, which leading-index slices are ranked (1 = filters of 4-D tensors, 2 = rows of 2-D tensors)
-void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, int kinds = 1, int bh = 4, int bw = 4)
+// What a structured call ranks: for OP_FILTER which leading-index slices (1 = filters of 4-D tensors,
+// 2 = rows of 2-D tensors); for OP_BLOCKGEN the block extents, one per dimension of the tensors
+// that are cut; and the criterion.
+struct HostSpec {
+    int kinds = 1;
+    int nd = 2;
+    long long bs[4] = {4, 4, 1, 1};
+    int crit = CRIT_L2;
+};
+
+void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, const HostSpec &sp = HostSpec())
 {
+    const int kinds = sp.kinds;
     pl.td.resize(T);
     pl.prefix_a.assign(T + 1, 0);
     pl.prefix_b.assign(T + 1, 0);
@@ -215,14 +227,25 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, int kinds = 
                 items_a = d.d0 * ((d.d1 + SEG - 1) / SEG);
             }
         } else if (op == OP_BLOCKGEN) {
-            d.ranked = (x.ndim == 2 && x.numel > 0) ? 1 : 0;
+            d.ranked = (x.ndim == sp.nd && x.numel > 0) ? 1 : 0;
             if (d.ranked) {
-                d.d0 = x.shape[0];
-                d.d1 = x.shape[1];
-                d.bh = bh;
-                d.bw = bw;
-                d.nbc = (d.d1 + bw - 1) / bw;
-                d.n_units = ((d.d0 + bh - 1) / bh) * d.nbc;
+                d.nd = sp.nd;
+                d.n_units = 1;
+                for (int q = 0; q < 4; ++q) { d.sh[q] = 1; d.bs[q] = 1; d.nb[q] = 1; }
+                for (int q = 0; q < sp.nd; ++q) {          // right-aligned to four dimensions
+                    const int r = 4 - sp.nd + q;
+                    d.sh[r] = (int)x.shape[q];
+                    d.bs[r] = (int)std::min<long long>(sp.bs[q], x.shape[q]);
+                    d.nb[r] = (int)((x.shape[q] + sp.bs[q] - 1) / sp.bs[q]);
+                    d.n_units *= d.nb[r];
+                }
+                if (sp.nd == 2) {
+                    d.d0 = x.shape[0];
+                    d.d1 = x.shape[1];
+                    d.bh = d.bs[2];
+                    d.bw = d.bs[3];
+                    d.nbc = d.nb[3];
+                }
                 items_a = (d.n_units + BLOCKS_PER_ITEM - 1) / BLOCKS_PER_ITEM;
             }
         } else if (op == OP_BLOCK) {
@@ -290,7 +313,7 @@ Layout make_layout(int T, const Plan &pl, bool ranking, bool filter, int journal
     return L;
 }
 
-int ensure_workspace(condensa_ctx *ctx, size_t bytes, cudaStream_t stream)
+int ensure_workspace(condensa_ctx *ctx, size_t bytes, cudaStream_t stream, bool exact = false)
 {
     if (bytes <= ctx->ws_bytes) return CONDENSA_OK;
     CU_TRY(ctx, cudaStreamSynchronize(stream));
@@ -302,7 +325,7 @@ int ensure_workspace(condensa_ctx *ctx, size_t bytes, cudaStream_t stream)
     ctx->last_upload_dst = nullptr;
     ctx->has_result = false;       // the record of an earlier call lived in the old workspace
     ctx->ctl = nullptr;
-    const size_t want = align_up(bytes + bytes / 4, 1 << 20);
+    const size_t want = exact ? align_up(bytes, 256) : align_up(bytes + bytes / 4, 1 << 20);
     cudaError_t e = cudaMalloc((void **)&ctx->ws, want);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -460,17 +483,14 @@ Sel initial_state(long long S, long long k, int bits_key)
     return s;
 }
 
-int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double sparsity, float mu,
-           unsigned fuse, cudaStream_t stream, int kinds = 1, int bh = 4, int bw = 4)
+// Work decomposition and workspace layout of one call (no device work).
+Layout plan_call(int op, const condensa_tensor *ts, int T, unsigned fuse, const HostSpec &sp, Plan &pl,
+                 bool &ranking, bool &sampling)
 {
-    int rc = validate(ctx, op == OP_BLOCKGEN ? OP_BLOCK : op, ts, T, sparsity, mu, fuse);
-    if (rc) return rc;
-    CU_TRY(ctx, cudaSetDevice(ctx->device));
-    Plan pl;
-    build_plan(op, ts, T, pl, kinds, bh, bw);
-    const bool ranking = op <= OP_BLOCK || op == OP_BLOCKGEN;
+    build_plan(op, ts, T, pl, sp);
+    ranking = op <= OP_BLOCK || op == OP_BLOCKGEN;
     // single-pass path: unstructured and block pruning of lists too large to list whole
-    const bool sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) &&
+    sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) &&
                           (u64)pl.S > pl.cap && pl.S >= 8ll * N_SAMPLE;
     if (sampling && op == OP_BLOCK && pl.cap > (1ull << 20)) pl.cap = 1ull << 20;   // bounds the journal
     const int journal_floats = sampling ? (op == OP_BLOCK ? 16 : 1) : 0;
@@ -489,7 +509,23 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             }
         }
     }
-    const Layout L = make_layout(T, pl, ranking, op == OP_FILTER || op == OP_BLOCKGEN, journal_floats);
+    return make_layout(T, pl, ranking, op == OP_FILTER || op == OP_BLOCKGEN, journal_floats);
+}
+
+int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double sparsity, float mu,
+           unsigned fuse, cudaStream_t stream, const HostSpec &sp = HostSpec())
+{
+    int rc = validate(ctx, op == OP_BLOCKGEN ? OP_BLOCK : op, ts, T, sparsity, mu, fuse);
+    if (rc) return rc;
+    if (op == OP_BLOCKGEN)
+        for (int t = 0; t < T; ++t)
+            for (int q = 0; q < ts[t].ndim; ++q)
+                if (ts[t].ndim == sp.nd && ts[t].shape[q] > 0x7FFFFFFFll)
+                    return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "tensor %d: an extent above 2^31 - 1 cannot be cut into blocks", t);
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    Plan pl;
+    bool ranking = false, sampling = false;
+    const Layout L = plan_call(op, ts, T, fuse, sp, pl, ranking, sampling);
     rc = ensure_workspace(ctx, L.total, stream);
     if (rc) return rc;
     char *ws = ctx->ws;
@@ -504,9 +540,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     const long long *pb = pe + pl.edge_items.size();         // projection prefix, right behind it
     P.T = T;
     P.mu = mu;
-    P.fuse = fuse & 15u;
-    if (op == OP_QUANTIZE && !(P.fuse & FUSE_BF16)) P.fuse |= FUSE_FP16;
-    if (op == OP_LAGRANGE) P.fuse &= ~(unsigned)(FUSE_FP16 | FUSE_BF16);
+    P.fuse = fuse & FUSE_KERNEL_BITS;
+    if (op == OP_QUANTIZE && !(P.fuse & FUSE_QUANT)) P.fuse |= FUSE_FP16;
+    if (op == OP_LAGRANGE) P.fuse &= ~FUSE_QUANT;
     P.ctl = (Ctl *)(ws + L.ctl);
     P.hist = (u64 *)(ws + L.hist);
     P.fin_key = (u64 *)(ws + L.fin_key);
@@ -527,6 +563,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     P.n_sample = N_SAMPLE;
     P.jr_lam = (float *)(ws + L.journal);
     P.onepass_cap = pl.cap;
+    P.crit = sp.crit;
     P.seed = ctx->seed;
     {
         // a missed sample bracket can be repaired inside the call unless the first pass
@@ -536,7 +573,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             for (int t = 0; t < T; ++t) lam_in_place = lam_in_place || (ts[t].lambda != nullptr && ts[t].numel > 0);
         P.miss_fallback = lam_in_place ? 0 : 1;
     }
-    bool need_h = (fuse & (CONDENSA_FUSE_FP16 | CONDENSA_FUSE_BF16)) != 0;
+    bool need_h = (fuse & FUSE_QUANT) != 0;
     for (int t = 0; t < T; ++t) need_h = need_h || ts[t].theta_h != nullptr;
     ctx->ctl = P.ctl;
     // the workspace is shared by all calls of the context: a call on another stream
@@ -738,7 +775,7 @@ int condensa_create(condensa_ctx **out, int device, size_t workspace_bytes)
         c->seed = z;
     }
     if (workspace_bytes) {
-        int rc = ensure_workspace(c, workspace_bytes, nullptr);
+        int rc = ensure_workspace(c, workspace_bytes, nullptr, true);
         if (rc) {
             g_create_error = c->err;
             cudaEventDestroy(c->stage_ev);
@@ -767,6 +804,33 @@ int condensa_destroy(condensa_ctx *ctx)
     return CONDENSA_OK;
 }
 
+int condensa_workspace_bytes(int op, const condensa_tensor *tensors, int T, const condensa_structure_spec *spec,
+                             unsigned fuse, size_t *bytes)
+{
+    if (!bytes || !tensors || T <= 0 || op < CONDENSA_OP_PRUNE || op > CONDENSA_OP_LAGRANGE)
+        return fail(nullptr, CONDENSA_ERR_INVALID_ARG, "condensa_workspace_bytes: bad argument");
+    HostSpec sp;
+    int iop = op;
+    if (op == CONDENSA_OP_FILTER || op == CONDENSA_OP_BLOCK) {
+        if (spec) {
+            sp.crit = spec->criterion;
+            if (spec->kind == CONDENSA_SPEC_SLICES) { iop = OP_FILTER; sp.kinds = spec->kinds; }
+            else {
+                if (spec->ndim < 1 || spec->ndim > 4) return fail(nullptr, CONDENSA_ERR_INVALID_ARG, "blocks have 1 to 4 dimensions");
+                sp.nd = spec->ndim;
+                for (int q = 0; q < 4; ++q) sp.bs[q] = q < spec->ndim ? spec->block[q] : 1;
+                const bool fast = sp.nd == 2 && sp.bs[0] == 4 && sp.bs[1] == 4 && sp.crit == CRIT_L2;
+                iop = fast ? OP_BLOCK : OP_BLOCKGEN;
+            }
+        }
+    }
+    Plan pl;
+    bool ranking = false, sampling = false;
+    const Layout L = plan_call(iop, tensors, T, fuse, sp, pl, ranking, sampling);
+    *bytes = align_up(L.total + L.total / 4, 1 << 20);      // what a call of this shape makes the context hold
+    return CONDENSA_OK;
+}
+
 int condensa_set_seed(condensa_ctx *ctx, uint64_t seed)
 {
     if (!ctx) return CONDENSA_ERR_INVALID_ARG;
@@ -792,7 +856,9 @@ int condensa_cstep_structure(condensa_ctx *ctx, const condensa_tensor *tensors, 
     if (!ctx) return CONDENSA_ERR_INVALID_ARG;
     if (kinds < 1 || kinds > (CONDENSA_STRUCT_FILTER | CONDENSA_STRUCT_NEURON))
         return fail(ctx, CONDENSA_ERR_INVALID_ARG, "kinds must be CONDENSA_STRUCT_FILTER and/or CONDENSA_STRUCT_NEURON");
-    return run_op(ctx, OP_FILTER, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, kinds);
+    HostSpec sp;
+    sp.kinds = kinds;
+    return run_op(ctx, OP_FILTER, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, sp);
 }
 
 int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T, double sparsity,
@@ -801,20 +867,55 @@ int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int 
     if (!ctx) return CONDENSA_ERR_INVALID_ARG;
     if (bh < 1 || bw < 1) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "block shape must be positive");
     if (bh > 4096 || bw > 4096) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "block sides above 4096 are not built");
-    if (bh != 4 || bw != 4)      // general shapes: norms per block, selection on the norm array, elementwise projection
-        return run_op(ctx, OP_BLOCKGEN, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, 1, bh, bw);
+    if (bh != 4 || bw != 4) {    // general shapes: norms per block, selection on the norm array, elementwise projection
+        HostSpec sp;
+        sp.nd = 2; sp.bs[0] = bh; sp.bs[1] = bw;
+        return run_op(ctx, OP_BLOCKGEN, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, sp);
+    }
     return run_op(ctx, OP_BLOCK, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream);
+}
+
+int condensa_cstep_structured(condensa_ctx *ctx, const condensa_tensor *tensors, int T, double sparsity,
+                              float mu, const condensa_structure_spec *spec, unsigned fuse, void *stream)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    if (!spec) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "spec is NULL");
+    if (spec->criterion < CONDENSA_CRIT_L2 || spec->criterion > CONDENSA_CRIT_MAX)
+        return fail(ctx, CONDENSA_ERR_INVALID_ARG, "criterion must be CONDENSA_CRIT_L2, _L1 or _MAX");
+    HostSpec sp;
+    sp.crit = spec->criterion;
+    if (spec->kind == CONDENSA_SPEC_SLICES) {
+        if (spec->kinds < 1 || spec->kinds > (CONDENSA_STRUCT_FILTER | CONDENSA_STRUCT_NEURON))
+            return fail(ctx, CONDENSA_ERR_INVALID_ARG, "kinds must be CONDENSA_STRUCT_FILTER and/or CONDENSA_STRUCT_NEURON");
+        sp.kinds = spec->kinds;
+        return run_op(ctx, OP_FILTER, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, sp);
+    }
+    if (spec->kind != CONDENSA_SPEC_BLOCKS) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "kind must be CONDENSA_SPEC_SLICES or CONDENSA_SPEC_BLOCKS");
+    if (spec->ndim < 1 || spec->ndim > 4) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "blocks have 1 to 4 dimensions");
+    sp.nd = spec->ndim;
+    for (int q = 0; q < 4; ++q) sp.bs[q] = 1;
+    for (int q = 0; q < spec->ndim; ++q) {
+        if (spec->block[q] < 1) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "block extents must be positive");
+        if (spec->block[q] > 4096) return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "block extents above 4096 are not built");
+        sp.bs[q] = spec->block[q];
+    }
+    // 4 x 4 blocks of matrices by the L2 norm take the single-pass kernels
+    if (sp.nd == 2 && sp.bs[0] == 4 && sp.bs[1] == 4 && sp.crit == CRIT_L2)
+        return run_op(ctx, OP_BLOCK, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream);
+    return run_op(ctx, OP_BLOCKGEN, tensors, T, sparsity, mu, fuse, (cudaStream_t)stream, sp);
 }
 
 int condensa_cstep_quantize(condensa_ctx *ctx, const condensa_tensor *tensors, int T, float mu,
                             int dtype, unsigned fuse, void *stream)
 {
     if (!ctx) return CONDENSA_ERR_INVALID_ARG;
-    if (dtype != CONDENSA_DTYPE_FP16 && dtype != CONDENSA_DTYPE_BF16)
-        return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "only fp16 and bf16 are built");
-    if (fuse & (CONDENSA_FUSE_FP16 | CONDENSA_FUSE_BF16))
+    if (dtype < CONDENSA_DTYPE_FP16 || dtype > CONDENSA_DTYPE_FP8_E5M2)
+        return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "dtype must be one of CONDENSA_DTYPE_FP16 / BF16 / FP8_E4M3 / FP8_E5M2");
+    if (fuse & FUSE_QUANT)
         return fail(ctx, CONDENSA_ERR_INVALID_ARG, "the type is given by dtype, not by fuse bits");
     if (dtype == CONDENSA_DTYPE_BF16) fuse |= CONDENSA_FUSE_BF16;
+    if (dtype == CONDENSA_DTYPE_FP8_E4M3) fuse |= CONDENSA_FUSE_E4M3;
+    if (dtype == CONDENSA_DTYPE_FP8_E5M2) fuse |= CONDENSA_FUSE_E5M2;
     return run_op(ctx, OP_QUANTIZE, tensors, T, 0.0, mu, fuse, (cudaStream_t)stream);
 }
 
@@ -1268,7 +1369,7 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
     long long *prefix = (long long *)(ws + L.desc + sizeof(TensorDesc));
     P.T = 1;
     P.mu = mu;
-    P.fuse = fuse & 15u;
+    P.fuse = fuse & FUSE_KERNEL_BITS;
     P.ctl = (Ctl *)(ws + L.ctl);
     P.hist = (u64 *)(ws + L.hist);
     P.fin_key = (u64 *)(ws + L.fin_key);

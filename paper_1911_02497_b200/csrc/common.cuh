@@ -23,8 +23,11 @@ constexpr int MAX_SELECT_ITERS = 24;
 constexpr u64 KEY_NONE = ~0ull;          // cut-off key that keeps nothing
 
 enum { OP_PRUNE = 0, OP_FILTER = 1, OP_BLOCK = 2, OP_QUANTIZE = 3, OP_LAGRANGE = 4, OP_BLOCKGEN = 5 };
-enum { FUSE_FP16 = 1, FUSE_LAMBDA = 2, FUSE_PENALTY = 4, FUSE_BF16 = 8, NO_SAMPLING = 64 };
+enum { FUSE_FP16 = 1, FUSE_LAMBDA = 2, FUSE_PENALTY = 4, FUSE_BF16 = 8, FUSE_E4M3 = 16, FUSE_E5M2 = 32, NO_SAMPLING = 64 };
+constexpr unsigned FUSE_QUANT = FUSE_FP16 | FUSE_BF16 | FUSE_E4M3 | FUSE_E5M2;
+constexpr unsigned FUSE_KERNEL_BITS = 63u;      // the fuse bits the kernels see
 enum { SRC_ELEM = 0, SRC_BLOCK = 1, SRC_ARRAY = 2 };
+enum { CRIT_L2 = 0, CRIT_L1 = 1, CRIT_MAX = 2 };
 
 // One tensor of the list as the kernels see it.
 struct TensorDesc {
@@ -44,8 +47,12 @@ struct TensorDesc {
     int vec_ok;              // linear path may use 128-bit accesses
     int blk_vec_ok;          // block path may use 128-bit accesses
     int ranked;              // takes part in the ranking of the current call
-    int bh, bw;              // general block pruning: block height and width
+    int bh, bw;              // general block pruning of matrices: block height and width
+    int nd;                  // general n-D block pruning: dimensions cut (2: the fields above serve)
+    int sh[4], bs[4], nb[4]; // ... extents, block extents and blocks per dimension, right-aligned to four
+    int pad2;
 };
+static_assert(sizeof(TensorDesc) % 8 == 0, "descriptor tables are copied word by word");
 
 // Device-resident record of one ranking call.
 struct Result {
@@ -122,6 +129,7 @@ struct Params {
     u64 *fin_idx;                   // [FIN] list position of each entry of the final buffer
     const long long *tile_prefix;   // [T+1] warp tiles per tensor of the tiled block kernel
     long long n_tiles;
+    int crit;                       // structured pruning: value a structure is ranked by (CRIT_*)
     int miss_fallback;              // a missed sample bracket may be repaired by the two-pass route inside the
                                     // same call: nothing the first pass wrote is needed again (no multiplier
                                     // is updated in place)
@@ -185,6 +193,60 @@ __device__ __forceinline__ unsigned short f32_to_bf16_bits(float x)
 
 __device__ __forceinline__ float bf16_bits_to_f32(unsigned short h) { return __uint_as_float((u32)h << 16); }
 
+// Quantisation of theta named by the fuse bits: 0 none, 1 binary16, 2 bfloat16, 3 E4M3, 4 E5M2.
+__device__ __forceinline__ int quant_code(unsigned fuse)
+{
+    return (fuse & FUSE_E5M2) ? 4 : (fuse & FUSE_E4M3) ? 3 : (fuse & FUSE_BF16) ? 2 : (fuse & FUSE_FP16) ? 1 : 0;
+}
+
+// binary32 -> 8-bit floating point (fmt 0: E4M3, bias 7, no infinity, largest finite 448;
+// fmt 1: E5M2, bias 15, largest finite 57344), round to nearest even, saturating: what
+// rounds beyond the largest finite value, infinity included, becomes that value; NaN
+// becomes S.1111111. In the normal range the fraction is rounded by one integer addition
+// (a carry runs into the exponent, as it should) and the exponent rebiased; below the
+// smallest normal one IEEE addition of the power of two whose unit in the last place is
+// the smallest subnormal does the rounding, and the low bits of the sum are the code.
+__device__ __forceinline__ unsigned short f32_to_fp8_bits(float x, int fmt)
+{
+    const u32 b = __float_as_uint(x), a = b & 0x7FFFFFFFu, sign = (b >> 24) & 0x80u;
+    if (a > 0x7F800000u) return (unsigned short)(sign | 0x7Fu);
+    const int drop = fmt ? 21 : 20;                               // fraction bits that go
+    const u32 maxcode = fmt ? 0x7Bu : 0x7Eu;
+    const u32 min_normal = fmt ? 0x38800000u : 0x3C800000u;       // 2^-14, 2^-6
+    u32 q;
+    if (a >= min_normal) {
+        const u32 r = a + ((1u << (drop - 1)) - 1u) + ((a >> drop) & 1u);
+        q = (r - ((fmt ? 112u : 120u) << 23)) >> drop;
+        if (q > maxcode) q = maxcode;
+    } else {
+        const float magic = fmt ? 128.0f : 16384.0f;              // 2^7, 2^14: ulp 2^-16, 2^-9
+        q = __float_as_uint(__fadd_rn(__uint_as_float(a), magic)) - __float_as_uint(magic);
+    }
+    return (unsigned short)(sign | q);
+}
+
+// 8-bit floating point -> binary32, exact: the code's bits, moved to the place of a binary32
+// exponent and fraction, times the power of two between the two exponent biases (this also
+// turns the format's subnormals into the right values).
+__device__ __forceinline__ float fp8_bits_to_f32(unsigned short h, int fmt)
+{
+    const u32 mag = (u32)h & 0x7Fu, sign = ((u32)h & 0x80u) << 24;
+    if (fmt == 0 && mag == 0x7Fu) return __uint_as_float(sign | 0x7FC00000u);
+    if (fmt == 1 && mag >= 0x7Cu) return __uint_as_float(sign | 0x7F800000u | (mag > 0x7Cu ? 0x400000u : 0u));
+    const float f = __fmul_rn(__uint_as_float(mag << (fmt ? 21 : 20)), fmt ? 5.192296858534828e33f : 1.329227995784916e36f);   // 2^112, 2^120
+    return __uint_as_float(__float_as_uint(f) | sign);
+}
+
+// Code and widened value for quantisation q (1..4) of x.
+__device__ __forceinline__ unsigned short quant_bits(float x, int q)
+{
+    return q == 1 ? f32_to_f16_bits(x) : q == 2 ? f32_to_bf16_bits(x) : f32_to_fp8_bits(x, q - 3);
+}
+__device__ __forceinline__ float quant_widen(unsigned short h, int q)
+{
+    return q == 1 ? f16_bits_to_f32(h) : q == 2 ? bf16_bits_to_f32(h) : fp8_bits_to_f32(h, q - 3);
+}
+
 struct Out {
     float theta, lam, grad;
     unsigned short th;
@@ -196,9 +258,9 @@ __device__ __forceinline__ Out finish(float w, float lam, float u, bool keep, fl
                                       unsigned fuse, bool has_lam)
 {
     Out o;
-    const bool bf = (fuse & FUSE_BF16) != 0;
-    unsigned short hb = keep ? (bf ? f32_to_bf16_bits(u) : f32_to_f16_bits(u)) : (unsigned short)0;
-    float th = keep ? (bf ? bf16_bits_to_f32(hb) : (fuse & FUSE_FP16) ? f16_bits_to_f32(hb) : u) : 0.0f;
+    const int q = quant_code(fuse);
+    unsigned short hb = keep ? quant_bits(u, q ? q : 1) : (unsigned short)0;
+    float th = keep ? (q ? quant_widen(hb, q) : u) : 0.0f;
     float d = __fsub_rn(w, th);
     float p = __fmul_rn(mu, d);
     float lu = has_lam ? lam : 0.0f;
@@ -222,10 +284,9 @@ __device__ __forceinline__ Out finish_lean(float w, float lam, float u, bool kee
     float th = keep ? u : 0.0f;
     o.th = 0;
     if (H) {
-        const unsigned short hb = keep ? (q == 2 ? f32_to_bf16_bits(u) : f32_to_f16_bits(u)) : (unsigned short)0;
+        const unsigned short hb = keep ? quant_bits(u, q ? q : 1) : (unsigned short)0;
         o.th = hb;
-        if (q == 1) th = keep ? f16_bits_to_f32(hb) : 0.0f;
-        if (q == 2) th = keep ? bf16_bits_to_f32(hb) : 0.0f;
+        if (q) th = keep ? quant_widen(hb, q) : 0.0f;
     }
     const float p = __fmul_rn(mu, __fsub_rn(w, th));
     const float lu = upd ? __fsub_rn(lam, p) : lam;
@@ -254,9 +315,9 @@ __device__ __forceinline__ void form_u4(const float *w, const float *l, float mu
 // NaN (whose sign must be kept) is patched on a side path.
 __device__ __forceinline__ void half4(const float *x, unsigned short *h, int q = 1)
 {
-    if (q == 2) {        // bfloat16: integer rounding, NaN included
+    if (q >= 2) {        // bfloat16 and the 8-bit formats: integer rounding, NaN included
 #pragma unroll
-        for (int j = 0; j < 4; ++j) h[j] = f32_to_bf16_bits(x[j]);
+        for (int j = 0; j < 4; ++j) h[j] = quant_bits(x[j], q);
         return;
     }
 #pragma unroll
@@ -270,9 +331,9 @@ __device__ __forceinline__ void half4(const float *x, unsigned short *h, int q =
 
 __device__ __forceinline__ void widen4(const unsigned short *h, const float *x, float *o, int q = 1)
 {
-    if (q == 2) {
+    if (q >= 2) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) o[j] = bf16_bits_to_f32(h[j]);
+        for (int j = 0; j < 4; ++j) o[j] = quant_widen(h[j], q);
         return;
     }
 #pragma unroll
@@ -308,6 +369,22 @@ __device__ __forceinline__ Out finish_given(float w, float lam, float th, float 
     o.lam = lu;
     o.grad = __fsub_rn(p, lu);
     return o;
+}
+
+// One element's contribution to the value a structure is ranked by, and the combination of
+// two partial values (sums for the norms, the larger one for the maximum; a NaN stays).
+__device__ __forceinline__ double crit_add(double acc, float u, int crit)
+{
+    const double x = (double)u;
+    if (crit == CRIT_L2) return __fma_rn(x, x, acc);         // x*x is exact in fp64: (acc + x*x) rounded once
+    const double a = fabs(x);
+    if (crit == CRIT_L1) return __dadd_rn(acc, a);
+    return (a > acc || a != a) ? a : acc;
+}
+__device__ __forceinline__ double crit_join(double a, double b, int crit)
+{
+    if (crit != CRIT_MAX) return __dadd_rn(a, b);
+    return (b > a || b != b) ? b : a;
 }
 
 __device__ __forceinline__ u64 key_of_u(float u) { return (u64)(__float_as_uint(u) & 0x7FFFFFFFu); }

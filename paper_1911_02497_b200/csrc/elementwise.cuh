@@ -9,19 +9,26 @@ namespace cs {
 
 enum { M_KEEPALL = 0, M_PRUNE = 1, M_FILTER = 2, M_LAGRANGE = 3, M_BLOCKGEN = 4 };
 
-// Structure id of element e of a 2-D tensor cut into bh x bw blocks (row-major block numbering).
+// Structure id of element e of a tensor cut into n-D blocks (row-major block numbering).
 __device__ __forceinline__ u64 blockgen_sid(const TensorDesc &d, long long e)
 {
-    long long r, c;
-    if (d.numel < 0x7FFFFFFFll) {
-        const u32 rr = (u32)e / (u32)d.d1;
-        r = rr;
-        c = (u32)e - rr * (u32)d.d1;
-        return (u64)d.unit_prefix + (u64)((u32)r / (u32)d.bh) * (u64)d.nbc + (u32)c / (u32)d.bw;
+    if (d.nd == 2) {
+        long long r, c;
+        if (d.numel < 0x7FFFFFFFll) {
+            const u32 rr = (u32)e / (u32)d.d1;
+            r = rr;
+            c = (u32)e - rr * (u32)d.d1;
+            return (u64)d.unit_prefix + (u64)((u32)r / (u32)d.bh) * (u64)d.nbc + (u32)c / (u32)d.bw;
+        }
+        r = e / d.d1;
+        c = e - r * d.d1;
+        return (u64)d.unit_prefix + (u64)(r / d.bh) * (u64)d.nbc + (u64)(c / d.bw);
     }
-    r = e / d.d1;
-    c = e - r * d.d1;
-    return (u64)d.unit_prefix + (u64)(r / d.bh) * (u64)d.nbc + (u64)(c / d.bw);
+    long long rest = e;
+    int bc[4];
+#pragma unroll
+    for (int q = 3; q >= 0; --q) { bc[q] = (int)(rest % d.sh[q]) / d.bs[q]; rest /= d.sh[q]; }
+    return (u64)d.unit_prefix + (u64)((((long long)bc[0] * d.nb[1] + bc[1]) * d.nb[2] + bc[2]) * d.nb[3] + bc[3]);
 }
 
 constexpr int LIN_UNROLL = GROUPS_PER_ITEM / THREADS;   // 4 groups per thread per item
@@ -177,7 +184,7 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
     const bool has_lam = d.lam != nullptr;
     const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
     const bool wr_grad = (P.fuse & FUSE_PENALTY) && d.grad != nullptr;
-    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
+    const int fp16 = quant_code(P.fuse);     // quantisation of theta
     const float mu = P.mu;
     const u32 tau32 = tau_key > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)tau_key;     // KEY_NONE keeps nothing
     const float4 *wp = reinterpret_cast<const float4 *>(d.w + e_base) + threadIdx.x;
@@ -234,7 +241,7 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
                 }
             }
             else if (MODE == M_BLOCKGEN) {
-                if (d.ranked && d.numel < 0x7FFFFFFFll) {
+                if (d.ranked && d.nd == 2 && d.numel < 0x7FFFFFFFll) {
                     // row, column and block coordinates once per group, then walked element by element
                     const u32 C = (u32)d.d1, bh = (u32)d.bh, bw = (u32)d.bw;
                     const u32 e0 = (u32)(e_base + eo);

@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
     for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
     if (threadIdx.x < WARPS) sh.wcount[threadIdx.x] = 0;
     __syncthreads();
-    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
+    const int fp16 = quant_code(P.fuse);     // quantisation of theta
     const u32 lo = (u32)br.lo, range = (u32)br.hi - (u32)br.lo, guess = (u32)br.guess;
     const float mu = P.mu;
     const int warp = threadIdx.x >> 5;
@@ -421,7 +421,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
     __syncthreads();
     const long long *tile_prefix = cached ? sh.tile_prefix : P.tile_prefix;
     const TensorDesc *td = cached ? sh.td : P.td;
-    const int fp16 = (P.fuse & FUSE_BF16) ? 2 : (P.fuse & FUSE_FP16) ? 1 : 0;     // quantisation of theta
+    const int fp16 = quant_code(P.fuse);     // quantisation of theta
     const float mu = P.mu;
     volatile int *abort_flag = &sh.abort;
     u64 na = 0;

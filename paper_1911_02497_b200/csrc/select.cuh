@@ -661,7 +661,10 @@ __device__ __forceinline__ void write_result(const Params &P, const Sel &s)
         r.n_gt = (long long)s.n_gt;
         r.n_tie = (long long)s.n_tie;
         r.n_tie_kept = (long long)(s.k - s.n_gt);
-        if (P.bits_key >= 63) r.tau_norm = (float)sqrt(__longlong_as_double((long long)s.lo_key));
+        if (P.bits_key >= 63) {     // structures: the norm for the L2 criterion, else the ranked value itself
+            const double v = __longlong_as_double((long long)s.lo_key);
+            r.tau_norm = P.crit == CRIT_L2 ? (float)sqrt(v) : (float)v;
+        }
     }
     r.n_repaired = 0;      // filled in by the host from the counter once the stream is idle
     r.seed = P.seed;

@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(SMALL_THREADS) k_select_small(Params P, Sel in
             const int nseg = sh.t_nseg[lo];
             const double *p = P.partial + sh.t_items[lo] + ((long long)i - sh.t_units[lo]) * nseg;
             double acc = 0.0;
-            for (int sgm = 0; sgm < nseg; ++sgm) acc = __dadd_rn(acc, p[sgm]);      // segment order, as k_filter_combine
+            for (int sgm = 0; sgm < nseg; ++sgm) acc = crit_join(acc, p[sgm], P.crit);      // segment order, as k_filter_combine
             const u64 key = (u64)__double_as_longlong(acc);
             P.arr_key[i] = key;
             skey[i] = key;

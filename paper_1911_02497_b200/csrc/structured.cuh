@@ -114,6 +114,7 @@ __device__ __noinline__ void apply_after_select(const Params &P, int need_h)
 __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int crit = P.crit;
     const long long n_work = P.n_items;
     for (long long base = (long long)blockIdx.x * WARPS; base < n_work; base += (long long)gridDim.x * WARPS) {
         const long long item = base + warp;
@@ -147,8 +148,7 @@ __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
                     const float l4[4] = {lv[q].x, lv[q].y, lv[q].z, lv[q].w};
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const double x = (double)form_u(w4[c], l4[c], P.mu, has_lam);
-                        acc = __fma_rn(x, x, acc);
+                        acc = crit_add(acc, form_u(w4[c], l4[c], P.mu, has_lam), crit);
                     }
                 }
             }
@@ -159,8 +159,7 @@ __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
                 const float l4[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const double x = (double)form_u(w4[c], l4[c], P.mu, has_lam);
-                    acc = __fma_rn(x, x, acc);
+                    acc = crit_add(acc, form_u(w4[c], l4[c], P.mu, has_lam), crit);
                 }
             }
         } else {
@@ -168,28 +167,27 @@ __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const int j = 4 * gidx + c;
-                    const double x = (double)form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam);
-                    acc = __fma_rn(x, x, acc);
+                    acc = crit_add(acc, form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam), crit);
                 }
             }
         }
         // the last, incomplete group belongs to the lane whose turn it is
         if ((n & 3) && lane == (ngroups & 31)) {
             for (int j = 4 * ngroups; j < n; ++j) {
-                const double x = (double)form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam);
-                acc = __fma_rn(x, x, acc);
+                acc = crit_add(acc, form_u(__ldg(wp + j), has_lam ? lp[j] : 0.0f, P.mu, has_lam), crit);
             }
         }
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        for (int o = 16; o > 0; o >>= 1) acc = crit_join(acc, __shfl_xor_sync(0xffffffffu, acc, o), crit);
         if (lane == 0) P.partial[item] = acc;
     }
 }
 
-// General bh x bw blocks: one thread per block adds the squares of the elements
-// that exist, row by row, in fp64 (the same order as the plain definition).
-// Work items: BLOCKS_PER_ITEM blocks of a ranked tensor.
+// General n-D blocks: one thread per block goes over the elements of the block that exist, in
+// row-major order (the order of the plain definition, so the fp64 value is bit-identical),
+// with the criterion of the call. Work items: BLOCKS_PER_ITEM blocks of a ranked tensor.
 __global__ void __launch_bounds__(THREADS) k_blockgen_norms(Params P)
 {
+    const int crit = P.crit;
     for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
         const int t = find_tensor(P.item_prefix, P.T, item);
         const TensorDesc d = P.td[t];
@@ -198,16 +196,26 @@ __global__ void __launch_bounds__(THREADS) k_blockgen_norms(Params P)
         for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it) {
             const long long b = local * BLOCKS_PER_ITEM + it * THREADS + threadIdx.x;
             if (b >= d.n_units) continue;
-            const long long br = b / d.nbc, bc = b - br * d.nbc;
-            const long long r1 = (br + 1) * d.bh < d.d0 ? (br + 1) * d.bh : d.d0;
-            const long long c1 = (bc + 1) * d.bw < d.d1 ? (bc + 1) * d.bw : d.d1;
+            long long rest = b;
+            int bc[4];
+#pragma unroll
+            for (int q = 3; q >= 0; --q) { bc[q] = (int)(rest % d.nb[q]); rest /= d.nb[q]; }
+            int lo[4], hi[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                lo[q] = bc[q] * d.bs[q];
+                hi[q] = lo[q] + d.bs[q] < d.sh[q] ? lo[q] + d.bs[q] : d.sh[q];
+            }
             double acc = 0.0;
-            for (long long r = br * d.bh; r < r1; ++r)
-                for (long long c = bc * d.bw; c < c1; ++c) {
-                    const long long e = r * d.d1 + c;
-                    const double x = (double)form_u(d.w[e], has_lam ? d.lam[e] : 0.0f, P.mu, has_lam);
-                    acc = __fma_rn(x, x, acc);
-                }
+            for (int i0 = lo[0]; i0 < hi[0]; ++i0)
+                for (int i1 = lo[1]; i1 < hi[1]; ++i1)
+                    for (int i2 = lo[2]; i2 < hi[2]; ++i2) {
+                        const long long row = (((long long)i0 * d.sh[1] + i1) * d.sh[2] + i2) * d.sh[3];
+                        for (int i3 = lo[3]; i3 < hi[3]; ++i3) {
+                            const long long e = row + i3;
+                            acc = crit_add(acc, form_u(d.w[e], has_lam ? d.lam[e] : 0.0f, P.mu, has_lam), crit);
+                        }
+                    }
             P.arr_key[d.unit_prefix + b] = (u64)__double_as_longlong(acc);
         }
     }
@@ -230,7 +238,7 @@ __device__ __forceinline__ u64 filter_norm_key(const Params &P, long long sid)
     const long long nseg = (d.d1 + SEG - 1) / SEG;
     const double *p = P.partial + P.item_prefix[t] + f * nseg;
     double acc = 0.0;
-    for (long long sgm = 0; sgm < nseg; ++sgm) acc = __dadd_rn(acc, p[sgm]);
+    for (long long sgm = 0; sgm < nseg; ++sgm) acc = crit_join(acc, p[sgm], P.crit);
     return (u64)__double_as_longlong(acc);
 }
 

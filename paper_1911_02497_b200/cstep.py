@@ -16,8 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libcondensa_cstep.so")
 
 FUSE_FP16, FUSE_LAMBDA, FUSE_PENALTY, NO_SAMPLING = 1, 2, 4, 64
 OP_PRUNE, OP_FILTER, OP_BLOCK, OP_QUANTIZE, OP_LAGRANGE = 0, 1, 2, 3, 4
-DTYPE_FP16, DTYPE_BF16 = 1, 2
-FUSE_BF16 = 8
+DTYPE_FP16, DTYPE_BF16, DTYPE_FP8_E4M3, DTYPE_FP8_E5M2 = 1, 2, 3, 4
+FUSE_BF16, FUSE_E4M3, FUSE_E5M2 = 8, 16, 32
 STRUCT_FILTER, STRUCT_NEURON = 1, 2
 OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_UNSUPPORTED, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
 ERR_TOO_LARGE = -6
@@ -29,7 +29,8 @@ EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "conde
            "condensa_last_error", "condensa_profile_enable", "condensa_profile_read",
            "condensa_cstep_prune_noalloc", "condensa_lstep_update",
            "condensa_cstep_structure", "condensa_thin_flags", "condensa_thin_compact",
-           "condensa_count_nonzero", "condensa_set_seed", "condensa_noalloc_status"]
+           "condensa_count_nonzero", "condensa_set_seed", "condensa_noalloc_status",
+           "condensa_cstep_structured", "condensa_workspace_bytes"]
 
 
 class CondensaError(RuntimeError):
@@ -55,6 +56,16 @@ class Result(C.Structure):
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class StructureSpec(C.Structure):
+    """Mirror of ``condensa_structure_spec``."""
+    _fields_ = [("kind", C.c_int32), ("kinds", C.c_int32), ("criterion", C.c_int32), ("ndim", C.c_int32),
+                ("block", C.c_int64 * 4)]
+
+
+SPEC_SLICES, SPEC_BLOCKS = 0, 1
+CRITERIA = {"l2": 0, "l1": 1, "max": 2}
 
 
 class OptTensor(C.Structure):
@@ -97,6 +108,7 @@ def load():
     L.condensa_cstep_block.argtypes = [vp, vp, i32, f64, f32, i32, i32, u32, vp]
     L.condensa_cstep_structure.argtypes = [vp, vp, i32, f64, f32, i32, u32, vp]
     L.condensa_cstep_quantize.argtypes = [vp, vp, i32, f32, i32, u32, vp]
+    L.condensa_cstep_structured.argtypes = [vp, vp, i32, f64, f32, C.POINTER(StructureSpec), u32, vp]
     L.condensa_cstep_lagrange_update.argtypes = [vp, vp, i32, f32, u32, vp]
     L.condensa_cstep_host.argtypes = [vp, i32, vp, i32, f64, f32, i32, i32, u32, vp]
     L.condensa_get_result.argtypes = [vp, C.POINTER(Result)]
@@ -104,6 +116,7 @@ def load():
     L.condensa_profile_read.argtypes = [vp, C.POINTER(KernelTime), i32, C.POINTER(i32)]
     L.condensa_cstep_prune_noalloc.argtypes = [vp, f64, f32, u32, vp]
     L.condensa_noalloc_status.argtypes = []
+    L.condensa_workspace_bytes.argtypes = [i32, vp, i32, C.POINTER(StructureSpec), u32, C.POINTER(C.c_size_t)]
     L.condensa_set_seed.argtypes = [vp, C.c_uint64]
     L.condensa_lstep_update.argtypes = [vp, vp, i32, f32, C.POINTER(Opt), vp]
     i64 = C.c_int64
@@ -124,7 +137,7 @@ def fuse_bits(fuse) -> int:
     if isinstance(fuse, int):
         return fuse
     table = {"fp16": FUSE_FP16, "lambda": FUSE_LAMBDA, "penalty": FUSE_PENALTY, "bf16": FUSE_BF16,
-             "no_sampling": NO_SAMPLING}
+             "e4m3": FUSE_E4M3, "e5m2": FUSE_E5M2, "no_sampling": NO_SAMPLING}
     b = 0
     for f in fuse:
         b |= table[f]
@@ -203,6 +216,17 @@ def cstep_prune_noalloc(tab, sparsity, mu, fuse=(), stream=None):
         raise CondensaError(rc, (L.condensa_last_error(None) or b"").decode())
 
 
+def workspace_bytes(op: int, tab, T: int, fuse=(), spec=None) -> int:
+    """``condensa_workspace_bytes``: what ``Context(device, workspace_bytes)`` must reserve so that
+    calls of this shape never allocate."""
+    L = load()
+    n = C.c_size_t(0)
+    rc = L.condensa_workspace_bytes(int(op), tab, int(T), spec, fuse_bits(fuse), C.byref(n))
+    if rc != OK:
+        raise CondensaError(rc, (L.condensa_last_error(None) or b"").decode())
+    return int(n.value)
+
+
 def noalloc_status():
     """``condensa_noalloc_status``: waits for the last allocation-free call on the current
     device and raises if one of its device-side checks failed."""
@@ -253,6 +277,19 @@ class Context:
         mask = sum({"filter": STRUCT_FILTER, "neuron": STRUCT_NEURON}[k] for k in set(kinds))
         self._check(self._lib.condensa_cstep_structure(self._h, tab, T, float(sparsity), float(mu), mask,
                                                        fuse_bits(fuse), _stream_handle(stream)))
+
+    def cstep_structured(self, tab, T, sparsity, mu, kind="filter", block=None, criterion="l2", fuse=(), stream=None):
+        """``kind``: 'filter', 'neuron', 'structure' (both) or 'block' with ``block`` = the extents."""
+        sp = StructureSpec()
+        sp.criterion = CRITERIA[criterion]
+        if kind == "block":
+            sp.kind, sp.ndim = SPEC_BLOCKS, len(block)
+            for d, b in enumerate(block):
+                sp.block[d] = int(b)
+        else:
+            sp.kind, sp.kinds = SPEC_SLICES, {"filter": 1, "neuron": 2, "structure": 3}[kind]
+        self._check(self._lib.condensa_cstep_structured(self._h, tab, T, float(sparsity), float(mu), C.byref(sp),
+                                                        fuse_bits(fuse), _stream_handle(stream)))
 
     def cstep_block(self, tab, T, sparsity, mu, bh=4, bw=4, fuse=(), stream=None):
         self._check(self._lib.condensa_cstep_block(self._h, tab, T, float(sparsity), float(mu),

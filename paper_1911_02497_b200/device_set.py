@@ -31,8 +31,13 @@ class DeviceSet:
         self._base = []            # keeps the padded allocations alive
 
         def alloc(n, dtype, shift):
+            # guard bands: `shift` elements before and 64 behind the data carry a canary that
+            # fetch() checks - a kernel that writes outside its tensor is caught here
             buf = torch.zeros(n + shift + 64, dtype=dtype, device=self.device)
-            self._base.append(buf)
+            canary = self._canary(dtype)
+            buf[:shift] = canary
+            buf[shift + n:] = canary
+            self._base.append((buf, shift, n, canary))
             return buf[shift:shift + n]
 
         def put(a, shift):
@@ -55,6 +60,17 @@ class DeviceSet:
         lam_ptrs = [None if l is None else l for l in self.lam]
         self.table = cstep.tensor_table(self.w, lam_ptrs, self.theta, self.mask, self.grad,
                                         self.theta_h, shapes=self.shapes)
+
+    @staticmethod
+    def _canary(dtype):
+        return {torch.float32: -12345.678, torch.uint8: 0xA5, torch.int16: 0x5A5A}[dtype]
+
+    def check_guard_bands(self):
+        """Raises if anything has been written next to a buffer."""
+        for i, (buf, shift, n, canary) in enumerate(self._base):
+            want = torch.tensor(canary, dtype=buf.dtype, device=buf.device)
+            if not (bool((buf[:shift] == want).all()) and bool((buf[shift + n:] == want).all())):
+                raise AssertionError("guard band of buffer %d (%s, %d elements) was overwritten" % (i, buf.dtype, n))
 
     # -- state ---------------------------------------------------------------
     def reset_lambda(self):
@@ -87,8 +103,9 @@ class DeviceSet:
             ctx.cstep_structure(self.table, self.T, sparsity, mu, kinds, fuse, stream)
         elif op == "block":
             ctx.cstep_block(self.table, self.T, sparsity, mu, block[0], block[1], fuse, stream)
-        elif op in ("quantize", "quantize_bf16"):
-            dt = cstep.DTYPE_BF16 if op == "quantize_bf16" else cstep.DTYPE_FP16
+        elif op.startswith("quantize"):
+            dt = {"quantize": cstep.DTYPE_FP16, "quantize_bf16": cstep.DTYPE_BF16,
+                  "quantize_e4m3": cstep.DTYPE_FP8_E4M3, "quantize_e5m2": cstep.DTYPE_FP8_E5M2}[op]
             ctx.cstep_quantize(self.table, self.T, mu, dt, fuse, stream)
         elif op == "lagrange":
             ctx.cstep_lagrange_update(self.table, self.T, mu, fuse, stream)
@@ -104,6 +121,7 @@ class DeviceSet:
 
     def fetch(self):
         torch.cuda.synchronize(self.device)
+        self.check_guard_bands()
         return {"theta": self._get(self.theta, np.float32), "mask": self._get(self.mask, np.uint8),
                 "lam": self._get(self.lam, np.float32), "grad": self._get(self.grad, np.float32),
                 "theta_h": self._get(self.theta_h, np.uint16)}

@@ -75,8 +75,8 @@ def run_oracle(op, w, lam, s, mu, fuse, block=(4, 4), theta=None):
         return oracle.cstep_block(w, lam, s, mu, block, fuse)
     if op == "quantize":
         return oracle.cstep_quantize(w, lam, mu, fuse)
-    if op == "quantize_bf16":
-        return oracle.cstep_quantize(w, lam, mu, tuple(fuse) + ("bf16",))
+    if op.startswith("quantize_"):
+        return oracle.cstep_quantize(w, lam, mu, tuple(fuse) + (op.split("_")[1],))
     return oracle.lagrange_update(w, theta, lam, mu, fuse)
 
 
@@ -158,10 +158,10 @@ def test_bf16_quantize_and_fused_paths(ctx):
         ds.run(ctx, "prune", 0.5, 1e-3, ("fp16", "bf16"))
 
 
-@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("dtype", ["fp16", "bf16", "e4m3", "e5m2"])
 def test_quantize_every_fp32_bit_pattern(ctx, dtype):
     """All 2^32 binary32 patterns through the quantise entry point against the oracle's
-    explicit-bit conversion (16-bit code and the widened theta)."""
+    explicit-bit conversion (the code and the widened theta)."""
     import torch
     from paper_1911_02497_b200 import cstep
     chunk = 1 << 27
@@ -171,22 +171,47 @@ def test_quantize_every_fp32_bit_pattern(ctx, dtype):
     th = torch.empty(chunk, dtype=torch.int16, device=dev)
     base = torch.arange(chunk, dtype=torch.int64, device=dev)
     tab = cstep.tensor_table([w], None, [theta], None, None, [th], shapes=[(chunk,)])
+    code = {"fp16": cstep.DTYPE_FP16, "bf16": cstep.DTYPE_BF16, "e4m3": cstep.DTYPE_FP8_E4M3,
+            "e5m2": cstep.DTYPE_FP8_E5M2}[dtype]
+    tdt = {"fp16": torch.float16, "bf16": torch.bfloat16, "e4m3": torch.float8_e4m3fn, "e5m2": torch.float8_e5m2}[dtype]
+    eight = dtype in ("e4m3", "e5m2")
     for c in range((1 << 32) // chunk):
         first = c * chunk
         w.copy_(((base + first) & 0xFFFFFFFF).to(torch.int64).sub_((base + first >= (1 << 31)).to(torch.int64) << 32).to(torch.int32))
-        ctx.cstep_quantize(tab, 1, 1.0, dtype=cstep.DTYPE_FP16 if dtype == "fp16" else cstep.DTYPE_BF16)
+        ctx.cstep_quantize(tab, 1, 1.0, dtype=code)
         got_h = th.cpu().numpy().view(np.uint16)
-        exp_h = (oracle.f32_to_f16_range if dtype == "fp16" else oracle.f32_to_bf16_range)(first, chunk)
+        if eight:
+            exp8 = oracle.f32_to_fp8_range(first, chunk, dtype)
+            exp_h = exp8.astype(np.uint16)
+        else:
+            exp_h = (oracle.f32_to_f16_range if dtype == "fp16" else oracle.f32_to_bf16_range)(first, chunk)
         assert np.array_equal(got_h, exp_h), "chunk %d" % c
-        # theta is the exact widening of those 16 bits (NaN: quiet, sign kept)
-        wide = torch.from_numpy(exp_h.view(np.int16)).to(dev).view(
-            torch.float16 if dtype == "fp16" else torch.bfloat16).to(torch.float32)
+        # theta is the exact widening of that code (NaN: quiet, sign kept); torch's widening is exact
+        src = torch.from_numpy(exp8.copy()).to(dev) if eight else torch.from_numpy(exp_h.view(np.int16)).to(dev)
+        wide = src.view(tdt).to(torch.float32)
         tb, wb = theta.view(torch.int32), wide.view(torch.int32)
         nan = torch.isnan(wide)
         assert bool(torch.equal(tb[~nan], wb[~nan]))
-        neg = torch.from_numpy((exp_h >> 15).astype(np.bool_)).to(dev)
+        neg = torch.from_numpy((exp_h >> (7 if eight else 15)).astype(np.bool_)).to(dev)
         assert bool(torch.isnan(theta[nan]).all()) and bool(torch.equal(tb[nan] < 0, neg[nan]))    # sign kept
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("q", ["e4m3", "e5m2"])
+def test_eight_bit_types_in_the_fused_paths(ctx, q):
+    """Compose([Prune, Quantize(8-bit)]) and the structured schemes with an 8-bit type: two-pass
+    sizes, single-pass sizes (elements and 4x4 blocks), filters, with multipliers and gradient."""
+    ws = W.random_set([(33, 17), (4099,), (5, 3, 3, 3)], seed=9, kind="normal", scale=2.0, lam_sigma=1e-2, mu=1e-2)
+    check(ctx, "quantize_" + q, ws.w, ws.lam, mu=ws.mu, fuse=("lambda", "penalty"), elem_offset=1)
+    check(ctx, "prune", ws.w, ws.lam, 0.7, ws.mu, (q, "lambda", "penalty"))
+    check(ctx, "filter", ws.w, ws.lam, 0.4, ws.mu, (q, "lambda"), exact_key=False)
+    check(ctx, "block", ws.w, ws.lam, 0.5, ws.mu, (q, "lambda"))
+    big = W.random_set([(300000,), (70001,)], seed=10, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
+    got, res, _ = check(ctx, "prune", big.w, big.lam, 0.9, big.mu, (q, "lambda", "penalty"))
+    assert res.sampled == 1
+    m = W.random_set([(1600, 1000), (602, 1000)], seed=11, kind="uniform", scale=0.1, lam_sigma=1e-3, mu=1e-2)
+    got, res, _ = check(ctx, "block", m.w, m.lam, 0.9, m.mu, (q, "lambda", "penalty"))
+    assert res.sampled == 1
 
 
 @pytest.mark.parametrize("fuse", [("lambda",), ("penalty",), ("lambda", "penalty")])
@@ -500,6 +525,83 @@ def test_single_pass_block_kernel_tiles_edges_and_many_tensors(ctx):
     ctx.set_seed(SEED)
 
 
+def check_structured(ctx, w, lam, s, mu, kind, block=None, criterion="l2", fuse=("lambda",), elem_offset=0,
+                     exact_key=True):
+    """The specification entry point against the oracle's: masks, theta, multipliers, gradient and
+    the record; the ranked value bit for bit where the summation order is the definition's."""
+    from paper_1911_02497_b200.device_set import DeviceSet
+    lam = lam if lam is not None else [None] * len(w)
+    ds = DeviceSet(w, lam, elem_offset=elem_offset)
+    ds.poison_outputs()
+    ctx.cstep_structured(ds.table, ds.T, s, mu, kind, block, criterion, fuse)
+    got, res = ds.fetch(), ctx.get_result()
+    exp = oracle.cstep_structured(w, lam, s, mu, kind, block, criterion, tuple(f for f in fuse if f != "no_sampling"))
+    for t in range(len(w)):
+        assert np.array_equal(got["mask"][t], exp.mask[t]), "mask, tensor %d" % t
+        assert same_f32(got["theta"][t], exp.theta[t]), "theta, tensor %d" % t
+        if lam[t] is not None:
+            assert same_f32(got["lam"][t], exp.lam[t]), "lambda, tensor %d" % t
+        if "penalty" in fuse:
+            assert same_f32(got["grad"][t], exp.grad[t]), "grad, tensor %d" % t
+    r = exp.result
+    assert res.status == 0 and (res.n_units, res.n_zero, res.n_keep, res.tau_id) == (r.n_units, r.n_zero, r.n_keep, r.tau_id)
+    assert (res.n_gt, res.n_tie, res.n_tie_kept) == (r.n_gt, r.n_tie, r.n_tie_kept)
+    if exact_key:
+        assert res.tau_key == r.tau_key
+    else:
+        a, b = (np.array([k], np.uint64).view(np.float64)[0] for k in (res.tau_key, r.tau_key))
+        assert a == b or abs(a - b) <= 1e-12 * abs(b)
+    if r.n_keep > 0:
+        assert abs(res.tau_norm - r.tau_norm) <= REL * abs(r.tau_norm)
+    return got, res, exp
+
+
+@pytest.mark.parametrize("crit", ["l2", "l1", "max"])
+def test_structure_criteria(ctx, crit):
+    """Filters, neurons, both, and 2-D blocks ranked by the L2, L1 or max criterion."""
+    ws = W.random_set([(300, 257), (7, 3, 3, 3), (64,), (40, 1024), (12, 20, 3, 3), (1, 9)], seed=45,
+                      kind="normal", scale=0.3, lam_sigma=1e-2, mu=1e-2)
+    for kind in ("filter", "neuron", "structure"):
+        for s in (0.0, 0.4, 1.0):
+            check_structured(ctx, ws.w, ws.lam, s, ws.mu, kind, None, crit, ("lambda", "penalty"), exact_key=(crit == "max"))
+    check_structured(ctx, ws.w, ws.lam, 0.7, ws.mu, "structure", None, crit, ("fp16", "lambda"), elem_offset=3,
+                     exact_key=(crit == "max"))
+    for block in ((5, 5), (4, 4), (1, 8)):
+        check_structured(ctx, ws.w, ws.lam, 0.6, ws.mu, "block", block, crit, ("lambda",))
+    # many equal values: ties settled by the structure index, in one CTA and grid-wide
+    rows = np.tile(np.array([[1.0, -2.0, 0.5, 2.0]], np.float32), (900, 1)) * np.repeat(
+        np.arange(1, 4, dtype=np.float32), 300)[:, None]
+    for extra in ((), ("no_sampling",)):
+        got, res, _ = check_structured(ctx, [rows], None, 0.5, 1.0, "neuron", None, crit, extra)
+        assert res.n_tie == 300
+    # the VGG-shaped set: the filter ranking with the other criteria
+    ws = W.config(3, scale=0.25)
+    check_structured(ctx, ws.w, ws.lam, 0.8, ws.mu, "filter", None, crit, ("lambda",), exact_key=(crit == "max"))
+
+
+@pytest.mark.parametrize("block", [(2, 2, 2), (1, 3, 2), (2, 1, 3, 3), (3, 2, 1, 2), (5,), (4, 4), (7, 3)])
+def test_nd_blocks(ctx, block):
+    """BlockPrune with n-D blocks: tensors of that rank are cut, the others pass through."""
+    nd = len(block)
+    shape = {1: (10007,), 2: (129, 70), 3: (33, 17, 9), 4: (20, 9, 5, 5)}[nd]
+    other = {1: (4, 4), 2: (6,), 3: (6, 5), 4: (7, 2, 2)}[nd]
+    ws = W.random_set([shape, other, shape, (5,) * nd], seed=50 + nd, kind="normal", scale=0.3, lam_sigma=1e-2, mu=1e-2)
+    for s in (0.0, 0.45, 0.9, 1.0):
+        check_structured(ctx, ws.w, ws.lam, s, ws.mu, "block", block, "l2", ("lambda", "penalty"))
+    check_structured(ctx, ws.w, ws.lam, 0.5, ws.mu, "block", block, "l1", ("bf16", "lambda"), elem_offset=1)
+    check_structured(ctx, ws.w, ws.lam, 0.5, ws.mu, "block", block, "max", ("lambda", "no_sampling"))
+
+
+def test_conv_weights_in_3d_blocks_at_size(ctx):
+    """3-D blocks over conv weights of a VGG-shaped set seen as [F, C, kh*kw] (more than 16384 blocks:
+    the grid-wide selection on the value array)."""
+    ws = W.config(3, scale=0.25)
+    w = [a.reshape(a.shape[0], a.shape[1], -1) if a.ndim == 4 else a for a in ws.w]
+    lam = [l.reshape(a.shape) for l, a in zip(ws.lam, w)]
+    got, res, _ = check_structured(ctx, w, lam, 0.7, ws.mu, "block", (2, 2, 9), "l2", ("lambda",))
+    assert res.n_units > 16384
+
+
 def test_block_size_five_on_the_lstm_shapes(ctx):
     ws = W.config("5", scale=0.1)
     got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.6, ws.mu, ("lambda",), block=(5, 5))
@@ -538,7 +640,7 @@ def test_argument_errors_leave_buffers_untouched(ctx):
     ds.poison_outputs()
     bad = [lambda: ds.run(ctx, "prune", 1.5, 1e-3), lambda: ds.run(ctx, "prune", float("nan"), 1e-3),
            lambda: ds.run(ctx, "prune", 0.5, 0.0), lambda: ds.run(ctx, "prune", 0.5, float("inf")),
-           lambda: ds.run(ctx, "prune", 0.5, -1.0), lambda: ds.run(ctx, "prune", 0.5, 1e-3, fuse=16),
+           lambda: ds.run(ctx, "prune", 0.5, -1.0), lambda: ds.run(ctx, "prune", 0.5, 1e-3, fuse=128), lambda: ds.run(ctx, "prune", 0.5, 1e-3, fuse=1 | 16),
            lambda: ds.run(ctx, "lagrange", 0.0, 1e-3, fuse=())]
     for f in bad:
         with pytest.raises(cstep.CondensaError) as e:
@@ -551,7 +653,7 @@ def test_argument_errors_leave_buffers_untouched(ctx):
         ds.run(ctx, "block", 0.5, 1e-3, block=(0, 4))
     assert e.value.code == cstep.ERR_INVALID_ARG
     with pytest.raises(cstep.CondensaError) as e:
-        ctx.cstep_quantize(ds.table, ds.T, 1e-3, dtype=3)
+        ctx.cstep_quantize(ds.table, ds.T, 1e-3, dtype=7)
     assert e.value.code == cstep.ERR_UNSUPPORTED
     # aliasing: theta on top of w; the same lambda twice
     tab = cstep.tensor_table(ds.w, ds.lam, ds.w, shapes=ds.shapes)
@@ -596,3 +698,27 @@ def test_deterministic_across_runs(ctx):
         for key in ("theta", "mask", "lam", "theta_h"):
             for a, b in zip(first[key], again[key]):
                 assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
+
+
+def test_workspace_query_sizes_a_context_that_never_allocates():
+    """condensa_workspace_bytes() tells how much condensa_create() must reserve: a context made
+    with that figure runs the call without touching the device allocator."""
+    import torch
+    from paper_1911_02497_b200 import cstep
+    from paper_1911_02497_b200.device_set import DeviceSet
+    ws = W.config("5", scale=0.2)
+    ds = DeviceSet(ws.w, ws.lam)
+    need = cstep.workspace_bytes(cstep.OP_BLOCK, ds.table, ds.T, ("lambda",))
+    assert need > 0
+    c = cstep.Context(0, need)
+    try:
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info(0)
+        ds.run(c, "block", ws.sparsity, ws.mu, ("lambda",))
+        assert c.get_result().sampled == 1
+        free1, _ = torch.cuda.mem_get_info(0)
+        assert free1 == free0
+    finally:
+        c.close()
+    with pytest.raises(cstep.CondensaError):
+        cstep.workspace_bytes(99, ds.table, ds.T)
