@@ -100,7 +100,7 @@ enum {
                                    positions (seed: condensa_set_seed), the pass decides everything
                                    outside the bracket for good and lists the rest, and the exact
                                    selection runs on that list. The bracket is checked exactly
-                                   afterwards. Should it miss (probability < 1e-18 for positions
+                                   afterwards. Should it miss (probability < 1e-16 for positions
                                    independent of the data), the call falls back to the two-pass
                                    route by itself and returns the exact result whenever the first
                                    pass has not destroyed an input, i.e. unless FUSE_LAMBDA is set
