@@ -388,7 +388,7 @@ def run_ours(args):
         kernels = {k: {"launches": n, "avg_us": 1e3 * ms / n} for k, (n, ms) in prof.items()}
         # the kernel that does the projection (reads w, lambda; writes theta, mask, lambda):
         # its algorithmic bytes are the step's
-        names = ("k_fused", "k_apply", "k_quantize", "k_lagrange", "k_select_all")   # k_select_all: the one-launch route
+        names = ("k_fused", "k_apply", "k_quantize", "k_lagrange", "k_select_all", "k_prune_small")   # the last two: one-launch routes
         movers = {k: v for k, v in prof.items() if k.startswith(names)
                   and v[1] / v[0] > 0.02}          # launches that return at once do not count
         if not movers:                             # small sets: every launch is short

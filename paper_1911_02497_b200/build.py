@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcondensa_cstep.so")
 SOURCES = ["api.cu"]
 HEADERS = ["common.cuh", "elementwise.cuh", "select.cuh", "structured.cuh", "fused.cuh", "fused_fast.cuh",
-           "sample.cuh", "lstep.cuh", "thin.cuh", "small_select.cuh",
+           "sample.cuh", "lstep.cuh", "thin.cuh", "small_select.cuh", "small_prune.cuh",
            os.path.join("..", "..", "include", "condensa_cstep.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",

@@ -24,6 +24,7 @@
 #include "lstep.cuh"
 #include "thin.cuh"
 #include "small_select.cuh"
+#include "small_prune.cuh"
 
 using namespace cs;
 
@@ -65,6 +66,7 @@ struct condensa_ctx {
     Ctl *ctl = nullptr;
     int occ_select[3] = {0, 0, 0};
     int occ_stream = 0;
+    int occ_prune_small = 0;        // resident CTAs per SM of the register-resident small-list kernel
     bool small_smem_set = false;    // dynamic shared memory limit of k_select_small raised on this device
     bool block_smem_set = false;    // the same for the tiled block kernel
     DeviceMirror mirror;
@@ -485,12 +487,15 @@ Sel initial_state(long long S, long long k, int bits_key)
 
 // Work decomposition and workspace layout of one call (no device work).
 Layout plan_call(int op, const condensa_tensor *ts, int T, unsigned fuse, const HostSpec &sp, Plan &pl,
-                 bool &ranking, bool &sampling)
+                 bool &ranking, bool &sampling, long long small_items_max = 0, bool *small_prune = nullptr)
 {
     build_plan(op, ts, T, pl, sp);
     ranking = op <= OP_BLOCK || op == OP_BLOCKGEN;
     // single-pass path: unstructured and block pruning of lists too large to list whole
-    sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) &&
+    // an unstructured list of at most one work item per resident CTA stays in registers for the whole call
+    const bool reg_resident = op == OP_PRUNE && pl.n_items_b > 0 && pl.n_items_b <= small_items_max;
+    if (small_prune) *small_prune = reg_resident;
+    sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) && !reg_resident &&
                           (u64)pl.S > pl.cap && pl.S >= 8ll * N_SAMPLE;
     if (sampling && op == OP_BLOCK && pl.cap > (1ull << 20)) pl.cap = 1ull << 20;   // bounds the journal
     const int journal_floats = sampling ? (op == OP_BLOCK ? 16 : 1) : 0;
@@ -524,8 +529,10 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
                     return fail(ctx, CONDENSA_ERR_UNSUPPORTED, "tensor %d: an extent above 2^31 - 1 cannot be cut into blocks", t);
     CU_TRY(ctx, cudaSetDevice(ctx->device));
     Plan pl;
-    bool ranking = false, sampling = false;
-    const Layout L = plan_call(op, ts, T, fuse, sp, pl, ranking, sampling);
+    bool ranking = false, sampling = false, small_prune = false;
+    if (op == OP_PRUNE && !ctx->occ_prune_small) ctx->occ_prune_small = occupancy(k_prune_small);
+    const long long small_items_max = (op == OP_PRUNE && ctx->occ_prune_small >= 2) ? 2ll * ctx->num_sms : 0;
+    const Layout L = plan_call(op, ts, T, fuse, sp, pl, ranking, sampling, small_items_max, &small_prune);
     rc = ensure_workspace(ctx, L.total, stream);
     if (rc) return rc;
     char *ws = ctx->ws;
@@ -584,6 +591,22 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     if (!ctx->occ_stream) ctx->occ_stream = 3;
 
     bool applied_in_select = false;
+    if (ranking && small_prune) {
+        const long long Z = (long long)std::min<double>((double)pl.S, std::max(0.0, std::floor(sparsity * (double)pl.S + 0.5)));
+        Sel init = initial_state(pl.S, pl.S - Z, P.bits_key);
+        Params Ps = P;
+        Ps.item_prefix = pb;
+        Ps.n_items = pl.n_items_b;
+        dim3 grid((unsigned)(2 * ctx->num_sms)), block(THREADS);
+        void *args[] = {(void *)&Ps, (void *)&init};
+        const int pa_ = prof_begin(ctx, "k_prune_small", stream);
+        CU_TRY(ctx, cudaLaunchCooperativeKernel((const void *)k_prune_small, grid, block, args, 0, stream));
+        ctx->launches += 1;
+        prof_end(ctx, pa_, stream);
+        ctx->has_result = true;
+        if (cudaEventRecord(ctx->tail_ev, stream) == cudaSuccess) ctx->tail_recorded = true;
+        return CONDENSA_OK;
+    }
     if (ranking) {
         const long long Z = (long long)std::min<double>((double)pl.S, std::max(0.0, std::floor(sparsity * (double)pl.S + 0.5)));
         const long long k = pl.S - Z;
@@ -1228,6 +1251,13 @@ int condensa_get_result(condensa_ctx *ctx, condensa_result *out)
         CU_TRY(ctx, cudaMemcpy(&rep, &ctx->ctl->n_repaired, sizeof(rep), cudaMemcpyDeviceToHost));
         out->n_repaired = (int64_t)rep;
     }
+    if (out->status == 0 && out->n_keep > 0) {
+        // the index of the weakest kept unit as the kernels left it in the control block (the
+        // register-resident route finds it by an atomic maximum when every tie is kept)
+        u64 tid = 0;
+        CU_TRY(ctx, cudaMemcpy(&tid, &ctx->ctl->tau_id, sizeof(tid), cudaMemcpyDeviceToHost));
+        out->tau_id = (int64_t)tid;
+    }
     if (out->status != 0) {
         int code = 0;
         cudaMemcpy(&code, &ctx->ctl->sel.error, sizeof(int), cudaMemcpyDeviceToHost);
@@ -1293,6 +1323,7 @@ constexpr int NOALLOC_MAX_DEVICES = 64;
 std::mutex g_noalloc_mutex;                          // guards the once-per-device set-up and the error text
 unsigned char *g_noalloc_ptr[NOALLOC_MAX_DEVICES];   // device address of the scratch, per device
 int g_noalloc_occ[NOALLOC_MAX_DEVICES];
+int g_noalloc_occ_small[NOALLOC_MAX_DEVICES];
 int g_noalloc_sms[NOALLOC_MAX_DEVICES];
 size_t g_noalloc_ctl_off[NOALLOC_MAX_DEVICES];       // where the last call on the device put its control block
 cudaStream_t g_noalloc_stream[NOALLOC_MAX_DEVICES];
@@ -1353,6 +1384,7 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
                                     e != cudaSuccess ? cudaGetErrorString(e) : "device lacks cooperative launch");
             }
             g_noalloc_occ[dev] = occupancy(k_select<SRC_ELEM>);
+            g_noalloc_occ_small[dev] = occupancy(k_prune_small);
             g_noalloc_sms[dev] = sms;
             g_noalloc_ptr[dev] = p;
         }
@@ -1390,7 +1422,15 @@ int condensa_cstep_prune_noalloc(const condensa_tensor *tensor, double sparsity,
 
     k_noalloc_setup<<<1, 32, 0, stream>>>(pl.td[0], pl.n_items_a, (TensorDesc *)(ws + L.desc), prefix);
     if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
-    {
+    if (pl.n_items_b > 0 && pl.n_items_b <= 2ll * sms && g_noalloc_occ_small[dev] >= 2) {
+        // at most one work item per resident CTA: the list stays in registers for the whole call
+        P.item_prefix = prefix + 2;
+        P.n_items = pl.n_items_b;
+        dim3 grid((unsigned)(2 * sms)), block(THREADS);
+        void *args[] = {(void *)&P, (void *)&init};
+        e = cudaLaunchCooperativeKernel((const void *)k_prune_small, grid, block, args, 0, stream);
+        if (e != cudaSuccess) return noalloc_fail(CONDENSA_ERR_CUDA, cudaGetErrorString(e));
+    } else {
         // one cooperative launch: clears what the last call left in the scratch, ranks, projects
         dim3 grid((unsigned)(sms * std::min(g_noalloc_occ[dev], 2))), block(THREADS);
         int pre_scan = 1, post_apply = 2, do_init = 1;

@@ -206,7 +206,7 @@ def test_eight_bit_types_in_the_fused_paths(ctx, q):
     check(ctx, "prune", ws.w, ws.lam, 0.7, ws.mu, (q, "lambda", "penalty"))
     check(ctx, "filter", ws.w, ws.lam, 0.4, ws.mu, (q, "lambda"), exact_key=False)
     check(ctx, "block", ws.w, ws.lam, 0.5, ws.mu, (q, "lambda"))
-    big = W.random_set([(300000,), (70001,)], seed=10, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
+    big = W.random_set([(1300000,), (270001,)], seed=10, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
     got, res, _ = check(ctx, "prune", big.w, big.lam, 0.9, big.mu, (q, "lambda", "penalty"))
     assert res.sampled == 1
     m = W.random_set([(1600, 1000), (602, 1000)], seed=11, kind="uniform", scale=0.1, lam_sigma=1e-3, mu=1e-2)
@@ -324,15 +324,15 @@ def test_two_pass_path_without_sampling(ctx, cfg, scale):
 
 
 def test_single_pass_path_is_taken_and_repairs(ctx):
-    ws = W.config(1)
-    got, res, _ = check(ctx, "prune", ws.w, ws.lam, ws.sparsity, ws.mu, ws.fuse)
+    ws = W.random_set([(1 << 21,)], seed=0, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)     # too long for the registers
+    got, res, _ = check(ctx, "prune", ws.w, ws.lam, 0.9, ws.mu, ("fp16", "lambda"))
     assert res.sampled == 1 and 0 < res.n_candidates < ws.numel // 8
     ws = W.config("5", scale=0.2)
     got, res, _ = check(ctx, "block", ws.w, ws.lam, ws.sparsity, ws.mu, ("fp16", "lambda", "penalty"))
     assert res.sampled == 1 and 0 < res.n_candidates < res.n_units // 8
 
 
-def _adversarial_for_seed(seed, n=1 << 20, m=16384):
+def _adversarial_for_seed(seed, n=3 << 19, m=16384):
     """An input built against the sample positions of `seed`: tiny values exactly there, so that
     the bracket taken from the sample cannot hold the threshold of the whole tensor."""
     w = W.draw(n, "normal", 1.0, 77, 0, 0)
@@ -380,7 +380,7 @@ def test_more_candidates_than_the_list_holds_falls_back(ctx):
     """A tie group that the sample cannot see but that overflows the candidate list: the values at
     the sampled positions are spread out, everything else within the bracket is one value."""
     seed = 0x1234ABCD
-    n, m = 1 << 20, 16384
+    n, m = 3 << 19, 16384
     w = np.full(n, 0.5, np.float32)
     w[::20] = 2.0                                    # 5 % clearly above the cut of s = 0.9
     pos = np.array([(W._mix64_scalar(W._mix64_scalar(seed) ^ j) * n) >> 64 for j in range(m)])
@@ -389,7 +389,7 @@ def test_more_candidates_than_the_list_holds_falls_back(ctx):
         ctx.set_seed(seed)
         for fuse in (("penalty",), ("fp16",)):
             got, res, _ = check(ctx, "prune", [w], [np.zeros_like(w)], 0.9, 1e-3, fuse)
-            assert res.sampled == 0 and res.n_tie > 900000
+            assert res.sampled == 0 and res.n_tie > 1400000
     finally:
         ctx.set_seed(SEED)
 
@@ -398,7 +398,7 @@ def test_single_pass_with_and_without_multipliers_in_one_list(ctx):
     """Tensors with and without a lambda buffer in one sampled call: the journal of a candidate
     must carry the multiplier of its own tensor (candidates staged by one tensor are flushed
     while the CTA already works on the next)."""
-    shapes = [(70001,), (50000,), (123457,), (4099,), (200003,)]
+    shapes = [(280001,), (200000,), (493457,), (4099,), (800003,)]
     ws = W.random_set(shapes, seed=91, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
     lam = [ws.lam[0], None, ws.lam[2], None, ws.lam[4]]
     for sd in (1, 2, 3):
@@ -722,3 +722,35 @@ def test_workspace_query_sizes_a_context_that_never_allocates():
         c.close()
     with pytest.raises(cstep.CondensaError):
         cstep.workspace_bytes(99, ds.table, ds.T)
+
+
+def test_register_resident_route_of_short_lists(ctx):
+    """Lists of at most one work item per resident CTA are pruned in one launch out of registers:
+    many small tensors with unaligned heads, every quantisation type, tie groups that are kept
+    whole, cut in the middle (index levels) and spread over tensors, k = 0 and k = S."""
+    shapes = [(4097,), (33, 17), (5, 3, 3, 3), (1,), (100003,), (64, 1500), (7,)]
+    ws = W.random_set(shapes, seed=60, kind="normal", scale=0.05, lam_sigma=1e-2, mu=1e-2)
+    for s_ in (0.0, 0.37, 0.9, 1.0, 1e-6, 1 - 1e-6):
+        got, res, _ = check(ctx, "prune", ws.w, ws.lam, s_, ws.mu, ("lambda", "penalty"))
+        assert res.sampled == 0 and res.n_candidates == 0
+    for q in ("fp16", "bf16", "e4m3", "e5m2"):
+        check(ctx, "prune", ws.w, ws.lam, 0.8, ws.mu, (q, "lambda"), elem_offset=1)
+    check(ctx, "prune", ws.w, [None] * len(shapes), 0.5, 1.0, (), skew=1)
+    # ties: integers, so that many units share the threshold key
+    ints = [np.round(a * 60).astype(np.float32) for a in ws.w]
+    for s_ in (0.3, 0.5, 0.77):
+        got, res, _ = check(ctx, "prune", ints, None, s_, 1.0, ("lambda",))
+        assert res.n_tie > 1
+    const = [np.full(n, v, np.float32) for n, v in ((5000, 0.5), (70001, -0.5), (3, 0.5))]
+    for s_ in (0.1, 0.5, 0.999):
+        got, res, _ = check(ctx, "prune", const, None, s_, 1.0, ())
+        assert res.n_tie == 75004
+    # the largest list the route takes on this device, and the first one it does not take
+    import torch
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for n_items, route in ((2 * sms, 0), (2 * sms + 1, None)):
+        n = 4096 * n_items
+        w = W.draw(n, "normal", 0.05, 61, 0, 0)
+        got, res, _ = check(ctx, "prune", [w], [np.zeros_like(w)], 0.9, 1e-3, ("fp16", "lambda"))
+        if route is not None:
+            assert res.sampled == route and res.n_candidates == 0
