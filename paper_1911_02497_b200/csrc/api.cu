@@ -665,15 +665,29 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
                 CU_TRY(ctx, cudaFuncSetAttribute(k_fused_block<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
                 ctx->block_smem_set = true;
             }
-#define CS_LAUNCH_FUSED(KERNEL, GRID, NTHR, SMEM)                                              \
+            // Programmatic dependent launch: the single-pass kernel may start while the sampler
+            // still runs; it sets itself up (and the block kernel already fetches its first tiles)
+            // and waits for the sampler's results with griddepcontrol.wait.
+            cudaLaunchConfig_t cfg;
+            memset(&cfg, 0, sizeof(cfg));
+            cudaLaunchAttribute pdl;
+            pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            pdl.val.programmaticStreamSerializationAllowed = 1;
+            cfg.gridDim = dim3((unsigned)gridf);
+            cfg.blockDim = dim3((unsigned)(op == OP_PRUNE ? THREADS : BT_THREADS));
+            cfg.dynamicSmemBytes = op == OP_PRUNE ? 0 : BLOCK_FAST_DYN_SMEM;
+            cfg.stream = stream;
+            cfg.attrs = &pdl;
+            cfg.numAttrs = ctx->prof_on ? 0 : 1;       // with an event pair around every kernel there is nothing to overlap
+#define CS_LAUNCH_FUSED(KERNEL)                                                                \
     do {                                                                                       \
-        if (need_h && need_g) KERNEL<true, true><<<GRID, NTHR, SMEM, stream>>>(Pf);            \
-        else if (need_h) KERNEL<true, false><<<GRID, NTHR, SMEM, stream>>>(Pf);                \
-        else if (need_g) KERNEL<false, true><<<GRID, NTHR, SMEM, stream>>>(Pf);                \
-        else KERNEL<false, false><<<GRID, NTHR, SMEM, stream>>>(Pf);                           \
+        if (need_h && need_g) CU_TRY(ctx, cudaLaunchKernelEx(&cfg, KERNEL<true, true>, Pf));   \
+        else if (need_h) CU_TRY(ctx, cudaLaunchKernelEx(&cfg, KERNEL<true, false>, Pf));       \
+        else if (need_g) CU_TRY(ctx, cudaLaunchKernelEx(&cfg, KERNEL<false, true>, Pf));       \
+        else CU_TRY(ctx, cudaLaunchKernelEx(&cfg, KERNEL<false, false>, Pf));                  \
     } while (0)
-            if (op == OP_PRUNE) CS_LAUNCH_FUSED(k_fused_elem, gridf, THREADS, 0);
-            else CS_LAUNCH_FUSED(k_fused_block, gridf, BT_THREADS, BLOCK_FAST_DYN_SMEM);
+            if (op == OP_PRUNE) CS_LAUNCH_FUSED(k_fused_elem);
+            else CS_LAUNCH_FUSED(k_fused_block);
 #undef CS_LAUNCH_FUSED
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);

@@ -405,6 +405,13 @@ __device__ __forceinline__ int find_tensor(const long long *__restrict__ prefix,
     return lo;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start before the kernel ahead of it in the stream has finished; pdl_wait() returns when that
+// kernel has completed and its writes are visible (a no-op for a normal launch);
+// pdl_launch_dependents() lets the kernel behind start as early as resources allow.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ int bit_length(u64 x) { return x ? 64 - __clzll((long long)x) : 0; }
 
 }  // namespace cs

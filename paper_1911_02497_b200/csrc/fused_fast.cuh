@@ -53,10 +53,11 @@ template <bool H, bool G>
 __global__ void __launch_bounds__(THREADS, 3) k_fused_elem(Params P)
 {
     __shared__ ElemFastShared sh;
-    if (!P.ctl->sel.onepass) return;
-    const Bracket br = load_bracket(P.ctl->sel);
     for (int i = threadIdx.x; i < NBINS; i += THREADS) sh.hist[i] = 0;
     if (threadIdx.x < WARPS) sh.wcount[threadIdx.x] = 0;
+    pdl_wait();                     // the sampler's bracket and cleared counters are needed from here on
+    if (!P.ctl->sel.onepass) return;
+    const Bracket br = load_bracket(P.ctl->sel);
     __syncthreads();
     const int fp16 = quant_code(P.fuse);     // quantisation of theta
     const u32 lo = (u32)br.lo, range = (u32)br.hi - (u32)br.lo, guess = (u32)br.guess;
@@ -397,8 +398,9 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
 {
     __shared__ BlockFastShared sh;
     extern __shared__ __align__(128) unsigned char dyn_smem[];      // tile buffers, then the candidate staging
-    if (!P.ctl->sel.onepass) return;
-    const Bracket br = load_bracket(P.ctl->sel);
+    // The kernel may have been launched while the sampler ahead of it still runs (programmatic
+    // dependent launch): until pdl_wait() nothing the sampler writes is read - the set-up below and
+    // the first tile loads need only w, lambda and the descriptors.
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned char *tile_buf = dyn_smem;
     BlockCand *cands = reinterpret_cast<BlockCand *>(dyn_smem + (size_t)BT_STAGES * BT_STAGE_BYTES);
@@ -425,12 +427,28 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
     const float mu = P.mu;
     volatile int *abort_flag = &sh.abort;
     u64 na = 0;
+    Bracket br;
+    memset(&br, 0, sizeof(br));
+    bool onepass = false;
+    if (warp < BT_CWARPS) {
+        pdl_wait();
+        onepass = P.ctl->sel.onepass != 0;      // else the sampler advised against the single pass: nothing to do here
+        br = load_bracket(P.ctl->sel);
+    }
 
     if (warp == BT_CWARPS) {
         // ------------------------------------------------------------ producer (one lane)
         if (lane == 0) {
             u32 k = 0;
-            bool ok = true;
+            bool ok = true, dep_seen = false, quiet = false;
+            // before the first store, and before leaving: the sampler must have finished and
+            // must have said that the single pass is on
+            auto see_dependency = [&]() {
+                if (dep_seen) return;
+                pdl_wait();
+                dep_seen = true;
+                if (!P.ctl->sel.onepass) { quiet = true; ok = false; }
+            };
             // writes the outputs of the tile that used buffer `stage` (tile number `tile`) back
             auto store_tile = [&](long long tile, int stage) {
                 const TileGeom g = tile_geom(tile_prefix, td, P.T, tile);
@@ -459,6 +477,8 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
             for (; tile < P.n_tiles && ok; tile += gridDim.x, ++k) {
                 const int stage = (int)(k % BT_STAGES);
                 if (k >= (u32)BT_STAGES) {
+                    see_dependency();
+                    if (!ok) break;
                     // the consumers have left theta / lambda / mask of the tile before in this buffer
                     ok = mbar_wait_bounded(smem_u32(&sh.done_bar[stage]), ((k / BT_STAGES) - 1u) & 1u, abort_flag);
                     if (!ok) break;
@@ -486,6 +506,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
             }
             // drain: the last tiles still sit in their buffers
             const u32 issued = k;                       // tiles whose loads have been issued
+            see_dependency();
             if (ok) {
                 const u32 first = issued > (u32)BT_STAGES ? issued - BT_STAGES : 0u;
                 for (u32 j = first; j < issued && ok; ++j) {
@@ -497,9 +518,10 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
             if (!ok) {
                 // A wait ran out: report it (the selection kernels turn it into an error status) and
                 // give the loads still in flight the same bounded time, so that none lands in shared
-                // memory after this CTA has gone. The consumers see the flag and stop.
+                // memory after this CTA has gone. The consumers see the flag and stop. (`quiet`: no
+                // error, the single pass is simply off; the loads fetched ahead are waited for too.)
                 *abort_flag = 1;
-                atomicExch(&P.ctl->async_error, 1);
+                if (!quiet) atomicExch(&P.ctl->async_error, 1);
                 const u32 first = issued > (u32)BT_STAGES ? issued - BT_STAGES : 0u;
                 for (u32 j = first; j < issued; ++j)
                     (void)mbar_wait_bounded(smem_u32(&sh.full_bar[j % BT_STAGES]), (j / BT_STAGES) & 1u, nullptr);
@@ -513,7 +535,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
         u32 n_above = 0, k = 0;
         bool ok = true;
 #pragma unroll 1
-        for (long long tile = blockIdx.x; tile < P.n_tiles; tile += gridDim.x, ++k) {
+        for (long long tile = blockIdx.x; onepass && tile < P.n_tiles; tile += gridDim.x, ++k) {
             const int stage = (int)(k % BT_STAGES);
             const TileGeom g = tile_geom(tile_prefix, td, P.T, tile);
             const TensorDesc &d = td[g.t];
@@ -602,7 +624,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
             if (lane == 0) mbar_arrive(smem_u32(&sh.done_bar[stage]));
             block_flush(P, sh, cd, cw, BSTG - 32);
         }
-        if (!ok && lane == 0) {
+        if (!ok && lane == 0 && !*abort_flag) {
             *abort_flag = 1;
             atomicExch(&P.ctl->async_error, 1);
         }
@@ -610,6 +632,8 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_block(Params P)
         na = n_above;
     }
     __syncthreads();
+    pdl_wait();
+    if (!P.ctl->sel.onepass) return;         // (the same for every thread)
     // the blocks outside the aligned interior (ragged last block rows, unaligned tensors) and
     // the tensors that pass through: work items listed by the host, done by generic code
     if (P.n_edge_items > 0) {

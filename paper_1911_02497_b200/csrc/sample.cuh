@@ -73,6 +73,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
 {
     __shared__ SampleShared sh;
     Ctl *ctl = P.ctl;
+    pdl_launch_dependents();        // the single-pass kernel behind may set itself up meanwhile
     // what the plain start kernel does: clear histograms (all CTAs share the work)
     for (int i = blockIdx.x * SAMPLE_THREADS + threadIdx.x; i < 3 * NBINS; i += gridDim.x * SAMPLE_THREADS)
         P.hist[i] = 0;
