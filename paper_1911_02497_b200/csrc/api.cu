@@ -66,6 +66,7 @@ struct condensa_ctx {
     Ctl *ctl = nullptr;
     int occ_select[3] = {0, 0, 0};
     int occ_stream = 0;
+    int occ_filter = 0;
     int occ_prune_small = 0;        // resident CTAs per SM of the register-resident small-list kernel
     bool small_smem_set = false;    // dynamic shared memory limit of k_select_small raised on this device
     bool block_smem_set = false;    // the same for the tiled block kernel
@@ -440,6 +441,25 @@ void prof_collect(condensa_ctx *ctx)
     ctx->prof_used = 0;
 }
 
+// Launch configuration with the programmatic-dependent-launch attribute (dropped while every
+// kernel is bracketed by an event pair: nothing can overlap then).
+struct PdlLaunch {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr;
+    PdlLaunch(const condensa_ctx *ctx, int grid, int block, size_t smem, cudaStream_t stream)
+    {
+        memset(&cfg, 0, sizeof(cfg));
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3((unsigned)block);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cfg.attrs = &attr;
+        cfg.numAttrs = ctx->prof_on ? 0 : 1;
+    }
+};
+
 #define LAUNCH_CHECK(ctx)                                                                    \
     do {                                                                                     \
         cudaError_t e_ = cudaGetLastError();                                                 \
@@ -631,7 +651,8 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         }
         if (op == OP_FILTER && pl.S > 0) {
             int pa_ = prof_begin(ctx, "k_filter_partial", stream);
-            k_filter_partial<<<stream_grid(ctx, (pl.n_items_a + WARPS - 1) / WARPS, 8), THREADS, 0, stream>>>(Pa);
+            if (!ctx->occ_filter) ctx->occ_filter = occupancy(k_filter_partial);       // one wave of resident CTAs
+            k_filter_partial<<<stream_grid(ctx, (pl.n_items_a + WARPS - 1) / WARPS, ctx->occ_filter), THREADS, 0, stream>>>(Pa);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pa_, stream);
             if (!small) {           // the one-CTA selection forms the norms itself
@@ -699,7 +720,11 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
                 ctx->small_smem_set = true;
             }
             const int pi_ = prof_begin(ctx, "k_select_small", stream);
-            k_select_small<<<1, SMALL_THREADS, sizeof(u64) * (size_t)pl.S, stream>>>(Pa, init, op == OP_FILTER ? 1 : 0);
+            {
+                PdlLaunch L2(ctx, 1, SMALL_THREADS, sizeof(u64) * (size_t)pl.S, stream);
+                const int combine = op == OP_FILTER ? 1 : 0;
+                CU_TRY(ctx, cudaLaunchKernelEx(&L2.cfg, k_select_small, Pa, init, combine));
+            }
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
         } else if (!one_launch) {
@@ -747,10 +772,12 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             if (need_h) k_apply_linear<M_PRUNE, true><<<grid, THREADS, 0, stream>>>(Pb);
             else k_apply_linear<M_PRUNE, false><<<grid, THREADS, 0, stream>>>(Pb);
             break;
-        case OP_FILTER:
-            if (need_h) k_apply_linear<M_FILTER, true><<<grid, THREADS, 0, stream>>>(Pb);
-            else k_apply_linear<M_FILTER, false><<<grid, THREADS, 0, stream>>>(Pb);
+        case OP_FILTER: {
+            PdlLaunch L2(ctx, grid, THREADS, 0, stream);
+            if (need_h) CU_TRY(ctx, cudaLaunchKernelEx(&L2.cfg, k_apply_linear<M_FILTER, true>, Pb));
+            else CU_TRY(ctx, cudaLaunchKernelEx(&L2.cfg, k_apply_linear<M_FILTER, false>, Pb));
             break;
+        }
         case OP_BLOCK: k_apply_block<<<grid, THREADS, 0, stream>>>(Pb); break;
         case OP_BLOCKGEN:
             if (need_h) k_apply_linear<M_BLOCKGEN, true><<<grid, THREADS, 0, stream>>>(Pb);

@@ -14,7 +14,8 @@ constexpr int THREADS = 256;             // every kernel here runs 256-thread CT
 constexpr int WARPS = THREADS / 32;
 constexpr int GROUPS_PER_ITEM = 1024;    // linear work item = 1024 groups of 4 elements
 constexpr int BLOCKS_PER_ITEM = 256;     // block work item = 256 4x4 blocks (one per thread: the smaller the item, the smaller the imbalance of the last round)
-constexpr int SEG = 2048;                // filter norm segment (elements)
+constexpr int SEG = 512;                 // filter norm segment (elements): one batch of four 128-bit loads per lane,
+                                         // and enough segments that the last round of the grid hardly matters
 constexpr int LOG_NBINS = 11;
 constexpr int NBINS = 1 << LOG_NBINS;    // histogram bins per selection pass
 constexpr int FIN = 4096;                // bracket population finished by ranking in shared memory

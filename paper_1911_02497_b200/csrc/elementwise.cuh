@@ -318,6 +318,7 @@ template <int MODE, bool H>
 __global__ void __launch_bounds__(THREADS, 3) k_apply_linear(Params P)
 {
     u64 tau_key = 0, tau_id = 0;
+    pdl_wait();                     // a no-op unless the launch was made dependent on the kernel ahead
     if (MODE == M_PRUNE || MODE == M_FILTER || MODE == M_BLOCKGEN) {
         if (P.ctl->sel.onepass) return;      // the single-pass kernel has written everything
         tau_key = P.ctl->tau_key;

@@ -56,6 +56,8 @@ __global__ void __launch_bounds__(SMALL_THREADS) k_select_small(Params P, Sel in
     extern __shared__ __align__(16) u64 skey[];        // [S]
     __shared__ SmallShared sh;
     Ctl *c = P.ctl;
+    pdl_launch_dependents();
+    pdl_wait();                     // the partial sums (or the value array) of the kernel ahead
     const u32 S = (u32)init.S;
     if (combine && P.T <= SMALL_T_CACHE) {
         // tensor ranges first (one round trip), then every key needs only its partial sums

@@ -115,6 +115,7 @@ __global__ void __launch_bounds__(THREADS) k_filter_partial(Params P)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int crit = P.crit;
+    pdl_launch_dependents();        // the kernels behind may set themselves up (they wait before reading the sums)
     const long long n_work = P.n_items;
     for (long long base = (long long)blockIdx.x * WARPS; base < n_work; base += (long long)gridDim.x * WARPS) {
         const long long item = base + warp;
