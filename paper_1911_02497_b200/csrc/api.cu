@@ -283,7 +283,10 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, const HostSp
     const u64 S = (u64)pl.S;
     u64 cap = S / 8;
     if (cap < 65536) cap = 65536;
-    if (cap > (1ull << 22)) cap = 1ull << 22;
+    // unstructured lists may list up to 16 Mi candidates (20 bytes each with the journal): the sample
+    // bracket of a list of more than 10^8 parameters at a moderate sparsity holds several million
+    const u64 cap_max = op == OP_PRUNE ? (1ull << 24) : (1ull << 22);
+    if (cap > cap_max) cap = cap_max;
     if (cap > S) cap = S ? S : 1;
     pl.cap = cap;
 }
