@@ -292,6 +292,8 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, const HostSp
 }
 
 constexpr int N_SAMPLE = SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD;
+constexpr int N_SAMPLE_BIG = SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD_BIG;
+constexpr long long SAMPLE_BIG_FROM = 1ll << 25;     // unstructured lists from this many units take the larger sample
 constexpr int SAMPLE_CTAS = 64;
 constexpr long long ONE_LAUNCH_MAX_N = 4ll << 20;    // parameters of a list that the one-launch route takes
 
@@ -313,7 +315,7 @@ Layout make_layout(int T, const Plan &pl, bool ranking, bool filter, int journal
     L.list_id = off; if (ranking) off = align_up(off + sizeof(u64) * pl.cap, 256);
     L.arr_key = off; if (filter) off = align_up(off + sizeof(u64) * (size_t)std::max<long long>(pl.S, 1), 256);
     L.partial = off; if (filter) off = align_up(off + sizeof(double) * (size_t)std::max<long long>(pl.n_seg, 1), 256);
-    L.sample = off; if (journal_floats) off = align_up(off + sizeof(u64) * N_SAMPLE, 256);
+    L.sample = off; if (journal_floats) off = align_up(off + sizeof(u64) * N_SAMPLE_BIG, 256);
     L.journal = off; if (journal_floats) off = align_up(off + sizeof(float) * (size_t)journal_floats * pl.cap, 256);
     L.total = off;
     return L;
@@ -590,7 +592,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     P.S = pl.S;
     P.bits_key = (op == OP_PRUNE) ? 31 : 63;
     P.sample_key = (u64 *)(ws + L.sample);
-    P.n_sample = N_SAMPLE;
+    // a longer list pays for a larger sample: bracket and wrong provisional decisions shrink with its square root
+    const bool big_sample = op == OP_PRUNE && pl.S >= SAMPLE_BIG_FROM;
+    P.n_sample = big_sample ? N_SAMPLE_BIG : N_SAMPLE;
     P.jr_lam = (float *)(ws + L.journal);
     P.onepass_cap = pl.cap;
     P.crit = sp.crit;
@@ -671,8 +675,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         if (sampling) Pa.n_edge_items = 0;     // the single-pass kernels do their edge items themselves
         if (sampling && !init.done) {
             int pi_ = prof_begin(ctx, "k_sample", stream);
-            if (op == OP_PRUNE) k_sample<SRC_ELEM><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
-            else k_sample<SRC_BLOCK><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            if (op == OP_PRUNE && big_sample) k_sample<SRC_ELEM, SAMPLE_KEYS_PER_THREAD_BIG><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            else if (op == OP_PRUNE) k_sample<SRC_ELEM, SAMPLE_KEYS_PER_THREAD><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            else k_sample<SRC_BLOCK, SAMPLE_KEYS_PER_THREAD><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
             pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : "k_fused_block", stream);

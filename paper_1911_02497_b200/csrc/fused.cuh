@@ -325,19 +325,42 @@ __device__ __noinline__ void repair_unit(const Params &P, u64 idx, u64 id, bool 
         jr = P.jr_lam + idx * 16 + 4 * part;
     }
     float w[4], l[4];
+    const bool vec = SRC == SRC_BLOCK && nv == 4 && d.blk_vec_ok;      // a whole aligned row of a block
+    if (vec) {
+        const float4 a = ld4_ro(d.w + off);
+        w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
+        const float4 q = has_lam ? __ldcg(reinterpret_cast<const float4 *>(jr)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        l[0] = q.x; l[1] = q.y; l[2] = q.z; l[3] = q.w;
+    } else {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        w[j] = j < nv ? __ldg(d.w + off + j) : 0.0f;
-        l[j] = (j < nv && has_lam) ? __ldcg(jr + j) : 0.0f;
+        for (int j = 0; j < 4; ++j) {
+            w[j] = j < nv ? __ldg(d.w + off + j) : 0.0f;
+            l[j] = (j < nv && has_lam) ? __ldcg(jr + j) : 0.0f;
+        }
     }
+    float th[4], ln[4], gr[4];
+    unsigned short hb[4];
+    unsigned char mk[4];
 #pragma unroll 1
     for (int j = 0; j < nv; ++j) {
         const Out o = finish(w[j], l[j], form_u(w[j], l[j], P.mu, has_lam), keep, P.mu, P.fuse, has_lam);
-        d.theta[off + j] = o.theta;
-        if (d.mask) d.mask[off + j] = o.m;
-        if (d.theta_h) d.theta_h[off + j] = o.th;
-        if (wr_lam) d.lam[off + j] = o.lam;
-        if (wr_grad) d.grad[off + j] = o.grad;
+        th[j] = o.theta; ln[j] = o.lam; gr[j] = o.grad; hb[j] = o.th; mk[j] = o.m;
+    }
+    if (vec) {
+        *reinterpret_cast<float4 *>(d.theta + off) = make_float4(th[0], th[1], th[2], th[3]);
+        if (d.mask) *reinterpret_cast<u32 *>(d.mask + off) = keep ? 0x01010101u : 0u;
+        if (d.theta_h) *reinterpret_cast<uint2 *>(d.theta_h + off) =
+            make_uint2((u32)hb[0] | ((u32)hb[1] << 16), (u32)hb[2] | ((u32)hb[3] << 16));
+        if (wr_lam) *reinterpret_cast<float4 *>(d.lam + off) = make_float4(ln[0], ln[1], ln[2], ln[3]);
+        if (wr_grad) *reinterpret_cast<float4 *>(d.grad + off) = make_float4(gr[0], gr[1], gr[2], gr[3]);
+    } else {
+        for (int j = 0; j < nv; ++j) {
+            d.theta[off + j] = th[j];
+            if (d.mask) d.mask[off + j] = mk[j];
+            if (d.theta_h) d.theta_h[off + j] = hb[j];
+            if (wr_lam) d.lam[off + j] = ln[j];
+            if (wr_grad) d.grad[off + j] = gr[j];
+        }
     }
 }
 

@@ -8,13 +8,15 @@
 // afterwards from the full pass's counts - the sample only decides how little
 // work the exact selection has to do, never the result.
 #pragma once
+#include <type_traits>
 #include "common.cuh"
 #include "select.cuh"
 
 namespace cs {
 
 constexpr int SAMPLE_THREADS = 1024;
-constexpr int SAMPLE_KEYS_PER_THREAD = 16;          // n_sample = 16384 keys for one CTA
+constexpr int SAMPLE_KEYS_PER_THREAD = 16;          // n_sample = 16384 keys for one CTA ...
+constexpr int SAMPLE_KEYS_PER_THREAD_BIG = 32;      // ... 32768 for long unstructured lists (31-bit keys: half the registers)
 
 constexpr int SAMPLE_TD_CACHE = 16;
 
@@ -68,9 +70,10 @@ __device__ __forceinline__ u64 cta_sum(u64 v, u64 *red)
     return t;
 }
 
-template <int SRC>
+template <int SRC, int KPT>
 __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
 {
+    typedef typename std::conditional<SRC == SRC_ELEM, u32, u64>::type KeyT;     // element keys have 31 bits
     __shared__ SampleShared sh;
     Ctl *ctl = P.ctl;
     pdl_launch_dependents();        // the single-pass kernel behind may set itself up meanwhile
@@ -107,12 +110,12 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
 
     // ---- last CTA: bracket from the sample ----
     const int m = P.n_sample;
-    u64 key[SAMPLE_KEYS_PER_THREAD];
+    KeyT key[KPT];
     u64 mn = ~0ull, mx = 0;
 #pragma unroll
-    for (int q = 0; q < SAMPLE_KEYS_PER_THREAD; ++q) {
+    for (int q = 0; q < KPT; ++q) {
         const int idx = q * SAMPLE_THREADS + threadIdx.x;
-        key[q] = idx < m ? __ldcg(&P.sample_key[idx]) : 0;
+        key[q] = idx < m ? (KeyT)__ldcg(&P.sample_key[idx]) : (KeyT)0;
         if (idx < m) { mn = key[q] < mn ? key[q] : mn; mx = key[q] > mx ? key[q] : mx; }
     }
     for (int o = 16; o > 0; o >>= 1) {
@@ -150,7 +153,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         if (threadIdx.x < 3) { sh.rank_bin[threadIdx.x] = 0; sh.rank_before[threadIdx.x] = 0; }
         __syncthreads();
 #pragma unroll
-        for (int q = 0; q < SAMPLE_KEYS_PER_THREAD; ++q) {
+        for (int q = 0; q < KPT; ++q) {
             const int idx = q * SAMPLE_THREADS + threadIdx.x;
             if (idx < m && key[q] >= lo && key[q] <= hi) {
                 u64 b = (hi - key[q]) >> shift;
@@ -186,7 +189,17 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
         const u64 e_lo = (lo_edge - lo >= width - 1) ? lo_edge - (width - 1) : lo;   // lower edge of b_lo
         const u64 mid_edge = hi - ((u64)b_mid << shift);
         const u64 e_mid = (mid_edge - lo >= width - 1) ? mid_edge - (width - 1) : lo;
-        hi0 = e_hi; lo0 = e_lo; guess = e_mid;
+        hi0 = e_hi; lo0 = e_lo;
+        {
+            // the guess: inside the bin of the sample's rank m*p, by linear interpolation over the
+            // bin's population (a whole bin width of bias would cost as many wrong provisional
+            // decisions as the bin holds units of the full list)
+            const u64 c_mid = sh.hist[b_mid];
+            const u64 pos = ranks[1] - above - sh.rank_before[1];           // 1 .. c_mid, counted from the upper edge
+            const u64 span = mid_edge - e_mid;
+            const u64 down = c_mid ? (u64)((double)span * (((double)pos - 0.5) / (double)c_mid)) : 0;
+            guess = mid_edge - (down > span ? span : down);
+        }
         const u64 before_hi = sh.rank_before[0];
         __syncthreads();
         if (b_lo - b_hi >= 16 || shift == 0) break;
@@ -200,7 +213,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) k_sample(Params P, Sel init)
     if (guess > hi0) guess = hi0;
     u64 inside = 0;
 #pragma unroll
-    for (int q = 0; q < SAMPLE_KEYS_PER_THREAD; ++q) {
+    for (int q = 0; q < KPT; ++q) {
         const int idx = q * SAMPLE_THREADS + threadIdx.x;
         inside += (idx < m && key[q] >= lo0 && key[q] <= hi0) ? 1 : 0;
     }

@@ -735,13 +735,23 @@ struct ListChunk {
     u64 key[LIST_ROUNDS], id[LIST_ROUNDS];
 };
 
-__device__ __forceinline__ void load_list_chunk(const Params &P, u64 base, u64 n_list, ListChunk &ch)
+// Entries per thread and chunk for a list of n_list entries: as many as give every CTA of the
+// grid one chunk, at most LIST_ROUNDS (a short list is then spread over all CTAs, and so are the
+// rewrites it causes).
+__device__ __forceinline__ int list_rounds(u64 n_list)
+{
+    const u64 per = (n_list + (u64)gridDim.x * THREADS - 1) / ((u64)gridDim.x * THREADS);
+    return per < 1 ? 1 : per > (u64)LIST_ROUNDS ? LIST_ROUNDS : (int)per;
+}
+
+__device__ __forceinline__ void load_list_chunk(const Params &P, u64 base, u64 n_list, int rounds, ListChunk &ch)
 {
 #pragma unroll
     for (int r = 0; r < LIST_ROUNDS; ++r) {
         const u64 i = base + (u64)r * THREADS + threadIdx.x;
-        ch.key[r] = i < n_list ? __ldcg(&P.list_key[i]) : 0;
-        ch.id[r] = i < n_list ? __ldcg(&P.list_id[i]) : 0;
+        const bool ok = r < rounds && i < n_list;
+        ch.key[r] = ok ? __ldcg(&P.list_key[i]) : 0;
+        ch.id[r] = ok ? __ldcg(&P.list_id[i]) : 0;
     }
 }
 
@@ -759,7 +769,8 @@ __device__ __noinline__ u64 list_walk(const Params &P, ScanShared &sh, bool gath
     Ctl *c = P.ctl;
     const Sel &s = sh.sel;
     const bool sk = s.lo_key == s.hi_key;
-    const u64 chunk = (u64)LIST_ROUNDS * THREADS;
+    const int rounds = list_rounds(n_list);
+    const u64 chunk = (u64)rounds * THREADS;
     constexpr u32 LPU = RepairLanes<SRC>::value;
     u64 fixed = 0;
     bool have_pre = pre != nullptr;
@@ -768,12 +779,12 @@ __device__ __noinline__ u64 list_walk(const Params &P, ScanShared &sh, bool gath
         __syncthreads();
         ListChunk ch;
         if (have_pre) ch = *pre;
-        else load_list_chunk(P, base, n_list, ch);
+        else load_list_chunk(P, base, n_list, rounds, ch);
         have_pre = false;
 #pragma unroll
         for (int r = 0; r < LIST_ROUNDS; ++r) {
             const u64 i = base + (u64)r * THREADS + threadIdx.x;
-            if (i >= n_list) continue;
+            if (r >= rounds || i >= n_list) continue;
             const u64 key = ch.key[r], id = ch.id[r];
             bool fin;
             if (gather) {
@@ -861,7 +872,8 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
         // single-pass path: this CTA's first chunk of the list is fetched while the pick is made
         const u64 n_all = __ldcg(&P.ctl->list_count[0]);
         if (n_all <= P.cap) {
-            load_list_chunk(P, (u64)blockIdx.x * LIST_ROUNDS * THREADS, n_all, pre);
+            const int rounds = list_rounds(n_all);
+            load_list_chunk(P, (u64)blockIdx.x * rounds * THREADS, n_all, rounds, pre);
             have_pre = true;
         }
     }
@@ -945,7 +957,7 @@ __global__ void __launch_bounds__(THREADS) k_select(Params P, int first_listed, 
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) write_result(P, sh.sel);
     if constexpr (SRC != SRC_ARRAY) {
-        if (post_apply && !sh.sel.onepass) {       // the same on every CTA: the sampler's verdict never changes
+        if (post_apply && !sh.sel.onepass) {       // the same on every CTA: all derive the state from the same global data
             __threadfence();
             grid.sync();
             Params Pb = P;
