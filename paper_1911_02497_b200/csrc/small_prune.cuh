@@ -4,8 +4,9 @@
 // about 1.2 M parameters on 148 SMs) is read from memory ONCE: every thread keeps its w, lambda
 // and u in registers across the grid barriers while the CTAs agree on the threshold by three
 // histogram levels over the 31-bit key (11 + 11 + 9 bits, most significant first; shared-memory
-// histograms with warp-aggregated updates - the first level is the exponent, where nearly all
-// lanes hit a handful of bins - merged into a global one, one grid barrier per level), then, only
+// histograms merged into a global one, one grid barrier per level; plain shared-memory atomics:
+// electing one lane per bin with match.any was measured slower, here and in the grid-wide scan,
+// although the first level is the exponent and most lanes hit a handful of bins), then, only
 // if the threshold key is shared by more units than may be kept, by two more levels over the
 // index (the tie rule). The projection is written from the same registers. No sample, no
 // candidate list, no second read: the configuration-1/2-sized lists are latency, not bandwidth.
@@ -42,12 +43,7 @@ __device__ __forceinline__ void ps_level(const Params &P, SmallPruneShared &sh, 
         const bool in = ((live >> j) & 1u) && (V)(val[j] >> (shift + bits)) == want_above;
         u32 b = (u32)(val[j] >> shift) & (nb - 1u);
         if (desc) b = nb - 1u - b;
-        // warp-aggregated update: lanes with the same bin elect one that adds their count
-        const unsigned act = __ballot_sync(0xffffffffu, in);
-        if (in) {
-            const unsigned same = __match_any_sync(act, b);
-            if (lane == __ffs(same) - 1) atomicAdd(&sh.hist[b], (u32)__popc(same));
-        }
+        if (in) atomicAdd(&sh.hist[b], 1u);
     }
     __syncthreads();
     u64 *gh = P.hist + (size_t)slot * NBINS;
