@@ -354,6 +354,26 @@ CONDENSA_API int condensa_thin_compact(condensa_ctx *ctx, const float *src, int6
                                        int64_t inner, const uint8_t *keep0, const uint8_t *keep1,
                                        float *dst, int64_t *dims_out, void *stream);
 
+/* The same for a whole list of tensors in three launches (flags of all, index lists of all,
+ * gather of all) instead of three per tensor: thinning a network is dozens of small tensors.
+ * For every layer l: keep0 (d0 bytes, DEVICE, out) receives the axis-0 flags of src (1 iff
+ * the slice holds a non-zero); dst receives src without the axis-0 slices whose flag is 0
+ * (if remove_axis0 != 0) and without the axis-1 slices whose flag in layer keep1_from's keep0
+ * is 0 (keep1_from = -1: the whole axis stays; that layer's d0 must equal this layer's d1 -
+ * e.g. a conv layer loses the input channels that the layer feeding it lost as filters);
+ * dims_out (DEVICE, two int64) receives the kept extents. `layers` is a HOST array.
+ * Extents and pointer rules as for condensa_thin_compact(). */
+typedef struct {
+    const float *src;      /* in : [d0][d1][inner], fp32                      */
+    int64_t d0, d1, inner;
+    uint8_t *keep0;        /* out: axis-0 flags, d0 bytes                     */
+    int32_t remove_axis0;  /* remove the axis-0 slices whose flag is 0        */
+    int32_t keep1_from;    /* layer whose keep0 removes axis-1 slices, or -1  */
+    float *dst;            /* out: the dense smaller tensor                   */
+    int64_t *dims_out;     /* out: d0', d1'                                   */
+} condensa_thin_layer;
+CONDENSA_API int condensa_thin_list(condensa_ctx *ctx, const condensa_thin_layer *layers, int L, void *stream);
+
 /* counts[t] = number of non-zero values of arrays[t] (numel[t] floats each),
  * counts[T] = their sum; the memory footprint is that count times the bytes of
  * a stored value. `arrays` and `numel` are HOST arrays of T entries (the

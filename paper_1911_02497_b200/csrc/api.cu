@@ -1172,6 +1172,87 @@ int condensa_thin_compact(condensa_ctx *ctx, const float *src, int64_t d0, int64
     return CONDENSA_OK;
 }
 
+int condensa_thin_list(condensa_ctx *ctx, const condensa_thin_layer *layers, int L, void *stream_)
+{
+    if (!ctx) return CONDENSA_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!layers || L <= 0 || L > 65535) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer list is empty, NULL or too long");
+    std::vector<ThinLayerDesc> td((size_t)L);
+    std::vector<long long> pre_f((size_t)L + 1, 0), pre_g((size_t)L + 1, 0);
+    size_t idx_bytes = 0;
+    std::vector<size_t> off0((size_t)L), off1((size_t)L);
+    for (int l = 0; l < L; ++l) {
+        const condensa_thin_layer &x = layers[l];
+        if (x.d0 < 0 || x.d1 < 0 || x.inner < 0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: negative extent", l);
+        if (x.d0 > 0x7FFFFFFFll || x.d1 > 0x7FFFFFFFll || (double)x.d1 * (double)x.inner >= 2147483648.0)
+            return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: d0, d1 and d1 * inner must be below 2^31", l);
+        const long long n = x.d0 * x.d1 * x.inner;
+        if (!x.dims_out || (uintptr_t)x.dims_out % 8) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: dims_out is NULL or misaligned", l);
+        if (n > 0 && (!x.src || !x.dst)) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: src or dst is NULL", l);
+        if (x.d0 > 0 && !x.keep0) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: keep0 is NULL", l);
+        if ((uintptr_t)x.src % 4 || (uintptr_t)x.dst % 4) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: misaligned pointer", l);
+        if (x.keep1_from >= L || (x.keep1_from >= 0 && layers[x.keep1_from].d0 != x.d1))
+            return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: keep1_from must name a layer whose d0 equals this layer's d1", l);
+        if (n > 0) {
+            const uintptr_t a = (uintptr_t)x.src, b = (uintptr_t)x.dst, bytes = (uintptr_t)n * 4;
+            if (a < b + bytes && b < a + bytes) return fail(ctx, CONDENSA_ERR_INVALID_ARG, "layer %d: src and dst overlap", l);
+        }
+        ThinLayerDesc d;
+        memset(&d, 0, sizeof(d));
+        d.src = x.src; d.dst = x.dst; d.keep0 = x.keep0;
+        d.keep1 = x.keep1_from >= 0 ? layers[x.keep1_from].keep0 : nullptr;
+        d.dims_out = (long long *)x.dims_out;
+        d.d0 = x.d0; d.d1 = x.d1; d.inner = x.inner;
+        d.use_keep0 = x.remove_axis0 ? 1 : 0;
+        td[l] = d;
+        off0[l] = idx_bytes; idx_bytes += align_up(sizeof(int) * (size_t)x.d0, 256);
+        off1[l] = idx_bytes; idx_bytes += align_up(sizeof(int) * (size_t)x.d1, 256);
+        pre_f[l + 1] = pre_f[l] + x.d0;            // a slice without values still gets its flag (0)
+        pre_g[l + 1] = pre_g[l] + (n > 0 ? x.d0 * ((x.d1 * x.inner + 1023) / 1024) : 0);
+    }
+    CU_TRY(ctx, cudaSetDevice(ctx->device));
+    Plan none;
+    none.cap = 1;
+    const Layout Lay = make_layout(0, none, false, false);
+    const size_t desc_bytes = align_up(sizeof(ThinLayerDesc) * (size_t)L + 2 * sizeof(long long) * (size_t)(L + 1), 256);
+    int rc = ensure_workspace(ctx, Lay.desc + desc_bytes + idx_bytes, stream);
+    if (rc) return rc;
+    char *base = ctx->ws + Lay.desc;
+    for (int l = 0; l < L; ++l) {
+        td[l].idx0 = (int *)(base + desc_bytes + off0[l]);
+        td[l].idx1 = (int *)(base + desc_bytes + off1[l]);
+    }
+    std::vector<char> img(sizeof(ThinLayerDesc) * (size_t)L + 2 * sizeof(long long) * (size_t)(L + 1));
+    memcpy(img.data(), td.data(), sizeof(ThinLayerDesc) * (size_t)L);
+    memcpy(img.data() + sizeof(ThinLayerDesc) * (size_t)L, pre_f.data(), sizeof(long long) * (size_t)(L + 1));
+    memcpy(img.data() + sizeof(ThinLayerDesc) * (size_t)L + sizeof(long long) * (size_t)(L + 1), pre_g.data(),
+           sizeof(long long) * (size_t)(L + 1));
+    rc = upload_image(ctx, img, base, stream);
+    if (rc) return rc;
+    const ThinLayerDesc *dtd = (const ThinLayerDesc *)base;
+    const long long *dpf = (const long long *)(base + sizeof(ThinLayerDesc) * (size_t)L);
+    const long long *dpg = dpf + (L + 1);
+    ctx->last_stream = stream;
+    int pa_ = prof_begin(ctx, "k_thin_list_flags", stream);
+    if (pre_f[L] > 0) {
+        k_thin_list_flags<<<stream_grid(ctx, (pre_f[L] + WARPS - 1) / WARPS, 8), THREADS, 0, stream>>>(dtd, dpf, L);
+        LAUNCH_CHECK(ctx);
+    }
+    prof_end(ctx, pa_, stream);
+    pa_ = prof_begin(ctx, "k_thin_list_index", stream);
+    k_thin_list_index<<<L, THIN_INDEX_THREADS, 0, stream>>>(dtd);
+    LAUNCH_CHECK(ctx);
+    prof_end(ctx, pa_, stream);
+    if (pre_g[L] > 0) {
+        pa_ = prof_begin(ctx, "k_thin_list_gather", stream);
+        k_thin_list_gather<<<stream_grid(ctx, pre_g[L], 8), THREADS, 0, stream>>>(dtd, dpg, L);
+        LAUNCH_CHECK(ctx);
+        prof_end(ctx, pa_, stream);
+    }
+    if (cudaEventRecord(ctx->tail_ev, stream) == cudaSuccess) ctx->tail_recorded = true;
+    return CONDENSA_OK;
+}
+
 int condensa_count_nonzero(condensa_ctx *ctx, const float *const *arrays, const int64_t *numel, int T,
                            int64_t *counts, void *stream_)
 {

@@ -179,4 +179,120 @@ __global__ void __launch_bounds__(THREADS) k_count_nonzero(const CountDesc *td, 
     }
 }
 
+// ---------------------------------------------------------------- a whole list of layers at once
+// The same three steps for a list of tensors in three launches instead of three per tensor
+// (thinning a network is dozens of small tensors: launch latency, not bandwidth).
+struct ThinLayerDesc {
+    const float *src;
+    float *dst;
+    uint8_t *keep0;            // out: axis-0 flags of this tensor (d0 bytes), written 0 / 1
+    const uint8_t *keep1;      // in : flags that remove axis-1 slices (another tensor's keep0), or NULL
+    long long *dims_out;       // out: d0', d1'
+    int *idx0, *idx1;          // scratch: ascending positions of the kept slices
+    long long d0, d1, inner;
+    int use_keep0;             // remove the axis-0 slices whose flag is 0
+    int pad;
+};
+
+// keep0[i] = 1 iff slice [i][:][:] of its tensor holds a non-zero value; one warp per slice.
+// Work items: slices, numbered through the list (`prefix[l]` = first slice of layer l).
+__global__ void __launch_bounds__(THREADS) k_thin_list_flags(const ThinLayerDesc *td, const long long *prefix, int L)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long n = prefix[L];
+    for (long long base = (long long)blockIdx.x * WARPS; base < n; base += (long long)gridDim.x * WARPS) {
+        const long long item = base + warp;
+        if (item >= n) continue;
+        const int l = find_tensor(prefix, L, item);
+        const ThinLayerDesc &d = td[l];
+        const long long i = item - prefix[l], len = d.d1 * d.inner;
+        const float *x = d.src + i * len;
+        bool nz = false;
+        for (long long j = lane; j < len && !nz; j += 32) nz = is_nonzero(__ldg(x + j));
+        nz = __any_sync(0xffffffffu, nz);
+        if (lane == 0) d.keep0[i] = nz ? 1 : 0;
+    }
+}
+
+// Index lists and kept extents of every layer: CTA l does layer l.
+__global__ void __launch_bounds__(THIN_INDEX_THREADS) k_thin_list_index(const ThinLayerDesc *td)
+{
+    const ThinLayerDesc &d = td[blockIdx.x];
+    __shared__ int wsum[THIN_INDEX_THREADS / 32];
+    __shared__ int carry;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int ax = 0; ax < 2; ++ax) {
+        const uint8_t *keep = ax ? d.keep1 : (d.use_keep0 ? d.keep0 : nullptr);
+        const long long n = ax ? d.d1 : d.d0;
+        int *idx = ax ? d.idx1 : d.idx0;
+        if (!keep) {
+            if (threadIdx.x == 0) d.dims_out[ax] = n;
+            continue;
+        }
+        if (threadIdx.x == 0) carry = 0;
+        __syncthreads();
+        for (long long c0 = 0; c0 < n; c0 += THIN_INDEX_THREADS) {
+            const long long i = c0 + threadIdx.x;
+            const int f = (i < n && keep[i]) ? 1 : 0;
+            int sc = f;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, sc, o);
+                if (lane >= o) sc += y;
+            }
+            if (lane == 31) wsum[warp] = sc;
+            __syncthreads();
+            if (warp == 0) {
+                int t = wsum[lane];
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(0xffffffffu, t, o);
+                    if (lane >= o) t += y;
+                }
+                wsum[lane] = t;
+            }
+            __syncthreads();
+            const int before = carry + (warp ? wsum[warp - 1] : 0) + sc - f;
+            if (f) idx[before] = (int)i;
+            __syncthreads();
+            if (threadIdx.x == 0) carry += wsum[THIN_INDEX_THREADS / 32 - 1];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) d.dims_out[ax] = carry;
+        __syncthreads();
+    }
+}
+
+// dst = src without the removed slices, for every layer. Work items: 1024 consecutive elements of
+// one INPUT row position (an upper bound of the output rows; `prefix[l]` = first item of layer l).
+__global__ void __launch_bounds__(THREADS) k_thin_list_gather(const ThinLayerDesc *td, const long long *prefix, int L)
+{
+    const long long n = prefix[L];
+    for (long long item = blockIdx.x; item < n; item += gridDim.x) {
+        const int l = find_tensor(prefix, L, item);
+        const ThinLayerDesc &d = td[l];
+        const long long n0 = d.dims_out[0], n1 = d.dims_out[1];
+        const long long L_in = d.d1 * d.inner, L_out = n1 * d.inner;
+        const long long tiles_per_row = (L_in + 1023) / 1024;        // of the input row: the bound the host used
+        const long long local = item - prefix[l];
+        const long long io = local / tiles_per_row, c = local - io * tiles_per_row;
+        if (io >= n0 || c * 1024 >= L_out) continue;
+        const bool rm0 = d.use_keep0 != 0;
+        const long long ii = rm0 ? (long long)d.idx0[io] : io;
+        const float *s = d.src + ii * L_in;
+        float *o = d.dst + io * L_out;
+        const u32 inner32 = (u32)d.inner;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const u32 r = (u32)(c * 1024) + (u32)q * THREADS + threadIdx.x;
+            if (r < (u32)L_out) {
+                u32 sr = r;
+                if (d.keep1) {
+                    const u32 jo = r / inner32;
+                    sr = (u32)d.idx1[jo] * inner32 + (r - jo * inner32);
+                }
+                o[r] = __ldg(s + sr);
+            }
+        }
+    }
+}
+
 }  // namespace cs

@@ -30,7 +30,7 @@ EXPORTS = ["condensa_create", "condensa_destroy", "condensa_cstep_prune", "conde
            "condensa_cstep_prune_noalloc", "condensa_lstep_update",
            "condensa_cstep_structure", "condensa_thin_flags", "condensa_thin_compact",
            "condensa_count_nonzero", "condensa_set_seed", "condensa_noalloc_status",
-           "condensa_cstep_structured", "condensa_workspace_bytes"]
+           "condensa_cstep_structured", "condensa_workspace_bytes", "condensa_thin_list"]
 
 
 class CondensaError(RuntimeError):
@@ -66,6 +66,13 @@ class StructureSpec(C.Structure):
 
 SPEC_SLICES, SPEC_BLOCKS = 0, 1
 CRITERIA = {"l2": 0, "l1": 1, "max": 2}
+
+
+class ThinLayer(C.Structure):
+    """Mirror of ``condensa_thin_layer``."""
+    _fields_ = [("src", C.c_void_p), ("d0", C.c_int64), ("d1", C.c_int64), ("inner", C.c_int64),
+                ("keep0", C.c_void_p), ("remove_axis0", C.c_int32), ("keep1_from", C.c_int32),
+                ("dst", C.c_void_p), ("dims_out", C.c_void_p)]
 
 
 class OptTensor(C.Structure):
@@ -123,6 +130,7 @@ def load():
     L.condensa_thin_flags.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp]
     L.condensa_thin_compact.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp, vp]
     L.condensa_count_nonzero.argtypes = [vp, C.POINTER(vp), C.POINTER(i64), i32, vp, vp]
+    L.condensa_thin_list.argtypes = [vp, C.POINTER(ThinLayer), i32, vp]
     L.condensa_launch_count.argtypes = [vp]
     L.condensa_launch_count.restype = C.c_int64
     L.condensa_last_error.argtypes = [vp]
@@ -323,6 +331,16 @@ class Context:
         self._check(self._lib.condensa_thin_compact(self._h, _addr(src), int(d0), int(d1), int(inner),
                                                     _addr(keep0), _addr(keep1), _addr(dst), _addr(dims_out),
                                                     _stream_handle(stream)))
+
+    def thin_list(self, layers, stream=None):
+        """``layers``: dicts with src, d0, d1, inner, keep0, remove_axis0, keep1_from, dst, dims_out."""
+        n = len(layers)
+        tab = (ThinLayer * max(n, 1))()
+        for e, x in zip(tab, layers):
+            e.src, e.dst, e.keep0, e.dims_out = _addr(x["src"]), _addr(x["dst"]), _addr(x["keep0"]), _addr(x["dims_out"])
+            e.d0, e.d1, e.inner = int(x["d0"]), int(x["d1"]), int(x["inner"])
+            e.remove_axis0, e.keep1_from = int(bool(x.get("remove_axis0", True))), int(x.get("keep1_from", -1))
+        self._check(self._lib.condensa_thin_list(self._h, tab, n, _stream_handle(stream)))
 
     def count_nonzero(self, arrays, counts, stream=None):
         """``arrays``: device float32 tensors; ``counts``: device int64 tensor of len(arrays) + 1."""

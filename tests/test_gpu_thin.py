@@ -170,3 +170,103 @@ def test_thin_vgg_after_filter_pruning_full_size():
     torch.cuda.synchronize()
     assert np.array_equal(counts.cpu().numpy(), oracle.count_nonzero(exp.theta))
     ctx.close()
+
+
+def _list_case(shapes, chain, seed, off=0):
+    """Layers for ``Context.thin_list``: ``shapes`` are (d0, d1, inner); ``chain[l]`` is the
+    layer whose axis-0 flags remove layer l's axis-1 slices (-1: none)."""
+    import torch
+    host, layers, keep = [], [], []
+    for l, shp in enumerate(shapes):
+        x = _structured_zeros(shp, seed + l)
+        if chain[l] >= 0:
+            assert shapes[chain[l]][0] == shp[1]
+        host.append(x)
+        src, buf = _dev(x, off)
+        n = max(x.size, 1)
+        layers.append(dict(src=src if x.size else None, d0=shp[0], d1=shp[1], inner=shp[2],
+                           keep0=torch.full((max(shp[0], 1),), 7, dtype=torch.uint8, device="cuda:0"),
+                           remove_axis0=(l % 3 != 2), keep1_from=chain[l],
+                           dst=torch.full((n + off + 16,), float("nan"), dtype=torch.float32, device="cuda:0")[off:],
+                           dims_out=torch.full((2,), -1, dtype=torch.int64, device="cuda:0"), _buf=buf))
+    return host, layers
+
+
+def _check_list(host, layers):
+    import torch
+    torch.cuda.synchronize()
+    flags = [oracle.thin_flags(x, 0) for x in host]
+    for l, (x, lay) in enumerate(zip(host, layers)):
+        d0 = x.shape[0]
+        got_flags = lay["keep0"][:d0].cpu().numpy()
+        assert np.array_equal(got_flags, flags[l]), l
+        k0 = flags[l] if lay["remove_axis0"] else None
+        k1 = flags[lay["keep1_from"]] if lay["keep1_from"] >= 0 else None
+        exp = oracle.thin_compact(x, k0, k1)
+        n0, n1 = (int(v) for v in lay["dims_out"].cpu())
+        assert (n0, n1) == exp.shape[:2], (l, n0, n1, exp.shape)
+        got = lay["dst"][:exp.size].cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), exp.reshape(-1).view(np.uint32)), l
+        rest = lay["dst"][exp.size:max(x.size, 1)].cpu().numpy()
+        assert np.all(np.isnan(rest)), (l, "wrote past the compacted tensor")
+
+
+@pytest.mark.parametrize("off", [0, 1])
+def test_thin_list_matches_oracle(off):
+    from paper_1911_02497_b200 import cstep
+    ctx = cstep.Context(0)
+    # a conv chain, a classifier fed by the last conv layer, a bias, ragged and empty extents
+    shapes = [(37, 3, 9), (64, 37, 9), (130, 64, 25), (300, 130, 1), (300, 1, 1), (2100, 300, 1),
+              (5, 0, 3), (0, 5, 3), (1, 1, 1), (3, 4100, 3), (1500, 2100, 1)]
+    chain = [-1, 0, 1, 2, -1, 3, -1, -1, -1, -1, 5]
+    host, layers = _list_case(shapes, chain, seed=50 + off, off=off)
+    for _ in range(2):                       # a second call on the same context reuses the workspace
+        ctx.thin_list(layers)
+    _check_list(host, layers)
+    ctx.close()
+
+
+def test_thin_list_refuses_bad_arguments():
+    from paper_1911_02497_b200 import cstep
+    ctx = cstep.Context(0)
+    host, layers = _list_case([(8, 4, 2), (6, 7, 2)], [-1, -1], seed=3)
+    with pytest.raises(cstep.CondensaError):
+        ctx.thin_list([])
+    bad = [dict(l) for l in layers]
+    bad[1]["keep1_from"] = 0                  # layer 0 has 8 filters, layer 1 has 7 input channels
+    with pytest.raises(cstep.CondensaError):
+        ctx.thin_list(bad)
+    bad = [dict(l) for l in layers]
+    bad[0]["dst"] = bad[0]["src"]
+    with pytest.raises(cstep.CondensaError):
+        ctx.thin_list(bad)
+    ctx.thin_list(layers)                     # the context is still usable
+    _check_list(host, layers)
+    ctx.close()
+
+
+def test_thin_list_vgg_full_size_equals_per_layer_calls():
+    """Config 3 after filter pruning: the chain strategy over all conv layers in one call
+    equals the oracle layer by layer."""
+    import torch
+    from paper_1911_02497_b200 import cstep
+    from paper_1911_02497_b200.device_set import DeviceSet
+    ws = W.config("3")
+    ctx = cstep.Context(0)
+    ds = DeviceSet(ws.w, ws.lam, device="cuda:0")
+    ds.run(ctx, ws.op, ws.sparsity, ws.mu, ws.fuse, ws.block)
+    torch.cuda.synchronize()
+    exp = oracle.run_config(ws)
+    convs = [t for t in range(len(ws.w)) if len(ws.shapes[t]) == 4]
+    host, layers = [], []
+    for i, t in enumerate(convs):
+        Fo, Ci, kh, kw = ws.shapes[t]
+        host.append(exp.theta[t].reshape(Fo, Ci, kh * kw))
+        layers.append(dict(src=ds.theta[t], d0=Fo, d1=Ci, inner=kh * kw,
+                           keep0=torch.empty(Fo, dtype=torch.uint8, device="cuda:0"), remove_axis0=True,
+                           keep1_from=i - 1,
+                           dst=torch.full((Fo * Ci * kh * kw,), float("nan"), dtype=torch.float32, device="cuda:0"),
+                           dims_out=torch.zeros(2, dtype=torch.int64, device="cuda:0")))
+    ctx.thin_list(layers)
+    _check_list(host, layers)
+    ctx.close()
