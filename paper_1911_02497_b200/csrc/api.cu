@@ -293,7 +293,7 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, const HostSp
 
 constexpr int N_SAMPLE = SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD;
 constexpr int N_SAMPLE_BIG = SAMPLE_THREADS * SAMPLE_KEYS_PER_THREAD_BIG;
-constexpr long long SAMPLE_BIG_FROM = 1ll << 25;     // unstructured lists from this many units take the larger sample
+constexpr long long SAMPLE_BIG_FROM = 1ll << 26;     // unstructured lists from this many units take the larger sample
 constexpr int SAMPLE_CTAS = 64;
 constexpr long long ONE_LAUNCH_MAX_N = 4ll << 20;    // parameters of a list that the one-launch route takes
 
