@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcondensa_cstep.so")
 SOURCES = ["api.cu"]
-HEADERS = ["common.cuh", "elementwise.cuh", "select.cuh", "structured.cuh", "fused.cuh", "fused_fast.cuh",
+HEADERS = ["common.cuh", "elementwise.cuh", "select.cuh", "structured.cuh", "fused.cuh", "fused_fast.cuh", "fused_blockg.cuh",
            "sample.cuh", "lstep.cuh", "thin.cuh", "small_select.cuh", "small_prune.cuh",
            os.path.join("..", "..", "include", "condensa_cstep.h")]
 

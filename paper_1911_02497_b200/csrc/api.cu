@@ -20,6 +20,7 @@
 #include "structured.cuh"
 #include "fused.cuh"
 #include "fused_fast.cuh"
+#include "fused_blockg.cuh"
 #include "sample.cuh"
 #include "lstep.cuh"
 #include "thin.cuh"
@@ -64,12 +65,13 @@ struct condensa_ctx {
     cudaStream_t last_stream = nullptr;
     bool has_result = false;
     Ctl *ctl = nullptr;
-    int occ_select[3] = {0, 0, 0};
+    int occ_select[4] = {0, 0, 0, 0};
     int occ_stream = 0;
     int occ_filter = 0;
     int occ_prune_small = 0;        // resident CTAs per SM of the register-resident small-list kernel
     bool small_smem_set = false;    // dynamic shared memory limit of k_select_small raised on this device
     bool block_smem_set = false;    // the same for the tiled block kernel
+    size_t blockg_smem_set = 0;     // ... and for the tiled bh x bw kernel (bytes it has been allowed so far)
     DeviceMirror mirror;
     // optional per-kernel timing (event pair around every launch)
     bool prof_on = false;
@@ -122,6 +124,8 @@ struct Plan {
     u64 cap = 0;
     std::vector<long long> edge_items;           // projection items outside the aligned fast path
     std::vector<long long> tile_prefix;          // block pruning: warp tiles of the aligned interior per tensor
+    int bt_arr = 0, bt_stages = 0;               // tiled bh x bw kernel: bytes of one array in a tile buffer, buffers
+    int jr_floats = 0;                           // journal floats per listed unit
 };
 
 int validate(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s, float mu,
@@ -250,6 +254,24 @@ void build_plan(int op, const condensa_tensor *ts, int T, Plan &pl, const HostSp
                     d.nbc = d.nb[3];
                 }
                 items_a = (d.n_units + BLOCKS_PER_ITEM - 1) / BLOCKS_PER_ITEM;
+            }
+        } else if (op == OP_BLOCKG1) {
+            d.ranked = (x.ndim == 2 && x.numel > 0) ? 1 : 0;
+            if (d.ranked) {
+                d.nd = 2;
+                d.d0 = x.shape[0];
+                d.d1 = x.shape[1];
+                d.bh = (int)sp.bs[0];            // (not cut down to the shape: the kernels are built for bh x bw)
+                d.bw = (int)sp.bs[1];
+                d.nbc = (d.d1 + d.bw - 1) / d.bw;
+                d.n_units = ((d.d0 + d.bh - 1) / d.bh) * d.nbc;
+                // whole block rows go through shared memory by bulk copies: 16-byte rule for every row start
+                bool bok = (d.d1 % 4) == 0 && (aw % 16) == 0;
+                for (int i = 0; i < 2; ++i)
+                    if (f32p[i] % 16) bok = false;
+                d.blk_vec_ok = bok ? 1 : 0;
+                items_a = (d.n_units + BLOCKS_PER_ITEM - 1) / BLOCKS_PER_ITEM;
+                items_b = items_a;
             }
         } else if (op == OP_BLOCK) {
             d.ranked = (x.ndim == 2 && x.numel > 0) ? 1 : 0;
@@ -510,21 +532,90 @@ Sel initial_state(long long S, long long k, int bits_key)
     return s;
 }
 
+// Tile buffers of the tiled bh x bw kernel for this plan: three buffers if a block row of every
+// large matrix fits then, else two; false when even two do not hold the widest block row or a
+// large matrix is not aligned (the caller then takes the route over the norm array).
+constexpr size_t SMEM_OPTIN_BYTES = 232448;      // shared memory one CTA may have on this architecture
+bool blockg_ring_config(Plan &pl, int T)
+{
+    const size_t fixed = sizeof(BlockFastShared) + 1024 + (size_t)BT_CWARPS * blockg_cand_bytes(pl.jr_floats);
+    if (fixed >= SMEM_OPTIN_BYTES) return false;
+    int best_arr = 0, best_stages = 0;
+    long long best_chunked = -1;
+    for (int stages = BT_STAGES; stages >= 2; --stages) {
+        // stages * (2.25 * arr + 16) <= what is left
+        const size_t per = (SMEM_OPTIN_BYTES - fixed) / (size_t)stages;
+        if (per < 1024) continue;
+        long long arr = (long long)((per - 16) * 4 / 9);
+        arr -= arr % 64;
+        long long chunked = 0, tiled = 0;               // parameters in column chunks; units the tiles cover
+        for (int t = 0; t < T; ++t) {
+            const TensorDesc &d = pl.td[t];
+            if (!d.ranked) continue;
+            const long long fe = blockg_fast_end(d, (int)arr);
+            tiled += fe;
+            if (fe > 0 && (long long)d.bh * d.d1 * 4 > arr) chunked += d.numel;
+        }
+        if (2 * tiled < pl.S) continue;                 // mostly unaligned matrices: the generic code would do the work
+        if (best_chunked < 0 || chunked < best_chunked) {      // whole block rows beat a deeper ring
+            best_chunked = chunked;
+            best_arr = (int)arr;
+            best_stages = stages;
+        }
+    }
+    if (best_chunked < 0) return false;
+    pl.bt_arr = best_arr;
+    pl.bt_stages = best_stages;
+    return true;
+}
+
+// May this structured call take the single-pass kernels for bh x bw blocks?
+// Block shapes the tiled bh x bw kernel is built for (the per-block code is unrolled at compile
+// time; 5 x 5 is the block size of the paper's LSTM experiment). Other shapes take the route
+// over the norm array.
+#define CS_BLOCKG_SHAPES(X) X(5, 5) X(3, 3) X(2, 2) X(1, 8) X(8, 1)
+bool blockg_shape_built(long long bh, long long bw)
+{
+#define CS_X(BH, BW) if (bh == BH && bw == BW) return true;
+    CS_BLOCKG_SHAPES(CS_X)
+#undef CS_X
+    return false;
+}
+
+bool blockg_single_pass_candidate(int op, const HostSpec &sp, unsigned fuse)
+{
+    return op == OP_BLOCKGEN && sp.nd == 2 && sp.crit == CRIT_L2 && blockg_shape_built(sp.bs[0], sp.bs[1]) &&
+           !(fuse & CONDENSA_NO_SAMPLING);
+}
+
 // Work decomposition and workspace layout of one call (no device work).
 Layout plan_call(int op, const condensa_tensor *ts, int T, unsigned fuse, const HostSpec &sp, Plan &pl,
                  bool &ranking, bool &sampling, long long small_items_max = 0, bool *small_prune = nullptr)
 {
     build_plan(op, ts, T, pl, sp);
-    ranking = op <= OP_BLOCK || op == OP_BLOCKGEN;
+    ranking = op <= OP_BLOCK || op == OP_BLOCKGEN || op == OP_BLOCKG1;
     // single-pass path: unstructured and block pruning of lists too large to list whole
     // an unstructured list of at most one work item per resident CTA stays in registers for the whole call
     const bool reg_resident = op == OP_PRUNE && pl.n_items_b > 0 && pl.n_items_b <= small_items_max;
     if (small_prune) *small_prune = reg_resident;
-    sampling = (op == OP_PRUNE || op == OP_BLOCK) && !(fuse & CONDENSA_NO_SAMPLING) && !reg_resident &&
+    sampling = (op == OP_PRUNE || op == OP_BLOCK || op == OP_BLOCKG1) && !(fuse & CONDENSA_NO_SAMPLING) && !reg_resident &&
                           (u64)pl.S > pl.cap && pl.S >= 8ll * N_SAMPLE;
     if (sampling && op == OP_BLOCK && pl.cap > (1ull << 20)) pl.cap = 1ull << 20;   // bounds the journal
-    const int journal_floats = sampling ? (op == OP_BLOCK ? 16 : 1) : 0;
-    if (sampling) {
+    if (op == OP_BLOCKG1) {
+        pl.jr_floats = (int)(sp.bs[0] * sp.bs[1]);
+        const u64 cap_j = (16ull << 20) / (u64)pl.jr_floats;                        // journal of at most 64 MB
+        if (sampling && pl.cap > cap_j) pl.cap = cap_j;
+        sampling = sampling && (u64)pl.S > pl.cap && blockg_ring_config(pl, T);
+    }
+    const int journal_floats = sampling ? (op == OP_BLOCK ? 16 : op == OP_BLOCKG1 ? pl.jr_floats : 1) : 0;
+    if (sampling && op == OP_BLOCKG1) {
+        pl.tile_prefix.assign((size_t)T + 1, 0);
+        for (int t = 0; t < T; ++t) {
+            for (long long j = 0; j < pl.prefix_b[t + 1] - pl.prefix_b[t]; ++j)
+                if (!blockg_item_is_fast(pl.td[t], j, pl.bt_arr)) pl.edge_items.push_back(pl.prefix_b[t] + j);
+            pl.tile_prefix[t + 1] = pl.tile_prefix[t] + blockg_tile_count(pl.td[t], pl.bt_arr);
+        }
+    } else if (sampling) {
         for (int t = 0; t < T; ++t)
             for (long long j = 0; j < pl.prefix_b[t + 1] - pl.prefix_b[t]; ++j) {
                 const bool fast = op == OP_BLOCK ? block_item_is_fast(pl.td[t], j) : elem_item_is_fast(pl.td[t], j);
@@ -557,7 +648,21 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     bool ranking = false, sampling = false, small_prune = false;
     if (op == OP_PRUNE && !ctx->occ_prune_small) ctx->occ_prune_small = occupancy(k_prune_small);
     const long long small_items_max = (op == OP_PRUNE && ctx->occ_prune_small >= 2) ? 2ll * ctx->num_sms : 0;
-    const Layout L = plan_call(op, ts, T, fuse, sp, pl, ranking, sampling, small_items_max, &small_prune);
+    Layout L;
+    bool planned = false;
+    if (blockg_single_pass_candidate(op, sp, fuse)) {
+        // bh x bw blocks of matrices by the L2 norm: the single-pass kernels, when the list is long
+        // enough for a sample, at least one unit is kept and a block row fits the tile buffers
+        L = plan_call(OP_BLOCKG1, ts, T, fuse, sp, pl, ranking, sampling, 0, nullptr);
+        const long long Z = (long long)std::min<double>((double)pl.S, std::max(0.0, std::floor(sparsity * (double)pl.S + 0.5)));
+        if (sampling && pl.S - Z > 0) {
+            op = OP_BLOCKG1;
+            planned = true;
+        } else {
+            pl = Plan();
+        }
+    }
+    if (!planned) L = plan_call(op, ts, T, fuse, sp, pl, ranking, sampling, small_items_max, &small_prune);
     rc = ensure_workspace(ctx, L.total, stream);
     if (rc) return rc;
     char *ws = ctx->ws;
@@ -596,6 +701,9 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     const bool big_sample = op == OP_PRUNE && pl.S >= SAMPLE_BIG_FROM;
     P.n_sample = big_sample ? N_SAMPLE_BIG : N_SAMPLE;
     P.jr_lam = (float *)(ws + L.journal);
+    P.jr_floats = op == OP_BLOCKG1 ? pl.jr_floats : op == OP_BLOCK ? 16 : 1;
+    P.bt_arr_bytes = pl.bt_arr;
+    P.bt_stages = pl.bt_stages;
     P.onepass_cap = pl.cap;
     P.crit = sp.crit;
     P.seed = ctx->seed;
@@ -677,14 +785,27 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             int pi_ = prof_begin(ctx, "k_sample", stream);
             if (op == OP_PRUNE && big_sample) k_sample<SRC_ELEM, SAMPLE_KEYS_PER_THREAD_BIG><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
             else if (op == OP_PRUNE) k_sample<SRC_ELEM, SAMPLE_KEYS_PER_THREAD><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
+            else if (op == OP_BLOCKG1) k_sample<SRC_BLOCKG, SAMPLE_KEYS_PER_THREAD><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
             else k_sample<SRC_BLOCK, SAMPLE_KEYS_PER_THREAD><<<SAMPLE_CTAS, SAMPLE_THREADS, 0, stream>>>(Pa, init);
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
-            pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : "k_fused_block", stream);
+            pi_ = prof_begin(ctx, op == OP_PRUNE ? "k_fused_elem" : op == OP_BLOCKG1 ? "k_fused_blockg" : "k_fused_block", stream);
             // block pruning: one CTA per WARPS warp tiles at least, and enough CTAs for the edge items
-            const long long work = op == OP_BLOCK ? std::max<long long>(Pf.n_tiles, (long long)pl.edge_items.size())
-                                                  : pl.n_items_b;
-            const int gridf = stream_grid(ctx, work, op == OP_BLOCK ? 1 : 3);
+            const bool tiled = op == OP_BLOCK || op == OP_BLOCKG1;
+            const long long work = tiled ? std::max<long long>(Pf.n_tiles, (long long)pl.edge_items.size()) : pl.n_items_b;
+            const int gridf = stream_grid(ctx, work, tiled ? 1 : 3);
+            const size_t dyn_g = op == OP_BLOCKG1 ? blockg_dyn_smem(pl.bt_arr, pl.bt_stages, pl.jr_floats) : 0;
+            if (op == OP_BLOCKG1 && dyn_g > ctx->blockg_smem_set) {
+                const int dyn = (int)dyn_g;
+#define CS_X(BH, BW)                                                                                                          \
+    CU_TRY(ctx, cudaFuncSetAttribute(k_fused_blockg<true, true, BH, BW>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));   \
+    CU_TRY(ctx, cudaFuncSetAttribute(k_fused_blockg<true, false, BH, BW>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));  \
+    CU_TRY(ctx, cudaFuncSetAttribute(k_fused_blockg<false, true, BH, BW>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));  \
+    CU_TRY(ctx, cudaFuncSetAttribute(k_fused_blockg<false, false, BH, BW>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+                CS_BLOCKG_SHAPES(CS_X)
+#undef CS_X
+                ctx->blockg_smem_set = dyn_g;
+            }
             const bool need_g = (fuse & CONDENSA_FUSE_PENALTY) != 0;
             if (op == OP_BLOCK && !ctx->block_smem_set) {
                 const int dyn = (int)BLOCK_FAST_DYN_SMEM;
@@ -704,7 +825,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             pdl.val.programmaticStreamSerializationAllowed = 1;
             cfg.gridDim = dim3((unsigned)gridf);
             cfg.blockDim = dim3((unsigned)(op == OP_PRUNE ? THREADS : BT_THREADS));
-            cfg.dynamicSmemBytes = op == OP_PRUNE ? 0 : BLOCK_FAST_DYN_SMEM;
+            cfg.dynamicSmemBytes = op == OP_PRUNE ? 0 : op == OP_BLOCKG1 ? dyn_g : BLOCK_FAST_DYN_SMEM;
             cfg.stream = stream;
             cfg.attrs = &pdl;
             cfg.numAttrs = ctx->prof_on ? 0 : 1;       // with an event pair around every kernel there is nothing to overlap
@@ -716,7 +837,17 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         else CU_TRY(ctx, cudaLaunchKernelEx(&cfg, KERNEL<false, false>, Pf));                  \
     } while (0)
             if (op == OP_PRUNE) CS_LAUNCH_FUSED(k_fused_elem);
-            else CS_LAUNCH_FUSED(k_fused_block);
+            else if (op == OP_BLOCKG1) {
+#define CS_X(BH, BW)                                                                                            \
+    if (sp.bs[0] == BH && sp.bs[1] == BW) {                                                                     \
+        if (need_h && need_g) CU_TRY(ctx, cudaLaunchKernelEx(&cfg, k_fused_blockg<true, true, BH, BW>, Pf));    \
+        else if (need_h) CU_TRY(ctx, cudaLaunchKernelEx(&cfg, k_fused_blockg<true, false, BH, BW>, Pf));        \
+        else if (need_g) CU_TRY(ctx, cudaLaunchKernelEx(&cfg, k_fused_blockg<false, true, BH, BW>, Pf));        \
+        else CU_TRY(ctx, cudaLaunchKernelEx(&cfg, k_fused_blockg<false, false, BH, BW>, Pf));                   \
+    }
+                CS_BLOCKG_SHAPES(CS_X)
+#undef CS_X
+            } else CS_LAUNCH_FUSED(k_fused_block);
 #undef CS_LAUNCH_FUSED
             LAUNCH_CHECK(ctx);
             prof_end(ctx, pi_, stream);
@@ -763,6 +894,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
         if (small) rc = CONDENSA_OK;
         else if (op == OP_PRUNE) rc = launch_select<SRC_ELEM>(ctx, Pa, do_list0, pre_scan, stream, pb, pl.n_items_b, post_apply, init_p);
         else if (op == OP_BLOCK) rc = launch_select<SRC_BLOCK>(ctx, Pa, do_list0, pre_scan, stream, pb, pl.n_items_b, post_apply, init_p);
+        else if (op == OP_BLOCKG1) rc = launch_select<SRC_BLOCKG>(ctx, Pa, do_list0, pre_scan, stream, pb, pl.n_items_b, post_apply, init_p);
         else rc = launch_select<SRC_ARRAY>(ctx, Pa, do_list0, 0, stream);
         if (rc) return rc;
         ctx->has_result = true;
@@ -773,7 +905,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
     Pb.n_items = pl.n_items_b;
     if (pl.n_items_b > 0 && !applied_in_select) {
         const int grid = stream_grid(ctx, pl.n_items_b, ctx->occ_stream);
-        static const char *apply_names[6] = {"k_apply_prune", "k_apply_filter", "k_apply_block", "k_quantize", "k_lagrange", "k_apply_blockgen"};
+        static const char *apply_names[7] = {"k_apply_prune", "k_apply_filter", "k_apply_block", "k_quantize", "k_lagrange", "k_apply_blockgen", "k_apply_blockgen"};
         const int pa_ = prof_begin(ctx, apply_names[op], stream);
         switch (op) {
         case OP_PRUNE:
@@ -899,7 +1031,13 @@ int condensa_workspace_bytes(int op, const condensa_tensor *tensors, int T, cons
     Plan pl;
     bool ranking = false, sampling = false;
     const Layout L = plan_call(iop, tensors, T, fuse, sp, pl, ranking, sampling);
-    *bytes = align_up(L.total + L.total / 4, 1 << 20);      // what a call of this shape makes the context hold
+    size_t total = L.total;
+    if (blockg_single_pass_candidate(iop, sp, fuse)) {      // the call may take the single-pass kernels instead
+        Plan pg;
+        const Layout Lg = plan_call(OP_BLOCKG1, tensors, T, fuse, sp, pg, ranking, sampling);
+        if (sampling) total = std::max(total, Lg.total);
+    }
+    *bytes = align_up(total + total / 4, 1 << 20);      // what a call of this shape makes the context hold
     return CONDENSA_OK;
 }
 

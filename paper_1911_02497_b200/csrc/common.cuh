@@ -23,11 +23,12 @@ constexpr int WSTG = 256;                // staged list entries per warp
 constexpr int MAX_SELECT_ITERS = 24;
 constexpr u64 KEY_NONE = ~0ull;          // cut-off key that keeps nothing
 
-enum { OP_PRUNE = 0, OP_FILTER = 1, OP_BLOCK = 2, OP_QUANTIZE = 3, OP_LAGRANGE = 4, OP_BLOCKGEN = 5 };
+enum { OP_PRUNE = 0, OP_FILTER = 1, OP_BLOCK = 2, OP_QUANTIZE = 3, OP_LAGRANGE = 4, OP_BLOCKGEN = 5,
+       OP_BLOCKG1 = 6 };      // OP_BLOCKG1: bh x bw blocks of matrices by the single-pass kernels
 enum { FUSE_FP16 = 1, FUSE_LAMBDA = 2, FUSE_PENALTY = 4, FUSE_BF16 = 8, FUSE_E4M3 = 16, FUSE_E5M2 = 32, NO_SAMPLING = 64 };
 constexpr unsigned FUSE_QUANT = FUSE_FP16 | FUSE_BF16 | FUSE_E4M3 | FUSE_E5M2;
 constexpr unsigned FUSE_KERNEL_BITS = 63u;      // the fuse bits the kernels see
-enum { SRC_ELEM = 0, SRC_BLOCK = 1, SRC_ARRAY = 2 };
+enum { SRC_ELEM = 0, SRC_BLOCK = 1, SRC_ARRAY = 2, SRC_BLOCKG = 3 };    // SRC_BLOCKG: bh x bw blocks of matrices
 enum { CRIT_L2 = 0, CRIT_L1 = 1, CRIT_MAX = 2 };
 
 // One tensor of the list as the kernels see it.
@@ -134,6 +135,9 @@ struct Params {
     int miss_fallback;              // a missed sample bracket may be repaired by the two-pass route inside the
                                     // same call: nothing the first pass wrote is needed again (no multiplier
                                     // is updated in place)
+    int jr_floats;                  // journal floats per listed unit (1, 16, or bh * bw of the call)
+    int bt_arr_bytes;               // tiled bh x bw kernel: bytes of w (or lambda) one tile buffer holds ...
+    int bt_stages;                  // ... and the number of tile buffers
 };
 
 // Which projection work items the fast single-pass kernels take (host and device
@@ -155,6 +159,34 @@ __host__ __device__ inline long long block_fast_end(const TensorDesc &d)
 __host__ __device__ inline bool block_item_is_fast(const TensorDesc &d, long long local)
 {
     return d.ranked && (local + 1) * BLOCKS_PER_ITEM <= block_fast_end(d);
+}
+
+// The same for bh x bw blocks: complete block rows of an aligned matrix. A tile buffer of
+// `arr_bytes` bytes per array takes whole block rows when one fits, else a column chunk of one
+// block row: a multiple of bw and of 4 columns (blockg_chunk_cols; 0 = not even one fits).
+__host__ __device__ inline long long blockg_chunk_cols(const TensorDesc &d, int arr_bytes)
+{
+    long long a = d.bw, b = 4;
+    while (b) { const long long r = a % b; a = b; b = r; }       // a = gcd(bw, 4)
+    const long long step = (long long)d.bw * 4 / a;                // lcm(bw, 4)
+    const long long room = ((long long)arr_bytes - 64ll * d.bh) / (4ll * d.bh);
+    if (room < step) return 0;
+    const long long most = room - room % step;                     // widest chunk that fits
+    const long long cpr = (d.d1 + most - 1) / most;                // chunks per block row
+    const long long even = ((d.d1 + cpr - 1) / cpr + step - 1) / step * step;      // ... of about equal width
+    return even < most ? even : most;
+}
+
+__host__ __device__ inline long long blockg_fast_end(const TensorDesc &d, int arr_bytes)
+{
+    if (!d.ranked || !d.blk_vec_ok || d.numel >= 0xFFFFFFFFll) return 0;
+    if ((long long)d.bh * d.d1 * 4 > (long long)arr_bytes && blockg_chunk_cols(d, arr_bytes) == 0) return 0;
+    return (d.d0 / d.bh) * d.nbc;
+}
+
+__host__ __device__ inline bool blockg_item_is_fast(const TensorDesc &d, long long local, int arr_bytes)
+{
+    return d.ranked && (local + 1) * BLOCKS_PER_ITEM <= blockg_fast_end(d, arr_bytes);
 }
 
 // ---------------------------------------------------------------- arithmetic

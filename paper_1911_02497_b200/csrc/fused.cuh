@@ -302,6 +302,12 @@ __device__ __noinline__ void repair_unit(const Params &P, u64 idx, u64 id, bool 
         if ((u64)pre <= id) lo = mid; else hi = mid - 1;
     }
     const TensorDesc &d = tdc ? tdc[lo] : P.td[lo];
+    if (SRC == SRC_BLOCKG) {                    // rows part, part + 8, ... of a bh x bw block
+        const long long b = (long long)id - d.unit_prefix;
+        if (b < 0 || b >= d.n_units) return;
+        blockg_write_global(P, d, b, keep, P.jr_lam + idx * (u64)P.jr_floats, part, (int)RepairLanes<SRC_BLOCKG>::value);
+        return;
+    }
     const bool has_lam = d.lam != nullptr;
     const bool wr_lam = (P.fuse & FUSE_LAMBDA) && has_lam;
     const bool wr_grad = (P.fuse & FUSE_PENALTY) && d.grad != nullptr;

@@ -1,0 +1,464 @@
+// Single-pass projection for bh x bw blocks of matrices (any block shape but 4 x 4, which has
+// its own kernel): the sample bracket, one pass that writes everything, the exact selection
+// on the listed candidates. A block row - bh matrix rows - is one contiguous range of memory,
+// so the pass moves whole block rows through shared memory exactly like the 4 x 4 kernel
+// does; only the per-block arithmetic differs (runtime loops over the rows and columns of a
+// block that exist, in row-major order: the order of the plain definition).
+#pragma once
+#include "fused_fast.cuh"
+
+namespace cs {
+
+// Shared memory of a CTA: `stages` tile buffers (w, lambda: `arr` bytes each; mask: arr / 4 + 16
+// bytes, the tile's mask starts at the byte offset its global address has inside a 16-byte line,
+// so that the aligned interior can leave by one bulk copy), then the candidate staging of each
+// consumer warp (BSTG keys, BSTG ids, BSTG x jr_floats original multipliers).
+__host__ __device__ inline size_t blockg_stage_bytes(int arr) { return (size_t)arr * 2 + (size_t)arr / 4 + 16; }
+__host__ __device__ inline size_t blockg_cand_bytes(int jr_floats) { return (size_t)BSTG * (16 + 4 * (size_t)jr_floats); }
+__host__ __device__ inline size_t blockg_dyn_smem(int arr, int stages, int jr_floats)
+{
+    return (size_t)stages * blockg_stage_bytes(arr) + (size_t)BT_CWARPS * blockg_cand_bytes(jr_floats);
+}
+
+// Tiles of the aligned interior of tensor d: as many complete block rows as fit a buffer, or,
+// for a matrix too wide for that, column chunks of one block row.
+__host__ __device__ inline long long blockg_tile_count(const TensorDesc &d, int arr)
+{
+    if (blockg_fast_end(d, arr) <= 0) return 0;
+    const long long nbr = d.d0 / d.bh;
+    const long long row_bytes = (long long)d.bh * d.d1 * 4;
+    if (row_bytes <= arr) {
+        const long long rpt = (long long)arr / row_bytes;
+        return (nbr + rpt - 1) / rpt;
+    }
+    const long long cc = blockg_chunk_cols(d, arr);
+    return nbr * ((d.d1 + cc - 1) / cc);
+}
+
+struct TileG {
+    int t;              // owning tensor
+    u32 b0;             // first block (number inside the tensor); block q of the tile is b0 + q
+    u32 nq;             // blocks in the tile
+    u32 nbpr;           // blocks per row piece
+    u32 nrows;          // matrix rows in the tile
+    u32 cols;           // columns of a row piece (= its pitch in shared memory)
+    u32 c_start;        // first column
+    u32 off0;           // element offset of the first row piece
+    bool whole;         // whole block rows: one contiguous range
+};
+
+__device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const TensorDesc *td, int T, long long tile, int arr)
+{
+    TileG g;
+    g.t = find_tensor(tile_prefix, T, tile);
+    const TensorDesc &d = td[g.t];
+    const u32 bh = (u32)d.bh, bw = (u32)d.bw, C = (u32)d.d1, nbc = (u32)d.nbc, nbr = (u32)(d.d0 / d.bh);
+    const u32 local = (u32)(tile - tile_prefix[g.t]);
+    g.whole = (long long)bh * C * 4 <= (long long)arr;
+    if (g.whole) {
+        const u32 rpt = (u32)arr / (bh * C * 4u);
+        const u32 brow0 = local * rpt;
+        const u32 brows = nbr - brow0 < rpt ? nbr - brow0 : rpt;
+        g.nbpr = nbc;
+        g.nq = brows * nbc;
+        g.nrows = bh * brows;
+        g.cols = C;
+        g.c_start = 0;
+        g.b0 = brow0 * nbc;
+        g.off0 = bh * brow0 * C;
+    } else {
+        const u32 cc = (u32)blockg_chunk_cols(d, arr);
+        const u32 cpr = (C + cc - 1) / cc;
+        const u32 brow = local / cpr, chunk = local - brow * cpr;
+        g.c_start = chunk * cc;
+        g.cols = C - g.c_start < cc ? C - g.c_start : cc;
+        g.nbpr = (g.cols + bw - 1) / bw;
+        g.nq = g.nbpr;
+        g.nrows = bh;
+        g.b0 = brow * nbc + g.c_start / bw;
+        g.off0 = bh * brow * C + g.c_start;
+    }
+    return g;
+}
+
+// Appends the candidates a consumer warp has staged to the list (one global atomic per flush).
+__device__ __forceinline__ void blockg_flush(const Params &P, u32 *wcount, const u64 *ckey, const u64 *cid, const float *clam,
+                                             u32 limit)
+{
+    const int lane = threadIdx.x & 31;
+    __syncwarp();
+    const u32 c = *wcount;
+    if (c > limit) {
+        u64 base = 0;
+        if (lane == 0) base = atomicAdd(&P.ctl->list_count[0], (u64)c);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        for (u32 i = lane; i < c; i += 32) {
+            const u64 pos = base + i;
+            if (pos < P.cap) {
+                P.list_key[pos] = ckey[i];
+                P.list_id[pos] = cid[i];
+            }
+        }
+        const u32 J = (u32)P.jr_floats;
+        for (u32 i = lane; i < c * J; i += 32) {
+            const u64 pos = base + i / J;
+            if (pos < P.cap) P.jr_lam[pos * J + (i % J)] = clam[i];
+        }
+        __syncwarp();
+        if (lane == 0) *wcount = 0;
+    }
+    __syncwarp();
+}
+
+// One block of a tile in shared memory: norm, decision, outputs in place. BH x BW (when not 0)
+// is the block shape at compile time: blocks of full width then run without loops or address
+// arithmetic, with u kept in registers between the norm and the outputs.
+struct BlockJob {
+    u32 nc, bh, bw, pitch, C;       // columns that exist; block shape; row pitch in shared memory and in the tensor
+    u32 base, gbase;                // element offset of the block in the tile buffer / in the tensor
+    u64 id;
+    float *sw, *sl;
+    unsigned char *sm;
+    bool mstage, has_lam, upd;
+};
+
+template <bool H, bool G, int BH, int BW>
+__device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, const BlockJob &jb, const Bracket &br,
+                                          float mu, int fp16, BlockFastShared &sh, int cw, u64 *ckey, u64 *cid, float *clam)
+{
+    const u32 J = (u32)P.jr_floats;
+    if (BH > 0 && jb.nc == (u32)BW) {
+        constexpr int N = BH > 0 ? BH * BW : 1;
+        float w[N], l[N], u[N];
+        u32 nz = 0;
+#pragma unroll
+        for (int r = 0; r < (BH > 0 ? BH : 1); ++r)
+#pragma unroll
+            for (int c = 0; c < (BW > 0 ? BW : 1); ++c) {
+                const u32 o = jb.base + r * jb.pitch + c;
+                w[r * BW + c] = jb.sw[o];
+                l[r * BW + c] = jb.has_lam ? jb.sl[o] : 0.0f;
+                nz |= __float_as_uint(l[r * BW + c]);
+            }
+        if (nz) {
+#pragma unroll
+            for (int i = 0; i < N; ++i) u[i] = form_u(w[i], l[i], mu, true);
+        } else {                        // every lambda is +0: u is w, bit for bit
+#pragma unroll
+            for (int i = 0; i < N; ++i) u[i] = w[i];
+        }
+        double acc = 0.0;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const double x = (double)u[i];
+            acc = __fma_rn(x, x, acc);
+        }
+        const u64 key = (u64)__double_as_longlong(acc);
+        const bool keep = key >= br.guess;
+        if (key >= br.lo && key <= br.hi) {
+            const u32 slot = atomicAdd(&sh.wcount[cw], 1u);
+            ckey[slot] = key;
+            cid[slot] = jb.id;
+#pragma unroll
+            for (int i = 0; i < N; ++i) clam[slot * J + i] = l[i];
+            atomicAdd(&sh.hist[bracket_bin(br, key, jb.id)], 1u);
+        }
+#pragma unroll
+        for (int r = 0; r < (BH > 0 ? BH : 1); ++r)
+#pragma unroll
+            for (int c = 0; c < (BW > 0 ? BW : 1); ++c) {
+                const int i = r * BW + c;
+                const u32 o = jb.base + r * jb.pitch + c, go = jb.gbase + r * jb.C + c;
+                const Out out = finish_lean<H>(w[i], l[i], u[i], keep, mu, fp16, jb.upd);
+                jb.sw[o] = out.theta;
+                if (jb.upd) jb.sl[o] = out.lam;
+                if (jb.mstage) jb.sm[o] = out.m;
+                else if (d.mask) d.mask[go] = out.m;
+                if (H && d.theta_h) d.theta_h[go] = out.th;
+                if (G && d.grad) d.grad[go] = out.grad;
+            }
+        return key > br.hi ? 1u : 0u;
+    }
+    // any shape, ragged width: loops over the rows and the columns that exist
+    double acc = 0.0;
+    for (u32 r = 0; r < jb.bh; ++r)
+        for (u32 c = 0; c < jb.nc; ++c) {
+            const u32 o = jb.base + r * jb.pitch + c;
+            const double x = (double)form_u(jb.sw[o], jb.has_lam ? jb.sl[o] : 0.0f, mu, jb.has_lam);
+            acc = __fma_rn(x, x, acc);
+        }
+    const u64 key = (u64)__double_as_longlong(acc);
+    const bool keep = key >= br.guess;
+    if (key >= br.lo && key <= br.hi) {
+        const u32 slot = atomicAdd(&sh.wcount[cw], 1u);
+        ckey[slot] = key;
+        cid[slot] = jb.id;
+        for (u32 r = 0; r < jb.bh; ++r)
+            for (u32 c = 0; c < jb.nc; ++c)
+                clam[slot * J + r * jb.bw + c] = jb.has_lam ? jb.sl[jb.base + r * jb.pitch + c] : 0.0f;
+        atomicAdd(&sh.hist[bracket_bin(br, key, jb.id)], 1u);
+    }
+    for (u32 r = 0; r < jb.bh; ++r)
+        for (u32 c = 0; c < jb.nc; ++c) {
+            const u32 o = jb.base + r * jb.pitch + c, go = jb.gbase + r * jb.C + c;
+            const float w = jb.sw[o], l = jb.has_lam ? jb.sl[o] : 0.0f;
+            const Out out = finish_lean<H>(w, l, form_u(w, l, mu, jb.has_lam), keep, mu, fp16, jb.upd);
+            jb.sw[o] = out.theta;
+            if (jb.upd) jb.sl[o] = out.lam;
+            if (jb.mstage) jb.sm[o] = out.m;
+            else if (d.mask) d.mask[go] = out.m;
+            if (H && d.theta_h) d.theta_h[go] = out.th;
+            if (G && d.grad) d.grad[go] = out.grad;
+        }
+    return key > br.hi ? 1u : 0u;
+}
+
+template <bool H, bool G, int BH, int BW>
+__global__ void __launch_bounds__(BT_THREADS, 1) k_fused_blockg(Params P)
+{
+    __shared__ BlockFastShared sh;
+    extern __shared__ __align__(128) unsigned char dyn_smem[];      // tile buffers, then the candidate staging
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int arr = P.bt_arr_bytes, n_stages = P.bt_stages;
+    const size_t stage_bytes = blockg_stage_bytes(arr);
+    unsigned char *tile_buf = dyn_smem;
+    unsigned char *cand_buf = dyn_smem + (size_t)n_stages * stage_bytes;
+    for (int i = threadIdx.x; i < NBINS; i += BT_THREADS) sh.hist[i] = 0;
+    if (threadIdx.x < BT_CWARPS) sh.wcount[threadIdx.x] = 0;
+    if (threadIdx.x == 0) sh.abort = 0;
+    const bool cached = P.T <= BT_TD_CACHE;
+    if (cached) {
+        for (int i = threadIdx.x; i <= P.T; i += BT_THREADS) sh.tile_prefix[i] = P.tile_prefix[i];
+        const int words = P.T * (int)(sizeof(TensorDesc) / sizeof(u32));
+        const u32 *src = reinterpret_cast<const u32 *>(P.td);
+        u32 *dst = reinterpret_cast<u32 *>(sh.td);
+        for (int i = threadIdx.x; i < words; i += BT_THREADS) dst[i] = src[i];
+    }
+    if (threadIdx.x < n_stages) {
+        mbar_init(smem_u32(&sh.full_bar[threadIdx.x]), 1);
+        mbar_init(smem_u32(&sh.done_bar[threadIdx.x]), BT_CWARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    const long long *tile_prefix = cached ? sh.tile_prefix : P.tile_prefix;
+    const TensorDesc *td = cached ? sh.td : P.td;
+    const int fp16 = quant_code(P.fuse);
+    const float mu = P.mu;
+    volatile int *abort_flag = &sh.abort;
+    u64 na = 0;
+    Bracket br;
+    memset(&br, 0, sizeof(br));
+    bool onepass = false;
+    if (warp < BT_CWARPS) {
+        pdl_wait();
+        onepass = P.ctl->sel.onepass != 0;      // else the sampler advised against the single pass
+        br = load_bracket(P.ctl->sel);
+    }
+    const u32 S_ = (u32)n_stages;
+
+    if (warp == BT_CWARPS) {
+        // ------------------------------------------------------------ producer (one lane)
+        if (lane == 0) {
+            u32 k = 0;
+            bool ok = true, dep_seen = false, quiet = false;
+            auto see_dependency = [&]() {       // before the first store and before leaving
+                if (dep_seen) return;
+                pdl_wait();
+                dep_seen = true;
+                if (!P.ctl->sel.onepass) { quiet = true; ok = false; }
+            };
+            auto store_tile = [&](long long tile, int stage) {
+                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
+                const TensorDesc &d = td[g.t];
+                const bool upd = (P.fuse & FUSE_LAMBDA) && d.lam != nullptr;
+                const u32 C = (u32)d.d1, pitch = g.cols * 4u, bytes = g.nrows * pitch;
+                unsigned char *sbp = tile_buf + (size_t)stage * stage_bytes;
+                const u32 sb = smem_u32(sbp);
+                if (!g.whole) {                 // one copy per matrix row; the consumers have written the mask themselves
+                    for (u32 r = 0; r < g.nrows; ++r) {
+                        bulk_store_1d(d.theta + g.off0 + r * C, sb + r * pitch, pitch);
+                        if (upd) bulk_store_1d(d.lam + g.off0 + r * C, sb + (u32)arr + r * pitch, pitch);
+                    }
+                    bulk_commit();
+                    return;
+                }
+                bulk_store_1d(d.theta + g.off0, sb, bytes);
+                if (upd) bulk_store_1d(d.lam + g.off0, sb + (u32)arr, bytes);
+                if (d.mask && ((uintptr_t)d.mask & 15u) == 0) {
+                    // the 16-byte aligned interior of the tile's mask by one bulk copy, the ragged ends byte by byte
+                    const u32 n = bytes / 4u, m0 = g.off0, m1 = g.off0 + n;
+                    const u32 a = (m0 + 15u) & ~15u, e = m1 & ~15u;
+                    const unsigned char *smk = sbp + 2 * (size_t)arr + (m0 & 15u);     // mask byte of element m0
+                    if (e > a) {
+                        bulk_store_1d(d.mask + a, sb + 2u * (u32)arr + (m0 & 15u) + (a - m0), e - a);
+                        for (u32 i = m0; i < a; ++i) d.mask[i] = smk[i - m0];
+                        for (u32 i = e; i < m1; ++i) d.mask[i] = smk[i - m0];
+                    } else {
+                        for (u32 i = m0; i < m1; ++i) d.mask[i] = smk[i - m0];
+                    }
+                }
+                bulk_commit();
+            };
+            long long tile = blockIdx.x;
+#pragma unroll 1
+            for (; tile < P.n_tiles && ok; tile += gridDim.x, ++k) {
+                const int stage = (int)(k % S_);
+                if (k >= S_) {
+                    see_dependency();
+                    if (!ok) break;
+                    ok = mbar_wait_bounded(smem_u32(&sh.done_bar[stage]), ((k / S_) - 1u) & 1u, abort_flag);
+                    if (!ok) break;
+                    store_tile(tile - (long long)S_ * gridDim.x, stage);
+                    bulk_wait_read_all();               // shared memory has been read: the buffer is free
+                }
+                if (*abort_flag) { ok = false; break; }
+                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
+                const TensorDesc &d = td[g.t];
+                const bool has_lam = d.lam != nullptr;
+                const u32 C = (u32)d.d1, pitch = g.cols * 4u, bytes = g.nrows * pitch;
+                const u32 bar = smem_u32(&sh.full_bar[stage]);
+                const u32 sb = smem_u32(tile_buf + (size_t)stage * stage_bytes);
+                mbar_arrive_expect_tx(bar, (has_lam ? 2u : 1u) * bytes);
+                if (g.whole) {
+                    bulk_load_1d(sb, d.w + g.off0, bytes, bar);
+                    if (has_lam) bulk_load_1d(sb + (u32)arr, d.lam + g.off0, bytes, bar);
+                } else {
+                    for (u32 r = 0; r < g.nrows; ++r) {
+                        bulk_load_1d(sb + r * pitch, d.w + g.off0 + r * C, pitch, bar);
+                        if (has_lam) bulk_load_1d(sb + (u32)arr + r * pitch, d.lam + g.off0 + r * C, pitch, bar);
+                    }
+                }
+            }
+            const u32 issued = k;                       // tiles whose loads have been issued
+            see_dependency();
+            if (ok) {                                   // drain: the last tiles still sit in their buffers
+                const u32 first = issued > S_ ? issued - S_ : 0u;
+                for (u32 j = first; j < issued && ok; ++j) {
+                    const int stage = (int)(j % S_);
+                    ok = mbar_wait_bounded(smem_u32(&sh.done_bar[stage]), (j / S_) & 1u, abort_flag);
+                    if (ok) store_tile((long long)blockIdx.x + (long long)j * gridDim.x, stage);
+                }
+            }
+            if (!ok) {
+                // a wait ran out (or the single pass is off: `quiet`): the loads still in flight get the
+                // same bounded time, so that none lands in shared memory after this CTA has gone
+                *abort_flag = 1;
+                if (!quiet) atomicExch(&P.ctl->async_error, 1);
+                const u32 first = issued > S_ ? issued - S_ : 0u;
+                for (u32 j = first; j < issued; ++j)
+                    (void)mbar_wait_bounded(smem_u32(&sh.full_bar[j % S_]), (j / S_) & 1u, nullptr);
+            }
+            bulk_wait_all();                            // every store has left shared memory and is performed
+        }
+    } else {
+        // ------------------------------------------------------------ consumers
+        const int cw = warp;
+        const u32 J = (u32)P.jr_floats;
+        unsigned char *cb = cand_buf + (size_t)cw * blockg_cand_bytes(P.jr_floats);
+        u64 *ckey = reinterpret_cast<u64 *>(cb);
+        u64 *cid = ckey + BSTG;
+        float *clam = reinterpret_cast<float *>(cid + BSTG);
+        u32 n_above = 0, k = 0;
+        bool ok = true;
+#pragma unroll 1
+        for (long long tile = blockIdx.x; onepass && tile < P.n_tiles; tile += gridDim.x, ++k) {
+            const int stage = (int)(k % S_);
+            const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
+            const TensorDesc &d = td[g.t];
+            const bool has_lam = d.lam != nullptr;
+            const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
+            const bool mstage = g.whole && d.mask && ((uintptr_t)d.mask & 15u) == 0;      // the producer stores the mask
+            const u32 C = (u32)d.d1, bh = (u32)d.bh, bw = (u32)d.bw, P_ = g.cols;
+            if (*abort_flag || !mbar_wait_bounded(smem_u32(&sh.full_bar[stage]), (k / S_) & 1u, abort_flag)) { ok = false; break; }
+            unsigned char *sbp = tile_buf + (size_t)stage * stage_bytes;
+            float *sw = reinterpret_cast<float *>(sbp);
+            float *sl = reinterpret_cast<float *>(sbp + arr);
+            unsigned char *sm = sbp + 2 * (size_t)arr + (g.off0 & 15u);
+#pragma unroll 1
+            for (u32 q0 = (u32)cw * 32u; q0 < g.nq; q0 += (u32)BT_BLOCKS) {
+                const u32 q = q0 + (u32)lane;
+                if (q < g.nq) {
+                    BlockJob jb;
+                    const u32 brl = q / g.nbpr, bcol = q - brl * g.nbpr;
+                    const u32 c0 = bcol * bw;
+                    jb.nc = g.cols - c0 < bw ? g.cols - c0 : bw;
+                    jb.bh = bh; jb.bw = bw; jb.pitch = P_; jb.C = C;
+                    jb.base = brl * bh * P_ + c0;
+                    jb.gbase = g.off0 + brl * bh * C + c0;
+                    jb.id = (u64)d.unit_prefix + g.b0 + q;
+                    jb.sw = sw; jb.sl = sl; jb.sm = sm;
+                    jb.mstage = mstage; jb.has_lam = has_lam; jb.upd = upd;
+                    n_above += blockg_one<H, G, BH, BW>(P, d, jb, br, mu, fp16, sh, cw, ckey, cid, clam);
+                }
+                blockg_flush(P, &sh.wcount[cw], ckey, cid, clam, BSTG - 32);
+            }
+            fence_proxy_async();                        // the bulk stores of the producer read these writes
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh.done_bar[stage]));
+        }
+        if (!ok && lane == 0 && !*abort_flag) {
+            *abort_flag = 1;
+            atomicExch(&P.ctl->async_error, 1);
+        }
+        blockg_flush(P, &sh.wcount[cw], ckey, cid, clam, 0);
+        na = n_above;
+    }
+    __syncthreads();
+    pdl_wait();
+    if (!P.ctl->sel.onepass) return;         // (the same for every thread)
+    // the blocks outside the aligned interior (ragged last block rows, unaligned or too wide
+    // tensors) and the tensors that pass through: work items listed by the host, generic code
+    if (P.n_edge_items > 0) {
+        const u32 J = (u32)P.jr_floats;
+        for (long long i = blockIdx.x; i < P.n_edge_items; i += gridDim.x) {
+            const long long item = P.edge_items[i];
+            const int t = find_tensor(P.item_prefix, P.T, item);
+            const TensorDesc g = P.td[t];
+            const long long local = item - P.item_prefix[t];
+            if (!g.ranked) {
+                if (threadIdx.x < THREADS) process_linear_item<M_KEEPALL>(P, g, local, 0, 0);
+                continue;
+            }
+            if (warp >= BLOCKS_PER_ITEM / 32) continue;             // 8 warps x 32 blocks make one item
+            const int cw = warp;
+            unsigned char *cb = cand_buf + (size_t)cw * blockg_cand_bytes(P.jr_floats);
+            u64 *ckey = reinterpret_cast<u64 *>(cb);
+            u64 *cid = ckey + BSTG;
+            float *clam = reinterpret_cast<float *>(cid + BSTG);
+            const long long b = local * BLOCKS_PER_ITEM + warp * 32 + lane;
+            if (b < g.n_units && b >= blockg_fast_end(g, arr)) {
+                const u64 key = blockg_key_global(g, b, mu);
+                const u64 id = (u64)(g.unit_prefix + b);
+                na += key > br.hi ? 1 : 0;
+                if (key >= br.lo && key <= br.hi) {
+                    const u32 slot = atomicAdd(&sh.wcount[cw], 1u);
+                    ckey[slot] = key;
+                    cid[slot] = id;
+                    const BlockExt e = blockg_ext(g, b);
+                    for (int r = 0; r < e.nr; ++r)
+                        for (int c = 0; c < e.nc; ++c)
+                            clam[slot * J + r * g.bw + c] = g.lam ? g.lam[(e.r0 + r) * g.d1 + e.c0 + c] : 0.0f;
+                    atomicAdd(&sh.hist[bracket_bin(br, key, id)], 1u);
+                }
+                blockg_write_global(P, g, b, key >= br.guess, nullptr, 0, 1);
+            }
+            blockg_flush(P, &sh.wcount[cw], ckey, cid, clam, 0);
+        }
+    }
+    if (warp < BT_CWARPS) {
+        for (int o = 16; o > 0; o >>= 1) na += __shfl_xor_sync(0xffffffffu, na, o);
+        if (lane == 0) sh.red[warp] = na;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        u64 tot = 0;
+        for (int i = 0; i < BT_CWARPS; ++i) tot += sh.red[i];
+        if (tot) atomicAdd(&P.ctl->scan_above[0], tot);
+    }
+    for (int i = threadIdx.x; i < NBINS; i += BT_THREADS) {
+        const u32 hc = sh.hist[i];
+        if (hc) atomicAdd(&P.hist[i], (u64)hc);
+    }
+}
+
+}  // namespace cs

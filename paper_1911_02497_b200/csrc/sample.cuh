@@ -48,6 +48,10 @@ __device__ __forceinline__ u64 unit_key(const Params &P, u64 unit, const TensorD
         const long long e = (long long)unit - d.elem_prefix;
         if (e < 0 || e >= d.numel) return 0;
         return key_of_u(form_u(d.w[e], has_lam ? d.lam[e] : 0.0f, P.mu, has_lam));
+    } else if (SRC == SRC_BLOCKG) {
+        const long long b = (long long)unit - d.unit_prefix;
+        if (b < 0 || b >= d.n_units) return 0;
+        return blockg_key_global(d, b, P.mu);
     } else {
         const long long b = (long long)unit - d.unit_prefix;
         if (b < 0 || b >= d.n_units) return 0;

@@ -243,6 +243,82 @@ __device__ __forceinline__ u64 block_key(const BlockData &bd, float mu, bool has
     return (u64)__double_as_longlong(acc);
 }
 
+// Block b of tensor d: first row and column, rows and columns that exist.
+struct BlockExt {
+    long long r0, c0;
+    int nr, nc;
+};
+
+__device__ __forceinline__ BlockExt blockg_ext(const TensorDesc &d, long long b)
+{
+    BlockExt e;
+    const long long br = d.n_units < 0x7FFFFFFFll ? (long long)((u32)b / (u32)d.nbc) : b / d.nbc;
+    const long long bc = b - br * d.nbc;
+    e.r0 = br * d.bh;
+    e.c0 = bc * d.bw;
+    e.nr = (int)(d.d0 - e.r0 < d.bh ? d.d0 - e.r0 : d.bh);
+    e.nc = (int)(d.d1 - e.c0 < d.bw ? d.d1 - e.c0 : d.bw);
+    return e;
+}
+
+// nu of block b straight from global memory: fp64 sum of u^2 over the elements that exist,
+// row by row. Returns the fp64 bit pattern.
+__device__ __forceinline__ u64 blockg_key_global(const TensorDesc &d, long long b, float mu)
+{
+    const BlockExt e = blockg_ext(d, b);
+    const bool has_lam = d.lam != nullptr;
+    double acc = 0.0;
+    for (int r = 0; r < e.nr; ++r) {
+        const long long off = (e.r0 + r) * d.d1 + e.c0;
+        for (int c = 0; c < e.nc; ++c) {
+            const double x = (double)form_u(__ldg(d.w + off + c), has_lam ? d.lam[off + c] : 0.0f, mu, has_lam);
+            acc = __fma_rn(x, x, acc);
+        }
+    }
+    return (u64)__double_as_longlong(acc);
+}
+
+// Final write of the rows r_first, r_first + r_step, ... of block b from global memory. `jr`,
+// when given, holds the block's original multipliers (row-major, d.bw floats per row) and is
+// read instead of lambda, which an earlier pass may have updated in place.
+__device__ __forceinline__ void blockg_write_global(const Params &P, const TensorDesc &d, long long b, bool keep,
+                                                    const float *jr, int r_first, int r_step)
+{
+    const BlockExt e = blockg_ext(d, b);
+    const bool has_lam = d.lam != nullptr;
+    const bool wr_lam = (P.fuse & FUSE_LAMBDA) && has_lam;
+    const bool wr_grad = (P.fuse & FUSE_PENALTY) && d.grad != nullptr;
+    for (int r = r_first; r < e.nr; r += r_step) {
+        const long long off = (e.r0 + r) * d.d1 + e.c0;
+        for (int c = 0; c < e.nc; ++c) {
+            const float w = __ldg(d.w + off + c);
+            const float l = has_lam ? (jr ? __ldcg(jr + r * d.bw + c) : d.lam[off + c]) : 0.0f;
+            const Out o = finish(w, l, form_u(w, l, P.mu, has_lam), keep, P.mu, P.fuse, has_lam);
+            d.theta[off + c] = o.theta;
+            if (d.mask) d.mask[off + c] = o.m;
+            if (d.theta_h) d.theta_h[off + c] = o.th;
+            if (wr_lam) d.lam[off + c] = o.lam;
+            if (wr_grad) d.grad[off + c] = o.grad;
+        }
+    }
+}
+
+// The same scan for bh x bw blocks.
+__device__ __forceinline__ void scan_source_blockg(const Params &P, ScanShared &sh, ScanCtx &c)
+{
+    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        const long long b0 = (item - P.item_prefix[t]) * BLOCKS_PER_ITEM;
+#pragma unroll 1
+        for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it) {
+            const long long b = b0 + it * THREADS + threadIdx.x;
+            const bool ok = b < d.n_units;
+            scan_emit(P, sh, c, ok ? blockg_key_global(d, b, P.mu) : 0, (u64)(d.unit_prefix + b), ok);
+        }
+    }
+}
+
 // Block items exist for ranked (2-D) tensors only in the scan decomposition.
 __device__ __forceinline__ void scan_source_block(const Params &P, ScanShared &sh, ScanCtx &c)
 {
@@ -284,6 +360,7 @@ __device__ __noinline__ void scan_source(const Params &P, ScanShared &sh, bool d
     scan_begin(sh, c, do_list);
     if (SRC == SRC_ELEM) scan_source_elem(P, sh, c);
     else if (SRC == SRC_BLOCK) scan_source_block(P, sh, c);
+    else if (SRC == SRC_BLOCKG) scan_source_blockg(P, sh, c);
     else scan_source_array(P, sh, c);
     scan_end(P, sh, c, slot);
 }
@@ -683,10 +760,10 @@ template <int SRC>
 __device__ __noinline__ void repair_unit(const Params &P, u64 idx, u64 id, bool keep, int part, const long long *pre_s,
                                          const TensorDesc *tdc);
 
-// Threads per rewritten unit: a block is rewritten by four threads, a row each, which keeps the
-// dependent chain of one rewrite short.
+// Threads per rewritten unit: a 4 x 4 block is rewritten by four threads, a row each, which keeps
+// the dependent chain of one rewrite short; a bh x bw block by eight (rows part, part + 8, ...).
 template <int SRC>
-struct RepairLanes { static constexpr u32 value = (SRC == SRC_BLOCK) ? 4u : 1u; };
+struct RepairLanes { static constexpr u32 value = (SRC == SRC_BLOCK) ? 4u : (SRC == SRC_BLOCKG) ? 8u : 1u; };
 
 // Fills the shared-memory copies used by the rewrites (all threads; a barrier must follow).
 template <int SRC>

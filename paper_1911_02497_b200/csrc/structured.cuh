@@ -83,6 +83,27 @@ __device__ __forceinline__ void apply_block_items(const Params &P, u64 tau_key, 
     }
 }
 
+// The same for bh x bw blocks (the fall-back of the single-pass route).
+__device__ __forceinline__ void apply_blockg_items(const Params &P, u64 tau_key, u64 tau_id)
+{
+    for (long long item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        const int t = find_tensor(P.item_prefix, P.T, item);
+        const TensorDesc d = P.td[t];
+        const long long local = item - P.item_prefix[t];
+        if (!d.ranked) {
+            process_linear_item<M_KEEPALL>(P, d, local, 0, 0);
+            continue;
+        }
+#pragma unroll 1
+        for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it) {
+            const long long b = local * BLOCKS_PER_ITEM + it * THREADS + threadIdx.x;
+            if (b >= d.n_units) continue;
+            const u64 key = blockg_key_global(d, b, P.mu);
+            blockg_write_global(P, d, b, keep_by_cutoff(key, (u64)(d.unit_prefix + b), tau_key, tau_id), nullptr, 0, 1);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(THREADS) k_apply_block(Params P)
 {
     if (P.ctl->sel.onepass) return;          // the single-pass kernel has written everything
@@ -101,6 +122,8 @@ __device__ __noinline__ void apply_after_select(const Params &P, int need_h)
         else apply_linear_items<M_PRUNE, false>(P, tau_key, tau_id);
     } else if (SRC == SRC_BLOCK) {
         apply_block_items(P, tau_key, tau_id);
+    } else if (SRC == SRC_BLOCKG) {
+        apply_blockg_items(P, tau_key, tau_id);
     }
 }
 

@@ -525,6 +525,44 @@ def test_single_pass_block_kernel_tiles_edges_and_many_tensors(ctx):
     ctx.set_seed(SEED)
 
 
+@pytest.mark.parametrize("block", [(5, 5), (3, 3), (1, 8), (8, 1), (2, 2), (3, 2), (7, 3)])
+def test_single_pass_general_blocks(ctx, block):
+    """bh x bw blocks at a size that takes the tiled single-pass kernel (more than 131072 blocks):
+    several block rows per tile and one per tile, ragged last block rows, widths that are no
+    multiple of bw, a matrix whose width is no multiple of 4, a vector and a 4-D tensor (pass
+    through), tensors without multipliers, 16-bit codes and gradient. The kernel is built for the
+    first five shapes; the others take the route over the norm array at the same size."""
+    bh, bw = block
+    tiled = 1 if block in ((5, 5), (3, 3), (1, 8), (8, 1), (2, 2)) else 0
+    shapes = [(bh * 37 + bh // 2, 1500), (203 * bh, 8 * bw * 4), (61, 1001), (4097,), (401, 2004), (3, 2, 4, 4),
+              (bh + 1, 1024 * bw)]
+    need = 140000 * bh * bw - sum(r * c for r, c in [sh for sh in shapes if len(sh) == 2])
+    shapes.append((max(need // 1000 + 1, bh), 1000))
+    ws = W.random_set(shapes, seed=31 + bh * 9 + bw, kind="uniform", scale=0.1, lam_sigma=1e-3, mu=1e-2)
+    for sd in (5, 6):
+        ctx.set_seed(sd)
+        got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.9, ws.mu, ("lambda", "penalty"), block=block)
+        assert res.sampled == tiled and res.n_units > 131072
+        assert not tiled or (res.n_candidates > 0 and res.n_repaired > 0)
+    got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.5, ws.mu, ("fp16", "lambda"), block=block)
+    assert res.sampled == tiled
+    lam = [l if t % 3 else None for t, l in enumerate(ws.lam)]
+    got, res, _ = check(ctx, "block", ws.w, lam, 0.8, ws.mu, ("bf16", "lambda", "penalty"), block=block)
+    assert res.sampled == tiled
+    got, res, _ = check(ctx, "block", ws.w, ws.lam, 0.9, ws.mu, (), block=block)     # nothing updated in place
+    assert res.sampled == tiled
+    ctx.set_seed(SEED)
+
+
+def test_single_pass_general_blocks_fall_back(ctx):
+    """A list whose block norms are nearly all equal: the sample advises against the single pass and
+    the selection kernel does the two-pass job for bh x bw blocks itself."""
+    rng = np.random.default_rng(12)
+    w = [np.full((3000, 1500), 0.25, np.float32), rng.standard_normal((100, 200)).astype(np.float32)]
+    got, res, _ = check(ctx, "block", w, None, 0.5, 1e-2, ("penalty",), block=(5, 5))
+    assert res.sampled == 0 and res.n_units == 600 * 300 + 20 * 40
+
+
 def check_structured(ctx, w, lam, s, mu, kind, block=None, criterion="l2", fuse=("lambda",), elem_offset=0,
                      exact_key=True):
     """The specification entry point against the oracle's: masks, theta, multipliers, gradient and
@@ -710,6 +748,13 @@ def test_workspace_query_sizes_a_context_that_never_allocates():
     ds = DeviceSet(ws.w, ws.lam)
     need = cstep.workspace_bytes(cstep.OP_BLOCK, ds.table, ds.T, ("lambda",))
     assert need > 0
+    # the first launch of a kernel in a process makes the CUDA runtime load its code, which takes
+    # device memory of its own: a throw-away context runs the same call first
+    c0 = cstep.Context(0)
+    ds.run(c0, "block", ws.sparsity, ws.mu, ("lambda",))
+    torch.cuda.synchronize()
+    c0.close()
+    ds.reset_lambda()
     c = cstep.Context(0, need)
     try:
         torch.cuda.synchronize()
