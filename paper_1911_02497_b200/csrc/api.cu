@@ -538,11 +538,11 @@ Sel initial_state(long long S, long long k, int bits_key)
 constexpr size_t SMEM_OPTIN_BYTES = 232448;      // shared memory one CTA may have on this architecture
 bool blockg_ring_config(Plan &pl, int T)
 {
-    const size_t fixed = sizeof(BlockFastShared) + 1024 + (size_t)BT_CWARPS * blockg_cand_bytes(pl.jr_floats);
+    const size_t fixed = sizeof(BlockGShared) + 1024 + (size_t)BG_GROUPS * blockg_cand_bytes(pl.jr_floats);
     if (fixed >= SMEM_OPTIN_BYTES) return false;
     int best_arr = 0, best_stages = 0;
     long long best_chunked = -1;
-    for (int stages = BT_STAGES; stages >= 2; --stages) {
+    for (int stages = BG_MAX_STAGES; stages >= 2; --stages) {
         // stages * (2.25 * arr + 16) <= what is left
         const size_t per = (SMEM_OPTIN_BYTES - fixed) / (size_t)stages;
         if (per < 1024) continue;
@@ -824,7 +824,7 @@ int run_op(condensa_ctx *ctx, int op, const condensa_tensor *ts, int T, double s
             pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
             pdl.val.programmaticStreamSerializationAllowed = 1;
             cfg.gridDim = dim3((unsigned)gridf);
-            cfg.blockDim = dim3((unsigned)(op == OP_PRUNE ? THREADS : BT_THREADS));
+            cfg.blockDim = dim3((unsigned)(op == OP_PRUNE ? THREADS : op == OP_BLOCKG1 ? BG_THREADS : BT_THREADS));
             cfg.dynamicSmemBytes = op == OP_PRUNE ? 0 : op == OP_BLOCKG1 ? dyn_g : BLOCK_FAST_DYN_SMEM;
             cfg.stream = stream;
             cfg.attrs = &pdl;

@@ -12,12 +12,35 @@ namespace cs {
 // Shared memory of a CTA: `stages` tile buffers (w, lambda: `arr` bytes each; mask: arr / 4 + 16
 // bytes, the tile's mask starts at the byte offset its global address has inside a 16-byte line,
 // so that the aligned interior can leave by one bulk copy), then the candidate staging of each
-// consumer warp (BSTG keys, BSTG ids, BSTG x jr_floats original multipliers).
+// consumer group (BG_CAND keys, ids and blocks of jr_floats original multipliers; a candidate
+// that finds it full goes to the list directly).
+// The consumer warps may form several groups that work on different tiles at the same time
+// (measured on 5 x 5 blocks of 1500-column matrices: two groups of ten warps at 80 registers
+// were slower than one group of twelve at 128).
+constexpr int BG_GROUPS = 1;
+constexpr int BG_GWARPS = 12;                                   // warps of a group: 384 blocks of a tile at a time
+constexpr int BG_CWARPS = BG_GROUPS * BG_GWARPS;                // consumer warps
+constexpr int BG_THREADS = (BG_CWARPS + 1) * 32;                // + the producer warp
+constexpr int BG_MAX_STAGES = 4;
+constexpr u32 BG_CAND = 64;         // staged candidates of a group
+constexpr u32 BG_FLUSH = 24;        // ... appended to the list once there are more than this many
+
+struct BlockGShared {
+    u32 hist[NBINS];
+    u64 red[BG_CWARPS];
+    u64 flush_base[BG_GROUPS];
+    u32 ccount[BG_GROUPS];                       // staged candidates of each group
+    unsigned long long full_bar[BG_MAX_STAGES];  // bytes of a tile have arrived
+    unsigned long long done_bar[BG_MAX_STAGES];  // every warp of the tile's group has finished with the buffer
+    int abort;                                   // a bounded wait ran out somewhere in this CTA
+    long long tile_prefix[BT_TD_CACHE + 1];
+    TensorDesc td[BT_TD_CACHE];
+};
 __host__ __device__ inline size_t blockg_stage_bytes(int arr) { return (size_t)arr * 2 + (size_t)arr / 4 + 16; }
-__host__ __device__ inline size_t blockg_cand_bytes(int jr_floats) { return (size_t)BSTG * (16 + 4 * (size_t)jr_floats); }
+__host__ __device__ inline size_t blockg_cand_bytes(int jr_floats) { return (size_t)BG_CAND * (16 + 4 * (size_t)jr_floats); }
 __host__ __device__ inline size_t blockg_dyn_smem(int arr, int stages, int jr_floats)
 {
-    return (size_t)stages * blockg_stage_bytes(arr) + (size_t)BT_CWARPS * blockg_cand_bytes(jr_floats);
+    return (size_t)stages * blockg_stage_bytes(arr) + (size_t)BG_GROUPS * blockg_cand_bytes(jr_floats);
 }
 
 // Tiles of the aligned interior of tensor d: as many complete block rows as fit a buffer, or,
@@ -81,33 +104,75 @@ __device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const
     return g;
 }
 
-// Appends the candidates a consumer warp has staged to the list (one global atomic per flush).
-__device__ __forceinline__ void blockg_flush(const Params &P, u32 *wcount, const u64 *ckey, const u64 *cid, const float *clam,
-                                             u32 limit)
+__device__ __forceinline__ void bar_sync_named(int id, int nthreads)
 {
-    const int lane = threadIdx.x & 31;
-    __syncwarp();
-    const u32 c = *wcount;
-    if (c > limit) {
-        u64 base = 0;
-        if (lane == 0) base = atomicAdd(&P.ctl->list_count[0], (u64)c);
-        base = __shfl_sync(0xffffffffu, base, 0);
-        for (u32 i = lane; i < c; i += 32) {
-            const u64 pos = base + i;
-            if (pos < P.cap) {
-                P.list_key[pos] = ckey[i];
-                P.list_id[pos] = cid[i];
-            }
-        }
-        const u32 J = (u32)P.jr_floats;
-        for (u32 i = lane; i < c * J; i += 32) {
-            const u64 pos = base + i / J;
-            if (pos < P.cap) P.jr_lam[pos * J + (i % J)] = clam[i];
-        }
-        __syncwarp();
-        if (lane == 0) *wcount = 0;
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Candidate (key, id) with the original multipliers `lam` of its block (row-major, `n` floats):
+// into the CTA's staging, or straight to the list when the staging is full.
+struct CandStage {
+    u64 *key, *id;
+    float *lam;
+    u32 *count;         // entries staged so far (may run past BG_CAND: those went to the list directly)
+    u64 *base;          // scratch word of the flush
+};
+__device__ __forceinline__ CandStage blockg_stage_of(unsigned char *cand_buf, int jr_floats, BlockGShared &sh, int group)
+{
+    CandStage cs;
+    cs.key = reinterpret_cast<u64 *>(cand_buf + (size_t)group * blockg_cand_bytes(jr_floats));
+    cs.id = cs.key + BG_CAND;
+    cs.lam = reinterpret_cast<float *>(cs.id + BG_CAND);
+    cs.count = &sh.ccount[group];
+    cs.base = &sh.flush_base[group];
+    return cs;
+}
+__device__ __forceinline__ float *blockg_cand_slot(const Params &P, const CandStage &cs, u64 key, u64 id)
+{
+    const u32 J = (u32)P.jr_floats;
+    const u32 slot = atomicAdd(cs.count, 1u);
+    if (slot < BG_CAND) {
+        cs.key[slot] = key;
+        cs.id[slot] = id;
+        return cs.lam + slot * J;
     }
-    __syncwarp();
+    const u64 pos = atomicAdd(&P.ctl->list_count[0], 1ull);
+    if (pos >= P.cap) return nullptr;            // (the selection reports the overflow)
+    P.list_key[pos] = key;
+    P.list_id[pos] = id;
+    return P.jr_lam + pos * J;
+}
+
+// Appends the staged candidates to the list when there are more than `limit`: `nthreads` threads
+// (numbered tid) call this together, synchronised by the named barrier `bar`. Every thread takes
+// the same decision, and every call runs the same barriers whatever the outcome.
+__device__ __forceinline__ void blockg_cta_flush(const Params &P, const CandStage &cs, int bar, int nthreads, int tid,
+                                                 u32 limit)
+{
+    bar_sync_named(bar, nthreads);              // the staged entries are complete
+    const u32 cnt = *cs.count;
+    const u32 c = cnt < BG_CAND ? cnt : BG_CAND;
+    bar_sync_named(bar, nthreads);              // everybody has read the count
+    if (c <= limit) return;
+    if (tid == 0) {
+        *cs.base = atomicAdd(&P.ctl->list_count[0], (u64)c);
+        *cs.count = 0;
+    }
+    bar_sync_named(bar, nthreads);
+    const u64 base = *cs.base;
+    for (u32 i = tid; i < c; i += nthreads) {
+        const u64 pos = base + i;
+        if (pos < P.cap) {
+            P.list_key[pos] = cs.key[i];
+            P.list_id[pos] = cs.id[i];
+        }
+    }
+    const u32 J = (u32)P.jr_floats;
+    for (u32 i = tid; i < c * J; i += nthreads) {
+        const u64 pos = base + i / J;
+        if (pos < P.cap) P.jr_lam[pos * J + (i % J)] = cs.lam[i];
+    }
+    bar_sync_named(bar, nthreads);              // the staging may be filled again
 }
 
 // One block of a tile in shared memory: norm, decision, outputs in place. BH x BW (when not 0)
@@ -124,25 +189,24 @@ struct BlockJob {
 
 template <bool H, bool G, int BH, int BW>
 __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, const BlockJob &jb, const Bracket &br,
-                                          float mu, int fp16, BlockFastShared &sh, int cw, u64 *ckey, u64 *cid, float *clam)
+                                          float mu, int fp16, u32 *hist, const CandStage &cs)
 {
-    const u32 J = (u32)P.jr_floats;
     if (BH > 0 && jb.nc == (u32)BW) {
-        constexpr int N = BH > 0 ? BH * BW : 1;
+        constexpr int RB = BH > 0 ? BH : 1, CB = BW > 0 ? BW : 1, N = RB * CB;
         float w[N], l[N], u[N];
         u32 nz = 0;
 #pragma unroll
-        for (int r = 0; r < (BH > 0 ? BH : 1); ++r)
+        for (int r = 0; r < RB; ++r)
 #pragma unroll
-            for (int c = 0; c < (BW > 0 ? BW : 1); ++c) {
+            for (int c = 0; c < CB; ++c) {
                 const u32 o = jb.base + r * jb.pitch + c;
-                w[r * BW + c] = jb.sw[o];
-                l[r * BW + c] = jb.has_lam ? jb.sl[o] : 0.0f;
-                nz |= __float_as_uint(l[r * BW + c]);
+                w[r * CB + c] = jb.sw[o];
+                l[r * CB + c] = jb.has_lam ? jb.sl[o] : 0.0f;
+                nz |= __float_as_uint(l[r * CB + c]);
             }
-        if (nz) {
+        if (nz) {                       // one decision per block keeps the code free of branches per element
 #pragma unroll
-            for (int i = 0; i < N; ++i) u[i] = form_u(w[i], l[i], mu, true);
+            for (int i = 0; i < N; ++i) u[i] = __fsub_rn(w[i], __fdiv_rn(l[i], mu));
         } else {                        // every lambda is +0: u is w, bit for bit
 #pragma unroll
             for (int i = 0; i < N; ++i) u[i] = w[i];
@@ -156,18 +220,33 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
         const u64 key = (u64)__double_as_longlong(acc);
         const bool keep = key >= br.guess;
         if (key >= br.lo && key <= br.hi) {
-            const u32 slot = atomicAdd(&sh.wcount[cw], 1u);
-            ckey[slot] = key;
-            cid[slot] = jb.id;
+            float *jl = blockg_cand_slot(P, cs, key, jb.id);
+            if (jl) {
 #pragma unroll
-            for (int i = 0; i < N; ++i) clam[slot * J + i] = l[i];
-            atomicAdd(&sh.hist[bracket_bin(br, key, jb.id)], 1u);
+                for (int i = 0; i < N; ++i) jl[i] = l[i];
+            }
+            atomicAdd(&hist[bracket_bin(br, key, jb.id)], 1u);
+        }
+        if (jb.mstage && jb.upd && !H && !G) {
+            // the common case without side outputs: everything stays in shared memory
+#pragma unroll
+            for (int r = 0; r < RB; ++r)
+#pragma unroll
+                for (int c = 0; c < CB; ++c) {
+                    const int i = r * CB + c;
+                    const u32 o = jb.base + r * jb.pitch + c;
+                    const float th = keep ? u[i] : 0.0f;
+                    jb.sw[o] = th;
+                    jb.sl[o] = __fsub_rn(l[i], __fmul_rn(mu, __fsub_rn(w[i], th)));
+                    jb.sm[o] = keep ? 1 : 0;
+                }
+            return key > br.hi ? 1u : 0u;
         }
 #pragma unroll
-        for (int r = 0; r < (BH > 0 ? BH : 1); ++r)
+        for (int r = 0; r < RB; ++r)
 #pragma unroll
-            for (int c = 0; c < (BW > 0 ? BW : 1); ++c) {
-                const int i = r * BW + c;
+            for (int c = 0; c < CB; ++c) {
+                const int i = r * CB + c;
                 const u32 o = jb.base + r * jb.pitch + c, go = jb.gbase + r * jb.C + c;
                 const Out out = finish_lean<H>(w[i], l[i], u[i], keep, mu, fp16, jb.upd);
                 jb.sw[o] = out.theta;
@@ -190,13 +269,12 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
     const u64 key = (u64)__double_as_longlong(acc);
     const bool keep = key >= br.guess;
     if (key >= br.lo && key <= br.hi) {
-        const u32 slot = atomicAdd(&sh.wcount[cw], 1u);
-        ckey[slot] = key;
-        cid[slot] = jb.id;
-        for (u32 r = 0; r < jb.bh; ++r)
-            for (u32 c = 0; c < jb.nc; ++c)
-                clam[slot * J + r * jb.bw + c] = jb.has_lam ? jb.sl[jb.base + r * jb.pitch + c] : 0.0f;
-        atomicAdd(&sh.hist[bracket_bin(br, key, jb.id)], 1u);
+        float *jl = blockg_cand_slot(P, cs, key, jb.id);
+        if (jl)
+            for (u32 r = 0; r < jb.bh; ++r)
+                for (u32 c = 0; c < jb.nc; ++c)
+                    jl[r * jb.bw + c] = jb.has_lam ? jb.sl[jb.base + r * jb.pitch + c] : 0.0f;
+        atomicAdd(&hist[bracket_bin(br, key, jb.id)], 1u);
     }
     for (u32 r = 0; r < jb.bh; ++r)
         for (u32 c = 0; c < jb.nc; ++c) {
@@ -214,29 +292,29 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
 }
 
 template <bool H, bool G, int BH, int BW>
-__global__ void __launch_bounds__(BT_THREADS, 1) k_fused_blockg(Params P)
+__global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
 {
-    __shared__ BlockFastShared sh;
+    __shared__ BlockGShared sh;
     extern __shared__ __align__(128) unsigned char dyn_smem[];      // tile buffers, then the candidate staging
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int arr = P.bt_arr_bytes, n_stages = P.bt_stages;
     const size_t stage_bytes = blockg_stage_bytes(arr);
     unsigned char *tile_buf = dyn_smem;
-    unsigned char *cand_buf = dyn_smem + (size_t)n_stages * stage_bytes;
-    for (int i = threadIdx.x; i < NBINS; i += BT_THREADS) sh.hist[i] = 0;
-    if (threadIdx.x < BT_CWARPS) sh.wcount[threadIdx.x] = 0;
+    unsigned char *cand_buf = dyn_smem + (size_t)n_stages * stage_bytes;      // candidate staging of the CTA
+    for (int i = threadIdx.x; i < NBINS; i += BG_THREADS) sh.hist[i] = 0;
+    if (threadIdx.x < BG_GROUPS) sh.ccount[threadIdx.x] = 0;
     if (threadIdx.x == 0) sh.abort = 0;
     const bool cached = P.T <= BT_TD_CACHE;
     if (cached) {
-        for (int i = threadIdx.x; i <= P.T; i += BT_THREADS) sh.tile_prefix[i] = P.tile_prefix[i];
+        for (int i = threadIdx.x; i <= P.T; i += BG_THREADS) sh.tile_prefix[i] = P.tile_prefix[i];
         const int words = P.T * (int)(sizeof(TensorDesc) / sizeof(u32));
         const u32 *src = reinterpret_cast<const u32 *>(P.td);
         u32 *dst = reinterpret_cast<u32 *>(sh.td);
-        for (int i = threadIdx.x; i < words; i += BT_THREADS) dst[i] = src[i];
+        for (int i = threadIdx.x; i < words; i += BG_THREADS) dst[i] = src[i];
     }
     if (threadIdx.x < n_stages) {
         mbar_init(smem_u32(&sh.full_bar[threadIdx.x]), 1);
-        mbar_init(smem_u32(&sh.done_bar[threadIdx.x]), BT_CWARPS);
+        mbar_init(smem_u32(&sh.done_bar[threadIdx.x]), BG_GWARPS);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
@@ -249,14 +327,14 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_blockg(Params P)
     Bracket br;
     memset(&br, 0, sizeof(br));
     bool onepass = false;
-    if (warp < BT_CWARPS) {
+    if (warp < BG_CWARPS) {
         pdl_wait();
         onepass = P.ctl->sel.onepass != 0;      // else the sampler advised against the single pass
         br = load_bracket(P.ctl->sel);
     }
     const u32 S_ = (u32)n_stages;
 
-    if (warp == BT_CWARPS) {
+    if (warp == BG_CWARPS) {
         // ------------------------------------------------------------ producer (one lane)
         if (lane == 0) {
             u32 k = 0;
@@ -352,32 +430,38 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_blockg(Params P)
         }
     } else {
         // ------------------------------------------------------------ consumers
-        const int cw = warp;
-        const u32 J = (u32)P.jr_floats;
-        unsigned char *cb = cand_buf + (size_t)cw * blockg_cand_bytes(P.jr_floats);
-        u64 *ckey = reinterpret_cast<u64 *>(cb);
-        u64 *cid = ckey + BSTG;
-        float *clam = reinterpret_cast<float *>(cid + BSTG);
-        u32 n_above = 0, k = 0;
+        // Group `grp` takes the tiles k = grp, grp + BG_GROUPS, ... of this CTA. Every warp of a
+        // group runs every iteration and every barrier of its loop, also after a wait has run
+        // out (it then only skips the work): the flush below synchronises the group.
+        const int grp = warp / BG_GWARPS, gw = warp - grp * BG_GWARPS;
+        const int gtid = gw * 32 + lane, gthreads = BG_GWARPS * 32;
+        const CandStage cs = blockg_stage_of(cand_buf, P.jr_floats, sh, grp);
+        u32 n_above = 0;
         bool ok = true;
 #pragma unroll 1
-        for (long long tile = blockIdx.x; onepass && tile < P.n_tiles; tile += gridDim.x, ++k) {
+        for (u32 k = (u32)grp; onepass && (long long)blockIdx.x + (long long)k * gridDim.x < P.n_tiles; k += (u32)BG_GROUPS) {
+            const long long tile = (long long)blockIdx.x + (long long)k * gridDim.x;
             const int stage = (int)(k % S_);
-            const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
-            const TensorDesc &d = td[g.t];
-            const bool has_lam = d.lam != nullptr;
-            const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
-            const bool mstage = g.whole && d.mask && ((uintptr_t)d.mask & 15u) == 0;      // the producer stores the mask
-            const u32 C = (u32)d.d1, bh = (u32)d.bh, bw = (u32)d.bw, P_ = g.cols;
-            if (*abort_flag || !mbar_wait_bounded(smem_u32(&sh.full_bar[stage]), (k / S_) & 1u, abort_flag)) { ok = false; break; }
-            unsigned char *sbp = tile_buf + (size_t)stage * stage_bytes;
-            float *sw = reinterpret_cast<float *>(sbp);
-            float *sl = reinterpret_cast<float *>(sbp + arr);
-            unsigned char *sm = sbp + 2 * (size_t)arr + (g.off0 & 15u);
+            if (ok && (*abort_flag || !mbar_wait_bounded(smem_u32(&sh.full_bar[stage]), (k / S_) & 1u, abort_flag))) {
+                ok = false;
+                if (lane == 0 && !*abort_flag) {
+                    *abort_flag = 1;
+                    atomicExch(&P.ctl->async_error, 1);
+                }
+            }
+            if (ok) {
+                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
+                const TensorDesc &d = td[g.t];
+                const bool has_lam = d.lam != nullptr;
+                const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
+                const bool mstage = g.whole && d.mask && ((uintptr_t)d.mask & 15u) == 0;      // the producer stores the mask
+                const u32 C = (u32)d.d1, bh = (u32)d.bh, bw = (u32)d.bw, P_ = g.cols;
+                unsigned char *sbp = tile_buf + (size_t)stage * stage_bytes;
+                float *sw = reinterpret_cast<float *>(sbp);
+                float *sl = reinterpret_cast<float *>(sbp + arr);
+                unsigned char *sm = sbp + 2 * (size_t)arr + (g.off0 & 15u);
 #pragma unroll 1
-            for (u32 q0 = (u32)cw * 32u; q0 < g.nq; q0 += (u32)BT_BLOCKS) {
-                const u32 q = q0 + (u32)lane;
-                if (q < g.nq) {
+                for (u32 q = (u32)gtid; q < g.nq; q += (u32)gthreads) {
                     BlockJob jb;
                     const u32 brl = q / g.nbpr, bcol = q - brl * g.nbpr;
                     const u32 c0 = bcol * bw;
@@ -388,19 +472,15 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_blockg(Params P)
                     jb.id = (u64)d.unit_prefix + g.b0 + q;
                     jb.sw = sw; jb.sl = sl; jb.sm = sm;
                     jb.mstage = mstage; jb.has_lam = has_lam; jb.upd = upd;
-                    n_above += blockg_one<H, G, BH, BW>(P, d, jb, br, mu, fp16, sh, cw, ckey, cid, clam);
+                    n_above += blockg_one<H, G, BH, BW>(P, d, jb, br, mu, fp16, sh.hist, cs);
                 }
-                blockg_flush(P, &sh.wcount[cw], ckey, cid, clam, BSTG - 32);
+                fence_proxy_async();                    // the bulk stores of the producer read these writes
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.done_bar[stage]));
             }
-            fence_proxy_async();                        // the bulk stores of the producer read these writes
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh.done_bar[stage]));
+            blockg_cta_flush(P, cs, 1 + grp, gthreads, gtid, BG_FLUSH);
         }
-        if (!ok && lane == 0 && !*abort_flag) {
-            *abort_flag = 1;
-            atomicExch(&P.ctl->async_error, 1);
-        }
-        blockg_flush(P, &sh.wcount[cw], ckey, cid, clam, 0);
+        blockg_cta_flush(P, cs, 1 + grp, gthreads, gtid, 0);
         na = n_above;
     }
     __syncthreads();
@@ -409,7 +489,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_blockg(Params P)
     // the blocks outside the aligned interior (ragged last block rows, unaligned or too wide
     // tensors) and the tensors that pass through: work items listed by the host, generic code
     if (P.n_edge_items > 0) {
-        const u32 J = (u32)P.jr_floats;
+        const CandStage cs = blockg_stage_of(cand_buf, P.jr_floats, sh, 0);
         for (long long i = blockIdx.x; i < P.n_edge_items; i += gridDim.x) {
             const long long item = P.edge_items[i];
             const int t = find_tensor(P.item_prefix, P.T, item);
@@ -419,43 +499,36 @@ __global__ void __launch_bounds__(BT_THREADS, 1) k_fused_blockg(Params P)
                 if (threadIdx.x < THREADS) process_linear_item<M_KEEPALL>(P, g, local, 0, 0);
                 continue;
             }
-            if (warp >= BLOCKS_PER_ITEM / 32) continue;             // 8 warps x 32 blocks make one item
-            const int cw = warp;
-            unsigned char *cb = cand_buf + (size_t)cw * blockg_cand_bytes(P.jr_floats);
-            u64 *ckey = reinterpret_cast<u64 *>(cb);
-            u64 *cid = ckey + BSTG;
-            float *clam = reinterpret_cast<float *>(cid + BSTG);
-            const long long b = local * BLOCKS_PER_ITEM + warp * 32 + lane;
-            if (b < g.n_units && b >= blockg_fast_end(g, arr)) {
+            const long long b = local * BLOCKS_PER_ITEM + warp * 32 + lane;         // 8 warps x 32 blocks make one item
+            if (warp < BLOCKS_PER_ITEM / 32 && b < g.n_units && b >= blockg_fast_end(g, arr)) {
                 const u64 key = blockg_key_global(g, b, mu);
                 const u64 id = (u64)(g.unit_prefix + b);
                 na += key > br.hi ? 1 : 0;
                 if (key >= br.lo && key <= br.hi) {
-                    const u32 slot = atomicAdd(&sh.wcount[cw], 1u);
-                    ckey[slot] = key;
-                    cid[slot] = id;
+                    float *jl = blockg_cand_slot(P, cs, key, id);
                     const BlockExt e = blockg_ext(g, b);
-                    for (int r = 0; r < e.nr; ++r)
-                        for (int c = 0; c < e.nc; ++c)
-                            clam[slot * J + r * g.bw + c] = g.lam ? g.lam[(e.r0 + r) * g.d1 + e.c0 + c] : 0.0f;
+                    if (jl)
+                        for (int r = 0; r < e.nr; ++r)
+                            for (int c = 0; c < e.nc; ++c)
+                                jl[r * g.bw + c] = g.lam ? g.lam[(e.r0 + r) * g.d1 + e.c0 + c] : 0.0f;
                     atomicAdd(&sh.hist[bracket_bin(br, key, id)], 1u);
                 }
                 blockg_write_global(P, g, b, key >= br.guess, nullptr, 0, 1);
             }
-            blockg_flush(P, &sh.wcount[cw], ckey, cid, clam, 0);
+            blockg_cta_flush(P, cs, 1 + BG_GROUPS, BG_THREADS, threadIdx.x, 0);
         }
     }
-    if (warp < BT_CWARPS) {
+    if (warp < BG_CWARPS) {
         for (int o = 16; o > 0; o >>= 1) na += __shfl_xor_sync(0xffffffffu, na, o);
         if (lane == 0) sh.red[warp] = na;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         u64 tot = 0;
-        for (int i = 0; i < BT_CWARPS; ++i) tot += sh.red[i];
+        for (int i = 0; i < BG_CWARPS; ++i) tot += sh.red[i];
         if (tot) atomicAdd(&P.ctl->scan_above[0], tot);
     }
-    for (int i = threadIdx.x; i < NBINS; i += BT_THREADS) {
+    for (int i = threadIdx.x; i < NBINS; i += BG_THREADS) {
         const u32 hc = sh.hist[i];
         if (hc) atomicAdd(&P.hist[i], (u64)hc);
     }

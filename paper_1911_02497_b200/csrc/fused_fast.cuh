@@ -287,6 +287,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(u32 bar, u32 parity, volatile 
     for (u32 i = 0; i < BT_WAIT_POLLS; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 1023u) == 1023u && abort_flag && *abort_flag) return false;
+        __nanosleep(64);        // a tight polling loop takes issue slots and pipe time from the warps that work
     }
     return false;
 }

@@ -267,6 +267,17 @@ __device__ __forceinline__ u64 blockg_key_global(const TensorDesc &d, long long 
 {
     const BlockExt e = blockg_ext(d, b);
     const bool has_lam = d.lam != nullptr;
+    // the rows are fetched one after the other by the loop below (its bounds are not known at
+    // compile time): ask for all of them first, so that the loop finds them on the way
+    for (int r = 0; r < e.nr; ++r) {
+        const long long off = (e.r0 + r) * d.d1 + e.c0;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(d.w + off));
+        if (has_lam) asm volatile("prefetch.global.L2 [%0];" ::"l"(d.lam + off));
+        if (((uintptr_t)(d.w + off) & 127u) + 4u * (u32)e.nc > 128u) {       // the row piece crosses a 128-byte line
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(d.w + off + e.nc - 1));
+            if (has_lam) asm volatile("prefetch.global.L2 [%0];" ::"l"(d.lam + off + e.nc - 1));
+        }
+    }
     double acc = 0.0;
     for (int r = 0; r < e.nr; ++r) {
         const long long off = (e.r0 + r) * d.d1 + e.c0;
