@@ -186,10 +186,14 @@ CONDENSA_API int condensa_cstep_structure(condensa_ctx *ctx, const condensa_tens
 /* BlockPrune - every 2-D tensor is cut into bh x bw blocks (row-major numbering,
  * blocks that stick out over an edge hold fewer elements) ranked on the fp64 sum
  * of u^2 taken row by row inside the block (Table 1, "n-D blocks of size bs").
- * bh = bw = 4 takes the single-pass kernels; every other shape with sides up to 4096
- * (the paper's LSTM run uses bs = 5) is ranked in three steps - norms per block,
- * selection on the norm array, elementwise projection - with the same results
- * contract. Tensors with ndim != 2 pass through. */
+ * bh = bw = 4 takes the single-pass kernels, and so do 5 x 5 (the block size of the
+ * paper's LSTM run), 3 x 3, 2 x 2, 1 x 8 and 8 x 1 on lists of at least 131072 blocks
+ * whose matrices are mostly 16-byte aligned with a width that is a multiple of 4 (the
+ * sample-bracket rules of condensa_cstep_prune() then apply: CONDENSA_NO_SAMPLING,
+ * result fields `sampled`, `n_candidates`, `n_repaired`). Every other shape with sides
+ * up to 4096, and every list the single pass does not take, is ranked in three steps -
+ * norms per block, selection on the norm array, elementwise projection - with the same
+ * results contract. Tensors with ndim != 2 pass through. */
 CONDENSA_API int condensa_cstep_block(condensa_ctx *ctx, const condensa_tensor *tensors, int T,
                          double sparsity, float mu, int bh, int bw, unsigned fuse, void *stream);
 

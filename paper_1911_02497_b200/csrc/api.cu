@@ -540,36 +540,26 @@ bool blockg_ring_config(Plan &pl, int T)
 {
     const size_t fixed = sizeof(BlockGShared) + 1024 + (size_t)BG_GROUPS * blockg_cand_bytes(pl.jr_floats);
     if (fixed >= SMEM_OPTIN_BYTES) return false;
-    int best_arr = 0, best_stages = 0;
-    long long best_chunked = -1;
+    long long best_tiled = 0;
     for (int stages = BG_MAX_STAGES; stages >= 2; --stages) {
         // stages * (2.25 * arr + 16) <= what is left
         const size_t per = (SMEM_OPTIN_BYTES - fixed) / (size_t)stages;
         if (per < 1024) continue;
         long long arr = (long long)((per - 16) * 4 / 9);
         arr -= arr % 64;
-        long long chunked = 0, tiled = 0;               // parameters in column chunks; units the tiles cover
-        for (int t = 0; t < T; ++t) {
-            const TensorDesc &d = pl.td[t];
-            if (!d.ranked) continue;
-            const long long fe = blockg_fast_end(d, (int)arr);
-            tiled += fe;
-            if (fe > 0 && (long long)d.bh * d.d1 * 4 > arr) chunked += d.numel;
-        }
-        if (2 * tiled < pl.S) continue;                 // mostly unaligned matrices: the generic code would do the work
-        if (best_chunked < 0 || chunked < best_chunked) {      // whole block rows beat a deeper ring
-            best_chunked = chunked;
-            best_arr = (int)arr;
-            best_stages = stages;
+        long long tiled = 0;                            // units the tiles cover
+        for (int t = 0; t < T; ++t) tiled += blockg_fast_end(pl.td[t], (int)arr);
+        if (tiled > best_tiled) {                       // more buffers win when they cover the same matrices
+            best_tiled = tiled;
+            pl.bt_arr = (int)arr;
+            pl.bt_stages = stages;
         }
     }
-    if (best_chunked < 0) return false;
-    pl.bt_arr = best_arr;
-    pl.bt_stages = best_stages;
-    return true;
+    // (mostly unaligned or very wide matrices: the generic code would do the work, at the speed
+    // of the route over the norm array at best)
+    return best_tiled > 0 && 2 * best_tiled >= pl.S;
 }
 
-// May this structured call take the single-pass kernels for bh x bw blocks?
 // Block shapes the tiled bh x bw kernel is built for (the per-block code is unrolled at compile
 // time; 5 x 5 is the block size of the paper's LSTM experiment). Other shapes take the route
 // over the norm array.

@@ -161,26 +161,14 @@ __host__ __device__ inline bool block_item_is_fast(const TensorDesc &d, long lon
     return d.ranked && (local + 1) * BLOCKS_PER_ITEM <= block_fast_end(d);
 }
 
-// The same for bh x bw blocks: complete block rows of an aligned matrix. A tile buffer of
-// `arr_bytes` bytes per array takes whole block rows when one fits, else a column chunk of one
-// block row: a multiple of bw and of 4 columns (blockg_chunk_cols; 0 = not even one fits).
-__host__ __device__ inline long long blockg_chunk_cols(const TensorDesc &d, int arr_bytes)
-{
-    long long a = d.bw, b = 4;
-    while (b) { const long long r = a % b; a = b; b = r; }       // a = gcd(bw, 4)
-    const long long step = (long long)d.bw * 4 / a;                // lcm(bw, 4)
-    const long long room = ((long long)arr_bytes - 64ll * d.bh) / (4ll * d.bh);
-    if (room < step) return 0;
-    const long long most = room - room % step;                     // widest chunk that fits
-    const long long cpr = (d.d1 + most - 1) / most;                // chunks per block row
-    const long long even = ((d.d1 + cpr - 1) / cpr + step - 1) / step * step;      // ... of about equal width
-    return even < most ? even : most;
-}
-
+// The same for bh x bw blocks: complete block rows of an aligned matrix, when one block row
+// (bh matrix rows) fits a tile buffer of `arr_bytes` bytes per array. (Tiles that are column
+// chunks of a block row were measured too: the time of a tile hardly depends on its size, so
+// twice as many tiles took twice as long, more than the route over the norm array.)
 __host__ __device__ inline long long blockg_fast_end(const TensorDesc &d, int arr_bytes)
 {
     if (!d.ranked || !d.blk_vec_ok || d.numel >= 0xFFFFFFFFll) return 0;
-    if ((long long)d.bh * d.d1 * 4 > (long long)arr_bytes && blockg_chunk_cols(d, arr_bytes) == 0) return 0;
+    if ((long long)d.bh * d.d1 * 4 > (long long)arr_bytes) return 0;
     return (d.d0 / d.bh) * d.nbc;
 }
 

@@ -43,31 +43,21 @@ __host__ __device__ inline size_t blockg_dyn_smem(int arr, int stages, int jr_fl
     return (size_t)stages * blockg_stage_bytes(arr) + (size_t)BG_GROUPS * blockg_cand_bytes(jr_floats);
 }
 
-// Tiles of the aligned interior of tensor d: as many complete block rows as fit a buffer, or,
-// for a matrix too wide for that, column chunks of one block row.
+// Tiles of the aligned interior of tensor d: as many complete block rows as fit a buffer.
 __host__ __device__ inline long long blockg_tile_count(const TensorDesc &d, int arr)
 {
     if (blockg_fast_end(d, arr) <= 0) return 0;
     const long long nbr = d.d0 / d.bh;
-    const long long row_bytes = (long long)d.bh * d.d1 * 4;
-    if (row_bytes <= arr) {
-        const long long rpt = (long long)arr / row_bytes;
-        return (nbr + rpt - 1) / rpt;
-    }
-    const long long cc = blockg_chunk_cols(d, arr);
-    return nbr * ((d.d1 + cc - 1) / cc);
+    const long long rpt = (long long)arr / ((long long)d.bh * d.d1 * 4);       // >= 1 by blockg_fast_end
+    return (nbr + rpt - 1) / rpt;
 }
 
 struct TileG {
     int t;              // owning tensor
     u32 b0;             // first block (number inside the tensor); block q of the tile is b0 + q
     u32 nq;             // blocks in the tile
-    u32 nbpr;           // blocks per row piece
     u32 nrows;          // matrix rows in the tile
-    u32 cols;           // columns of a row piece (= its pitch in shared memory)
-    u32 c_start;        // first column
-    u32 off0;           // element offset of the first row piece
-    bool whole;         // whole block rows: one contiguous range
+    u32 off0;           // element offset of the tile's first row
 };
 
 __device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const TensorDesc *td, int T, long long tile, int arr)
@@ -75,32 +65,15 @@ __device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const
     TileG g;
     g.t = find_tensor(tile_prefix, T, tile);
     const TensorDesc &d = td[g.t];
-    const u32 bh = (u32)d.bh, bw = (u32)d.bw, C = (u32)d.d1, nbc = (u32)d.nbc, nbr = (u32)(d.d0 / d.bh);
+    const u32 bh = (u32)d.bh, C = (u32)d.d1, nbc = (u32)d.nbc, nbr = (u32)(d.d0 / d.bh);
     const u32 local = (u32)(tile - tile_prefix[g.t]);
-    g.whole = (long long)bh * C * 4 <= (long long)arr;
-    if (g.whole) {
-        const u32 rpt = (u32)arr / (bh * C * 4u);
-        const u32 brow0 = local * rpt;
-        const u32 brows = nbr - brow0 < rpt ? nbr - brow0 : rpt;
-        g.nbpr = nbc;
-        g.nq = brows * nbc;
-        g.nrows = bh * brows;
-        g.cols = C;
-        g.c_start = 0;
-        g.b0 = brow0 * nbc;
-        g.off0 = bh * brow0 * C;
-    } else {
-        const u32 cc = (u32)blockg_chunk_cols(d, arr);
-        const u32 cpr = (C + cc - 1) / cc;
-        const u32 brow = local / cpr, chunk = local - brow * cpr;
-        g.c_start = chunk * cc;
-        g.cols = C - g.c_start < cc ? C - g.c_start : cc;
-        g.nbpr = (g.cols + bw - 1) / bw;
-        g.nq = g.nbpr;
-        g.nrows = bh;
-        g.b0 = brow * nbc + g.c_start / bw;
-        g.off0 = bh * brow * C + g.c_start;
-    }
+    const u32 rpt = (u32)arr / (bh * C * 4u);
+    const u32 brow0 = local * rpt;
+    const u32 brows = nbr - brow0 < rpt ? nbr - brow0 : rpt;
+    g.nq = brows * nbc;
+    g.nrows = bh * brows;
+    g.b0 = brow0 * nbc;
+    g.off0 = bh * brow0 * C;
     return g;
 }
 
@@ -179,8 +152,8 @@ __device__ __forceinline__ void blockg_cta_flush(const Params &P, const CandStag
 // is the block shape at compile time: blocks of full width then run without loops or address
 // arithmetic, with u kept in registers between the norm and the outputs.
 struct BlockJob {
-    u32 nc, bh, bw, pitch, C;       // columns that exist; block shape; row pitch in shared memory and in the tensor
-    u32 base, gbase;                // element offset of the block in the tile buffer / in the tensor
+    u32 nc, bh, bw, C;              // columns that exist; block shape; row pitch (the matrix width)
+    u32 base, goff;                 // element offset of the block in the tile; of the tile in the tensor
     u64 id;
     float *sw, *sl;
     unsigned char *sm;
@@ -199,7 +172,7 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
         for (int r = 0; r < RB; ++r)
 #pragma unroll
             for (int c = 0; c < CB; ++c) {
-                const u32 o = jb.base + r * jb.pitch + c;
+                const u32 o = jb.base + r * jb.C + c;
                 w[r * CB + c] = jb.sw[o];
                 l[r * CB + c] = jb.has_lam ? jb.sl[o] : 0.0f;
                 nz |= __float_as_uint(l[r * CB + c]);
@@ -234,7 +207,7 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
 #pragma unroll
                 for (int c = 0; c < CB; ++c) {
                     const int i = r * CB + c;
-                    const u32 o = jb.base + r * jb.pitch + c;
+                    const u32 o = jb.base + r * jb.C + c;
                     const float th = keep ? u[i] : 0.0f;
                     jb.sw[o] = th;
                     jb.sl[o] = __fsub_rn(l[i], __fmul_rn(mu, __fsub_rn(w[i], th)));
@@ -247,7 +220,7 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
 #pragma unroll
             for (int c = 0; c < CB; ++c) {
                 const int i = r * CB + c;
-                const u32 o = jb.base + r * jb.pitch + c, go = jb.gbase + r * jb.C + c;
+                const u32 o = jb.base + r * jb.C + c, go = jb.goff + jb.base + r * jb.C + c;
                 const Out out = finish_lean<H>(w[i], l[i], u[i], keep, mu, fp16, jb.upd);
                 jb.sw[o] = out.theta;
                 if (jb.upd) jb.sl[o] = out.lam;
@@ -262,7 +235,7 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
     double acc = 0.0;
     for (u32 r = 0; r < jb.bh; ++r)
         for (u32 c = 0; c < jb.nc; ++c) {
-            const u32 o = jb.base + r * jb.pitch + c;
+            const u32 o = jb.base + r * jb.C + c;
             const double x = (double)form_u(jb.sw[o], jb.has_lam ? jb.sl[o] : 0.0f, mu, jb.has_lam);
             acc = __fma_rn(x, x, acc);
         }
@@ -273,12 +246,12 @@ __device__ __forceinline__ u32 blockg_one(const Params &P, const TensorDesc &d, 
         if (jl)
             for (u32 r = 0; r < jb.bh; ++r)
                 for (u32 c = 0; c < jb.nc; ++c)
-                    jl[r * jb.bw + c] = jb.has_lam ? jb.sl[jb.base + r * jb.pitch + c] : 0.0f;
+                    jl[r * jb.bw + c] = jb.has_lam ? jb.sl[jb.base + r * jb.C + c] : 0.0f;
         atomicAdd(&hist[bracket_bin(br, key, jb.id)], 1u);
     }
     for (u32 r = 0; r < jb.bh; ++r)
         for (u32 c = 0; c < jb.nc; ++c) {
-            const u32 o = jb.base + r * jb.pitch + c, go = jb.gbase + r * jb.C + c;
+            const u32 o = jb.base + r * jb.C + c, go = jb.goff + jb.base + r * jb.C + c;
             const float w = jb.sw[o], l = jb.has_lam ? jb.sl[o] : 0.0f;
             const Out out = finish_lean<H>(w, l, form_u(w, l, mu, jb.has_lam), keep, mu, fp16, jb.upd);
             jb.sw[o] = out.theta;
@@ -349,17 +322,9 @@ __global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
                 const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
                 const TensorDesc &d = td[g.t];
                 const bool upd = (P.fuse & FUSE_LAMBDA) && d.lam != nullptr;
-                const u32 C = (u32)d.d1, pitch = g.cols * 4u, bytes = g.nrows * pitch;
+                const u32 bytes = g.nrows * (u32)d.d1 * 4u;
                 unsigned char *sbp = tile_buf + (size_t)stage * stage_bytes;
                 const u32 sb = smem_u32(sbp);
-                if (!g.whole) {                 // one copy per matrix row; the consumers have written the mask themselves
-                    for (u32 r = 0; r < g.nrows; ++r) {
-                        bulk_store_1d(d.theta + g.off0 + r * C, sb + r * pitch, pitch);
-                        if (upd) bulk_store_1d(d.lam + g.off0 + r * C, sb + (u32)arr + r * pitch, pitch);
-                    }
-                    bulk_commit();
-                    return;
-                }
                 bulk_store_1d(d.theta + g.off0, sb, bytes);
                 if (upd) bulk_store_1d(d.lam + g.off0, sb + (u32)arr, bytes);
                 if (d.mask && ((uintptr_t)d.mask & 15u) == 0) {
@@ -393,19 +358,12 @@ __global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
                 const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
                 const TensorDesc &d = td[g.t];
                 const bool has_lam = d.lam != nullptr;
-                const u32 C = (u32)d.d1, pitch = g.cols * 4u, bytes = g.nrows * pitch;
+                const u32 bytes = g.nrows * (u32)d.d1 * 4u;
                 const u32 bar = smem_u32(&sh.full_bar[stage]);
                 const u32 sb = smem_u32(tile_buf + (size_t)stage * stage_bytes);
                 mbar_arrive_expect_tx(bar, (has_lam ? 2u : 1u) * bytes);
-                if (g.whole) {
-                    bulk_load_1d(sb, d.w + g.off0, bytes, bar);
-                    if (has_lam) bulk_load_1d(sb + (u32)arr, d.lam + g.off0, bytes, bar);
-                } else {
-                    for (u32 r = 0; r < g.nrows; ++r) {
-                        bulk_load_1d(sb + r * pitch, d.w + g.off0 + r * C, pitch, bar);
-                        if (has_lam) bulk_load_1d(sb + (u32)arr + r * pitch, d.lam + g.off0 + r * C, pitch, bar);
-                    }
-                }
+                bulk_load_1d(sb, d.w + g.off0, bytes, bar);
+                if (has_lam) bulk_load_1d(sb + (u32)arr, d.lam + g.off0, bytes, bar);
             }
             const u32 issued = k;                       // tiles whose loads have been issued
             see_dependency();
@@ -454,8 +412,8 @@ __global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
                 const TensorDesc &d = td[g.t];
                 const bool has_lam = d.lam != nullptr;
                 const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
-                const bool mstage = g.whole && d.mask && ((uintptr_t)d.mask & 15u) == 0;      // the producer stores the mask
-                const u32 C = (u32)d.d1, bh = (u32)d.bh, bw = (u32)d.bw, P_ = g.cols;
+                const bool mstage = d.mask && ((uintptr_t)d.mask & 15u) == 0;      // the producer stores the mask
+                const u32 C = (u32)d.d1, bh = (u32)d.bh, bw = (u32)d.bw, nbc = (u32)d.nbc;
                 unsigned char *sbp = tile_buf + (size_t)stage * stage_bytes;
                 float *sw = reinterpret_cast<float *>(sbp);
                 float *sl = reinterpret_cast<float *>(sbp + arr);
@@ -463,12 +421,12 @@ __global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
 #pragma unroll 1
                 for (u32 q = (u32)gtid; q < g.nq; q += (u32)gthreads) {
                     BlockJob jb;
-                    const u32 brl = q / g.nbpr, bcol = q - brl * g.nbpr;
+                    const u32 brl = q / nbc, bcol = q - brl * nbc;
                     const u32 c0 = bcol * bw;
-                    jb.nc = g.cols - c0 < bw ? g.cols - c0 : bw;
-                    jb.bh = bh; jb.bw = bw; jb.pitch = P_; jb.C = C;
-                    jb.base = brl * bh * P_ + c0;
-                    jb.gbase = g.off0 + brl * bh * C + c0;
+                    jb.nc = C - c0 < bw ? C - c0 : bw;
+                    jb.bh = bh; jb.bw = bw; jb.C = C;
+                    jb.base = brl * bh * C + c0;
+                    jb.goff = g.off0;
                     jb.id = (u64)d.unit_prefix + g.b0 + q;
                     jb.sw = sw; jb.sl = sl; jb.sm = sm;
                     jb.mstage = mstage; jb.has_lam = has_lam; jb.upd = upd;

@@ -534,7 +534,7 @@ def test_single_pass_general_blocks(ctx, block):
     first five shapes; the others take the route over the norm array at the same size."""
     bh, bw = block
     tiled = 1 if block in ((5, 5), (3, 3), (1, 8), (8, 1), (2, 2)) else 0
-    shapes = [(bh * 37 + bh // 2, 1500), (203 * bh, 8 * bw * 4), (61, 1001), (4097,), (401, 2004), (3, 2, 4, 4),
+    shapes = [(bh * 37 + bh // 2, 1500), (203 * bh, 8 * bw * 4), (61, 1001), (4097,), (401, 1204), (3, 2, 4, 4),
               (bh + 1, 1024 * bw)]
     need = 140000 * bh * bw - sum(r * c for r, c in [sh for sh in shapes if len(sh) == 2])
     shapes.append((max(need // 1000 + 1, bh), 1000))
