@@ -22,8 +22,13 @@ constexpr int BG_GWARPS = 12;                                   // warps of a gr
 constexpr int BG_CWARPS = BG_GROUPS * BG_GWARPS;                // consumer warps
 constexpr int BG_THREADS = (BG_CWARPS + 1) * 32;                // + the producer warp
 constexpr int BG_MAX_STAGES = 4;
-constexpr u32 BG_CAND = 64;         // staged candidates of a group
-constexpr u32 BG_FLUSH = 24;        // ... appended to the list once there are more than this many
+// (The append stops the whole group for the round trip of one atomic on a word every CTA of the
+// grid adds to - microseconds - so it should be rare: 64 / 24 entries instead of 144 / 104 cost
+// 7 % of the kernel's time on 5 x 5 blocks. Two variants that take the wait off the group - the
+// answer of the atomic picked up one tile later, or the copy done by one warp while the others
+// go on - were measured slower: that warp is then late for the next tile's barriers.)
+constexpr u32 BG_CAND = 144;        // staged candidates of a group
+constexpr u32 BG_FLUSH = 104;       // ... appended to the list once there are more than this many
 
 struct BlockGShared {
     u32 hist[NBINS];
