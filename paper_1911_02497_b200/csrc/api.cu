@@ -540,17 +540,23 @@ bool blockg_ring_config(Plan &pl, int T)
 {
     const size_t fixed = sizeof(BlockGShared) + 1024 + (size_t)BG_GROUPS * blockg_cand_bytes(pl.jr_floats);
     if (fixed >= SMEM_OPTIN_BYTES) return false;
-    long long best_tiled = 0;
+    long long best_tiled = 0, best_rounds = 0;
     for (int stages = BG_MAX_STAGES; stages >= 2; --stages) {
         // stages * (2.25 * arr + 16) <= what is left
         const size_t per = (SMEM_OPTIN_BYTES - fixed) / (size_t)stages;
         if (per < 1024) continue;
         long long arr = (long long)((per - 16) * 4 / 9);
         arr -= arr % 64;
-        long long tiled = 0;                            // units the tiles cover
-        for (int t = 0; t < T; ++t) tiled += blockg_fast_end(pl.td[t], (int)arr);
-        if (tiled > best_tiled) {                       // more buffers win when they cover the same matrices
+        long long tiled = 0, rounds = 0;                // units the tiles cover; rounds of one block per thread
+        for (int t = 0; t < T; ++t) {
+            tiled += blockg_fast_end(pl.td[t], (int)arr);
+            rounds += blockg_tile_rounds(pl.td[t], (int)arr);
+        }
+        // coverage first, then the fewest rounds (the kernel's time follows them, not the bytes of
+        // a tile), then the most buffers
+        if (tiled > best_tiled || (tiled == best_tiled && tiled > 0 && rounds < best_rounds)) {
             best_tiled = tiled;
+            best_rounds = rounds;
             pl.bt_arr = (int)arr;
             pl.bt_stages = stages;
         }

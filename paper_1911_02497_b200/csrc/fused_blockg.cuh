@@ -48,13 +48,31 @@ __host__ __device__ inline size_t blockg_dyn_smem(int arr, int stages, int jr_fl
     return (size_t)stages * blockg_stage_bytes(arr) + (size_t)BG_GROUPS * blockg_cand_bytes(jr_floats);
 }
 
-// Tiles of the aligned interior of tensor d: as many complete block rows as fit a buffer.
+// Block rows of one tile of tensor d: as many as fit a buffer, but no more blocks than the group
+// has threads where one block row has fewer (the time of a tile is the time of the longest
+// thread: a second block per thread costs as much as another tile).
+__host__ __device__ inline long long blockg_rows_per_tile(const TensorDesc &d, int arr)
+{
+    const long long fit = (long long)arr / ((long long)d.bh * d.d1 * 4);       // >= 1 by blockg_fast_end
+    const long long lanes = (long long)(BG_GWARPS * 32) / d.nbc;
+    return lanes >= 1 && lanes < fit ? lanes : fit;
+}
+
+// Tiles of the aligned interior of tensor d.
 __host__ __device__ inline long long blockg_tile_count(const TensorDesc &d, int arr)
 {
     if (blockg_fast_end(d, arr) <= 0) return 0;
     const long long nbr = d.d0 / d.bh;
-    const long long rpt = (long long)arr / ((long long)d.bh * d.d1 * 4);       // >= 1 by blockg_fast_end
+    const long long rpt = blockg_rows_per_tile(d, arr);
     return (nbr + rpt - 1) / rpt;
+}
+
+// Rounds of one block per thread that the tiles of tensor d take (what the kernel's time follows).
+__host__ __device__ inline long long blockg_tile_rounds(const TensorDesc &d, int arr)
+{
+    if (blockg_fast_end(d, arr) <= 0) return 0;
+    const long long per_tile = (blockg_rows_per_tile(d, arr) * d.nbc + BG_GWARPS * 32 - 1) / (BG_GWARPS * 32);
+    return blockg_tile_count(d, arr) * per_tile;
 }
 
 struct TileG {
@@ -72,7 +90,7 @@ __device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const
     const TensorDesc &d = td[g.t];
     const u32 bh = (u32)d.bh, C = (u32)d.d1, nbc = (u32)d.nbc, nbr = (u32)(d.d0 / d.bh);
     const u32 local = (u32)(tile - tile_prefix[g.t]);
-    const u32 rpt = (u32)arr / (bh * C * 4u);
+    const u32 rpt = (u32)blockg_rows_per_tile(d, arr);
     const u32 brow0 = local * rpt;
     const u32 brows = nbr - brow0 < rpt ? nbr - brow0 : rpt;
     g.nq = brows * nbc;
