@@ -607,6 +607,7 @@ Layout plan_call(int op, const condensa_tensor *ts, int T, unsigned fuse, const 
     if (sampling && op == OP_BLOCKG1) {
         pl.tile_prefix.assign((size_t)T + 1, 0);
         for (int t = 0; t < T; ++t) {
+            pl.td[t].tile_rows = blockg_fast_end(pl.td[t], pl.bt_arr) > 0 ? (int)blockg_rows_per_tile(pl.td[t], pl.bt_arr) : 0;
             for (long long j = 0; j < pl.prefix_b[t + 1] - pl.prefix_b[t]; ++j)
                 if (!blockg_item_is_fast(pl.td[t], j, pl.bt_arr)) pl.edge_items.push_back(pl.prefix_b[t] + j);
             pl.tile_prefix[t + 1] = pl.tile_prefix[t] + blockg_tile_count(pl.td[t], pl.bt_arr);

@@ -52,7 +52,7 @@ struct TensorDesc {
     int bh, bw;              // general block pruning of matrices: block height and width
     int nd;                  // general n-D block pruning: dimensions cut (2: the fields above serve)
     int sh[4], bs[4], nb[4]; // ... extents, block extents and blocks per dimension, right-aligned to four
-    int pad2;
+    int tile_rows;           // tiled bh x bw kernel: block rows of one tile of this tensor (set by the host)
 };
 static_assert(sizeof(TensorDesc) % 8 == 0, "descriptor tables are copied word by word");
 

@@ -88,9 +88,9 @@ __device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const
     TileG g;
     g.t = find_tensor(tile_prefix, T, tile);
     const TensorDesc &d = td[g.t];
-    const u32 bh = (u32)d.bh, C = (u32)d.d1, nbc = (u32)d.nbc, nbr = (u32)(d.d0 / d.bh);
+    const u32 bh = (u32)d.bh, C = (u32)d.d1, nbc = (u32)d.nbc, nbr = (u32)d.d0 / bh;     // (fewer than 2^32 elements)
     const u32 local = (u32)(tile - tile_prefix[g.t]);
-    const u32 rpt = (u32)blockg_rows_per_tile(d, arr);
+    const u32 rpt = (u32)d.tile_rows;               // = blockg_rows_per_tile(d, arr), worked out by the host
     const u32 brow0 = local * rpt;
     const u32 brows = nbr - brow0 < rpt ? nbr - brow0 : rpt;
     g.nq = brows * nbc;
