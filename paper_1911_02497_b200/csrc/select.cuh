@@ -279,6 +279,25 @@ __device__ __forceinline__ u64 blockg_key_global(const TensorDesc &d, long long 
         }
     }
     double acc = 0.0;
+    if (e.nc <= 8) {
+        // a row at a time: its loads leave together (one round trip per row, not one per element)
+        for (int r = 0; r < e.nr; ++r) {
+            const long long off = (e.r0 + r) * d.d1 + e.c0;
+            float wv[8], lv[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                wv[c] = c < e.nc ? __ldg(d.w + off + c) : 0.0f;
+                lv[c] = (c < e.nc && has_lam) ? d.lam[off + c] : 0.0f;
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                if (c < e.nc) {
+                    const double x = (double)form_u(wv[c], lv[c], mu, has_lam);
+                    acc = __fma_rn(x, x, acc);
+                }
+        }
+        return (u64)__double_as_longlong(acc);
+    }
     for (int r = 0; r < e.nr; ++r) {
         const long long off = (e.r0 + r) * d.d1 + e.c0;
         for (int c = 0; c < e.nc; ++c) {
