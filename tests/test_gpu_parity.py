@@ -2,6 +2,7 @@
 the same seeded inputs. Integer / bit results must be identical; fp32 values are
 produced by the same single IEEE operations, so they are compared bit for bit as
 well (and within 1e-6 relative as the stated bar)."""
+import ctypes as C
 import math
 
 import numpy as np
@@ -767,6 +768,26 @@ def test_workspace_query_sizes_a_context_that_never_allocates():
         c.close()
     with pytest.raises(cstep.CondensaError):
         cstep.workspace_bytes(99, ds.table, ds.T)
+    # the same for 5 x 5 blocks, which take a single-pass kernel of their own (larger journal)
+    spec = cstep.StructureSpec(cstep.SPEC_BLOCKS, 0, cstep.CRITERIA["l2"], 2, (5, 5, 1, 1))
+    need5 = cstep.workspace_bytes(cstep.OP_BLOCK, ds.table, ds.T, ("lambda",), C.byref(spec))
+    assert need5 >= need
+    c0 = cstep.Context(0)
+    ds.reset_lambda()
+    ds.run(c0, "block", ws.sparsity, ws.mu, ("lambda",), (5, 5))
+    torch.cuda.synchronize()
+    c0.close()
+    ds.reset_lambda()
+    c = cstep.Context(0, need5)
+    try:
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info(0)
+        ds.run(c, "block", ws.sparsity, ws.mu, ("lambda",), (5, 5))
+        assert c.get_result().sampled == 1
+        free1, _ = torch.cuda.mem_get_info(0)
+        assert free1 == free0
+    finally:
+        c.close()
 
 
 def test_register_resident_route_of_short_lists(ctx):
