@@ -220,6 +220,10 @@ __global__ void __launch_bounds__(THREADS) k_blockgen_norms(Params P)
         for (int it = 0; it < BLOCKS_PER_ITEM / THREADS; ++it) {
             const long long b = local * BLOCKS_PER_ITEM + it * THREADS + threadIdx.x;
             if (b >= d.n_units) continue;
+            if (d.nd == 2 && crit == CRIT_L2) {     // blocks of a matrix by the L2 norm: rows fetched ahead, a row's loads together
+                P.arr_key[d.unit_prefix + b] = blockg_key_global(d, b, P.mu);
+                continue;
+            }
             long long rest = b;
             int bc[4];
 #pragma unroll
