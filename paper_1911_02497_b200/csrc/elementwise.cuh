@@ -231,12 +231,18 @@ __device__ __forceinline__ void process_linear_item_fast(const Params &P, const 
                     const long long e0 = e_base + eo;
                     long long f = (d.numel < 0x7FFFFFFFll) ? (long long)((u32)e0 / (u32)d.d1) : e0 / d.d1;
                     long long r = e0 - f * d.d1;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (r >= d.d1) { r -= d.d1; ++f; while (r >= d.d1) { r -= d.d1; ++f; } }
+                    if (r + 3 < d.d1) {             // the four elements lie in one filter (nearly always): one decision
                         const u64 sid = (u64)(d.unit_prefix + f);
-                        keep[j] = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
-                        ++r;
+                        const bool kp = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
+                        keep[0] = keep[1] = keep[2] = keep[3] = kp;
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (r >= d.d1) { r -= d.d1; ++f; while (r >= d.d1) { r -= d.d1; ++f; } }
+                            const u64 sid = (u64)(d.unit_prefix + f);
+                            keep[j] = keep_by_cutoff(P.arr_key[sid], sid, tau_key, tau_id);
+                            ++r;
+                        }
                     }
                 }
             }
