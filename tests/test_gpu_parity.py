@@ -555,6 +555,22 @@ def test_single_pass_general_blocks(ctx, block):
     ctx.set_seed(SEED)
 
 
+def test_block_shapes_alternate_on_one_context(ctx):
+    """One context serves 4 x 4, 5 x 5 and 2 x 2 block calls and an unstructured call in turn, at sizes
+    that take the single-pass kernels: workspace layout, descriptor cache and shared-memory
+    configuration change from call to call."""
+    ws = W.random_set([(2500, 1200), (803, 1000), (77,), (1000, 640)], seed=91, kind="uniform", scale=0.1,
+                      lam_sigma=1e-3, mu=1e-2)
+    # (2 x 2 at s = 0.7: the sample's bracket would hold more blocks than the list takes, so the
+    # selection kernel does the two-pass job for that call)
+    for block, s, single in (((4, 4), 0.9, 1), ((5, 5), 0.9, 1), ((2, 2), 0.7, 0), ((5, 5), 0.5, 1), ((2, 2), 0.9, 1),
+                             ((4, 4), 0.6, 1)):
+        got, res, _ = check(ctx, "block", ws.w, ws.lam, s, ws.mu, ("lambda",), block=block)
+        assert res.sampled == single, block
+        got, res, _ = check(ctx, "prune", ws.w, ws.lam, 0.8, ws.mu, ("lambda", "penalty"))
+        assert res.sampled == 1
+
+
 def test_single_pass_general_blocks_fall_back(ctx):
     """A list whose block norms are nearly all equal: the sample advises against the single pass and
     the selection kernel does the two-pass job for bh x bw blocks itself."""
