@@ -1,9 +1,10 @@
-// Single-pass projection for bh x bw blocks of matrices (any block shape but 4 x 4, which has
-// its own kernel): the sample bracket, one pass that writes everything, the exact selection
+// Single-pass projection for bh x bw blocks of matrices (block shapes other than 4 x 4, which
+// has its own kernel): the sample bracket, one pass that writes everything, the exact selection
 // on the listed candidates. A block row - bh matrix rows - is one contiguous range of memory,
 // so the pass moves whole block rows through shared memory exactly like the 4 x 4 kernel
-// does; only the per-block arithmetic differs (runtime loops over the rows and columns of a
-// block that exist, in row-major order: the order of the plain definition).
+// does; only the per-block arithmetic differs: unrolled at compile time for the shapes the
+// kernel is built for, loops over the rows and columns that exist for a block of ragged width,
+// always in row-major order (the order of the plain definition).
 #pragma once
 #include "fused_fast.cuh"
 
@@ -83,14 +84,14 @@ struct TileG {
     u32 off0;           // element offset of the tile's first row
 };
 
-__device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const TensorDesc *td, int T, long long tile, int arr)
+__device__ __forceinline__ TileG tile_geom_g(const long long *tile_prefix, const TensorDesc *td, int T, long long tile)
 {
     TileG g;
     g.t = find_tensor(tile_prefix, T, tile);
     const TensorDesc &d = td[g.t];
     const u32 bh = (u32)d.bh, C = (u32)d.d1, nbc = (u32)d.nbc, nbr = (u32)d.d0 / bh;     // (fewer than 2^32 elements)
     const u32 local = (u32)(tile - tile_prefix[g.t]);
-    const u32 rpt = (u32)d.tile_rows;               // = blockg_rows_per_tile(d, arr), worked out by the host
+    const u32 rpt = (u32)d.tile_rows;               // = blockg_rows_per_tile(), worked out by the host
     const u32 brow0 = local * rpt;
     const u32 brows = nbr - brow0 < rpt ? nbr - brow0 : rpt;
     g.nq = brows * nbc;
@@ -342,7 +343,7 @@ __global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
                 if (!P.ctl->sel.onepass) { quiet = true; ok = false; }
             };
             auto store_tile = [&](long long tile, int stage) {
-                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
+                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile);
                 const TensorDesc &d = td[g.t];
                 const bool upd = (P.fuse & FUSE_LAMBDA) && d.lam != nullptr;
                 const u32 bytes = g.nrows * (u32)d.d1 * 4u;
@@ -378,7 +379,7 @@ __global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
                     bulk_wait_read_all();               // shared memory has been read: the buffer is free
                 }
                 if (*abort_flag) { ok = false; break; }
-                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
+                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile);
                 const TensorDesc &d = td[g.t];
                 const bool has_lam = d.lam != nullptr;
                 const u32 bytes = g.nrows * (u32)d.d1 * 4u;
@@ -431,7 +432,7 @@ __global__ void __launch_bounds__(BG_THREADS, 1) k_fused_blockg(Params P)
                 }
             }
             if (ok) {
-                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile, arr);
+                const TileG g = tile_geom_g(tile_prefix, td, P.T, tile);
                 const TensorDesc &d = td[g.t];
                 const bool has_lam = d.lam != nullptr;
                 const bool upd = (P.fuse & FUSE_LAMBDA) && has_lam;
